@@ -1,0 +1,120 @@
+/* hola_verify.h - C ABI of the B200 (sm_100a) library for the entropy-aware verify step of Hierarchical
+ * Speculative Decoding (HSD).
+ *
+ * One call verifies k draft tokens for each of B sequences:
+ *   1. LM-head projection of the verifier for the k+1 verify positions,  l[r,v] = sum_h hidden[r,h] * W_lm[v,h]
+ *      (the "higher-fidelity verifier" f_ver of the HSD section, restricted to its output layer);
+ *   2. softmax statistics and Shannon entropy per position,  H = -sum_i p_i log p_i  in nats (HSD section);
+ *   3. the entropy gate  g(t) = 1[H < tau]  and Eq. (1): a gated position keeps its draft token, any other
+ *      position falls back to the verifier (Algorithm 1, lines 4-8);
+ *   4. the fallback itself, which the paper leaves open, is the speculative-sampling test: accept draft token x
+ *      iff  u * q(x) < p(x)  (u < min(1, p/q)); the first position that is not accepted ends the run;
+ *   5. one new token per sequence: from the normalised residual max(0, p - q) at the first rejected position,
+ *      or from p at position k when every draft was accepted, by inverse CDF with the supplied uniform
+ *      (ascending token id, first token whose cumulative mass exceeds u * total).
+ *
+ * All pointers in hola_verify_args are DEVICE pointers unless a field says otherwise.  Every buffer is owned by
+ * the caller.  The library allocates device memory only inside hola_create and frees it in hola_destroy.
+ * No function throws, aborts or exits; each returns a hola_status.
+ */
+#ifndef HOLA_VERIFY_H_
+#define HOLA_VERIFY_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct hola_ctx hola_ctx; /* opaque: workspace, cached TMA descriptors, device properties */
+
+typedef enum {
+  HOLA_OK = 0,
+  HOLA_ERR_INVALID_ARG = 1,       /* null pointer, non-positive size, misaligned buffer */
+  HOLA_ERR_UNSUPPORTED_SHAPE = 2, /* H % 8 != 0, or B / k / H / V beyond what the context was created for */
+  HOLA_ERR_WORKSPACE = 3,         /* device allocation failed in hola_create */
+  HOLA_ERR_CUDA = 4,              /* a CUDA runtime or driver call failed; see hola_last_cuda_error */
+  HOLA_ERR_NO_DEVICE = 5          /* no sm_100 device, or the driver lacks tensor-map support */
+} hola_status;
+
+typedef enum { HOLA_Q_BF16 = 0, HOLA_Q_F32 = 1 } hola_q_dtype;
+
+/* Bits of the device status word (OR-ed by the kernels; the caller clears it). */
+#define HOLA_FLAG_BAD_TOKEN 1u   /* a draft token outside [0,V): treated as a rejection at that position    */
+#define HOLA_FLAG_BAD_UNIFORM 2u /* a uniform outside [0,1): clamped into [0, 1 - 2^-24]                     */
+#define HOLA_FLAG_TIMEOUT 4u     /* an on-chip wait ran out of iterations; outputs of this call are invalid  */
+#define HOLA_FLAG_R_ZERO 8u      /* residual mass was zero (p <= q everywhere): token drawn from p instead   */
+
+typedef struct {
+  int32_t B; /* sequences, >= 0 */
+  int32_t k; /* draft tokens per sequence, >= 0; k = 0 is a plain draw from p_0 */
+  int32_t H; /* hidden size, multiple of 8 (row pitch must be a multiple of 16 bytes) */
+  int32_t V; /* vocabulary size, >= 1 */
+  const void* hidden;      /* bf16 [B][k+1][H], contiguous, 16-byte aligned                                   */
+  const void* W_lm;        /* bf16 [V][H], contiguous, 16-byte aligned; read exactly once per call            */
+  const int32_t* draft_tok;/* int32 [B][k]                                                                    */
+  const void* draft_q;     /* [B][k][V] in q_dtype: the draft model's probabilities, used as given             */
+  int32_t q_dtype;         /* hola_q_dtype                                                                    */
+  const float* uniforms;   /* fp32 [B][k+1] in [0,1): [b][j<k] feeds accept test j, [b][k] feeds the one draw  */
+  float tau;               /* entropy threshold in nats (paper: 1.5).  tau <= 0 or NaN: gate off; +inf: all on */
+  int32_t* accept_len;     /* out int32 [B], 0..k: number of draft tokens kept                                */
+  int32_t* next_tok;       /* out int32 [B], 0..V-1: the token that follows them                              */
+  float* entropy;          /* out fp32 [B][k+1], nats, >= 0                                                    */
+  float* logZ;             /* out fp32 [B][k+1], log-sum-exp of the logits                                     */
+  float* logits_out;       /* out fp32 [B][k+1][V], optional (NULL: the context's own scratch is used)         */
+  uint32_t* status_word;   /* in/out uint32 [1], optional: HOLA_FLAG_* bits are OR-ed in                       */
+} hola_verify_args;
+
+/* Creates a context on `device` able to serve calls with B <= maxB, k <= maxK and exactly this H and V.
+ * Allocates the workspace (hola_workspace_bytes) once.  One context serves one stream at a time. */
+hola_status hola_create(hola_ctx** out, int device, int maxB, int maxK, int H, int V);
+hola_status hola_destroy(hola_ctx* ctx);
+
+/* Device bytes a context of these limits holds: fp32 logits scratch [B(k+1)][V], per-CTA softmax partials,
+ * staging for hola_verify_host, a status word. */
+size_t hola_workspace_bytes(int maxB, int maxK, int H, int V);
+
+/* Enqueues the whole verify step (steps 1-5 above) on `cuda_stream` (a cudaStream_t; NULL = default stream).
+ * Asynchronous: no synchronisation, no host read-back.  The return code covers host-detectable errors only;
+ * device-detected conditions are reported through status_word and never fault. */
+hola_status hola_verify(hola_ctx* ctx, const hola_verify_args* args, void* cuda_stream);
+
+/* End-to-end form for callers whose per-step data lives in host memory.  Same computation as hola_verify, but
+ * hidden, draft_tok, draft_q, uniforms are HOST pointers (pinned memory makes the copies asynchronous) and
+ * accept_len, next_tok, entropy, logZ, status_word are HOST outputs; logits_out is ignored.  W_lm stays a
+ * DEVICE pointer: weights are resident.  Copies in, runs, copies out and synchronises the stream. */
+hola_status hola_verify_host(hola_ctx* ctx, const hola_verify_args* args, void* cuda_stream);
+
+/* Partial entry points, the steps of the path exposed one by one (same argument struct).
+ * hola_lm_head_entropy: steps 1-2 only; fills logits (logits_out or scratch), entropy, logZ.
+ * hola_accept_sample:   steps 3-5 only, from fp32 logits in args->logits_out (required) and the entropy / logZ
+ *                       arrays already present in args->entropy / args->logZ (inputs here). */
+hola_status hola_lm_head_entropy(hola_ctx* ctx, const hola_verify_args* args, void* cuda_stream);
+hola_status hola_accept_sample(hola_ctx* ctx, const hola_verify_args* args, void* cuda_stream);
+
+/* Launch geometry chosen for a shape (for reports): vocab tile width, grid size, pipeline stages,
+ * row blocks of 128 positions per pass, passes over W_lm. */
+typedef struct {
+  int32_t tile_n, grid, stages, row_blocks, passes, kernels_per_call;
+} hola_plan_info;
+hola_status hola_plan(const hola_ctx* ctx, int B, int k, hola_plan_info* out);
+
+/* Per-kernel timing for reports.  Between hola_profile_begin and hola_profile_end every hola_verify call (at
+ * most max_calls of them, max_calls <= 4096) records CUDA events on its stream around the LM-head GEMM launches
+ * and around the accept/sample launch.  hola_profile_end synchronises the stream and returns the summed
+ * durations in milliseconds and the number of calls recorded.  Creates events (no device memory). */
+hola_status hola_profile_begin(hola_ctx* ctx, int max_calls);
+hola_status hola_profile_end(hola_ctx* ctx, void* cuda_stream, double* lm_head_ms, double* accept_sample_ms,
+                             int* calls);
+
+const char* hola_strerror(hola_status s);
+/* Text of the last CUDA error seen by this context (empty string if none). */
+const char* hola_last_cuda_error(const hola_ctx* ctx);
+/* Library version, "major.minor". */
+const char* hola_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HOLA_VERIFY_H_ */

@@ -1,0 +1,235 @@
+"""ctypes binding of libhola_verify.so: argument marshalling only, every step runs in the CUDA kernels.
+
+Function names mirror the C ABI (include/hola_verify.h).  Tensors are torch CUDA tensors; torch is used for
+device memory and streams, nothing else.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+from . import build as _build
+
+HOLA_OK = 0
+HOLA_Q_BF16, HOLA_Q_F32 = 0, 1
+FLAG_BAD_TOKEN, FLAG_BAD_UNIFORM, FLAG_TIMEOUT, FLAG_R_ZERO = 1, 2, 4, 8
+
+EXPORTS = ["hola_create", "hola_destroy", "hola_workspace_bytes", "hola_verify", "hola_verify_host",
+           "hola_lm_head_entropy", "hola_accept_sample", "hola_plan", "hola_profile_begin", "hola_profile_end", "hola_strerror", "hola_last_cuda_error",
+           "hola_version"]
+
+
+class HolaError(RuntimeError):
+    pass
+
+
+class hola_verify_args(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("k", ctypes.c_int32), ("H", ctypes.c_int32), ("V", ctypes.c_int32),
+                ("hidden", ctypes.c_void_p), ("W_lm", ctypes.c_void_p), ("draft_tok", ctypes.c_void_p),
+                ("draft_q", ctypes.c_void_p), ("q_dtype", ctypes.c_int32), ("uniforms", ctypes.c_void_p),
+                ("tau", ctypes.c_float), ("accept_len", ctypes.c_void_p), ("next_tok", ctypes.c_void_p),
+                ("entropy", ctypes.c_void_p), ("logZ", ctypes.c_void_p), ("logits_out", ctypes.c_void_p),
+                ("status_word", ctypes.c_void_p)]
+
+
+class hola_plan_info(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("tile_n", "grid", "stages", "row_blocks", "passes", "kernels_per_call")]
+
+
+_lib = None
+
+
+def load_library(path: str | None = None) -> ctypes.CDLL:
+    """Loads the C-ABI library (building it first if the source is newer).  Raises if it cannot be had."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    p = path or (_build.LIB if os.path.exists(_build.LIB) and not _build.needs_build() else _build.build())
+    lib = ctypes.CDLL(p)
+    lib.hola_create.restype = ctypes.c_int
+    lib.hola_create.argtypes = [ctypes.POINTER(ctypes.c_void_p), ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                ctypes.c_int, ctypes.c_int]
+    lib.hola_destroy.restype = ctypes.c_int
+    lib.hola_destroy.argtypes = [ctypes.c_void_p]
+    lib.hola_workspace_bytes.restype = ctypes.c_size_t
+    lib.hola_workspace_bytes.argtypes = [ctypes.c_int] * 4
+    for name in ("hola_verify", "hola_verify_host", "hola_lm_head_entropy", "hola_accept_sample"):
+        fn = getattr(lib, name)
+        fn.restype = ctypes.c_int
+        fn.argtypes = [ctypes.c_void_p, ctypes.POINTER(hola_verify_args), ctypes.c_void_p]
+    lib.hola_plan.restype = ctypes.c_int
+    lib.hola_plan.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.POINTER(hola_plan_info)]
+    lib.hola_profile_begin.restype = ctypes.c_int
+    lib.hola_profile_begin.argtypes = [ctypes.c_void_p, ctypes.c_int]
+    lib.hola_profile_end.restype = ctypes.c_int
+    lib.hola_profile_end.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(ctypes.c_double),
+                                     ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_int)]
+    lib.hola_strerror.restype = ctypes.c_char_p
+    lib.hola_strerror.argtypes = [ctypes.c_int]
+    lib.hola_last_cuda_error.restype = ctypes.c_char_p
+    lib.hola_last_cuda_error.argtypes = [ctypes.c_void_p]
+    lib.hola_version.restype = ctypes.c_char_p
+    if path is None:
+        _lib = lib
+    return lib
+
+
+def _check(lib, ctx, status: int, what: str):
+    if status != HOLA_OK:
+        msg = lib.hola_strerror(status).decode()
+        detail = lib.hola_last_cuda_error(ctx).decode() if ctx else ""
+        raise HolaError(f"{what}: {msg}" + (f" [{detail}]" if detail else ""))
+
+
+def _dptr(t: torch.Tensor | None):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream_ptr(stream) -> ctypes.c_void_p:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+@dataclass
+class VerifyOutputs:
+    accept_len: torch.Tensor   # int32 [B]
+    next_tok: torch.Tensor     # int32 [B]
+    entropy: torch.Tensor      # fp32 [B, k+1]
+    logZ: torch.Tensor         # fp32 [B, k+1]
+    logits: torch.Tensor | None
+    status: torch.Tensor       # uint32 as int32 [1]
+
+
+class HolaVerify:
+    """Owns one hola_ctx.  Methods are named after the C entry points they call."""
+
+    def __init__(self, maxB: int, maxK: int, H: int, V: int, device: int | None = None):
+        if not torch.cuda.is_available():
+            raise HolaError("hola_create: no CUDA device; this library has no CPU path")
+        self.lib = load_library()
+        self.device = torch.cuda.current_device() if device is None else int(device)
+        self.maxB, self.maxK, self.H, self.V = maxB, maxK, H, V
+        self._ctx = ctypes.c_void_p()
+        st = self.lib.hola_create(ctypes.byref(self._ctx), self.device, maxB, maxK, H, V)
+        _check(self.lib, None, st, "hola_create")
+
+    def close(self):
+        if getattr(self, "_ctx", None) and self._ctx.value:
+            self.lib.hola_destroy(self._ctx)
+            self._ctx = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+    # -------------------------------------------------------------------------------------------------
+    def hola_plan(self, B: int, k: int) -> dict:
+        info = hola_plan_info()
+        _check(self.lib, self._ctx, self.lib.hola_plan(self._ctx, B, k, ctypes.byref(info)), "hola_plan")
+        return {n: getattr(info, n) for n, _ in info._fields_}
+
+    def hola_profile_begin(self, max_calls: int):
+        _check(self.lib, self._ctx, self.lib.hola_profile_begin(self._ctx, max_calls), "hola_profile_begin")
+
+    def hola_profile_end(self, stream=None) -> dict:
+        a, b, n = ctypes.c_double(), ctypes.c_double(), ctypes.c_int()
+        st = self.lib.hola_profile_end(self._ctx, _stream_ptr(stream), ctypes.byref(a), ctypes.byref(b), ctypes.byref(n))
+        _check(self.lib, self._ctx, st, "hola_profile_end")
+        return {"lm_head_ms": a.value, "accept_sample_ms": b.value, "calls": n.value}
+
+    def _args(self, hidden, W_lm, draft_tok, draft_q, uniforms, tau, out: VerifyOutputs, B, k):
+        if hidden.dtype != torch.bfloat16 or W_lm.dtype != torch.bfloat16:
+            raise HolaError("hidden and W_lm must be bfloat16")
+        if draft_q is not None and draft_q.dtype not in (torch.bfloat16, torch.float32):
+            raise HolaError("draft_q must be bfloat16 or float32")
+        for t in (hidden, W_lm, draft_tok, draft_q, uniforms):
+            if t is not None and not t.is_contiguous():
+                raise HolaError("all inputs must be contiguous")
+        a = hola_verify_args()
+        a.B, a.k, a.H, a.V = B, k, self.H, self.V
+        a.hidden, a.W_lm = _dptr(hidden), _dptr(W_lm)
+        a.draft_tok = _dptr(draft_tok) if k > 0 else None
+        a.draft_q = _dptr(draft_q) if k > 0 else None
+        a.q_dtype = HOLA_Q_F32 if (draft_q is not None and draft_q.dtype == torch.float32) else HOLA_Q_BF16
+        a.uniforms = _dptr(uniforms)
+        a.tau = float(tau)
+        a.accept_len, a.next_tok = _dptr(out.accept_len), _dptr(out.next_tok)
+        a.entropy, a.logZ = _dptr(out.entropy), _dptr(out.logZ)
+        a.logits_out = _dptr(out.logits)
+        a.status_word = _dptr(out.status)
+        return a
+
+    def alloc_outputs(self, B: int, k: int, want_logits: bool = False, device=None) -> VerifyOutputs:
+        dev = torch.device("cuda", self.device) if device is None else device
+        return VerifyOutputs(
+            accept_len=torch.empty(B, dtype=torch.int32, device=dev),
+            next_tok=torch.empty(B, dtype=torch.int32, device=dev),
+            entropy=torch.empty((B, k + 1), dtype=torch.float32, device=dev),
+            logZ=torch.empty((B, k + 1), dtype=torch.float32, device=dev),
+            logits=torch.empty((B, k + 1, self.V), dtype=torch.float32, device=dev) if want_logits else None,
+            status=torch.zeros(1, dtype=torch.int32, device=dev))
+
+    def hola_verify(self, hidden, W_lm, draft_tok, draft_q, uniforms, tau, out: VerifyOutputs | None = None,
+                    want_logits: bool = False, stream=None) -> VerifyOutputs:
+        """The whole verify step on device tensors, asynchronous on the stream."""
+        B, k = hidden.shape[0], hidden.shape[1] - 1
+        out = out or self.alloc_outputs(B, k, want_logits)
+        a = self._args(hidden, W_lm, draft_tok, draft_q, uniforms, tau, out, B, k)
+        _check(self.lib, self._ctx, self.lib.hola_verify(self._ctx, ctypes.byref(a), _stream_ptr(stream)), "hola_verify")
+        return out
+
+    def hola_lm_head_entropy(self, hidden, W_lm, out: VerifyOutputs | None = None, want_logits: bool = True,
+                             stream=None) -> VerifyOutputs:
+        B, k = hidden.shape[0], hidden.shape[1] - 1
+        out = out or self.alloc_outputs(B, k, want_logits)
+        a = self._args(hidden, W_lm, None, None, None, 0.0, out, B, k)
+        _check(self.lib, self._ctx, self.lib.hola_lm_head_entropy(self._ctx, ctypes.byref(a), _stream_ptr(stream)),
+               "hola_lm_head_entropy")
+        return out
+
+    def hola_accept_sample(self, logits, entropy, logZ, draft_tok, draft_q, uniforms, tau, stream=None) -> VerifyOutputs:
+        """Steps 3-5 from given fp32 logits [B, k+1, V] and their entropy / logZ."""
+        B, k = logits.shape[0], logits.shape[1] - 1
+        out = self.alloc_outputs(B, k, False)
+        out.logits = logits
+        out.entropy.copy_(entropy)
+        out.logZ.copy_(logZ)
+        a = hola_verify_args()
+        a.B, a.k, a.H, a.V = B, k, self.H, self.V
+        a.draft_tok = _dptr(draft_tok) if k > 0 else None
+        a.draft_q = _dptr(draft_q) if k > 0 else None
+        a.q_dtype = HOLA_Q_F32 if (draft_q is not None and draft_q.dtype == torch.float32) else HOLA_Q_BF16
+        a.uniforms, a.tau = _dptr(uniforms), float(tau)
+        a.accept_len, a.next_tok = _dptr(out.accept_len), _dptr(out.next_tok)
+        a.entropy, a.logZ, a.logits_out, a.status_word = _dptr(out.entropy), _dptr(out.logZ), _dptr(logits), _dptr(out.status)
+        _check(self.lib, self._ctx, self.lib.hola_accept_sample(self._ctx, ctypes.byref(a), _stream_ptr(stream)),
+               "hola_accept_sample")
+        return out
+
+    def hola_verify_host(self, hidden, W_lm, draft_tok, draft_q, uniforms, tau, out: VerifyOutputs | None = None,
+                         stream=None) -> VerifyOutputs:
+        """End-to-end form: per-step inputs and all outputs are HOST tensors (pinned for async copies);
+        W_lm is the resident device weight.  Returns after the stream has been synchronised."""
+        B, k = hidden.shape[0], hidden.shape[1] - 1
+        if W_lm.device.type != "cuda":
+            raise HolaError("W_lm must be resident on the device")
+        for t in (hidden, draft_tok, draft_q, uniforms):
+            if t is not None and t.device.type != "cpu":
+                raise HolaError("hola_verify_host takes host tensors for the per-step inputs")
+        out = out or self.alloc_outputs(B, k, False, device=torch.device("cpu"))
+        a = self._args(hidden, W_lm, draft_tok, draft_q, uniforms, tau, out, B, k)
+        a.logits_out = None
+        _check(self.lib, self._ctx, self.lib.hola_verify_host(self._ctx, ctypes.byref(a), _stream_ptr(stream)),
+               "hola_verify_host")
+        return out

@@ -1,0 +1,1153 @@
+// hola_verify.cu - sm_100a kernels and C ABI for the entropy-aware verify step of Hierarchical Speculative
+// Decoding (HSD section, Eq. 1, Algorithm 1 lines 4-8).  See include/hola_verify.h for the contract.
+//
+// Kernels
+//   lm_head_entropy_kernel<RB>  persistent, warp-specialised weight-streaming GEMM.  One CTA per SM walks vocab
+//       tiles; a producer thread feeds a shared-memory ring with TMA (128-byte-swizzled K-major tiles of W_lm and
+//       of up to RB blocks of 128 verify positions); one thread issues tcgen05.mma (bf16 x bf16 -> fp32 in
+//       tensor memory); four epilogue warps read the accumulators with tcgen05.ld, store fp32 logits and keep,
+//       per verify position, the running softmax statistics (m, s, t) = (max, sum e^(l-m), sum e^(l-m)(l-m)) in
+//       registers across all of the CTA's tiles.  W_lm is read from HBM once per pass.
+//   finalize_kernel             merges the per-CTA statistics:  logZ = m + ln s,  H = ln s - t/s  (entropy
+//       definition of the HSD section, rearranged around the running maximum).
+//   accept_sample_kernel        one CTA per sequence: merges the statistics for its k+1 positions (warp
+//       shuffles), applies the entropy gate and the ratio test in draft order, then makes one vectorised pass
+//       over the logits row and the draft row of the first rejected position: residual max(0, p - q), per-chunk
+//       sums, a scan, and the inverse-CDF pick with the supplied uniform.
+//
+// Every on-chip wait is bounded: when a wait runs out the CTA raises HOLA_FLAG_TIMEOUT, leaves its loops,
+// releases its tensor memory and returns.
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <math_constants.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include "../../include/hola_verify.h"
+
+namespace {
+
+// ------------------------------------------------------------------------------------------------ constants
+constexpr int kBlockK = 64;                      // bf16 elements per K block = one 128-byte swizzle row
+constexpr int kRows = 128;                       // verify positions per row block = tensor-memory lanes
+constexpr int kABlockBytes = kRows * kBlockK * 2;
+constexpr int kK1Threads = 192;                  // warp 0 TMA, warp 1 MMA + tensor-memory owner, warps 2-5 epilogue
+constexpr int kTmemCols = 512;
+constexpr int kMaxStages = 8;
+constexpr int kMaxRowBlocks = 4;
+constexpr int kSmemBudget = 227 * 1024;          // dynamic shared memory per CTA on sm_100
+constexpr int kBarrierBytes = 256;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait, far above any legitimate wait
+
+constexpr int kK3Threads = 512;
+constexpr int kK3Warps = kK3Threads / 32;
+constexpr int kChunk = 128;                      // vocabulary entries per warp step (32 lanes x 4)
+constexpr int kMaxChunks = 4096;                 // => V <= 524288
+constexpr int kMaxK1 = 64;                       // k + 1 <= 64
+
+constexpr float kLog2e = 1.4426950408889634f;
+
+struct K1Params {
+  int M;          // total verify rows B(k+1)
+  int row0;       // first row of this pass
+  int V, tile_n, n_tiles, n_kblocks, stages, nbuf;
+  int ldl;        // row pitch of the logits buffer, in floats
+  int vec_ok;     // 16-byte stores allowed (pitch and base aligned)
+  float* logits;
+  float4* partials;   // [grid][part_stride] (m, s, t, unused)
+  int part_stride;
+  unsigned* status;
+};
+
+struct K3Params {
+  int B, k, V, ldl;
+  const float* logits;
+  const float4* partials;
+  int nparts, part_stride, combine;
+  const int* tok;
+  const void* q;
+  int q_dtype;
+  const float* u;
+  float tau;
+  int* accept_len;
+  int* next_tok;
+  float* entropy;
+  float* logZ;
+  unsigned* status;
+};
+
+// ------------------------------------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred P1;\n mbarrier.try_wait.parity.shared::cta.b64 P1, [%1], %2;\n selp.u32 %0, 1, 0, P1;\n}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
+// Bounded wait.  Returns false when the CTA is aborting (this wait or another one ran out of time).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                          unsigned* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = globaltimer_ns();
+  uint32_t spins = 0;
+  while (true) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((++spins & 63u) == 0u) {
+      if (*abort_flag) return false;
+      if (globaltimer_ns() - t0 > kWaitLimitNs) {
+        *abort_flag = 1u;
+        if (status) atomicOr(status, HOLA_FLAG_TIMEOUT);
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+
+// 2-D tiled TMA load, global -> this CTA's shared memory, completion counted on an mbarrier.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y,
+                                            uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%3, %4}], [%2], %5;"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "l"(policy)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t holder_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(holder_smem), "r"(ncols)
+               : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+
+// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate, issued by one thread.
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+      " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// mbarrier arrives once every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// 32 consecutive fp32 columns of this thread's tensor-memory lane.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// Shared-memory matrix descriptor: K-major tile whose rows are 128 bytes, 128-byte swizzle, 8-row groups
+// 1024 bytes apart (stride byte offset), descriptor version 1 (sm_100).
+__device__ __forceinline__ uint64_t make_kmajor_sw128_desc(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4);      // start address, 16-byte units
+  d |= static_cast<uint64_t>(1) << 16;                          // leading byte offset: unused with swizzled K-major
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;                  // stride byte offset
+  d |= static_cast<uint64_t>(1) << 46;                          // version
+  d |= static_cast<uint64_t>(2) << 61;                          // layout: 128-byte swizzle
+  return d;
+}
+
+// Instruction descriptor, kind::f16: D fp32, A and B bf16, both K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t make_idesc_bf16_m128(uint32_t n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((n >> 3) << 17) | ((128u >> 4) << 24);
+}
+
+// ------------------------------------------------------------------------------------------------ softmax statistics
+// Statistics of a set of logits around its maximum m:  s = sum e^(l-m),  t = sum e^(l-m) (l-m).
+// logZ = m + ln s;  H = -sum p ln p = ln s - t/s.
+struct Stats {
+  float m, s, t;
+};
+__device__ __forceinline__ Stats stats_empty() { return Stats{-CUDART_INF_F, 0.f, 0.f}; }
+
+__device__ __forceinline__ Stats stats_merge(Stats a, Stats b) {
+  if (b.m == -CUDART_INF_F) return a;
+  if (a.m == -CUDART_INF_F) return b;
+  const float m = fmaxf(a.m, b.m);
+  const float da = a.m - m, db = b.m - m;
+  const float ea = __expf(da), eb = __expf(db);
+  Stats r;
+  r.m = m;
+  r.s = ea * a.s + eb * b.s;
+  r.t = ea * (a.t + da * a.s) + eb * (b.t + db * b.s);
+  return r;
+}
+
+// Fold `n` (1..32) logits into the running statistics.
+template <bool kFull>
+__device__ __forceinline__ void stats_fold(const float* v, int n, Stats& st) {
+  float cmax = v[0];
+#pragma unroll
+  for (int i = 1; i < 32; ++i)
+    if (kFull || i < n) cmax = fmaxf(cmax, v[i]);
+  if (cmax > st.m) {
+    if (st.m != -CUDART_INF_F) {
+      const float d = st.m - cmax;
+      const float sc = ex2_approx(d * kLog2e);
+      st.t = sc * (st.t + d * st.s);
+      st.s *= sc;
+    }
+    st.m = cmax;
+  }
+  const float m = st.m;
+  const float mneg2 = -m * kLog2e;
+  float s = st.s, t = st.t;
+#pragma unroll
+  for (int i = 0; i < 32; ++i) {
+    if (kFull || i < n) {
+      const float e = ex2_approx(fmaf(v[i], kLog2e, mneg2));
+      s += e;
+      t = fmaf(e, v[i] - m, t);
+    }
+  }
+  st.s = s;
+  st.t = t;
+}
+
+// ------------------------------------------------------------------------------------------------ K1
+template <int RB>
+__global__ void __launch_bounds__(kK1Threads, 1)
+lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __grid_constant__ CUtensorMap tmap_w,
+                       const K1Params p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;          // 128-byte swizzle wants 1024-byte aligned tiles
+  uint8_t* smem = smem_raw + (base - raw);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t stage_bytes = RB * kABlockBytes + p.tile_n * 128;
+  const uint32_t bar_base = base + p.stages * stage_bytes;
+  // barrier area: full[8] | empty[8] | tmem_full[2] | tmem_empty[2] | tmem holder | abort flag
+  const uint32_t full_bar = bar_base, empty_bar = bar_base + 64, tfull_bar = bar_base + 128,
+                 tempty_bar = bar_base + 144;
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + p.stages * stage_bytes + 160);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + p.stages * stage_bytes + 164);
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < p.stages; ++i) {
+      mbar_init(full_bar + 8 * i, 1);
+      mbar_init(empty_bar + 8 * i, 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(tfull_bar + 8 * i, 1);
+      mbar_init(tempty_bar + 8 * i, 4);                  // one arrival per epilogue warp
+    }
+    *abort_flag = 0u;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_hidden) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_w) : "memory");
+  }
+  if (warp == 1) tmem_alloc(smem_u32(tmem_holder), kTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_holder;
+
+  const int acc_cols = RB * p.tile_n;
+  const int my_tiles = (p.n_tiles - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) /
+                       static_cast<int>(gridDim.x);
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      const uint64_t pol_w = l2_policy_evict_first();    // W_lm is streamed once
+      const uint64_t pol_h = l2_policy_evict_last();     // hidden is re-read by every CTA for every tile
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int t = 0; t < my_tiles && ok; ++t) {
+        const int tile = blockIdx.x + t * gridDim.x;
+        for (int kb = 0; kb < p.n_kblocks; ++kb) {
+          if (!mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
+          const uint32_t sa = base + stage * stage_bytes;
+          const uint32_t fb = full_bar + 8 * stage;
+          mbar_expect_tx(fb, stage_bytes);
+#pragma unroll
+          for (int a = 0; a < RB; ++a)
+            tma_load_2d(sa + a * kABlockBytes, &tmap_hidden, fb, kb * kBlockK, p.row0 + a * kRows, pol_h);
+          tma_load_2d(sa + RB * kABlockBytes, &tmap_w, fb, kb * kBlockK, tile * p.tile_n, pol_w);
+          if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = make_idesc_bf16_m128(static_cast<uint32_t>(p.tile_n));
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int t = 0; t < my_tiles && ok; ++t) {
+        const int buf = t % p.nbuf;
+        const uint32_t acc_phase = static_cast<uint32_t>(t / p.nbuf) & 1u;
+        if (!mbar_wait(tempty_bar + 8 * buf, acc_phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d0 = tmem_base + buf * acc_cols;
+        for (int kb = 0; kb < p.n_kblocks; ++kb) {
+          if (!mbar_wait(full_bar + 8 * stage, phase, abort_flag, p.status)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = base + stage * stage_bytes;
+          const uint64_t bdesc = make_kmajor_sw128_desc(sa + RB * kABlockBytes);
+#pragma unroll
+          for (int a = 0; a < RB; ++a) {
+            const uint64_t adesc = make_kmajor_sw128_desc(sa + a * kABlockBytes);
+#pragma unroll
+            for (int kk = 0; kk < kBlockK / 16; ++kk) {
+              // 16 bf16 = 32 bytes further along K inside the swizzled row: +2 in 16-byte address units
+              umma_bf16(d0 + a * p.tile_n, adesc + 2 * kk, bdesc + 2 * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
+            }
+          }
+          umma_commit(empty_bar + 8 * stage);            // frees the stage once these MMAs have read it
+          if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+        }
+        if (ok) umma_commit(tfull_bar + 8 * buf);        // accumulators of this tile are complete
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue warps 2..5
+    const int quarter = warp & 3;                        // tensor-memory lanes 32*quarter .. +31
+    Stats st[RB];
+    int row[RB];
+    bool row_ok[RB], warp_has_rows[RB];
+#pragma unroll
+    for (int a = 0; a < RB; ++a) {
+      st[a] = stats_empty();
+      row[a] = p.row0 + a * kRows + quarter * 32 + lane;
+      row_ok[a] = row[a] < p.M;
+      warp_has_rows[a] = (p.row0 + a * kRows + quarter * 32) < p.M;
+    }
+    bool ok = true;
+    for (int t = 0; t < my_tiles && ok; ++t) {
+      const int tile = blockIdx.x + t * gridDim.x;
+      const int buf = t % p.nbuf;
+      const uint32_t acc_phase = static_cast<uint32_t>(t / p.nbuf) & 1u;
+      if (!mbar_wait(tfull_bar + 8 * buf, acc_phase, abort_flag, p.status)) { ok = false; break; }
+      tc_fence_after();
+      const int col_tile = tile * p.tile_n;
+#pragma unroll
+      for (int a = 0; a < RB; ++a) {
+        if (!warp_has_rows[a]) continue;                 // warp-uniform
+        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
+                               static_cast<uint32_t>(buf * acc_cols + a * p.tile_n);
+        float* dst_row = p.logits + static_cast<size_t>(row[a]) * p.ldl;
+        for (int c0 = 0; c0 < p.tile_n; c0 += 32) {
+          const int col = col_tile + c0;
+          const int valid = p.V - col;                   // columns of this chunk inside the vocabulary
+          if (valid <= 0) break;                         // warp-uniform
+          float v[32];
+          __syncwarp();                                  // tcgen05.ld is warp-collective: reconverge first
+          tmem_ld32(taddr + c0, v);
+          if (row_ok[a]) {
+            if (valid >= 32) {
+              stats_fold<true>(v, 32, st[a]);
+              if (p.vec_ok) {
+                float4* d4 = reinterpret_cast<float4*>(dst_row + col);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) d4[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+              } else {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) dst_row[col + i] = v[i];
+              }
+            } else {
+              stats_fold<false>(v, valid, st[a]);
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                if (i < valid) dst_row[col + i] = v[i];
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar + 8 * buf);
+    }
+    if (ok) {
+#pragma unroll
+      for (int a = 0; a < RB; ++a)
+        if (row_ok[a])
+          p.partials[static_cast<size_t>(blockIdx.x) * p.part_stride + row[a]] =
+              make_float4(st[a].m, st[a].s, st[a].t, 0.f);
+    }
+  }
+
+  // ------------------------------------------------------------------ common tail
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    if (*abort_flag) __nanosleep(200000);                // let copies already in flight land before leaving
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------ K2
+__device__ __forceinline__ Stats warp_merge_partials(const float4* partials, int nparts, int part_stride, int row,
+                                                     int lane) {
+  Stats st = stats_empty();
+  for (int i = lane; i < nparts; i += 32) {
+    const float4 x = partials[static_cast<size_t>(i) * part_stride + row];
+    st = stats_merge(st, Stats{x.x, x.y, x.z});
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    Stats o;
+    o.m = __shfl_xor_sync(0xffffffffu, st.m, off);
+    o.s = __shfl_xor_sync(0xffffffffu, st.s, off);
+    o.t = __shfl_xor_sync(0xffffffffu, st.t, off);
+    // merge in a fixed (lower lane first) order so that every lane holds bit-identical results
+    st = ((lane & off) == 0) ? stats_merge(st, o) : stats_merge(o, st);
+  }
+  return st;
+}
+
+__device__ __forceinline__ void stats_to_outputs(Stats st, float* logZ, float* H) {
+  const float ls = logf(st.s);
+  *logZ = st.m + ls;
+  *H = fmaxf(0.f, ls - st.t / st.s);
+}
+
+__global__ void __launch_bounds__(256) finalize_kernel(const float4* partials, int nparts, int part_stride, int M,
+                                                       float* logZ, float* entropy) {
+  const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (row >= M) return;
+  Stats st = warp_merge_partials(partials, nparts, part_stride, row, lane);
+  if (lane == 0) stats_to_outputs(st, &logZ[row], &entropy[row]);
+}
+
+// ------------------------------------------------------------------------------------------------ K3
+__device__ __forceinline__ double warp_sum_f64(double x) {
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) x += __shfl_xor_sync(0xffffffffu, x, off);
+  return x;
+}
+
+// The four residual masses of vocabulary entries base..base+3 of one row.
+// residual = true:  r = max(0, p - q);  false: r = p.   Entries at or beyond V give 0.
+template <bool kVec>
+__device__ __forceinline__ void load_r4(const float* lrow, const void* qrow, int q_dtype, bool residual, int base,
+                                        int V, float logZ, float r[4]) {
+  float l[4], q[4] = {0.f, 0.f, 0.f, 0.f};
+  if (kVec && base + 3 < V) {
+    const float4 l4 = *reinterpret_cast<const float4*>(lrow + base);
+    l[0] = l4.x; l[1] = l4.y; l[2] = l4.z; l[3] = l4.w;
+    if (residual) {
+      if (q_dtype == HOLA_Q_BF16) {
+        const uint2 raw = *reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(qrow) + base);
+        q[0] = __uint_as_float(raw.x << 16); q[1] = __uint_as_float(raw.x & 0xFFFF0000u);
+        q[2] = __uint_as_float(raw.y << 16); q[3] = __uint_as_float(raw.y & 0xFFFF0000u);
+      } else {
+        const float4 q4 = *reinterpret_cast<const float4*>(static_cast<const float*>(qrow) + base);
+        q[0] = q4.x; q[1] = q4.y; q[2] = q4.z; q[3] = q4.w;
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) r[i] = fmaxf(0.f, expf(l[i] - logZ) - q[i]);
+  } else {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int v = base + i;
+      if (v < V) {
+        float qq = 0.f;
+        if (residual)
+          qq = (q_dtype == HOLA_Q_BF16) ? __bfloat162float(static_cast<const __nv_bfloat16*>(qrow)[v])
+                                        : static_cast<const float*>(qrow)[v];
+        r[i] = fmaxf(0.f, expf(lrow[v] - logZ) - qq);
+      } else {
+        r[i] = 0.f;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ float clamp_uniform(float u, unsigned& flags) {
+  if (!(u >= 0.f)) { flags |= HOLA_FLAG_BAD_UNIFORM; return 0.f; }
+  if (u >= 1.f) { flags |= HOLA_FLAG_BAD_UNIFORM; return 1.f - 5.9604645e-8f; }   // 1 - 2^-24
+  return u;
+}
+
+template <bool kVec>
+__global__ void __launch_bounds__(kK3Threads) accept_sample_kernel(const K3Params p) {
+  __shared__ double csum[kMaxChunks];
+  __shared__ float sh_logZ[kMaxK1], sh_H[kMaxK1], sh_lx[kMaxK1], sh_qx[kMaxK1];
+  __shared__ int sh_x[kMaxK1];
+  __shared__ int sh_n, sh_residual, sh_redo;
+  __shared__ unsigned sh_flags;
+
+  const int b = blockIdx.x;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int k = p.k, V = p.V;
+  const int row_first = b * (k + 1);
+
+  // ---- softmax statistics of this sequence's k+1 positions
+  if (p.combine) {
+    for (int j = warp; j <= k; j += kK3Warps) {
+      Stats st = warp_merge_partials(p.partials, p.nparts, p.part_stride, row_first + j, lane);
+      if (lane == 0) {
+        float lz, h;
+        stats_to_outputs(st, &lz, &h);
+        sh_logZ[j] = lz; sh_H[j] = h;
+        p.logZ[row_first + j] = lz;
+        p.entropy[row_first + j] = h;
+      }
+    }
+  } else {
+    for (int j = threadIdx.x; j <= k; j += kK3Threads) {
+      sh_logZ[j] = p.logZ[row_first + j];
+      sh_H[j] = p.entropy[row_first + j];
+    }
+  }
+  // ---- gather the k draft-token logits and draft probabilities
+  for (int j = threadIdx.x; j < k; j += kK3Threads) {
+    const int x = p.tok[b * k + j];
+    sh_x[j] = x;
+    float lx = 0.f, qx = 0.f;
+    if (x >= 0 && x < V) {
+      lx = p.logits[static_cast<size_t>(row_first + j) * p.ldl + x];
+      const size_t qi = (static_cast<size_t>(b) * k + j) * V + x;
+      qx = (p.q_dtype == HOLA_Q_BF16) ? __bfloat162float(static_cast<const __nv_bfloat16*>(p.q)[qi])
+                                      : static_cast<const float*>(p.q)[qi];
+    }
+    sh_lx[j] = lx; sh_qx[j] = qx;
+  }
+  __syncthreads();
+
+  // ---- gate and ratio test in draft order; stop at the first position that is not accepted
+  if (threadIdx.x == 0) {
+    unsigned flags = 0;
+    int n = k;
+    for (int j = 0; j < k; ++j) {
+      const int x = sh_x[j];
+      if (x < 0 || x >= V) { flags |= HOLA_FLAG_BAD_TOKEN; n = j; break; }
+      if (sh_H[j] < p.tau) continue;                     // entropy gate: fast path keeps the draft token
+      const float u = clamp_uniform(p.u[b * (k + 1) + j], flags);
+      const float px = expf(sh_lx[j] - sh_logZ[j]);
+      const float qx = sh_qx[j];
+      const bool accept = (qx > 0.f) ? (u * qx < px) : (px > 0.f);
+      if (!accept) { n = j; break; }
+    }
+    sh_n = n;
+    sh_residual = (n < k) ? 1 : 0;
+    sh_flags = flags;
+    p.accept_len[b] = n;
+  }
+  __syncthreads();
+
+  // ---- one pass over row n: per-chunk residual mass
+  const int n = sh_n;
+  const float logZ = sh_logZ[n];
+  const float* lrow = p.logits + static_cast<size_t>(row_first + n) * p.ldl;
+  const size_t q_elem = (p.q_dtype == HOLA_Q_BF16) ? 2 : 4;
+  const void* qrow = (n < k) ? static_cast<const void*>(static_cast<const char*>(p.q) +
+                                                        (static_cast<size_t>(b) * k + n) * V * q_elem)
+                             : nullptr;
+  const int nchunks = (V + kChunk - 1) / kChunk;
+  const int per_lane = (nchunks + 31) / 32;
+
+  for (int attempt = 0; attempt < 2; ++attempt) {
+    const bool residual = sh_residual != 0;
+    for (int c0 = warp; c0 < nchunks; c0 += 4 * kK3Warps) {
+      float r[4][4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int c = c0 + i * kK3Warps;
+        if (c < nchunks) load_r4<kVec>(lrow, qrow, p.q_dtype, residual, c * kChunk + lane * 4, V, logZ, r[i]);
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int c = c0 + i * kK3Warps;
+        if (c < nchunks) {
+          const double sum = warp_sum_f64(((static_cast<double>(r[i][0]) + r[i][1]) + r[i][2]) + r[i][3]);
+          if (lane == 0) csum[c] = sum;
+        }
+      }
+    }
+    __syncthreads();
+    if (warp == 0) {
+      const int lo = lane * per_lane, hi = min(nchunks, lo + per_lane);
+      double tot = 0.0;
+      for (int c = lo; c < hi; ++c) tot += csum[c];
+      double incl = tot;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const double o = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += o;
+      }
+      const double R = __shfl_sync(0xffffffffu, incl, 31);
+      if (!(R > 0.0) && residual) {
+        // p <= q everywhere: draw from p instead
+        if (lane == 0) { sh_residual = 0; sh_redo = 1; sh_flags |= HOLA_FLAG_R_ZERO; }
+      } else {
+        if (lane == 0) sh_redo = 0;
+        unsigned flags = 0;
+        const float uk = clamp_uniform(p.u[b * (k + 1) + k], flags);
+        const double target = static_cast<double>(uk) * R;
+        // lane whose range of chunks contains the target
+        const unsigned over = __ballot_sync(0xffffffffu, incl > target);
+        const unsigned has_mass = __ballot_sync(0xffffffffu, tot > 0.0);
+        int L;
+        bool take_last = false;
+        if (over) L = __ffs(over) - 1;
+        else { L = has_mass ? 31 - __clz(has_mass) : 0; take_last = true; }
+        int cstar = -1;
+        double before = 0.0;
+        if (lane == L) {
+          double cum = incl - tot;
+          int last_pos = lo;
+          for (int c = lo; c < hi; ++c) {
+            if (csum[c] > 0.0) last_pos = c;
+            if (!take_last && cum + csum[c] > target) { cstar = c; before = cum; break; }
+            cum += csum[c];
+          }
+          if (cstar < 0) { cstar = last_pos; before = cum - csum[last_pos]; take_last = true; }
+        }
+        cstar = __shfl_sync(0xffffffffu, cstar, L);
+        before = __shfl_sync(0xffffffffu, before, L);
+        take_last = __shfl_sync(0xffffffffu, take_last ? 1 : 0, L) != 0;
+        // inside the chunk: lane prefix, then the lane's four entries in ascending order
+        float r4[4];
+        load_r4<kVec>(lrow, qrow, p.q_dtype, residual, cstar * kChunk + lane * 4, V, logZ, r4);
+        const double mine = ((static_cast<double>(r4[0]) + r4[1]) + r4[2]) + r4[3];
+        double lincl = mine;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+          const double o = __shfl_up_sync(0xffffffffu, lincl, off);
+          if (lane >= off) lincl += o;
+        }
+        double cum = before + (lincl - mine);
+        int found = -1, last_mass = -1;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          cum += r4[i];
+          if (r4[i] > 0.f) last_mass = i;
+          if (found < 0 && !take_last && cum > target) found = i;
+        }
+        const unsigned hit = __ballot_sync(0xffffffffu, found >= 0);
+        const unsigned mass = __ballot_sync(0xffffffffu, last_mass >= 0);
+        int src, idx;
+        if (hit) { src = __ffs(hit) - 1; idx = found; }
+        else { src = mass ? 31 - __clz(mass) : 0; idx = last_mass < 0 ? 0 : last_mass; }
+        idx = __shfl_sync(0xffffffffu, idx, src);
+        if (lane == 0) {
+          int tokn = cstar * kChunk + src * 4 + idx;
+          if (tokn >= V) tokn = V - 1;
+          p.next_tok[b] = tokn;
+          const unsigned fl = sh_flags | flags;
+          if (fl && p.status) atomicOr(p.status, fl);
+        }
+      }
+    }
+    __syncthreads();
+    if (!sh_redo) break;
+  }
+}
+
+// ------------------------------------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct Plan {
+  int tile_n, grid, stages, row_blocks, passes, nbuf, n_tiles, n_kblocks, smem_bytes;
+};
+
+}  // namespace
+
+struct hola_ctx {
+  int device, num_sms, maxB, maxK, H, V, ldl, max_rows;
+  EncodeTiledFn encode;
+  char* ws;                 // one device allocation, carved below
+  size_t ws_bytes;
+  float* logits;            // [max_rows][ldl]
+  float4* partials;         // [num_sms][max_rows]
+  unsigned* status;         // [1]
+  // staging for hola_verify_host
+  void* st_hidden; int* st_tok; void* st_q; float* st_u;
+  int* st_accept; int* st_next; float* st_entropy; float* st_logZ;
+  int force_tile_n, force_stages;
+  // optional per-kernel timing (hola_profile_begin / hola_profile_end)
+  cudaEvent_t* prof_ev;     // 3 events per recorded call: before the GEMM, after it, after accept/sample
+  int prof_cap, prof_n, prof_on;
+  char last_error[256];
+};
+
+namespace {
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct WsLayout {
+  size_t logits, partials, status, st_hidden, st_tok, st_q, st_u, st_accept, st_next, st_entropy, st_logZ, total;
+};
+
+WsLayout ws_layout(int maxB, int maxK, int H, int V, int num_sms) {
+  const size_t rows = static_cast<size_t>(maxB) * (maxK + 1);
+  const size_t ldl = align_up(static_cast<size_t>(V), 4);
+  WsLayout w;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  w.logits = take(rows * ldl * 4);
+  w.partials = take(static_cast<size_t>(num_sms) * rows * 16);
+  w.status = take(4);
+  w.st_hidden = take(rows * H * 2);
+  w.st_tok = take(static_cast<size_t>(maxB) * maxK * 4);
+  w.st_q = take(static_cast<size_t>(maxB) * maxK * V * 4);
+  w.st_u = take(rows * 4);
+  w.st_accept = take(static_cast<size_t>(maxB) * 4);
+  w.st_next = take(static_cast<size_t>(maxB) * 4);
+  w.st_entropy = take(rows * 4);
+  w.st_logZ = take(rows * 4);
+  w.total = off;
+  return w;
+}
+
+constexpr int kAssumedSms = 148;
+
+void set_error(hola_ctx* ctx, const char* what, cudaError_t e) {
+  snprintf(ctx->last_error, sizeof ctx->last_error, "%s: %s", what, cudaGetErrorString(e));
+}
+
+// Chooses the vocab tile width and the split of row blocks into passes for M rows.
+// Cost model per pass, in SM cycles: rounds of tiles x max(tensor time, HBM time, L2 time of the hidden blocks).
+Plan make_plan(const hola_ctx* ctx, int M) {
+  Plan best{};
+  double best_cost = 1e300;
+  const int rb_total = M > 0 ? (M + kRows - 1) / kRows : 1;
+  const int nkb = (ctx->H + kBlockK - 1) / kBlockK;
+  for (int tn = 32; tn <= 256; tn += 32) {
+    if (ctx->force_tile_n && tn != ctx->force_tile_n) continue;
+    const int rb_max = kTmemCols / tn < kMaxRowBlocks ? kTmemCols / tn : kMaxRowBlocks;
+    const int passes = (rb_total + rb_max - 1) / rb_max;
+    const int rb = (rb_total + passes - 1) / passes;
+    const int stage_bytes = rb * kABlockBytes + tn * 128;
+    int stages = (kSmemBudget - 1024 - kBarrierBytes) / stage_bytes;
+    if (stages > kMaxStages) stages = kMaxStages;
+    if (ctx->force_stages && ctx->force_stages < stages) stages = ctx->force_stages;
+    if (stages < 2) continue;
+    const int n_tiles = (ctx->V + tn - 1) / tn;
+    const int grid = n_tiles < ctx->num_sms ? n_tiles : ctx->num_sms;
+    const int rounds = (n_tiles + grid - 1) / grid;
+    const double mma_instr = (tn / 2.0 > (kRows * 32 + tn * 32) / 128.0) ? tn / 2.0 : (kRows * 32 + tn * 32) / 128.0;
+    const double t_mma = rb * 4.0 * mma_instr * nkb;
+    const double t_hbm = tn * 128.0 * nkb / 26.0;        // ~26 B/clk/SM of HBM bandwidth
+    const double t_l2 = rb * kABlockBytes * static_cast<double>(nkb) / 64.0;
+    double t_tile = t_mma > t_hbm ? t_mma : t_hbm;
+    if (t_l2 > t_tile) t_tile = t_l2;
+    const int nbuf = (2 * rb * tn <= kTmemCols) ? 2 : 1;
+    const double t_epi = rb * tn * 12.0;                 // 4 warps, ~12 issue slots per logit per warp lane
+    const double cost = passes * (rounds * (t_tile + (nbuf == 1 ? t_epi : 0.0)) + 3000.0);
+    if (cost < best_cost * 0.999 || (cost <= best_cost * 1.001 && tn > best.tile_n)) {
+      if (cost < best_cost) best_cost = cost;
+      best.tile_n = tn; best.grid = grid; best.stages = stages; best.row_blocks = rb; best.passes = passes;
+      best.nbuf = nbuf; best.n_tiles = n_tiles; best.n_kblocks = nkb;
+      best.smem_bytes = stages * stage_bytes + kBarrierBytes + 1024;
+    }
+  }
+  return best;
+}
+
+hola_status encode_map(hola_ctx* ctx, CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols,
+                       uint32_t box_rows) {
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {cols * 2};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(kBlockK), box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = ctx->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides,
+                                 box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    snprintf(ctx->last_error, sizeof ctx->last_error, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+    return HOLA_ERR_CUDA;
+  }
+  return HOLA_OK;
+}
+
+template <int RB>
+hola_status launch_k1_rb(hola_ctx* ctx, const CUtensorMap& th, const CUtensorMap& tw, const K1Params& kp,
+                         const Plan& pl, cudaStream_t stream) {
+  cudaError_t e = cudaFuncSetAttribute(lm_head_entropy_kernel<RB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       pl.smem_bytes);
+  if (e != cudaSuccess) { set_error(ctx, "cudaFuncSetAttribute", e); return HOLA_ERR_CUDA; }
+  lm_head_entropy_kernel<RB><<<pl.grid, kK1Threads, pl.smem_bytes, stream>>>(th, tw, kp);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) { set_error(ctx, "launch lm_head_entropy_kernel", e); return HOLA_ERR_CUDA; }
+  return HOLA_OK;
+}
+
+hola_status check_common(const hola_ctx* ctx, const hola_verify_args* a) {
+  if (!ctx || !a) return HOLA_ERR_INVALID_ARG;
+  if (a->B < 0 || a->k < 0 || a->H <= 0 || a->V <= 0) return HOLA_ERR_INVALID_ARG;
+  if (a->H != ctx->H || a->V != ctx->V || a->B > ctx->maxB || a->k > ctx->maxK) return HOLA_ERR_UNSUPPORTED_SHAPE;
+  if (a->q_dtype != HOLA_Q_BF16 && a->q_dtype != HOLA_Q_F32) return HOLA_ERR_INVALID_ARG;
+  return HOLA_OK;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Steps 1-2: the LM-head GEMM with fused statistics, one launch per pass over W_lm.
+hola_status run_lm_head(hola_ctx* ctx, const hola_verify_args* a, float* logits, int ldl, const Plan& pl,
+                        cudaStream_t stream) {
+  const int M = a->B * (a->k + 1);
+  CUtensorMap th, tw;
+  hola_status s = encode_map(ctx, &th, a->hidden, static_cast<uint64_t>(M), static_cast<uint64_t>(a->H), kRows);
+  if (s != HOLA_OK) return s;
+  s = encode_map(ctx, &tw, a->W_lm, static_cast<uint64_t>(a->V), static_cast<uint64_t>(a->H),
+                 static_cast<uint32_t>(pl.tile_n));
+  if (s != HOLA_OK) return s;
+  K1Params kp;
+  kp.M = M; kp.V = a->V; kp.tile_n = pl.tile_n; kp.n_tiles = pl.n_tiles; kp.n_kblocks = pl.n_kblocks;
+  kp.stages = pl.stages; kp.nbuf = pl.nbuf; kp.ldl = ldl;
+  kp.vec_ok = (ldl % 4 == 0 && aligned16(logits)) ? 1 : 0;
+  kp.logits = logits; kp.partials = ctx->partials; kp.part_stride = ctx->max_rows;
+  kp.status = a->status_word ? a->status_word : ctx->status;
+  const int rb_total = (M + kRows - 1) / kRows;
+  for (int pass = 0, rb0 = 0; pass < pl.passes; ++pass) {
+    int rb = rb_total - rb0 < pl.row_blocks ? rb_total - rb0 : pl.row_blocks;
+    if (rb <= 0) break;
+    kp.row0 = rb0 * kRows;
+    // the kernel is compiled for 1..4 row blocks; a pass narrower than the plan still uses the plan's
+    // shared-memory stage size only if RB matches, so the plan is re-derived per width below
+    Plan p2 = pl;
+    if (rb != pl.row_blocks) {
+      const int stage_bytes = rb * kABlockBytes + pl.tile_n * 128;
+      int stages = (kSmemBudget - 1024 - kBarrierBytes) / stage_bytes;
+      if (stages > kMaxStages) stages = kMaxStages;
+      p2.stages = stages; p2.row_blocks = rb; p2.nbuf = (2 * rb * pl.tile_n <= kTmemCols) ? 2 : 1;
+      p2.smem_bytes = stages * stage_bytes + kBarrierBytes + 1024;
+      kp.stages = p2.stages; kp.nbuf = p2.nbuf;
+    }
+    switch (rb) {
+      case 1: s = launch_k1_rb<1>(ctx, th, tw, kp, p2, stream); break;
+      case 2: s = launch_k1_rb<2>(ctx, th, tw, kp, p2, stream); break;
+      case 3: s = launch_k1_rb<3>(ctx, th, tw, kp, p2, stream); break;
+      default: s = launch_k1_rb<4>(ctx, th, tw, kp, p2, stream); break;
+    }
+    if (s != HOLA_OK) return s;
+    rb0 += rb;
+  }
+  return HOLA_OK;
+}
+
+hola_status run_accept_sample(hola_ctx* ctx, const hola_verify_args* a, const float* logits, int ldl, int combine,
+                              int nparts, cudaStream_t stream) {
+  K3Params kp;
+  kp.B = a->B; kp.k = a->k; kp.V = a->V; kp.ldl = ldl; kp.logits = logits;
+  kp.partials = ctx->partials; kp.nparts = nparts; kp.part_stride = ctx->max_rows; kp.combine = combine;
+  kp.tok = a->draft_tok; kp.q = a->draft_q; kp.q_dtype = a->q_dtype; kp.u = a->uniforms; kp.tau = a->tau;
+  kp.accept_len = a->accept_len; kp.next_tok = a->next_tok; kp.entropy = a->entropy; kp.logZ = a->logZ;
+  kp.status = a->status_word ? a->status_word : ctx->status;
+  const bool vec = (a->V % 4 == 0) && (ldl % 4 == 0) && aligned16(logits) && (a->k == 0 || aligned16(a->draft_q));
+  if (vec) accept_sample_kernel<true><<<a->B, kK3Threads, 0, stream>>>(kp);
+  else accept_sample_kernel<false><<<a->B, kK3Threads, 0, stream>>>(kp);
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) { set_error(ctx, "launch accept_sample_kernel", e); return HOLA_ERR_CUDA; }
+  return HOLA_OK;
+}
+
+hola_status check_lm_head_args(const hola_ctx* ctx, const hola_verify_args* a) {
+  if (!a->hidden || !a->W_lm) return HOLA_ERR_INVALID_ARG;
+  if (!aligned16(a->hidden) || !aligned16(a->W_lm)) return HOLA_ERR_INVALID_ARG;
+  if (a->H % 8 != 0) return HOLA_ERR_UNSUPPORTED_SHAPE;
+  (void)ctx;
+  return HOLA_OK;
+}
+
+hola_status check_sample_args(const hola_verify_args* a) {
+  if (!a->uniforms || !a->accept_len || !a->next_tok || !a->entropy || !a->logZ) return HOLA_ERR_INVALID_ARG;
+  if (a->k > 0 && (!a->draft_tok || !a->draft_q)) return HOLA_ERR_INVALID_ARG;
+  return HOLA_OK;
+}
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+    if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+  }
+  ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------------ C ABI
+extern "C" {
+
+const char* hola_version(void) { return "0.1"; }
+
+const char* hola_strerror(hola_status s) {
+  switch (s) {
+    case HOLA_OK: return "ok";
+    case HOLA_ERR_INVALID_ARG: return "invalid argument (null pointer, bad size or misaligned buffer)";
+    case HOLA_ERR_UNSUPPORTED_SHAPE: return "unsupported shape (H % 8 != 0, or sizes beyond the context's limits)";
+    case HOLA_ERR_WORKSPACE: return "workspace allocation failed";
+    case HOLA_ERR_CUDA: return "CUDA call failed (see hola_last_cuda_error)";
+    case HOLA_ERR_NO_DEVICE: return "no usable sm_100 device";
+    default: return "unknown status";
+  }
+}
+
+const char* hola_last_cuda_error(const hola_ctx* ctx) { return ctx ? ctx->last_error : ""; }
+
+size_t hola_workspace_bytes(int maxB, int maxK, int H, int V) {
+  if (maxB <= 0 || maxK < 0 || H <= 0 || V <= 0) return 0;
+  return ws_layout(maxB, maxK, H, V, kAssumedSms).total;
+}
+
+hola_status hola_create(hola_ctx** out, int device, int maxB, int maxK, int H, int V) {
+  if (!out) return HOLA_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (maxB <= 0 || maxK < 0 || H <= 0 || V <= 0) return HOLA_ERR_INVALID_ARG;
+  if (H % 8 != 0 || maxK + 1 > kMaxK1 || V > kMaxChunks * kChunk) return HOLA_ERR_UNSUPPORTED_SHAPE;
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || device < 0 || device >= ndev) return HOLA_ERR_NO_DEVICE;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return HOLA_ERR_NO_DEVICE;
+  if (prop.major != 10) return HOLA_ERR_NO_DEVICE;       // the kernels are sm_100a only; there is no fallback
+  DeviceGuard guard(device);
+  if (!guard.ok) return HOLA_ERR_NO_DEVICE;
+
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+      qres != cudaDriverEntryPointSuccess)
+    return HOLA_ERR_NO_DEVICE;
+
+  hola_ctx* ctx = static_cast<hola_ctx*>(calloc(1, sizeof(hola_ctx)));
+  if (!ctx) return HOLA_ERR_WORKSPACE;
+  ctx->device = device; ctx->num_sms = prop.multiProcessorCount; ctx->maxB = maxB; ctx->maxK = maxK;
+  ctx->H = H; ctx->V = V; ctx->ldl = static_cast<int>(align_up(static_cast<size_t>(V), 4));
+  ctx->max_rows = maxB * (maxK + 1);
+  ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
+  if (const char* e = getenv("HOLA_PLAN")) {             // "tile_n,stages": tuning override for sweeps
+    int tn = 0, st = 0;
+    if (sscanf(e, "%d,%d", &tn, &st) >= 1 && tn >= 32 && tn <= 256 && tn % 32 == 0) ctx->force_tile_n = tn;
+    if (st >= 2 && st <= kMaxStages) ctx->force_stages = st;
+  }
+  const WsLayout w = ws_layout(maxB, maxK, H, V, ctx->num_sms);
+  const cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&ctx->ws), w.total);
+  if (e != cudaSuccess) { free(ctx); return HOLA_ERR_WORKSPACE; }
+  ctx->ws_bytes = w.total;
+  ctx->logits = reinterpret_cast<float*>(ctx->ws + w.logits);
+  ctx->partials = reinterpret_cast<float4*>(ctx->ws + w.partials);
+  ctx->status = reinterpret_cast<unsigned*>(ctx->ws + w.status);
+  ctx->st_hidden = ctx->ws + w.st_hidden; ctx->st_tok = reinterpret_cast<int*>(ctx->ws + w.st_tok);
+  ctx->st_q = ctx->ws + w.st_q; ctx->st_u = reinterpret_cast<float*>(ctx->ws + w.st_u);
+  ctx->st_accept = reinterpret_cast<int*>(ctx->ws + w.st_accept);
+  ctx->st_next = reinterpret_cast<int*>(ctx->ws + w.st_next);
+  ctx->st_entropy = reinterpret_cast<float*>(ctx->ws + w.st_entropy);
+  ctx->st_logZ = reinterpret_cast<float*>(ctx->ws + w.st_logZ);
+  cudaMemset(ctx->status, 0, 4);
+  *out = ctx;
+  return HOLA_OK;
+}
+
+hola_status hola_destroy(hola_ctx* ctx) {
+  if (!ctx) return HOLA_OK;
+  DeviceGuard guard(ctx->device);
+  for (int i = 0; i < 3 * ctx->prof_cap; ++i) cudaEventDestroy(ctx->prof_ev[i]);
+  free(ctx->prof_ev);
+  cudaFree(ctx->ws);
+  free(ctx);
+  return HOLA_OK;
+}
+
+hola_status hola_plan(const hola_ctx* ctx, int B, int k, hola_plan_info* out) {
+  if (!ctx || !out || B < 0 || k < 0) return HOLA_ERR_INVALID_ARG;
+  if (B > ctx->maxB || k > ctx->maxK) return HOLA_ERR_UNSUPPORTED_SHAPE;
+  const Plan pl = make_plan(ctx, B * (k + 1));
+  out->tile_n = pl.tile_n; out->grid = pl.grid; out->stages = pl.stages; out->row_blocks = pl.row_blocks;
+  out->passes = pl.passes; out->kernels_per_call = pl.passes + 1;
+  return HOLA_OK;
+}
+
+hola_status hola_lm_head_entropy(hola_ctx* ctx, const hola_verify_args* a, void* cuda_stream) {
+  hola_status s = check_common(ctx, a);
+  if (s != HOLA_OK) return s;
+  if (a->B == 0) return HOLA_OK;
+  if ((s = check_lm_head_args(ctx, a)) != HOLA_OK) return s;
+  if (!a->entropy || !a->logZ) return HOLA_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const int M = a->B * (a->k + 1);
+  const Plan pl = make_plan(ctx, M);
+  float* logits = a->logits_out ? a->logits_out : ctx->logits;
+  const int ldl = a->logits_out ? a->V : ctx->ldl;
+  if ((s = run_lm_head(ctx, a, logits, ldl, pl, stream)) != HOLA_OK) return s;
+  finalize_kernel<<<(M + 7) / 8, 256, 0, stream>>>(ctx->partials, pl.grid, ctx->max_rows, M, a->logZ, a->entropy);
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) { set_error(ctx, "launch finalize_kernel", e); return HOLA_ERR_CUDA; }
+  return HOLA_OK;
+}
+
+hola_status hola_accept_sample(hola_ctx* ctx, const hola_verify_args* a, void* cuda_stream) {
+  hola_status s = check_common(ctx, a);
+  if (s != HOLA_OK) return s;
+  if (a->B == 0) return HOLA_OK;
+  if ((s = check_sample_args(a)) != HOLA_OK) return s;
+  if (!a->logits_out) return HOLA_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  return run_accept_sample(ctx, a, a->logits_out, a->V, 0, 0, static_cast<cudaStream_t>(cuda_stream));
+}
+
+hola_status hola_verify(hola_ctx* ctx, const hola_verify_args* a, void* cuda_stream) {
+  hola_status s = check_common(ctx, a);
+  if (s != HOLA_OK) return s;
+  if (a->B == 0) return HOLA_OK;
+  if ((s = check_lm_head_args(ctx, a)) != HOLA_OK) return s;
+  if ((s = check_sample_args(a)) != HOLA_OK) return s;
+  DeviceGuard guard(ctx->device);
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const Plan pl = make_plan(ctx, a->B * (a->k + 1));
+  float* logits = a->logits_out ? a->logits_out : ctx->logits;
+  const int ldl = a->logits_out ? a->V : ctx->ldl;
+  const bool prof = ctx->prof_on && ctx->prof_n < ctx->prof_cap;
+  cudaEvent_t* ev = prof ? ctx->prof_ev + 3 * ctx->prof_n : nullptr;
+  if (prof) cudaEventRecord(ev[0], stream);
+  if ((s = run_lm_head(ctx, a, logits, ldl, pl, stream)) != HOLA_OK) return s;
+  if (prof) cudaEventRecord(ev[1], stream);
+  s = run_accept_sample(ctx, a, logits, ldl, 1, pl.grid, stream);
+  if (prof) { cudaEventRecord(ev[2], stream); ctx->prof_n++; }
+  return s;
+}
+
+hola_status hola_profile_begin(hola_ctx* ctx, int max_calls) {
+  if (!ctx || max_calls <= 0 || max_calls > 4096) return HOLA_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  if (ctx->prof_cap < max_calls) {
+    cudaEvent_t* ev = static_cast<cudaEvent_t*>(calloc(static_cast<size_t>(3) * max_calls, sizeof(cudaEvent_t)));
+    if (!ev) return HOLA_ERR_WORKSPACE;
+    for (int i = 0; i < 3 * max_calls; ++i) {
+      const cudaError_t e = cudaEventCreate(&ev[i]);
+      if (e != cudaSuccess) { set_error(ctx, "cudaEventCreate", e); free(ev); return HOLA_ERR_CUDA; }
+    }
+    for (int i = 0; i < 3 * ctx->prof_cap; ++i) cudaEventDestroy(ctx->prof_ev[i]);
+    free(ctx->prof_ev);
+    ctx->prof_ev = ev;
+    ctx->prof_cap = max_calls;
+  }
+  ctx->prof_n = 0;
+  ctx->prof_on = 1;
+  return HOLA_OK;
+}
+
+hola_status hola_profile_end(hola_ctx* ctx, void* cuda_stream, double* lm_head_ms, double* accept_sample_ms,
+                             int* calls) {
+  if (!ctx || !lm_head_ms || !accept_sample_ms || !calls) return HOLA_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  ctx->prof_on = 0;
+  cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream));
+  if (e != cudaSuccess) { set_error(ctx, "cudaStreamSynchronize", e); return HOLA_ERR_CUDA; }
+  double a = 0.0, b = 0.0;
+  for (int i = 0; i < ctx->prof_n; ++i) {
+    float ms1 = 0.f, ms2 = 0.f;
+    e = cudaEventElapsedTime(&ms1, ctx->prof_ev[3 * i], ctx->prof_ev[3 * i + 1]);
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms2, ctx->prof_ev[3 * i + 1], ctx->prof_ev[3 * i + 2]);
+    if (e != cudaSuccess) { set_error(ctx, "cudaEventElapsedTime", e); return HOLA_ERR_CUDA; }
+    a += ms1; b += ms2;
+  }
+  *lm_head_ms = a; *accept_sample_ms = b; *calls = ctx->prof_n;
+  return HOLA_OK;
+}
+
+hola_status hola_verify_host(hola_ctx* ctx, const hola_verify_args* a, void* cuda_stream) {
+  hola_status s = check_common(ctx, a);
+  if (s != HOLA_OK) return s;
+  if (a->B == 0) return HOLA_OK;
+  if (!a->hidden || !a->W_lm) return HOLA_ERR_INVALID_ARG;
+  if ((s = check_sample_args(a)) != HOLA_OK) return s;
+  DeviceGuard guard(ctx->device);
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const size_t rows = static_cast<size_t>(a->B) * (a->k + 1);
+  const size_t q_elem = a->q_dtype == HOLA_Q_BF16 ? 2 : 4;
+  cudaError_t e = cudaSuccess;
+  auto h2d = [&](void* dst, const void* src, size_t bytes) {
+    if (e == cudaSuccess && bytes) e = cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, stream);
+  };
+  auto d2h = [&](void* dst, const void* src, size_t bytes) {
+    if (e == cudaSuccess && bytes) e = cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToHost, stream);
+  };
+  h2d(ctx->st_hidden, a->hidden, rows * a->H * 2);
+  h2d(ctx->st_tok, a->draft_tok, static_cast<size_t>(a->B) * a->k * 4);
+  h2d(ctx->st_q, a->draft_q, static_cast<size_t>(a->B) * a->k * a->V * q_elem);
+  h2d(ctx->st_u, a->uniforms, rows * 4);
+  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->status, 0, 4, stream);
+  if (e != cudaSuccess) { set_error(ctx, "host-to-device copy", e); return HOLA_ERR_CUDA; }
+  hola_verify_args d = *a;
+  d.hidden = ctx->st_hidden; d.draft_tok = ctx->st_tok; d.draft_q = ctx->st_q; d.uniforms = ctx->st_u;
+  d.accept_len = ctx->st_accept; d.next_tok = ctx->st_next; d.entropy = ctx->st_entropy; d.logZ = ctx->st_logZ;
+  d.logits_out = nullptr; d.status_word = ctx->status;
+  if ((s = hola_verify(ctx, &d, cuda_stream)) != HOLA_OK) return s;
+  d2h(a->accept_len, ctx->st_accept, static_cast<size_t>(a->B) * 4);
+  d2h(a->next_tok, ctx->st_next, static_cast<size_t>(a->B) * 4);
+  d2h(a->entropy, ctx->st_entropy, rows * 4);
+  d2h(a->logZ, ctx->st_logZ, rows * 4);
+  if (a->status_word) d2h(a->status_word, ctx->status, 4);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+  if (e != cudaSuccess) { set_error(ctx, "device-to-host copy", e); return HOLA_ERR_CUDA; }
+  return HOLA_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,320 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on identical seeded inputs."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import compare, ref
+from paper_2506_18952_b200 import workloads
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda"
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_2506_18952_b200 import binding as b
+    b.load_library()
+    return b
+
+
+def _np(t):
+    return compare.torch_to_numpy(t)
+
+
+def run_gpu(binding, w, want_logits=False, tau=None, ctx=None):
+    own = ctx is None
+    ctx = ctx or binding.HolaVerify(max(w.B, 1), w.k, w.H, w.V)
+    try:
+        out = ctx.hola_verify(w.hidden, w.W_lm, w.draft_tok, w.draft_q, w.uniforms, w.tau if tau is None else tau,
+                              want_logits=want_logits)
+        torch.cuda.synchronize()
+    finally:
+        if own:
+            ctx.close()
+    return out
+
+
+def check_against_oracle(binding, w, seqs=None, want_logits=True, tau=None, out=None):
+    """Runs the GPU path on the whole workload and the oracle on `seqs` (all sequences when None)."""
+    tau = w.tau if tau is None else tau
+    out = out or run_gpu(binding, w, want_logits=want_logits, tau=tau)
+    status = int(out.status.item())
+    assert status & binding.FLAG_TIMEOUT == 0, "a device-side wait timed out"
+    sub = w if seqs is None else w.slice(seqs)
+    idx = np.arange(w.B) if seqs is None else np.asarray(list(seqs))
+    sub.tau = tau
+    orc = compare.run_oracle(sub, keep_logits=True)
+    rep = compare.compare(orc, _np(sub.draft_q), _np(sub.uniforms), _np(out.accept_len)[idx], _np(out.next_tok)[idx],
+                          _np(out.entropy)[idx], _np(out.logZ)[idx],
+                          _np(out.logits)[idx] if out.logits is not None else None)
+    print(w.name, "tau", tau, rep.summary())
+    assert rep.ok, rep.summary() + f" accept_fail={rep.accept_failures[:5]} token_fail={rep.token_failures[:5]}"
+    # margin cases are reported, and must stay rare
+    assert rep.accept_margin_cases <= max(1, rep.n_seq // 20)
+    assert rep.token_margin_cases <= max(1, rep.n_seq // 10)
+    return out, orc, rep
+
+
+def check_ranges(w, out):
+    a, t = _np(out.accept_len), _np(out.next_tok)
+    assert a.min() >= 0 and a.max() <= w.k
+    assert t.min() >= 0 and t.max() < w.V
+    H = _np(out.entropy)
+    assert np.isfinite(H).all() and H.min() >= 0 and H.max() <= math.log(w.V) + 1e-3
+    assert np.isfinite(_np(out.logZ)).all()
+
+
+# ------------------------------------------------------------------------------------------ the projection
+def _int_workload(B, k, H, V, seed, identity=False):
+    g = torch.Generator().manual_seed(seed)
+    hidden = torch.randint(-4, 5, (B, k + 1, H), generator=g).float()
+    W = torch.eye(V, H) if identity else torch.randint(-4, 5, (V, H), generator=g).float()
+    q = torch.full((B, k, V), 1.0 / V)
+    tok = torch.randint(0, V, (B, k), generator=g, dtype=torch.int32)
+    u = torch.rand((B, k + 1), generator=g)
+    return workloads.VerifyInputs("ints", B, k, H, V, 0.0, hidden.bfloat16().to(DEV), W.bfloat16().to(DEV),
+                                  tok.to(DEV), q.to(DEV), u.to(DEV))
+
+
+@pytest.mark.parametrize("B,k,H,V", [(7, 0, 128, 37), (2, 3, 64, 300), (40, 3, 192, 520), (150, 3, 64, 96)])
+def test_small_integer_logits_are_bit_exact(binding, B, k, H, V):
+    # |values| <= 4: every product and partial sum is an integer far below 2^24, so bf16 inputs, fp32 tensor-core
+    # accumulation and the fp64 oracle must agree exactly, tile tails and row-block tails included.
+    w = _int_workload(B, k, H, V, seed=B * 1000 + V)
+    with binding.HolaVerify(B, k, H, V) as ctx:
+        out = ctx.hola_lm_head_entropy(w.hidden, w.W_lm, want_logits=True)
+        torch.cuda.synchronize()
+    want = ref.logits(_np(w.hidden).reshape(-1, H), _np(w.W_lm)).reshape(B, k + 1, V)
+    assert np.array_equal(_np(out.logits).astype(np.float64), want)
+    logZ, Hn = ref.softmax_entropy(want.reshape(-1, V))
+    assert np.max(np.abs(_np(out.logZ).reshape(-1) - logZ)) < 2e-3
+    assert np.max(np.abs(_np(out.entropy).reshape(-1) - Hn)) < 2e-3
+
+
+def test_identity_weight_returns_hidden(binding):
+    w = _int_workload(5, 1, 64, 64, seed=5, identity=True)
+    with binding.HolaVerify(5, 1, 64, 64) as ctx:
+        out = ctx.hola_lm_head_entropy(w.hidden, w.W_lm, want_logits=True)
+        torch.cuda.synchronize()
+    assert torch.equal(out.logits, w.hidden.float())
+
+
+@pytest.mark.parametrize("V", [8, 16, 1000, 32000])
+def test_zero_weight_gives_uniform_entropy(binding, V):
+    B, k, H = 3, 2, 64
+    hidden = torch.randn((B, k + 1, H), device=DEV).bfloat16()
+    W = torch.zeros((V, H), device=DEV, dtype=torch.bfloat16)
+    with binding.HolaVerify(B, k, H, V) as ctx:
+        out = ctx.hola_lm_head_entropy(hidden, W, want_logits=False)
+        torch.cuda.synchronize()
+    assert torch.allclose(out.logZ, torch.full_like(out.logZ, math.log(V)), atol=1e-4)
+    assert torch.allclose(out.entropy, torch.full_like(out.entropy, math.log(V)), atol=1e-4)
+
+
+def test_peaked_rows_keep_entropy_accuracy(binding):
+    # one logit 15 above the rest at V = 32000: H = 0.1551462, logZ - l_max = ln(1 + (V-1) e^-15)
+    V, H = 32000, 64
+    W = torch.zeros((V, H)); W[12345, 0] = 1.0
+    hidden = torch.zeros((1, 1, H)); hidden[0, 0, 0] = 15.0
+    with binding.HolaVerify(1, 0, H, V) as ctx:
+        out = ctx.hola_lm_head_entropy(hidden.bfloat16().to(DEV), W.bfloat16().to(DEV), want_logits=False)
+        torch.cuda.synchronize()
+    tail = (V - 1) * math.exp(-15.0)
+    p = 1 / (1 + tail)
+    H_want = -p * math.log(p) - (1 - p) * math.log((1 - p) / (V - 1))
+    assert abs(out.entropy.item() - H_want) < 1e-4
+    assert abs(out.logZ.item() - (15.0 + math.log1p(tail))) < 1e-4
+
+
+# ------------------------------------------------------------------------------------------ whole path, small
+@pytest.mark.parametrize("tau", [None, 0.0, 1.5, float("inf"), float("nan")])
+def test_tiny_config(binding, tau):
+    w = workloads.make_config("tiny", DEV)
+    check_against_oracle(binding, w, tau=w.tau if tau is None else tau)
+
+
+@pytest.mark.parametrize("B,k,H,V,qd", [
+    (3, 4, 200, 1000, torch.float32),      # K tail (H not a multiple of 64), vocab tail
+    (37, 6, 256, 5000, torch.bfloat16),    # 259 rows: three row blocks, the last one ragged
+    (5, 2, 64, 1001, torch.bfloat16),      # odd V: scalar load/store paths
+    (130, 0, 64, 777, torch.bfloat16),     # k = 0: plain draw from p
+    (90, 7, 128, 640, torch.float32),      # 720 rows: more row blocks than one pass holds
+])
+def test_ragged_shapes(binding, B, k, H, V, qd):
+    w = workloads.gaussian_head("ragged", B, k, H, V, seed=B + V, device=DEV, w_std=0.3, sigma=1.0, q_dtype=qd,
+                                tau=1.5 + 0.1 * k, sigma_far=0.2)
+    out, _, _ = check_against_oracle(binding, w)
+    check_ranges(w, out)
+
+
+@pytest.mark.parametrize("V", [8, 16])
+def test_brute_force_grid_matches_oracle_and_p(binding, V):
+    # every draft token x, a grid of accept uniforms and of sampling uniforms, laid out as one batch; k = 1.
+    # The emitted-token histogram, weighted by q(x), reproduces p to the grid resolution (gate off).
+    rng = np.random.default_rng(V)
+    H, G = 8, 24
+    pw = rng.integers(1, 30, size=(2, V)).astype(np.float64); p = pw / pw.sum(-1, keepdims=True)
+    qw = rng.integers(1, 30, size=V).astype(np.float64); q = qw / qw.sum()
+    Wt = np.zeros((V, H), np.float32); Wt[:, 0] = np.log(p[0]); Wt[:, 1] = np.log(p[1])
+    xs, ua, us = np.meshgrid(np.arange(V), (np.arange(G) + 0.5) / G, (np.arange(G) + 0.5) / G, indexing="ij")
+    B = xs.size
+    hidden = np.zeros((B, 2, H), np.float32); hidden[:, 0, 0] = 1.0; hidden[:, 1, 1] = 1.0
+    w = workloads.VerifyInputs(
+        "grid", B, 1, H, V, 0.0, torch.from_numpy(hidden).bfloat16().to(DEV), torch.from_numpy(Wt).bfloat16().to(DEV),
+        torch.from_numpy(xs.reshape(B, 1).astype(np.int32)).to(DEV),
+        torch.from_numpy(np.tile(q.astype(np.float32), (B, 1, 1))).to(DEV),
+        torch.from_numpy(np.stack([ua.ravel(), us.ravel()], 1).astype(np.float32)).to(DEV))
+    out, orc, _ = check_against_oracle(binding, w)
+    # marginal of the emitted token at position 0, from the GPU outputs; p as the GPU sees it (bf16-rounded logs)
+    lw = ref.bf16_bits_to_f64(ref.f32_to_bf16_bits(Wt[:, 0])); p0 = np.exp(lw) / np.exp(lw).sum()
+    acc, nxt = _np(out.accept_len), _np(out.next_tok)
+    emitted = np.where(acc >= 1, xs.ravel(), nxt)
+    marg = np.bincount(emitted, weights=q[xs.ravel()] / (G * G), minlength=V)
+    np.testing.assert_allclose(marg, p0, atol=2.0 / G)
+
+
+def test_accept_sample_entry_from_oracle_logits(binding):
+    # steps 3-5 alone, fed with logits, entropy and logZ made by the oracle (rounded to fp32)
+    w = workloads.gaussian_head("k3", 48, 4, 64, 3000, seed=77, device="cpu", w_std=0.4, sigma=0.8, tau=0.0)
+    orc0 = compare.run_oracle(w, keep_logits=True)
+    l32 = orc0.logits.astype(np.float32)
+    lz, Hn = ref.softmax_entropy(l32.astype(np.float64).reshape(-1, w.V))
+    orc = ref.verify_from_logits(l32.astype(np.float64), _np(w.draft_tok), _np(w.draft_q), _np(w.uniforms), w.tau)
+    with binding.HolaVerify(w.B, w.k, w.H, w.V) as ctx:
+        out = ctx.hola_accept_sample(torch.from_numpy(l32).to(DEV), torch.from_numpy(Hn.astype(np.float32)).reshape(w.B, -1).to(DEV),
+                                     torch.from_numpy(lz.astype(np.float32)).reshape(w.B, -1).to(DEV), w.draft_tok.to(DEV),
+                                     w.draft_q.to(DEV), w.uniforms.to(DEV), w.tau)
+        torch.cuda.synchronize()
+    rep = compare.compare(orc, _np(w.draft_q), _np(w.uniforms), _np(out.accept_len), _np(out.next_tok),
+                          Hn.reshape(w.B, -1), lz.reshape(w.B, -1))
+    assert rep.ok and rep.accept_exact >= w.B - 1, rep.summary()
+    assert 0 < _np(out.accept_len).mean() < w.k       # both branches taken
+
+
+# ------------------------------------------------------------------------------------------ degenerate inputs
+def test_degenerate_inputs_are_flagged_not_fatal(binding):
+    B, k, H, V = 4, 2, 64, 500
+    w = workloads.gaussian_head("edge", B, k, H, V, seed=3, device=DEV, w_std=0.3, q_dtype=torch.float32, tau=0.0)
+    w.draft_tok[0, 0] = V              # bad token -> rejection at position 0
+    w.draft_tok[1, 1] = -3
+    w.uniforms[2, k] = 1.0             # clamped
+    w.draft_q[3] = 2.0 * torch.softmax(workloads._target_logits(w.hidden, w.W_lm)[3, :k], -1)   # q = 2p: R = 0
+    w.uniforms[3, 0] = 0.75
+    out, orc, _ = check_against_oracle(binding, w)
+    st = int(out.status.item())
+    assert st & binding.FLAG_BAD_TOKEN and st & binding.FLAG_BAD_UNIFORM and st & binding.FLAG_R_ZERO
+    assert _np(out.accept_len)[0] == 0 and _np(out.accept_len)[1] <= 1 and _np(out.accept_len)[3] == 0
+    assert orc.flags[3] & ref.FLAG_R_ZERO
+
+
+def test_empty_batch_and_argument_errors(binding):
+    import ctypes
+    lib = binding.load_library()
+    bad = ctypes.c_void_p()
+    assert lib.hola_create(ctypes.byref(bad), 0, 1, 1, 60, 100) == 2          # H % 8 != 0
+    assert lib.hola_create(ctypes.byref(bad), 0, 0, 1, 64, 100) == 1
+    assert lib.hola_create(ctypes.byref(bad), 0, 1, 80, 64, 100) == 2         # k + 1 > 64
+    with binding.HolaVerify(4, 2, 64, 100) as ctx:
+        w = workloads.gaussian_head("e", 4, 2, 64, 100, seed=1, device=DEV)
+        empty = w.slice([])
+        out = ctx.hola_verify(empty.hidden, w.W_lm, empty.draft_tok, empty.draft_q, empty.uniforms, 1.5)
+        assert out.accept_len.numel() == 0
+        big = workloads.gaussian_head("e", 5, 2, 64, 100, seed=1, device=DEV)
+        with pytest.raises(binding.HolaError, match="unsupported shape"):
+            ctx.hola_verify(big.hidden, big.W_lm, big.draft_tok, big.draft_q, big.uniforms, 1.5)
+        # misaligned hidden pointer
+        raw = torch.zeros(4 * 3 * 64 + 8, dtype=torch.bfloat16, device=DEV)
+        mis = raw[1:1 + 4 * 3 * 64].view(4, 3, 64)
+        with pytest.raises(binding.HolaError, match="invalid argument"):
+            ctx.hola_verify(mis, w.W_lm, w.draft_tok, w.draft_q, w.uniforms, 1.5)
+        a = binding.hola_verify_args()
+        assert lib.hola_verify(ctx._ctx, ctypes.byref(a), None) != 0          # all-null arguments
+        assert lib.hola_verify(None, ctypes.byref(a), None) == 1
+
+
+# ------------------------------------------------------------------------------------------ properties
+def test_deterministic_and_batch_order_equivariant(binding):
+    w = workloads.gaussian_head("perm", 33, 3, 128, 2048, seed=9, device=DEV, w_std=0.3, sigma=1.0, tau=4.0)
+    a = run_gpu(binding, w, want_logits=True)
+    b = run_gpu(binding, w, want_logits=True)
+    for x, y in [(a.accept_len, b.accept_len), (a.next_tok, b.next_tok), (a.entropy, b.entropy), (a.logZ, b.logZ),
+                 (a.logits, b.logits)]:
+        assert torch.equal(x, y)
+    perm = torch.randperm(w.B, generator=torch.Generator().manual_seed(1)).tolist()
+    c = run_gpu(binding, w.slice(perm))
+    idx = torch.tensor(perm, device=DEV)
+    assert torch.equal(c.accept_len, a.accept_len[idx]) and torch.equal(c.next_tok, a.next_tok[idx])
+    assert torch.allclose(c.entropy, a.entropy[idx], atol=1e-5)
+
+
+def test_outputs_stay_inside_their_buffers(binding):
+    # canary words before and after every output
+    B, k, H, V = 6, 3, 64, 333
+    w = workloads.gaussian_head("canary", B, k, H, V, seed=4, device=DEV, w_std=0.3)
+    pad = 64
+
+    def padded(n, dtype, fill):
+        buf = torch.full((n + 2 * pad,), fill, dtype=dtype, device=DEV)
+        return buf, buf[pad:pad + n]
+
+    bufs = {}
+    with binding.HolaVerify(B, k, H, V) as ctx:
+        out = ctx.alloc_outputs(B, k, True)
+        bufs["a"], a = padded(B, torch.int32, -7); out.accept_len = a
+        bufs["n"], n = padded(B, torch.int32, -7); out.next_tok = n
+        bufs["e"], e = padded(B * (k + 1), torch.float32, -7.0); out.entropy = e.view(B, k + 1)
+        bufs["z"], z = padded(B * (k + 1), torch.float32, -7.0); out.logZ = z.view(B, k + 1)
+        bufs["l"], l = padded(B * (k + 1) * V, torch.float32, -7.0); out.logits = l.view(B, k + 1, V)
+        ctx.hola_verify(w.hidden, w.W_lm, w.draft_tok, w.draft_q, w.uniforms, 1.5, out=out)
+        torch.cuda.synchronize()
+    for name, buf in bufs.items():
+        assert torch.all(buf[:pad] == -7) and torch.all(buf[-pad:] == -7), name
+    assert torch.all(out.accept_len >= 0) and torch.all(out.logits != -7.0)
+
+
+def test_host_entry_equals_device_entry(binding):
+    w = workloads.gaussian_head("host", 9, 3, 128, 4000, seed=12, device=DEV, w_std=0.3, tau=5.0)
+    with binding.HolaVerify(w.B, w.k, w.H, w.V) as ctx:
+        d = ctx.hola_verify(w.hidden, w.W_lm, w.draft_tok, w.draft_q, w.uniforms, w.tau)
+        torch.cuda.synchronize()
+        h = ctx.hola_verify_host(w.hidden.cpu().pin_memory(), w.W_lm, w.draft_tok.cpu().pin_memory(),
+                                 w.draft_q.cpu().pin_memory(), w.uniforms.cpu().pin_memory(), w.tau)
+    assert torch.equal(h.accept_len, d.accept_len.cpu()) and torch.equal(h.next_tok, d.next_tok.cpu())
+    assert torch.equal(h.entropy, d.entropy.cpu()) and torch.equal(h.logZ, d.logZ.cpu())
+
+
+# ------------------------------------------------------------------------------------------ the named workloads
+def test_edge_decode_config_full(binding):
+    w = workloads.make_config("edge", DEV)
+    out, _, rep = check_against_oracle(binding, w)
+    check_ranges(w, out)
+    assert rep.max_logit_rel_err < 1e-3
+
+
+def test_batched_serving_config(binding):
+    w = workloads.make_config("batched", DEV)
+    seqs = [0, 13, 31, 32, 47, 63]
+    out, orc, _ = check_against_oracle(binding, w, seqs=seqs)
+    check_ranges(w, out)
+    acc = _np(out.accept_len)
+    assert acc[:32].mean() > acc[32:].mean() + 1.0      # near-p half keeps more drafts than the far half
+
+
+@pytest.mark.parametrize("tau", [1.0, 2.0, 4.0])
+def test_large_vocab_config(binding, tau):
+    w = workloads.make_config("large_vocab", DEV)
+    out, _, _ = check_against_oracle(binding, w, seqs=[1, 22, 40, 63], tau=tau)
+    check_ranges(w, out)
+    H = _np(out.entropy)
+    assert H.min() < 1.0 and H.max() > 6.0              # the entropy spread the workload asks for
+
+
+def test_wide_head_config(binding):
+    w = workloads.make_config("wide", DEV)
+    out, _, _ = check_against_oracle(binding, w, seqs=[0, 101, 255], want_logits=False)
+    check_ranges(w, out)
+    H = _np(out.entropy).reshape(-1)
+    assert (H[0::2] < 1.5).mean() > 0.9 and (H[1::2] > 10).mean() > 0.9     # peaked and flat rows
