@@ -118,13 +118,15 @@ def algorithmic_work(w) -> dict:
 def oracle_positions_per_s(w, budget_s: float, nthreads: int = 0):
     """Times the CPU oracle, as it stands, on a bounded sample of the workload's sequences."""
     from oracle import compare, ref
-    t0 = time.perf_counter()
-    compare.run_oracle(w.slice([0]), keep_logits=False, nthreads=nthreads)
-    t_one = time.perf_counter() - t0
-    n = int(max(1, min(w.B, budget_s // max(t_one, 1e-3))))
-    t0 = time.perf_counter()
-    compare.run_oracle(w.slice(range(n)), keep_logits=False, nthreads=nthreads)
-    dt = time.perf_counter() - t0
+    compare.run_oracle(w.slice([0]), keep_logits=False, nthreads=nthreads)        # builds, loads, spins up threads
+    n, dt = 1, 0.0
+    while True:
+        t0 = time.perf_counter()
+        compare.run_oracle(w.slice(range(n)), keep_logits=False, nthreads=nthreads)
+        dt = time.perf_counter() - t0
+        if dt >= 0.6 * budget_s or n >= w.B:
+            break
+        n = int(min(w.B, max(n + 1, n * min(8.0, budget_s / max(dt, 1e-3)))))
     return n * (w.k + 1) / dt, n, dt, ref.max_threads()
 
 

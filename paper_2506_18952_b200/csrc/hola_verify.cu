@@ -10,7 +10,7 @@
 //       registers across all of the CTA's tiles.  W_lm is read from HBM once per pass.
 //   finalize_kernel             merges the per-CTA statistics:  logZ = m + ln s,  H = ln s - t/s  (entropy
 //       definition of the HSD section, rearranged around the running maximum).
-//   accept_sample_kernel        one CTA per sequence: merges the statistics for its k+1 positions (warp
+//   accept_sample_kernel        one cluster of CTAs per sequence: merges the statistics for its k+1 positions (warp
 //       shuffles), applies the entropy gate and the ratio test in draft order, then makes one vectorised pass
 //       over the logits row and the draft row of the first rejected position: residual max(0, p - q), per-chunk
 //       sums, a scan, and the inverse-CDF pick with the supplied uniform.
@@ -27,7 +27,11 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <cooperative_groups.h>
+
 #include "../../include/hola_verify.h"
+
+namespace cg = cooperative_groups;
 
 namespace {
 
@@ -43,7 +47,7 @@ constexpr int kSmemBudget = 227 * 1024;          // dynamic shared memory per CT
 constexpr int kBarrierBytes = 256;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait, far above any legitimate wait
 
-constexpr int kK3Threads = 512;
+constexpr int kK3Threads = 256;
 constexpr int kK3Warps = kK3Threads / 32;
 constexpr int kChunk = 128;                      // vocabulary entries per warp step (32 lanes x 4)
 constexpr int kMaxChunks = 4096;                 // => V <= 524288
@@ -529,38 +533,29 @@ __device__ __forceinline__ float clamp_uniform(float u, unsigned& flags) {
   return u;
 }
 
+// One cluster of S CTAs per sequence.  Every CTA derives accept_len on its own (same inputs, same arithmetic,
+// same result), sums the residual mass of its slice of the vocabulary chunk by chunk, and publishes its slice
+// total to all CTAs of the cluster through distributed shared memory.  After one cluster barrier each CTA knows
+// the total mass R and which slice holds the point u*R; that CTA alone finishes the inverse-CDF search.
 template <bool kVec>
 __global__ void __launch_bounds__(kK3Threads) accept_sample_kernel(const K3Params p) {
-  __shared__ double csum[kMaxChunks];
-  __shared__ float sh_logZ[kMaxK1], sh_H[kMaxK1], sh_lx[kMaxK1], sh_qx[kMaxK1];
+  extern __shared__ double csum[];                       // per-chunk residual mass of this CTA's slice
+  __shared__ double sh_tot[2][8];                        // slice totals of the whole cluster, per attempt
+  __shared__ float sh_logZ[kMaxK1], sh_H[kMaxK1], sh_lx[kMaxK1], sh_qx[kMaxK1], sh_u[kMaxK1];
   __shared__ int sh_x[kMaxK1];
-  __shared__ int sh_n, sh_residual, sh_redo;
+  __shared__ int sh_n;
   __shared__ unsigned sh_flags;
 
-  const int b = blockIdx.x;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int S = static_cast<int>(cluster.num_blocks());
+  const int rank = static_cast<int>(cluster.block_rank());
+  const int b = blockIdx.x / S;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int k = p.k, V = p.V;
   const int row_first = b * (k + 1);
 
-  // ---- softmax statistics of this sequence's k+1 positions
-  if (p.combine) {
-    for (int j = warp; j <= k; j += kK3Warps) {
-      Stats st = warp_merge_partials(p.partials, p.nparts, p.part_stride, row_first + j, lane);
-      if (lane == 0) {
-        float lz, h;
-        stats_to_outputs(st, &lz, &h);
-        sh_logZ[j] = lz; sh_H[j] = h;
-        p.logZ[row_first + j] = lz;
-        p.entropy[row_first + j] = h;
-      }
-    }
-  } else {
-    for (int j = threadIdx.x; j <= k; j += kK3Threads) {
-      sh_logZ[j] = p.logZ[row_first + j];
-      sh_H[j] = p.entropy[row_first + j];
-    }
-  }
-  // ---- gather the k draft-token logits and draft probabilities
+  // ---- gather the k draft-token logits, draft probabilities and the uniforms (independent of the statistics)
+  for (int j = threadIdx.x; j <= k; j += kK3Threads) sh_u[j] = p.u[b * (k + 1) + j];
   for (int j = threadIdx.x; j < k; j += kK3Threads) {
     const int x = p.tok[b * k + j];
     sh_x[j] = x;
@@ -573,6 +568,23 @@ __global__ void __launch_bounds__(kK3Threads) accept_sample_kernel(const K3Param
     }
     sh_lx[j] = lx; sh_qx[j] = qx;
   }
+  // ---- softmax statistics of this sequence's k+1 positions
+  if (p.combine) {
+    for (int j = warp; j <= k; j += kK3Warps) {
+      Stats st = warp_merge_partials(p.partials, p.nparts, p.part_stride, row_first + j, lane);
+      if (lane == 0) {
+        float lz, h;
+        stats_to_outputs(st, &lz, &h);
+        sh_logZ[j] = lz; sh_H[j] = h;
+        if (rank == 0) { p.logZ[row_first + j] = lz; p.entropy[row_first + j] = h; }
+      }
+    }
+  } else {
+    for (int j = threadIdx.x; j <= k; j += kK3Threads) {
+      sh_logZ[j] = p.logZ[row_first + j];
+      sh_H[j] = p.entropy[row_first + j];
+    }
+  }
   __syncthreads();
 
   // ---- gate and ratio test in draft order; stop at the first position that is not accepted
@@ -583,20 +595,19 @@ __global__ void __launch_bounds__(kK3Threads) accept_sample_kernel(const K3Param
       const int x = sh_x[j];
       if (x < 0 || x >= V) { flags |= HOLA_FLAG_BAD_TOKEN; n = j; break; }
       if (sh_H[j] < p.tau) continue;                     // entropy gate: fast path keeps the draft token
-      const float u = clamp_uniform(p.u[b * (k + 1) + j], flags);
+      const float u = clamp_uniform(sh_u[j], flags);
       const float px = expf(sh_lx[j] - sh_logZ[j]);
       const float qx = sh_qx[j];
       const bool accept = (qx > 0.f) ? (u * qx < px) : (px > 0.f);
       if (!accept) { n = j; break; }
     }
     sh_n = n;
-    sh_residual = (n < k) ? 1 : 0;
     sh_flags = flags;
-    p.accept_len[b] = n;
+    if (rank == 0) p.accept_len[b] = n;
   }
   __syncthreads();
 
-  // ---- one pass over row n: per-chunk residual mass
+  // ---- this CTA's slice of row n: per-chunk residual mass
   const int n = sh_n;
   const float logZ = sh_logZ[n];
   const float* lrow = p.logits + static_cast<size_t>(row_first + n) * p.ldl;
@@ -605,103 +616,128 @@ __global__ void __launch_bounds__(kK3Threads) accept_sample_kernel(const K3Param
                                                         (static_cast<size_t>(b) * k + n) * V * q_elem)
                              : nullptr;
   const int nchunks = (V + kChunk - 1) / kChunk;
-  const int per_lane = (nchunks + 31) / 32;
+  const int cpc = (nchunks + S - 1) / S;                 // chunks per CTA
+  const int c_first = rank * cpc;
+  const int mine = max(0, min(nchunks, c_first + cpc) - c_first);
+  const int per_lane = (mine + 31) / 32;
+  bool residual = n < k;
 
   for (int attempt = 0; attempt < 2; ++attempt) {
-    const bool residual = sh_residual != 0;
-    for (int c0 = warp; c0 < nchunks; c0 += 4 * kK3Warps) {
+    for (int c0 = warp; c0 < mine; c0 += 4 * kK3Warps) {
       float r[4][4];
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         const int c = c0 + i * kK3Warps;
-        if (c < nchunks) load_r4<kVec>(lrow, qrow, p.q_dtype, residual, c * kChunk + lane * 4, V, logZ, r[i]);
+        if (c < mine)
+          load_r4<kVec>(lrow, qrow, p.q_dtype, residual, (c_first + c) * kChunk + lane * 4, V, logZ, r[i]);
       }
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         const int c = c0 + i * kK3Warps;
-        if (c < nchunks) {
+        if (c < mine) {
           const double sum = warp_sum_f64(((static_cast<double>(r[i][0]) + r[i][1]) + r[i][2]) + r[i][3]);
           if (lane == 0) csum[c] = sum;
         }
       }
     }
     __syncthreads();
+    // warp 0: scan of the slice; lane L owns chunks [lo, hi)
+    double tot = 0.0, incl = 0.0;
+    const int lo = lane * per_lane, hi = min(mine, lo + per_lane);
     if (warp == 0) {
-      const int lo = lane * per_lane, hi = min(nchunks, lo + per_lane);
-      double tot = 0.0;
       for (int c = lo; c < hi; ++c) tot += csum[c];
-      double incl = tot;
+      incl = tot;
 #pragma unroll
       for (int off = 1; off < 32; off <<= 1) {
         const double o = __shfl_up_sync(0xffffffffu, incl, off);
         if (lane >= off) incl += o;
       }
-      const double R = __shfl_sync(0xffffffffu, incl, 31);
-      if (!(R > 0.0) && residual) {
-        // p <= q everywhere: draw from p instead
-        if (lane == 0) { sh_residual = 0; sh_redo = 1; sh_flags |= HOLA_FLAG_R_ZERO; }
-      } else {
-        if (lane == 0) sh_redo = 0;
-        unsigned flags = 0;
-        const float uk = clamp_uniform(p.u[b * (k + 1) + k], flags);
-        const double target = static_cast<double>(uk) * R;
-        // lane whose range of chunks contains the target
-        const unsigned over = __ballot_sync(0xffffffffu, incl > target);
-        const unsigned has_mass = __ballot_sync(0xffffffffu, tot > 0.0);
-        int L;
-        bool take_last = false;
-        if (over) L = __ffs(over) - 1;
-        else { L = has_mass ? 31 - __clz(has_mass) : 0; take_last = true; }
-        int cstar = -1;
-        double before = 0.0;
-        if (lane == L) {
-          double cum = incl - tot;
-          int last_pos = lo;
-          for (int c = lo; c < hi; ++c) {
-            if (csum[c] > 0.0) last_pos = c;
-            if (!take_last && cum + csum[c] > target) { cstar = c; before = cum; break; }
-            cum += csum[c];
-          }
-          if (cstar < 0) { cstar = last_pos; before = cum - csum[last_pos]; take_last = true; }
-        }
-        cstar = __shfl_sync(0xffffffffu, cstar, L);
-        before = __shfl_sync(0xffffffffu, before, L);
-        take_last = __shfl_sync(0xffffffffu, take_last ? 1 : 0, L) != 0;
-        // inside the chunk: lane prefix, then the lane's four entries in ascending order
-        float r4[4];
-        load_r4<kVec>(lrow, qrow, p.q_dtype, residual, cstar * kChunk + lane * 4, V, logZ, r4);
-        const double mine = ((static_cast<double>(r4[0]) + r4[1]) + r4[2]) + r4[3];
-        double lincl = mine;
-#pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-          const double o = __shfl_up_sync(0xffffffffu, lincl, off);
-          if (lane >= off) lincl += o;
-        }
-        double cum = before + (lincl - mine);
-        int found = -1, last_mass = -1;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          cum += r4[i];
-          if (r4[i] > 0.f) last_mass = i;
-          if (found < 0 && !take_last && cum > target) found = i;
-        }
-        const unsigned hit = __ballot_sync(0xffffffffu, found >= 0);
-        const unsigned mass = __ballot_sync(0xffffffffu, last_mass >= 0);
-        int src, idx;
-        if (hit) { src = __ffs(hit) - 1; idx = found; }
-        else { src = mass ? 31 - __clz(mass) : 0; idx = last_mass < 0 ? 0 : last_mass; }
-        idx = __shfl_sync(0xffffffffu, idx, src);
-        if (lane == 0) {
-          int tokn = cstar * kChunk + src * 4 + idx;
-          if (tokn >= V) tokn = V - 1;
-          p.next_tok[b] = tokn;
-          const unsigned fl = sh_flags | flags;
-          if (fl && p.status) atomicOr(p.status, fl);
-        }
+      const double slice_total = __shfl_sync(0xffffffffu, incl, 31);
+      if (lane < S) *cluster.map_shared_rank(&sh_tot[attempt][rank], lane) = slice_total;
+    }
+    cluster.sync();
+    // every CTA: total mass and the slice that holds u * R (identical arithmetic everywhere)
+    double R = 0.0;
+    for (int r2 = 0; r2 < S; ++r2) R += sh_tot[attempt][r2];
+    if (!(R > 0.0) && residual) {                        // p <= q everywhere: draw from p instead
+      residual = false;
+      if (threadIdx.x == 0) sh_flags |= HOLA_FLAG_R_ZERO;
+      __syncthreads();
+      continue;
+    }
+    unsigned uflags = 0;
+    const float uk = clamp_uniform(sh_u[k], uflags);
+    const double target = static_cast<double>(uk) * R;
+    int rstar = -1, last_mass = 0;
+    double before_slice = 0.0;
+    {
+      double cum = 0.0;
+      for (int r2 = 0; r2 < S; ++r2) {
+        const double t = sh_tot[attempt][r2];
+        if (t > 0.0) last_mass = r2;
+        if (rstar < 0 && cum + t > target) { rstar = r2; before_slice = cum; }
+        cum += t;
       }
     }
-    __syncthreads();
-    if (!sh_redo) break;
+    bool take_last = false;
+    if (rstar < 0) {                                     // rounding left the running sum a hair below u*R
+      rstar = last_mass;
+      take_last = true;
+    }
+    if (rank == rstar && warp == 0) {
+      const unsigned over = __ballot_sync(0xffffffffu, before_slice + incl > target);
+      const unsigned has_mass = __ballot_sync(0xffffffffu, tot > 0.0);
+      int L;
+      if (over && !take_last) L = __ffs(over) - 1;
+      else { L = has_mass ? 31 - __clz(has_mass) : 0; take_last = true; }
+      int cstar = -1;
+      double before = 0.0;
+      if (lane == L) {
+        double cum = before_slice + (incl - tot);
+        int last_pos = lo;
+        for (int c = lo; c < hi; ++c) {
+          if (csum[c] > 0.0) last_pos = c;
+          if (!take_last && cum + csum[c] > target) { cstar = c; before = cum; break; }
+          cum += csum[c];
+        }
+        if (cstar < 0) { cstar = last_pos; before = cum - csum[last_pos]; take_last = true; }
+      }
+      cstar = __shfl_sync(0xffffffffu, cstar, L);
+      before = __shfl_sync(0xffffffffu, before, L);
+      take_last = __shfl_sync(0xffffffffu, take_last ? 1 : 0, L) != 0;
+      // inside the chunk: lane prefix, then the lane's four entries in ascending order
+      float r4[4];
+      load_r4<kVec>(lrow, qrow, p.q_dtype, residual, (c_first + cstar) * kChunk + lane * 4, V, logZ, r4);
+      const double mine4 = ((static_cast<double>(r4[0]) + r4[1]) + r4[2]) + r4[3];
+      double lincl = mine4;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const double o = __shfl_up_sync(0xffffffffu, lincl, off);
+        if (lane >= off) lincl += o;
+      }
+      double cum = before + (lincl - mine4);
+      int found = -1, last4 = -1;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        cum += r4[i];
+        if (r4[i] > 0.f) last4 = i;
+        if (found < 0 && !take_last && cum > target) found = i;
+      }
+      const unsigned hit = __ballot_sync(0xffffffffu, found >= 0);
+      const unsigned mass = __ballot_sync(0xffffffffu, last4 >= 0);
+      int src, idx;
+      if (hit) { src = __ffs(hit) - 1; idx = found; }
+      else { src = mass ? 31 - __clz(mass) : 0; idx = last4 < 0 ? 0 : last4; }
+      idx = __shfl_sync(0xffffffffu, idx, src);
+      if (lane == 0) {
+        int tokn = (c_first + cstar) * kChunk + src * 4 + idx;
+        if (tokn >= V) tokn = V - 1;
+        p.next_tok[b] = tokn;
+        const unsigned fl = sh_flags | uflags;
+        if (fl && p.status) atomicOr(p.status, fl);
+      }
+    }
+    break;
   }
 }
 
@@ -899,9 +935,25 @@ hola_status run_accept_sample(hola_ctx* ctx, const hola_verify_args* a, const fl
   kp.accept_len = a->accept_len; kp.next_tok = a->next_tok; kp.entropy = a->entropy; kp.logZ = a->logZ;
   kp.status = a->status_word ? a->status_word : ctx->status;
   const bool vec = (a->V % 4 == 0) && (ldl % 4 == 0) && aligned16(logits) && (a->k == 0 || aligned16(a->draft_q));
-  if (vec) accept_sample_kernel<true><<<a->B, kK3Threads, 0, stream>>>(kp);
-  else accept_sample_kernel<false><<<a->B, kK3Threads, 0, stream>>>(kp);
-  const cudaError_t e = cudaGetLastError();
+  // cluster size: as many CTAs per sequence as keeps the grid within a few waves of the SMs
+  const int nchunks = (a->V + kChunk - 1) / kChunk;
+  int S = 8;
+  while (S > 1 && (a->B * S > 8 * ctx->num_sms || nchunks / S < 8)) S >>= 1;
+  const int cpc = (nchunks + S - 1) / S;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(a->B * S));
+  cfg.blockDim = dim3(kK3Threads);
+  cfg.dynamicSmemBytes = static_cast<size_t>(cpc) * sizeof(double);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = static_cast<unsigned>(S);
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const cudaError_t e = vec ? cudaLaunchKernelEx(&cfg, accept_sample_kernel<true>, kp)
+                            : cudaLaunchKernelEx(&cfg, accept_sample_kernel<false>, kp);
   if (e != cudaSuccess) { set_error(ctx, "launch accept_sample_kernel", e); return HOLA_ERR_CUDA; }
   return HOLA_OK;
 }
