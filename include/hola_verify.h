@@ -35,7 +35,8 @@ typedef enum {
   HOLA_ERR_UNSUPPORTED_SHAPE = 2, /* H % 8 != 0, or B / k / H / V beyond what the context was created for */
   HOLA_ERR_WORKSPACE = 3,         /* device allocation failed in hola_create */
   HOLA_ERR_CUDA = 4,              /* a CUDA runtime or driver call failed; see hola_last_cuda_error */
-  HOLA_ERR_NO_DEVICE = 5          /* no sm_100 device, or the driver lacks tensor-map support */
+  HOLA_ERR_NO_DEVICE = 5,         /* no sm_100 device, or the driver lacks tensor-map support */
+  HOLA_ERR_STATIC_LIMIT = 6       /* hola_lm_head_entropy_static only: more verify rows than its fixed scratch holds */
 } hola_status;
 
 typedef enum { HOLA_Q_BF16 = 0, HOLA_Q_F32 = 1 } hola_q_dtype;
@@ -92,6 +93,25 @@ hola_status hola_verify_host(hola_ctx* ctx, const hola_verify_args* args, void* 
  *                       arrays already present in args->entropy / args->logZ (inputs here). */
 hola_status hola_lm_head_entropy(hola_ctx* ctx, const hola_verify_args* args, void* cuda_stream);
 hola_status hola_accept_sample(hola_ctx* ctx, const hola_verify_args* args, void* cuda_stream);
+
+/* The paper has no counterpart of this entry point; it exists for callers that cannot allocate device memory.
+ * Some hosts of this library may not call cudaMalloc at all: a serving engine that hands every byte of HBM to its
+ * own pool at start-up, a plugin running inside someone else's process under a fixed memory budget, code between
+ * the begin and end of a region where the allocator is locked.  Such callers cannot use hola_create, whose
+ * workspace comes from cudaMalloc.  This call does steps 1-2 (LM-head projection, logZ, entropy) with no context:
+ * the per-CTA softmax statistics that the GEMM kernel leaves for the final merge live in a 1.25 MiB array that is
+ * part of the library image (every GPU that loads the library holds it until the process exits), and everything
+ * else is the caller's: hidden, W_lm (inputs), logits_out (REQUIRED here, fp32 [B][k+1][V]), entropy, logZ
+ * (outputs), all device pointers with the layouts given above; draft_*, uniforms, tau, accept_len, next_tok are
+ * ignored.  Limit: B*(k+1) <= 512 verify rows, else HOLA_ERR_STATIC_LIMIT and nothing is launched.
+ * Runs on the CURRENT device, asynchronously on cuda_stream.  It calls no cudaMalloc, cudaFree or other allocating
+ * routine.  The first call on each device also looks up the array's device address and the driver's tensor-map
+ * encoder; make that first call outside any stream capture.
+ * All calls on one GPU share the array, and it keeps the previous call's contents: the library clears the one word
+ * that must start at zero and overwrites the rest before reading it, so calls that follow each other on one stream
+ * are safe, but two calls that overlap on the GPU (issued on different streams, say) race on it and give
+ * wrong entropy / logZ.  Serialise them. */
+hola_status hola_lm_head_entropy_static(const hola_verify_args* args, void* cuda_stream);
 
 /* Launch geometry chosen for a shape (for reports): vocab tile width, grid size, pipeline stages,
  * row blocks of 128 positions per pass, passes over W_lm. */

@@ -18,7 +18,7 @@ HOLA_Q_BF16, HOLA_Q_F32 = 0, 1
 FLAG_BAD_TOKEN, FLAG_BAD_UNIFORM, FLAG_TIMEOUT, FLAG_R_ZERO = 1, 2, 4, 8
 
 EXPORTS = ["hola_create", "hola_destroy", "hola_workspace_bytes", "hola_verify", "hola_verify_host",
-           "hola_lm_head_entropy", "hola_accept_sample", "hola_plan", "hola_profile_begin", "hola_profile_end", "hola_strerror", "hola_last_cuda_error",
+           "hola_lm_head_entropy", "hola_accept_sample", "hola_lm_head_entropy_static", "hola_plan", "hola_profile_begin", "hola_profile_end", "hola_strerror", "hola_last_cuda_error",
            "hola_version"]
 
 
@@ -60,6 +60,8 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
         fn = getattr(lib, name)
         fn.restype = ctypes.c_int
         fn.argtypes = [ctypes.c_void_p, ctypes.POINTER(hola_verify_args), ctypes.c_void_p]
+    lib.hola_lm_head_entropy_static.restype = ctypes.c_int
+    lib.hola_lm_head_entropy_static.argtypes = [ctypes.POINTER(hola_verify_args), ctypes.c_void_p]
     lib.hola_plan.restype = ctypes.c_int
     lib.hola_plan.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.POINTER(hola_plan_info)]
     lib.hola_profile_begin.restype = ctypes.c_int
@@ -91,6 +93,26 @@ def _dptr(t: torch.Tensor | None):
 def _stream_ptr(stream) -> ctypes.c_void_p:
     s = torch.cuda.current_stream() if stream is None else stream
     return ctypes.c_void_p(s.cuda_stream)
+
+
+def hola_lm_head_entropy_static(hidden, W_lm, logits, entropy, logZ, stream=None) -> None:
+    """Steps 1-2 through the entry point that allocates no device memory (no context needed).
+
+    For callers that cannot call cudaMalloc (all of HBM already handed to their own pool, a fixed memory budget,
+    an allocator that is locked at this point): the library's only scratch for this call is a 1.25 MiB array
+    built into it.  Every tensor is the caller's and lives on the current device: hidden bf16 [B, k+1, H],
+    W_lm bf16 [V, H], and the outputs logits fp32 [B, k+1, V], entropy and logZ fp32 [B, k+1].
+    At most 512 verify rows (B * (k+1)); larger calls raise HolaError and launch nothing.  Calls share the
+    built-in array, so do not let two of them overlap on one GPU.
+    """
+    lib = load_library()
+    B, k1, H = hidden.shape
+    a = hola_verify_args()
+    a.B, a.k, a.H, a.V = B, k1 - 1, H, W_lm.shape[0]
+    a.hidden, a.W_lm = _dptr(hidden), _dptr(W_lm)
+    a.logits_out, a.entropy, a.logZ = _dptr(logits), _dptr(entropy), _dptr(logZ)
+    _check(lib, None, lib.hola_lm_head_entropy_static(ctypes.byref(a), _stream_ptr(stream)),
+           "hola_lm_head_entropy_static")
 
 
 @dataclass

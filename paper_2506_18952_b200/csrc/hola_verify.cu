@@ -29,6 +29,8 @@
 
 #include <cooperative_groups.h>
 
+#include <mutex>
+
 #include "../../include/hola_verify.h"
 
 namespace cg = cooperative_groups;
@@ -997,6 +999,8 @@ const char* hola_strerror(hola_status s) {
     case HOLA_ERR_WORKSPACE: return "workspace allocation failed";
     case HOLA_ERR_CUDA: return "CUDA call failed (see hola_last_cuda_error)";
     case HOLA_ERR_NO_DEVICE: return "no usable sm_100 device";
+    case HOLA_ERR_STATIC_LIMIT:
+      return "problem too large for the fixed scratch of hola_lm_head_entropy_static (more than 512 verify rows)";
     default: return "unknown status";
   }
 }
@@ -1203,3 +1207,87 @@ hola_status hola_verify_host(hola_ctx* ctx, const hola_verify_args* a, void* cud
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------------------------------ no-allocation entry
+// hola_lm_head_entropy_static: steps 1-2 for callers that must not allocate device memory.  The per-CTA softmax
+// statistics, which hola_lm_head_entropy keeps in the context's cudaMalloc'ed workspace, live here in a fixed
+// array inside the library image; logits, entropy and logZ go to the caller's buffers as usual.
+
+namespace {
+
+constexpr int kStaticMaxRows = 512;    // verify rows B(k+1) one call may have
+constexpr int kStaticMaxCtas = 160;    // CTAs of the GEMM kernel that may leave statistics (one per SM; B200 has 148)
+constexpr size_t kStaticStatusBytes = 256;
+constexpr size_t kStaticScratchBytes =
+    kStaticStatusBytes + static_cast<size_t>(kStaticMaxCtas) * kStaticMaxRows * sizeof(float4);   // 1 310 976 bytes
+
+}  // namespace
+
+// Every GPU that loads the library holds this array until the process exits.  In host code the name is only a
+// handle for cudaGetSymbolAddress, never a device address.
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+namespace {
+
+constexpr int kStaticMaxDevices = 64;
+std::mutex g_static_mu;
+hola_ctx g_static_ctx[kStaticMaxDevices];      // host-side descriptors only; they own no memory
+bool g_static_ready[kStaticMaxDevices];
+
+// Once per device, with that device current: where the array lives on this device, the tensor-map encoder of the
+// driver, and the SM count.  Allocates nothing.
+hola_status static_setup(int dev, hola_ctx* out) {
+  std::lock_guard<std::mutex> lock(g_static_mu);
+  hola_ctx* c = &g_static_ctx[dev];
+  if (!g_static_ready[dev]) {
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess || prop.major != 10) return HOLA_ERR_NO_DEVICE;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+        qres != cudaDriverEntryPointSuccess)
+      return HOLA_ERR_NO_DEVICE;
+    void* base = nullptr;
+    const cudaError_t e = cudaGetSymbolAddress(&base, g_static_scratch);
+    if (e != cudaSuccess || !base) return HOLA_ERR_CUDA;
+    memset(c, 0, sizeof *c);
+    c->device = dev;
+    c->num_sms = prop.multiProcessorCount;
+    c->encode = reinterpret_cast<EncodeTiledFn>(fn);
+    c->status = reinterpret_cast<unsigned*>(base);
+    c->partials = reinterpret_cast<float4*>(static_cast<unsigned char*>(base) + kStaticStatusBytes);
+    c->max_rows = kStaticMaxRows;
+    g_static_ready[dev] = true;
+  }
+  *out = *c;
+  return HOLA_OK;
+}
+
+}  // namespace
+
+extern "C" hola_status hola_lm_head_entropy_static(const hola_verify_args* a, void* cuda_stream) {
+  if (!a) return HOLA_ERR_INVALID_ARG;
+  if (a->B < 0 || a->k < 0 || a->H <= 0 || a->V <= 0) return HOLA_ERR_INVALID_ARG;
+  if (a->B == 0) return HOLA_OK;
+  if (!a->hidden || !a->W_lm || !a->logits_out || !a->entropy || !a->logZ) return HOLA_ERR_INVALID_ARG;
+  if (!aligned16(a->hidden) || !aligned16(a->W_lm)) return HOLA_ERR_INVALID_ARG;
+  if (a->H % 8 != 0) return HOLA_ERR_UNSUPPORTED_SHAPE;
+  const long long rows = static_cast<long long>(a->B) * (a->k + 1);
+  if (rows > kStaticMaxRows) return HOLA_ERR_STATIC_LIMIT;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kStaticMaxDevices) return HOLA_ERR_NO_DEVICE;
+  hola_ctx local;                      // a per-call copy: concurrent host threads do not share host state
+  hola_status s = static_setup(dev, &local);
+  if (s != HOLA_OK) return s;
+  local.H = a->H; local.V = a->V; local.maxB = a->B; local.maxK = a->k;
+  const int M = static_cast<int>(rows);
+  const Plan pl = make_plan(&local, M);
+  if (pl.grid > kStaticMaxCtas) return HOLA_ERR_STATIC_LIMIT;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  // The array keeps whatever the last call left.  The statistics slots are fully overwritten for the rows of this
+  // call before they are read; the internal status word is the one thing that must start at zero.
+  if (cudaMemsetAsync(local.status, 0, sizeof(unsigned), stream) != cudaSuccess) return HOLA_ERR_CUDA;
+  if ((s = run_lm_head(&local, a, a->logits_out, a->V, pl, stream)) != HOLA_OK) return s;
+  finalize_kernel<<<(M + 7) / 8, 256, 0, stream>>>(local.partials, pl.grid, local.max_rows, M, a->logZ, a->entropy);
+  return cudaGetLastError() == cudaSuccess ? HOLA_OK : HOLA_ERR_CUDA;
+}
