@@ -113,10 +113,10 @@ hola_status hola_accept_sample(hola_ctx* ctx, const hola_verify_args* args, void
  * wrong entropy / logZ.  Serialise them. */
 hola_status hola_lm_head_entropy_static(const hola_verify_args* args, void* cuda_stream);
 
-/* Launch geometry chosen for a shape (for reports): vocab tile width, grid size, pipeline stages,
- * row blocks of 128 positions per pass, passes over W_lm. */
+/* Launch geometry chosen for a shape (for reports): vocabulary rows per tile of a CTA pair, grid size (CTAs),
+ * shared-memory ring slots, verify rows per pass, passes over W_lm, kernel launches per hola_verify call. */
 typedef struct {
-  int32_t tile_n, grid, stages, row_blocks, passes, kernels_per_call;
+  int32_t tile_v, grid, stages, rows_per_pass, passes, kernels_per_call;
 } hola_plan_info;
 hola_status hola_plan(const hola_ctx* ctx, int B, int k, hola_plan_info* out);
 

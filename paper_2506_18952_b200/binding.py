@@ -36,7 +36,7 @@ class hola_verify_args(ctypes.Structure):
 
 
 class hola_plan_info(ctypes.Structure):
-    _fields_ = [(n, ctypes.c_int32) for n in ("tile_n", "grid", "stages", "row_blocks", "passes", "kernels_per_call")]
+    _fields_ = [(n, ctypes.c_int32) for n in ("tile_v", "grid", "stages", "rows_per_pass", "passes", "kernels_per_call")]
 
 
 _lib = None

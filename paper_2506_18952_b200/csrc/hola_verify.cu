@@ -2,12 +2,15 @@
 // Decoding (HSD section, Eq. 1, Algorithm 1 lines 4-8).  See include/hola_verify.h for the contract.
 //
 // Kernels
-//   lm_head_entropy_kernel<RB>  persistent, warp-specialised weight-streaming GEMM.  One CTA per SM walks vocab
-//       tiles; a producer thread feeds a shared-memory ring with TMA (128-byte-swizzled K-major tiles of W_lm and
-//       of up to RB blocks of 128 verify positions); one thread issues tcgen05.mma (bf16 x bf16 -> fp32 in
-//       tensor memory); four epilogue warps read the accumulators with tcgen05.ld, store fp32 logits and keep,
-//       per verify position, the running softmax statistics (m, s, t) = (max, sum e^(l-m), sum e^(l-m)(l-m)) in
-//       registers across all of the CTA's tiles.  W_lm is read from HBM once per pass.
+//   lm_head_entropy_kernel      persistent, warp-specialised weight-streaming GEMM run by pairs of CTAs (clusters of
+//       two).  The vocabulary lies on the 128 tensor-memory lanes of each CTA, the verify positions on the N
+//       dimension of the MMA:  D[v, r] = sum_h W_lm[v, h] * hidden[r, h].  A pair owns 256 vocabulary rows per
+//       tile; each CTA streams its 128 rows of W_lm and HALF of the hidden rows per K block with TMA, and one
+//       thread of the leader CTA issues tcgen05.mma.cta_group::2 (bf16 x bf16 -> fp32 in tensor memory) that reads
+//       both halves.  Drain warps copy finished accumulators to the fp32 logits buffer; statistics warps re-read
+//       that tile row-wise (it is still in L2) and keep, per verify position, the running softmax statistics
+//       (m, s, t) = (max, sum e^(l-m), sum e^(l-m)(l-m)) in registers, in the shadow of the next tile's MMAs.
+//       W_lm is read from HBM once per pass.
 //   finalize_kernel             merges the per-CTA statistics:  logZ = m + ln s,  H = ln s - t/s  (entropy
 //       definition of the HSD section, rearranged around the running maximum).
 //   accept_sample_kernel        one cluster of CTAs per sequence: merges the statistics for its k+1 positions (warp
@@ -39,15 +42,22 @@ namespace {
 
 // ------------------------------------------------------------------------------------------------ constants
 constexpr int kBlockK = 64;                      // bf16 elements per K block = one 128-byte swizzle row
-constexpr int kRows = 128;                       // verify positions per row block = tensor-memory lanes
-constexpr int kABlockBytes = kRows * kBlockK * 2;
-constexpr int kK1Threads = 192;                  // warp 0 TMA, warp 1 MMA + tensor-memory owner, warps 2-5 epilogue
+constexpr int kLanes = 128;                      // vocabulary rows per CTA per tile = tensor-memory lanes
+constexpr int kPairTile = 2 * kLanes;            // vocabulary rows per CTA pair per tile
+constexpr int kWBlockBytes = kLanes * kBlockK * 2;
+constexpr int kMaxN = 256;                       // verify rows per MMA
+constexpr int kMaxRowsPerPass = 2 * kMaxN;       // two MMAs per K step fill the 512 tensor-memory columns
+constexpr int kDrainWarps = 8;                   // warps 2..9: tensor memory -> logits buffer
+constexpr int kStatsWarps = 8;                   // warps 10..17: softmax statistics from the stored tile
+constexpr int kStatsThreads = kStatsWarps * 32;
+constexpr int kK1Warps = 2 + kDrainWarps + kStatsWarps;   // warp 0 TMA, warp 1 MMA + tensor-memory owner
+constexpr int kK1Threads = kK1Warps * 32;
+constexpr int kStatsRowsPerThread = kMaxRowsPerPass * 4 / kStatsThreads;   // four threads share a row
 constexpr int kTmemCols = 512;
-constexpr int kMaxStages = 8;
-constexpr int kMaxRowBlocks = 4;
+constexpr int kMaxStages = 12;
 constexpr int kSmemBudget = 227 * 1024;          // dynamic shared memory per CTA on sm_100
-constexpr int kBarrierBytes = 256;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait, far above any legitimate wait
+constexpr int kBarrierBytes = 512;
+constexpr long long kWaitLimitCycles = 4000000000ll;   // about 2 s of SM clock per wait, far above any legitimate wait
 
 constexpr int kK3Threads = 256;
 constexpr int kK3Warps = kK3Threads / 32;
@@ -60,9 +70,11 @@ constexpr float kLog2e = 1.4426950408889634f;
 struct K1Params {
   int M;          // total verify rows B(k+1)
   int row0;       // first row of this pass
-  int V, tile_n, n_tiles, n_kblocks, stages, nbuf;
+  int rows;       // rows of this pass (<= n_sub * N)
+  int V, n_ptiles, n_kblocks, stages, nbuf;
+  int n_sub, N;   // MMAs per K step and their N (verify rows each; multiple of 16)
   int ldl;        // row pitch of the logits buffer, in floats
-  int vec_ok;     // 16-byte stores allowed (pitch and base aligned)
+  int vec_ok;     // 16-byte loads of the logits buffer allowed (pitch and base aligned)
   float* logits;
   float4* partials;   // [grid][part_stride] (m, s, t, unused)
   int part_stride;
@@ -89,20 +101,37 @@ struct K3Params {
 // ------------------------------------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
 
-__device__ __forceinline__ unsigned long long globaltimer_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
+__device__ __forceinline__ uint32_t cluster_cta_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// Address, in the cluster's shared window, of the same shared-memory offset in CTA `rank` of this cluster.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
 }
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// Arrivals on a barrier that may live in the peer CTA (address from map_to_cta).  Default (CTA-scope release)
+// semantics on purpose: a cluster-scope release here acts as a fence that waits for the thread's earlier
+// outstanding operations and serialises the pipeline.
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx_cluster(uint32_t cluster_bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_bar), "r"(bytes)
+               : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
@@ -115,22 +144,34 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 
 // Bounded wait.  Returns false when the CTA is aborting (this wait or another one ran out of time).
+// The clock is the SM's cycle counter (cheap to read), looked at only every 256 unsuccessful polls.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
                                           unsigned* status) {
   if (mbar_try_wait(bar, parity)) return true;
-  const unsigned long long t0 = globaltimer_ns();
+  long long t0 = 0;
   uint32_t spins = 0;
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((++spins & 63u) == 0u) {
+    if ((++spins & 255u) == 0u) {
       if (*abort_flag) return false;
-      if (globaltimer_ns() - t0 > kWaitLimitNs) {
+      const long long now = clock64();
+      if (t0 == 0) t0 = now;
+      if (now - t0 > kWaitLimitCycles) {
         *abort_flag = 1u;
         if (status) atomicOr(status, HOLA_FLAG_TIMEOUT);
         return false;
       }
     }
   }
+}
+
+// Whole-warp form: lane 0 polls, every lane gets the same answer (and, through the shuffle, the same ordering).
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                               unsigned* status) {
+  int r = 1;
+  if ((threadIdx.x & 31) == 0) r = mbar_wait(bar, parity, abort_flag, status) ? 1 : 0;
+  r = __shfl_sync(0xffffffffu, r, 0);
+  return r != 0;
 }
 
 __device__ __forceinline__ uint64_t l2_policy_evict_first() {
@@ -144,40 +185,47 @@ __device__ __forceinline__ uint64_t l2_policy_evict_last() {
   return pol;
 }
 
-// 2-D tiled TMA load, global -> this CTA's shared memory, completion counted on an mbarrier.
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y,
+// 2-D tiled TMA load, global -> this CTA's shared memory.  The completion is counted on an mbarrier that may
+// live in either CTA of the pair (cta_group::2 form); no multicast: each CTA fetches its own bytes.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t cluster_bar, int x, int y,
                                             uint64_t policy) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
       " [%0], [%1, {%3, %4}], [%2], %5;"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "l"(policy)
+      ::"r"(dst), "l"(map), "r"(cluster_bar), "r"(x), "r"(y), "l"(policy)
       : "memory");
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
+// Tensor memory of the CTA pair: executed by one warp of EACH CTA of the pair.
 __device__ __forceinline__ void tmem_alloc(uint32_t holder_smem, uint32_t ncols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(holder_smem), "r"(ncols)
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(holder_smem), "r"(ncols)
                : "memory");
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
 }
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
 }
 
-// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate, issued by one thread.
+// D[tmem of both CTAs] (+)= A[smem of both CTAs] * B[smem of both CTAs]^T, bf16 inputs, fp32 accumulate.
+// Issued by one thread of the pair's leader CTA; descriptors are shared-memory offsets valid in both CTAs.
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
                                           uint32_t accumulate) {
   asm volatile(
       "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
-      " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+      " tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}"
       ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
-// mbarrier arrives once every MMA issued so far by this thread has completed.
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+// The mbarrier at this shared-memory offset in BOTH CTAs of the pair gets one arrival once every MMA issued so far
+// by this thread has completed.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  const uint16_t mask = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(mask)
+               : "memory");
 }
 
 // 32 consecutive fp32 columns of this thread's tensor-memory lane.
@@ -216,9 +264,9 @@ __device__ __forceinline__ uint64_t make_kmajor_sw128_desc(uint32_t smem_addr) {
   return d;
 }
 
-// Instruction descriptor, kind::f16: D fp32, A and B bf16, both K-major, M = 128, N = n.
-__device__ __forceinline__ uint32_t make_idesc_bf16_m128(uint32_t n) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((n >> 3) << 17) | ((128u >> 4) << 24);
+// Instruction descriptor, kind::f16: D fp32, A and B bf16, both K-major, M = 256 (the pair), N = n.
+__device__ __forceinline__ uint32_t make_idesc_bf16_m256(uint32_t n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((n >> 3) << 17) | ((256u >> 4) << 24);
 }
 
 // ------------------------------------------------------------------------------------------------ softmax statistics
@@ -274,7 +322,15 @@ __device__ __forceinline__ void stats_fold(const float* v, int n, Stats& st) {
 }
 
 // ------------------------------------------------------------------------------------------------ K1
-template <int RB>
+// Shared memory: `stages` ring slots of [W_lm block 128 x 64 | hidden block(s) n_sub x (N/2) x 64], then the
+// barrier area.  Barriers (8 bytes each, offsets in the barrier area):
+//   full[12]   @0    leader CTA's copy is the live one: 2 arrivals (one producer per CTA) + the bytes of both CTAs
+//   empty[12]  @96   per CTA: the MMAs that read this slot have completed (commit, delivered to both CTAs)
+//   tfull[2]   @192  per CTA: the accumulators of a tile are complete (commit, delivered to both CTAs)
+//   tempty[2]  @208  leader's copy: all 16 drain warps of the pair have read their accumulators
+//   lready[2]  @224  per CTA: the 8 drain warps have stored the tile's logits (by tile parity)
+//   sfree[2]   @240  per CTA: the 8 statistics warps are done with that tile (keeps lready from lapping)
+//   tensor-memory base @256, abort flag @260
 __global__ void __launch_bounds__(kK1Threads, 1)
 lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __grid_constant__ CUtensorMap tmap_w,
                        const K1Params p) {
@@ -285,65 +341,74 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const uint32_t stage_bytes = RB * kABlockBytes + p.tile_n * 128;
+  const uint32_t rank = cluster_cta_rank();              // 0 = leader of the pair
+  const int pair = blockIdx.x >> 1;
+  const int npairs = gridDim.x >> 1;
+  const int half_n = p.N >> 1;                           // hidden rows this CTA supplies per MMA
+  const uint32_t hid_block_bytes = static_cast<uint32_t>(half_n) * 128u;
+  const uint32_t stage_bytes = kWBlockBytes + p.n_sub * hid_block_bytes;
   const uint32_t bar_base = base + p.stages * stage_bytes;
-  // barrier area: full[8] | empty[8] | tmem_full[2] | tmem_empty[2] | tmem holder | abort flag
-  const uint32_t full_bar = bar_base, empty_bar = bar_base + 64, tfull_bar = bar_base + 128,
-                 tempty_bar = bar_base + 144;
-  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + p.stages * stage_bytes + 160);
-  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + p.stages * stage_bytes + 164);
+  const uint32_t full_bar = bar_base, empty_bar = bar_base + 96, tfull_bar = bar_base + 192,
+                 tempty_bar = bar_base + 208, lready_bar = bar_base + 224, sfree_bar = bar_base + 240;
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + p.stages * stage_bytes + 256);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + p.stages * stage_bytes + 260);
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < p.stages; ++i) {
-      mbar_init(full_bar + 8 * i, 1);
+      mbar_init(full_bar + 8 * i, 2);
       mbar_init(empty_bar + 8 * i, 1);
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(tfull_bar + 8 * i, 1);
-      mbar_init(tempty_bar + 8 * i, 4);                  // one arrival per epilogue warp
+      mbar_init(tempty_bar + 8 * i, 2 * kDrainWarps);
+      mbar_init(lready_bar + 8 * i, kDrainWarps);
+      mbar_init(sfree_bar + 8 * i, kStatsWarps);
     }
     *abort_flag = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_hidden) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_w) : "memory");
   }
+  __syncwarp();
   if (warp == 1) tmem_alloc(smem_u32(tmem_holder), kTmemCols);
   tc_fence_before();
   __syncthreads();
+  cluster_sync_all();                                    // the peer's barriers are initialised too
   tc_fence_after();
   const uint32_t tmem_base = *tmem_holder;
 
-  const int acc_cols = RB * p.tile_n;
-  const int my_tiles = (p.n_tiles - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) /
-                       static_cast<int>(gridDim.x);
+  const int my_tiles = (p.n_ptiles - pair + npairs - 1) / npairs;
+  const int sub_chunks = (p.N + 31) >> 5;                // 32-column chunks per MMA's accumulator
+  // accumulator of MMA s of buffer b starts at column b * 256 + s * 256 (two buffers only when n_sub == 1)
 
   if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
+    // ------------------------------------------------------------------ TMA producer (one per CTA)
     if (lane == 0) {
       const uint64_t pol_w = l2_policy_evict_first();    // W_lm is streamed once
-      const uint64_t pol_h = l2_policy_evict_last();     // hidden is re-read by every CTA for every tile
+      const uint64_t pol_h = l2_policy_evict_last();     // hidden is re-read for every tile
+      const uint32_t leader_full = map_to_cta(full_bar, 0);
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
       for (int t = 0; t < my_tiles && ok; ++t) {
-        const int tile = blockIdx.x + t * gridDim.x;
+        const int v0 = (pair + t * npairs) * kPairTile + static_cast<int>(rank) * kLanes;
         for (int kb = 0; kb < p.n_kblocks; ++kb) {
           if (!mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
           const uint32_t sa = base + stage * stage_bytes;
-          const uint32_t fb = full_bar + 8 * stage;
-          mbar_expect_tx(fb, stage_bytes);
-#pragma unroll
-          for (int a = 0; a < RB; ++a)
-            tma_load_2d(sa + a * kABlockBytes, &tmap_hidden, fb, kb * kBlockK, p.row0 + a * kRows, pol_h);
-          tma_load_2d(sa + RB * kABlockBytes, &tmap_w, fb, kb * kBlockK, tile * p.tile_n, pol_w);
+          const uint32_t fb = leader_full + 8 * stage;
+          mbar_expect_tx_cluster(fb, stage_bytes);
+          tma_load_2d(sa, &tmap_w, fb, kb * kBlockK, v0, pol_w);
+          for (int s = 0; s < p.n_sub; ++s)
+            tma_load_2d(sa + kWBlockBytes + s * hid_block_bytes, &tmap_hidden, fb, kb * kBlockK,
+                        p.row0 + s * p.N + static_cast<int>(rank) * half_n, pol_h);
           if (++stage == p.stages) { stage = 0; phase ^= 1u; }
         }
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      const uint32_t idesc = make_idesc_bf16_m128(static_cast<uint32_t>(p.tile_n));
+    // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+    if (lane == 0 && rank == 0) {
+      const uint32_t idesc = make_idesc_bf16_m256(static_cast<uint32_t>(p.N));
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
@@ -352,97 +417,143 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
         const uint32_t acc_phase = static_cast<uint32_t>(t / p.nbuf) & 1u;
         if (!mbar_wait(tempty_bar + 8 * buf, acc_phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t d0 = tmem_base + buf * acc_cols;
+        const uint32_t d0 = tmem_base + buf * 256;
         for (int kb = 0; kb < p.n_kblocks; ++kb) {
           if (!mbar_wait(full_bar + 8 * stage, phase, abort_flag, p.status)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = base + stage * stage_bytes;
-          const uint64_t bdesc = make_kmajor_sw128_desc(sa + RB * kABlockBytes);
+          const uint64_t adesc = make_kmajor_sw128_desc(sa);
 #pragma unroll
-          for (int a = 0; a < RB; ++a) {
-            const uint64_t adesc = make_kmajor_sw128_desc(sa + a * kABlockBytes);
-#pragma unroll
-            for (int kk = 0; kk < kBlockK / 16; ++kk) {
-              // 16 bf16 = 32 bytes further along K inside the swizzled row: +2 in 16-byte address units
-              umma_bf16(d0 + a * p.tile_n, adesc + 2 * kk, bdesc + 2 * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
+          for (int kk = 0; kk < kBlockK / 16; ++kk) {
+            // 16 bf16 = 32 bytes further along K inside the swizzled row: +2 in 16-byte address units
+            for (int s = 0; s < p.n_sub; ++s) {
+              const uint64_t bdesc = make_kmajor_sw128_desc(sa + kWBlockBytes + s * hid_block_bytes);
+              umma_bf16(d0 + s * 256, adesc + 2 * kk, bdesc + 2 * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
             }
           }
-          umma_commit(empty_bar + 8 * stage);            // frees the stage once these MMAs have read it
+          umma_commit_pair(empty_bar + 8 * stage);       // frees the slot in both CTAs once these MMAs have read it
           if (++stage == p.stages) { stage = 0; phase ^= 1u; }
         }
-        if (ok) umma_commit(tfull_bar + 8 * buf);        // accumulators of this tile are complete
+        if (ok) umma_commit_pair(tfull_bar + 8 * buf);   // accumulators of this tile are complete in both CTAs
       }
     }
-  } else {
-    // ------------------------------------------------------------------ epilogue warps 2..5
-    const int quarter = warp & 3;                        // tensor-memory lanes 32*quarter .. +31
-    Stats st[RB];
-    int row[RB];
-    bool row_ok[RB], warp_has_rows[RB];
-#pragma unroll
-    for (int a = 0; a < RB; ++a) {
-      st[a] = stats_empty();
-      row[a] = p.row0 + a * kRows + quarter * 32 + lane;
-      row_ok[a] = row[a] < p.M;
-      warp_has_rows[a] = (p.row0 + a * kRows + quarter * 32) < p.M;
-    }
+  } else if (warp < 2 + kDrainWarps) {
+    // ------------------------------------------------------------------ drain warps: tensor memory -> logits
+    const int quarter = warp & 3;                        // tensor-memory lanes 32*quarter .. +31 (fixed by warp id)
+    const int group = (warp - 2) >> 2;                   // the two warps of a quarter alternate over the chunks
+    const uint32_t leader_tempty = map_to_cta(tempty_bar, 0);
+    const int n_chunks = p.n_sub * sub_chunks;
     bool ok = true;
     for (int t = 0; t < my_tiles && ok; ++t) {
-      const int tile = blockIdx.x + t * gridDim.x;
       const int buf = t % p.nbuf;
       const uint32_t acc_phase = static_cast<uint32_t>(t / p.nbuf) & 1u;
-      if (!mbar_wait(tfull_bar + 8 * buf, acc_phase, abort_flag, p.status)) { ok = false; break; }
+      const int par = t & 1;
+      if (!mbar_wait_warp(tfull_bar + 8 * buf, acc_phase, abort_flag, p.status)) { ok = false; break; }
       tc_fence_after();
-      const int col_tile = tile * p.tile_n;
+      const int vocab = (pair + t * npairs) * kPairTile + static_cast<int>(rank) * kLanes + quarter * 32 + lane;
+      const bool vocab_ok = vocab < p.V;
+      const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * 256;
+      for (int ch = group; ch < n_chunks; ch += 2) {
+        const int s = ch / sub_chunks, j = ch - s * sub_chunks;
+        float v[32];
+        __syncwarp();                                    // tcgen05.ld is warp-collective: reconverge first
+        tmem_ld32(lane_addr + s * 256 + j * 32, v);
+        const int c0 = j * 32;                           // first column of the chunk inside its MMA
+        const int r0 = p.row0 + s * p.N + c0;            // verify row of column c0
+        int n_ok = min(p.N - c0, p.M - r0);              // columns that are real rows
+        n_ok = min(n_ok, 32);
+        if (vocab_ok && n_ok > 0) {
+          float* dst = p.logits + static_cast<size_t>(r0) * p.ldl + vocab;
+          if (n_ok == 32) {
 #pragma unroll
-      for (int a = 0; a < RB; ++a) {
-        if (!warp_has_rows[a]) continue;                 // warp-uniform
-        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
-                               static_cast<uint32_t>(buf * acc_cols + a * p.tile_n);
-        float* dst_row = p.logits + static_cast<size_t>(row[a]) * p.ldl;
-        for (int c0 = 0; c0 < p.tile_n; c0 += 32) {
-          const int col = col_tile + c0;
-          const int valid = p.V - col;                   // columns of this chunk inside the vocabulary
-          if (valid <= 0) break;                         // warp-uniform
-          float v[32];
-          __syncwarp();                                  // tcgen05.ld is warp-collective: reconverge first
-          tmem_ld32(taddr + c0, v);
-          if (row_ok[a]) {
-            if (valid >= 32) {
-              stats_fold<true>(v, 32, st[a]);
-              if (p.vec_ok) {
-                float4* d4 = reinterpret_cast<float4*>(dst_row + col);
+            for (int i = 0; i < 32; ++i) dst[static_cast<size_t>(i) * p.ldl] = v[i];
+          } else {
 #pragma unroll
-                for (int i = 0; i < 8; ++i) d4[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-              } else {
-#pragma unroll
-                for (int i = 0; i < 32; ++i) dst_row[col + i] = v[i];
-              }
-            } else {
-              stats_fold<false>(v, valid, st[a]);
-#pragma unroll
-              for (int i = 0; i < 32; ++i)
-                if (i < valid) dst_row[col + i] = v[i];
-            }
+            for (int i = 0; i < 32; ++i)
+              if (i < n_ok) dst[static_cast<size_t>(i) * p.ldl] = v[i];
           }
         }
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(tempty_bar + 8 * buf);
+      if (lane == 0) mbar_arrive_cluster(leader_tempty + 8 * buf);     // this warp's accumulators may be overwritten
+      // the statistics warps must have finished the tile that used this parity before it is announced again
+      if (t >= 2 && !mbar_wait_warp(sfree_bar + 8 * par, static_cast<uint32_t>((t >> 1) - 1) & 1u, abort_flag, p.status)) {
+        ok = false;
+        break;
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(lready_bar + 8 * par);  // release: this warp's stores are visible to the CTA
+    }
+  } else {
+    // ------------------------------------------------------------------ statistics warps
+    // Four threads share a verify row: thread `part` takes floats 16*it + 4*part .. +3 (it = 0..7) of the row's 128
+    // logits of this tile, so a warp's load covers 8 rows x 64 contiguous bytes.
+    const int ts = threadIdx.x - (2 + kDrainWarps) * 32;
+    const int part = ts & 3, rsub = ts >> 2;
+    Stats st[kStatsRowsPerThread];
+#pragma unroll
+    for (int i = 0; i < kStatsRowsPerThread; ++i) st[i] = stats_empty();
+    bool ok = true;
+    for (int t = 0; t < my_tiles && ok; ++t) {
+      const int par = t & 1;
+      if (!mbar_wait_warp(lready_bar + 8 * par, static_cast<uint32_t>(t >> 1) & 1u, abort_flag, p.status)) { ok = false; break; }
+      const int vbase = (pair + t * npairs) * kPairTile + static_cast<int>(rank) * kLanes;
+      const int lim = p.V - vbase;                       // logits of this tile inside the vocabulary
+      if (lim > 0) {
+#pragma unroll
+        for (int i = 0; i < kStatsRowsPerThread; ++i) {
+          const int r = rsub + (kStatsThreads / 4) * i;
+          if (r < p.rows) {
+            const float* src = p.logits + static_cast<size_t>(p.row0 + r) * p.ldl + vbase;
+            float v[32];
+            if (p.vec_ok && lim >= kLanes) {
+#pragma unroll
+              for (int it = 0; it < 8; ++it) {
+                const float4 x = __ldcg(reinterpret_cast<const float4*>(src + 16 * it + 4 * part));
+                v[4 * it] = x.x; v[4 * it + 1] = x.y; v[4 * it + 2] = x.z; v[4 * it + 3] = x.w;
+              }
+              stats_fold<true>(v, 32, st[i]);
+            } else {
+              int n = 0;                                 // this thread's columns ascend with the index: a prefix is valid
+#pragma unroll
+              for (int idx = 0; idx < 32; ++idx) {
+                const int col = 16 * (idx >> 2) + 4 * part + (idx & 3);
+                const bool in = col < lim;
+                v[idx] = in ? __ldcg(src + col) : 0.f;
+                n += in ? 1 : 0;
+              }
+              if (n > 0) stats_fold<false>(v, n, st[i]);
+            }
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(sfree_bar + 8 * par);
     }
     if (ok) {
 #pragma unroll
-      for (int a = 0; a < RB; ++a)
-        if (row_ok[a])
-          p.partials[static_cast<size_t>(blockIdx.x) * p.part_stride + row[a]] =
-              make_float4(st[a].m, st[a].s, st[a].t, 0.f);
+      for (int i = 0; i < kStatsRowsPerThread; ++i) {
+        Stats a = st[i];
+#pragma unroll
+        for (int off = 1; off <= 2; off <<= 1) {
+          Stats o;
+          o.m = __shfl_xor_sync(0xffffffffu, a.m, off);
+          o.s = __shfl_xor_sync(0xffffffffu, a.s, off);
+          o.t = __shfl_xor_sync(0xffffffffu, a.t, off);
+          a = ((lane & off) == 0) ? stats_merge(a, o) : stats_merge(o, a);
+        }
+        const int r = rsub + (kStatsThreads / 4) * i;
+        if (part == 0 && r < p.rows)
+          p.partials[static_cast<size_t>(blockIdx.x) * p.part_stride + p.row0 + r] = make_float4(a.m, a.s, a.t, 0.f);
+      }
     }
   }
 
   // ------------------------------------------------------------------ common tail
   tc_fence_before();
   __syncthreads();
+  cluster_sync_all();                                    // the peer no longer signals this CTA's barriers or tensor memory
   if (warp == 1) {
     if (*abort_flag) __nanosleep(200000);                // let copies already in flight land before leaving
     tmem_dealloc(tmem_base, kTmemCols);
@@ -749,7 +860,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 struct Plan {
-  int tile_n, grid, stages, row_blocks, passes, nbuf, n_tiles, n_kblocks, smem_bytes;
+  int n_sub, N, rows_per_pass, passes, grid, stages, nbuf, n_ptiles, n_kblocks, smem_bytes;
 };
 
 }  // namespace
@@ -765,7 +876,7 @@ struct hola_ctx {
   // staging for hola_verify_host
   void* st_hidden; int* st_tok; void* st_q; float* st_u;
   int* st_accept; int* st_next; float* st_entropy; float* st_logZ;
-  int force_tile_n, force_stages;
+  int force_stages;
   // optional per-kernel timing (hola_profile_begin / hola_profile_end)
   cudaEvent_t* prof_ev;     // 3 events per recorded call: before the GEMM, after it, after accept/sample
   int prof_cap, prof_n, prof_on;
@@ -807,42 +918,41 @@ void set_error(hola_ctx* ctx, const char* what, cudaError_t e) {
   snprintf(ctx->last_error, sizeof ctx->last_error, "%s: %s", what, cudaGetErrorString(e));
 }
 
-// Chooses the vocab tile width and the split of row blocks into passes for M rows.
-// Cost model per pass, in SM cycles: rounds of tiles x max(tensor time, HBM time, L2 time of the hidden blocks).
+int round_up(int x, int a) { return (x + a - 1) / a * a; }
+
+// Splits M verify rows into passes over W_lm and each pass into one or two MMAs per K step.
+// A pass holds at most 512 rows (two MMAs of N <= 256 fill the tensor memory); N is a multiple of 16.
+// Cost per pass: the slower of streaming W_lm once and the padded rows' tensor time, plus a fixed launch cost.
 Plan make_plan(const hola_ctx* ctx, int M) {
   Plan best{};
   double best_cost = 1e300;
-  const int rb_total = M > 0 ? (M + kRows - 1) / kRows : 1;
-  const int nkb = (ctx->H + kBlockK - 1) / kBlockK;
-  for (int tn = 32; tn <= 256; tn += 32) {
-    if (ctx->force_tile_n && tn != ctx->force_tile_n) continue;
-    const int rb_max = kTmemCols / tn < kMaxRowBlocks ? kTmemCols / tn : kMaxRowBlocks;
-    const int passes = (rb_total + rb_max - 1) / rb_max;
-    const int rb = (rb_total + passes - 1) / passes;
-    const int stage_bytes = rb * kABlockBytes + tn * 128;
-    int stages = (kSmemBudget - 1024 - kBarrierBytes) / stage_bytes;
-    if (stages > kMaxStages) stages = kMaxStages;
-    if (ctx->force_stages && ctx->force_stages < stages) stages = ctx->force_stages;
-    if (stages < 2) continue;
-    const int n_tiles = (ctx->V + tn - 1) / tn;
-    const int grid = n_tiles < ctx->num_sms ? n_tiles : ctx->num_sms;
-    const int rounds = (n_tiles + grid - 1) / grid;
-    const double mma_instr = (tn / 2.0 > (kRows * 32 + tn * 32) / 128.0) ? tn / 2.0 : (kRows * 32 + tn * 32) / 128.0;
-    const double t_mma = rb * 4.0 * mma_instr * nkb;
-    const double t_hbm = tn * 128.0 * nkb / 26.0;        // ~26 B/clk/SM of HBM bandwidth
-    const double t_l2 = rb * kABlockBytes * static_cast<double>(nkb) / 64.0;
-    double t_tile = t_mma > t_hbm ? t_mma : t_hbm;
-    if (t_l2 > t_tile) t_tile = t_l2;
-    const int nbuf = (2 * rb * tn <= kTmemCols) ? 2 : 1;
-    const double t_epi = rb * tn * 12.0;                 // 4 warps, ~12 issue slots per logit per warp lane
-    const double cost = passes * (rounds * (t_tile + (nbuf == 1 ? t_epi : 0.0)) + 3000.0);
-    if (cost < best_cost * 0.999 || (cost <= best_cost * 1.001 && tn > best.tile_n)) {
-      if (cost < best_cost) best_cost = cost;
-      best.tile_n = tn; best.grid = grid; best.stages = stages; best.row_blocks = rb; best.passes = passes;
-      best.nbuf = nbuf; best.n_tiles = n_tiles; best.n_kblocks = nkb;
-      best.smem_bytes = stages * stage_bytes + kBarrierBytes + 1024;
+  const int rows = M > 0 ? M : 1;
+  const int p_min = (rows + kMaxRowsPerPass - 1) / kMaxRowsPerPass;
+  const double t_hbm = 2.0 * ctx->V * static_cast<double>(ctx->H) / 6.4e12;
+  for (int passes = p_min; passes <= p_min + 3; ++passes) {
+    const int r = (rows + passes - 1) / passes;
+    const int n_sub = r > kMaxN ? 2 : 1;
+    const int N = round_up((r + n_sub - 1) / n_sub, 16);
+    const double t_mma = 2.0 * n_sub * N * static_cast<double>(ctx->V) * ctx->H / 1.4e15;
+    const double cost = passes * ((t_mma > t_hbm ? t_mma : t_hbm) + 6e-6);
+    if (cost < best_cost) {
+      best_cost = cost;
+      best.n_sub = n_sub; best.N = N; best.rows_per_pass = n_sub * N; best.passes = passes;
     }
   }
+  // a pass may end up empty when rows_per_pass * (passes - 1) already covers M
+  best.passes = (rows + best.rows_per_pass - 1) / best.rows_per_pass;
+  const int stage_bytes = kWBlockBytes + best.n_sub * (best.N / 2) * 128;
+  int stages = (kSmemBudget - 1024 - kBarrierBytes) / stage_bytes;
+  if (stages > kMaxStages) stages = kMaxStages;
+  if (ctx->force_stages && ctx->force_stages < stages) stages = ctx->force_stages;
+  best.stages = stages;
+  best.nbuf = best.n_sub == 1 ? 2 : 1;
+  best.n_ptiles = (ctx->V + kPairTile - 1) / kPairTile;
+  const int pairs = ctx->num_sms / 2 > 0 ? ctx->num_sms / 2 : 1;
+  best.grid = 2 * (best.n_ptiles < pairs ? best.n_ptiles : pairs);
+  best.n_kblocks = (ctx->H + kBlockK - 1) / kBlockK;
+  best.smem_bytes = stages * stage_bytes + kBarrierBytes + 1024;
   return best;
 }
 
@@ -862,18 +972,6 @@ hola_status encode_map(hola_ctx* ctx, CUtensorMap* map, const void* ptr, uint64_
   return HOLA_OK;
 }
 
-template <int RB>
-hola_status launch_k1_rb(hola_ctx* ctx, const CUtensorMap& th, const CUtensorMap& tw, const K1Params& kp,
-                         const Plan& pl, cudaStream_t stream) {
-  cudaError_t e = cudaFuncSetAttribute(lm_head_entropy_kernel<RB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       pl.smem_bytes);
-  if (e != cudaSuccess) { set_error(ctx, "cudaFuncSetAttribute", e); return HOLA_ERR_CUDA; }
-  lm_head_entropy_kernel<RB><<<pl.grid, kK1Threads, pl.smem_bytes, stream>>>(th, tw, kp);
-  e = cudaGetLastError();
-  if (e != cudaSuccess) { set_error(ctx, "launch lm_head_entropy_kernel", e); return HOLA_ERR_CUDA; }
-  return HOLA_OK;
-}
-
 hola_status check_common(const hola_ctx* ctx, const hola_verify_args* a) {
   if (!ctx || !a) return HOLA_ERR_INVALID_ARG;
   if (a->B < 0 || a->k < 0 || a->H <= 0 || a->V <= 0) return HOLA_ERR_INVALID_ARG;
@@ -884,46 +982,43 @@ hola_status check_common(const hola_ctx* ctx, const hola_verify_args* a) {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-// Steps 1-2: the LM-head GEMM with fused statistics, one launch per pass over W_lm.
+// Steps 1-2: the LM-head GEMM with fused statistics, one launch (clusters of two CTAs) per pass over W_lm.
 hola_status run_lm_head(hola_ctx* ctx, const hola_verify_args* a, float* logits, int ldl, const Plan& pl,
                         cudaStream_t stream) {
   const int M = a->B * (a->k + 1);
   CUtensorMap th, tw;
-  hola_status s = encode_map(ctx, &th, a->hidden, static_cast<uint64_t>(M), static_cast<uint64_t>(a->H), kRows);
+  hola_status s = encode_map(ctx, &th, a->hidden, static_cast<uint64_t>(M), static_cast<uint64_t>(a->H),
+                             static_cast<uint32_t>(pl.N / 2));
   if (s != HOLA_OK) return s;
-  s = encode_map(ctx, &tw, a->W_lm, static_cast<uint64_t>(a->V), static_cast<uint64_t>(a->H),
-                 static_cast<uint32_t>(pl.tile_n));
+  s = encode_map(ctx, &tw, a->W_lm, static_cast<uint64_t>(a->V), static_cast<uint64_t>(a->H), kLanes);
   if (s != HOLA_OK) return s;
   K1Params kp;
-  kp.M = M; kp.V = a->V; kp.tile_n = pl.tile_n; kp.n_tiles = pl.n_tiles; kp.n_kblocks = pl.n_kblocks;
-  kp.stages = pl.stages; kp.nbuf = pl.nbuf; kp.ldl = ldl;
+  kp.M = M; kp.V = a->V; kp.n_ptiles = pl.n_ptiles; kp.n_kblocks = pl.n_kblocks;
+  kp.stages = pl.stages; kp.nbuf = pl.nbuf; kp.n_sub = pl.n_sub; kp.N = pl.N; kp.ldl = ldl;
   kp.vec_ok = (ldl % 4 == 0 && aligned16(logits)) ? 1 : 0;
   kp.logits = logits; kp.partials = ctx->partials; kp.part_stride = ctx->max_rows;
   kp.status = a->status_word ? a->status_word : ctx->status;
-  const int rb_total = (M + kRows - 1) / kRows;
-  for (int pass = 0, rb0 = 0; pass < pl.passes; ++pass) {
-    int rb = rb_total - rb0 < pl.row_blocks ? rb_total - rb0 : pl.row_blocks;
-    if (rb <= 0) break;
-    kp.row0 = rb0 * kRows;
-    // the kernel is compiled for 1..4 row blocks; a pass narrower than the plan still uses the plan's
-    // shared-memory stage size only if RB matches, so the plan is re-derived per width below
-    Plan p2 = pl;
-    if (rb != pl.row_blocks) {
-      const int stage_bytes = rb * kABlockBytes + pl.tile_n * 128;
-      int stages = (kSmemBudget - 1024 - kBarrierBytes) / stage_bytes;
-      if (stages > kMaxStages) stages = kMaxStages;
-      p2.stages = stages; p2.row_blocks = rb; p2.nbuf = (2 * rb * pl.tile_n <= kTmemCols) ? 2 : 1;
-      p2.smem_bytes = stages * stage_bytes + kBarrierBytes + 1024;
-      kp.stages = p2.stages; kp.nbuf = p2.nbuf;
-    }
-    switch (rb) {
-      case 1: s = launch_k1_rb<1>(ctx, th, tw, kp, p2, stream); break;
-      case 2: s = launch_k1_rb<2>(ctx, th, tw, kp, p2, stream); break;
-      case 3: s = launch_k1_rb<3>(ctx, th, tw, kp, p2, stream); break;
-      default: s = launch_k1_rb<4>(ctx, th, tw, kp, p2, stream); break;
-    }
-    if (s != HOLA_OK) return s;
-    rb0 += rb;
+  cudaError_t e = cudaFuncSetAttribute(lm_head_entropy_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       pl.smem_bytes);
+  if (e != cudaSuccess) { set_error(ctx, "cudaFuncSetAttribute", e); return HOLA_ERR_CUDA; }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(pl.grid));
+  cfg.blockDim = dim3(kK1Threads);
+  cfg.dynamicSmemBytes = static_cast<size_t>(pl.smem_bytes);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  for (int pass = 0; pass < pl.passes; ++pass) {
+    kp.row0 = pass * pl.rows_per_pass;
+    kp.rows = M - kp.row0 < pl.rows_per_pass ? M - kp.row0 : pl.rows_per_pass;
+    if (kp.rows <= 0) break;
+    e = cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel, th, tw, kp);
+    if (e != cudaSuccess) { set_error(ctx, "launch lm_head_entropy_kernel", e); return HOLA_ERR_CUDA; }
   }
   return HOLA_OK;
 }
@@ -1037,9 +1132,8 @@ hola_status hola_create(hola_ctx** out, int device, int maxB, int maxK, int H, i
   ctx->H = H; ctx->V = V; ctx->ldl = static_cast<int>(align_up(static_cast<size_t>(V), 4));
   ctx->max_rows = maxB * (maxK + 1);
   ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
-  if (const char* e = getenv("HOLA_PLAN")) {             // "tile_n,stages": tuning override for sweeps
-    int tn = 0, st = 0;
-    if (sscanf(e, "%d,%d", &tn, &st) >= 1 && tn >= 32 && tn <= 256 && tn % 32 == 0) ctx->force_tile_n = tn;
+  if (const char* e = getenv("HOLA_STAGES")) {           // tuning override for sweeps: fewer ring slots
+    const int st = atoi(e);
     if (st >= 2 && st <= kMaxStages) ctx->force_stages = st;
   }
   const WsLayout w = ws_layout(maxB, maxK, H, V, ctx->num_sms);
@@ -1074,7 +1168,7 @@ hola_status hola_plan(const hola_ctx* ctx, int B, int k, hola_plan_info* out) {
   if (!ctx || !out || B < 0 || k < 0) return HOLA_ERR_INVALID_ARG;
   if (B > ctx->maxB || k > ctx->maxK) return HOLA_ERR_UNSUPPORTED_SHAPE;
   const Plan pl = make_plan(ctx, B * (k + 1));
-  out->tile_n = pl.tile_n; out->grid = pl.grid; out->stages = pl.stages; out->row_blocks = pl.row_blocks;
+  out->tile_v = kPairTile; out->grid = pl.grid; out->stages = pl.stages; out->rows_per_pass = pl.rows_per_pass;
   out->passes = pl.passes; out->kernels_per_call = pl.passes + 1;
   return HOLA_OK;
 }
