@@ -35,7 +35,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of lm_head_entropy_kernel, from the ncu captures
 # summarised under profiles/ (None: not captured for that workload).
-NCU_TRAFFIC_BYTES = {"batched": 275003136}
+NCU_TRAFFIC_BYTES = {}
 
 
 def load_peaks():

@@ -117,6 +117,14 @@ __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
 }
 
+// True in exactly one lane of a converged warp.  Unlike a lane-id test, the compiler knows that a single thread
+// runs the guarded region, so TMA / tcgen05 operands can stay in uniform registers.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{\n .reg .pred P;\n elect.sync _|P, 0xffffffff;\n selp.u32 %0, 1, 0, P;\n}" : "=r"(pred));
+  return pred != 0;
+}
+
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
@@ -339,7 +347,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
   const uint32_t base = (raw + 1023u) & ~1023u;          // 128-byte swizzle wants 1024-byte aligned tiles
   uint8_t* smem = smem_raw + (base - raw);
 
-  const int warp = threadIdx.x >> 5;
+  const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0);   // same value in all lanes, and the compiler knows it
   const int lane = threadIdx.x & 31;
   const uint32_t rank = cluster_cta_rank();              // 0 = leader of the pair
   const int pair = blockIdx.x >> 1;
@@ -383,7 +391,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (one per CTA)
-    if (lane == 0) {
+    if (elect_one()) {
       const uint64_t pol_w = l2_policy_evict_first();    // W_lm is streamed once
       const uint64_t pol_h = l2_policy_evict_last();     // hidden is re-read for every tile
       const uint32_t leader_full = map_to_cta(full_bar, 0);
@@ -392,14 +400,15 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
       bool ok = true;
       for (int t = 0; t < my_tiles && ok; ++t) {
         const int v0 = (pair + t * npairs) * kPairTile + static_cast<int>(rank) * kLanes;
-        for (int kb = 0; kb < p.n_kblocks; ++kb) {
+        int kx = 0;                                      // K coordinate of the block, in elements
+        for (int kb = 0; kb < p.n_kblocks; ++kb, kx += kBlockK) {
           if (!mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
           const uint32_t sa = base + stage * stage_bytes;
           const uint32_t fb = leader_full + 8 * stage;
           mbar_expect_tx_cluster(fb, stage_bytes);
-          tma_load_2d(sa, &tmap_w, fb, kb * kBlockK, v0, pol_w);
+          tma_load_2d(sa, &tmap_w, fb, kx, v0, pol_w);
           for (int s = 0; s < p.n_sub; ++s)
-            tma_load_2d(sa + kWBlockBytes + s * hid_block_bytes, &tmap_hidden, fb, kb * kBlockK,
+            tma_load_2d(sa + kWBlockBytes + s * hid_block_bytes, &tmap_hidden, fb, kx,
                         p.row0 + s * p.N + static_cast<int>(rank) * half_n, pol_h);
           if (++stage == p.stages) { stage = 0; phase ^= 1u; }
         }
@@ -407,8 +416,10 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (leader CTA only)
-    if (lane == 0 && rank == 0) {
+    if (rank == 0 && elect_one()) {
       const uint32_t idesc = make_idesc_bf16_m256(static_cast<uint32_t>(p.N));
+      const uint64_t desc0 = make_kmajor_sw128_desc(base);
+      const bool two_mmas = p.n_sub == 2;
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
@@ -421,15 +432,24 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
         for (int kb = 0; kb < p.n_kblocks; ++kb) {
           if (!mbar_wait(full_bar + 8 * stage, phase, abort_flag, p.status)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t sa = base + stage * stage_bytes;
-          const uint64_t adesc = make_kmajor_sw128_desc(sa);
+          // descriptors of this slot: only the 14-bit address field changes (16-byte units)
+          const uint64_t adesc = desc0 + ((stage * stage_bytes) >> 4);
+          const uint64_t bdesc0 = adesc + (kWBlockBytes >> 4);
+          const uint32_t acc = kb != 0 ? 1u : 0u;
+          // 16 bf16 = 32 bytes further along K inside the swizzled row: +2 in 16-byte address units
+          if (two_mmas) {
+            const uint64_t bdesc1 = bdesc0 + (hid_block_bytes >> 4);
+            umma_bf16(d0, adesc, bdesc0, idesc, acc);
+            umma_bf16(d0 + 256, adesc, bdesc1, idesc, acc);
 #pragma unroll
-          for (int kk = 0; kk < kBlockK / 16; ++kk) {
-            // 16 bf16 = 32 bytes further along K inside the swizzled row: +2 in 16-byte address units
-            for (int s = 0; s < p.n_sub; ++s) {
-              const uint64_t bdesc = make_kmajor_sw128_desc(sa + kWBlockBytes + s * hid_block_bytes);
-              umma_bf16(d0 + s * 256, adesc + 2 * kk, bdesc + 2 * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
+            for (int kk = 1; kk < kBlockK / 16; ++kk) {
+              umma_bf16(d0, adesc + 2 * kk, bdesc0 + 2 * kk, idesc, 1u);
+              umma_bf16(d0 + 256, adesc + 2 * kk, bdesc1 + 2 * kk, idesc, 1u);
             }
+          } else {
+            umma_bf16(d0, adesc, bdesc0, idesc, acc);
+#pragma unroll
+            for (int kk = 1; kk < kBlockK / 16; ++kk) umma_bf16(d0, adesc + 2 * kk, bdesc0 + 2 * kk, idesc, 1u);
           }
           umma_commit_pair(empty_bar + 8 * stage);       // frees the slot in both CTAs once these MMAs have read it
           if (++stage == p.stages) { stage = 0; phase ^= 1u; }
@@ -551,6 +571,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
   }
 
   // ------------------------------------------------------------------ common tail
+  __syncwarp();                                          // warps 0 and 1 ran one lane apart from the others
   tc_fence_before();
   __syncthreads();
   cluster_sync_all();                                    // the peer no longer signals this CTA's barriers or tensor memory
