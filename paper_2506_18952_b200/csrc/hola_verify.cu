@@ -4,8 +4,8 @@
 // Kernels
 //   lm_head_entropy_kernel      persistent, warp-specialised weight-streaming GEMM run by pairs of CTAs (clusters of
 //       two).  The vocabulary lies on the 128 tensor-memory lanes of each CTA, the verify positions on the N
-//       dimension of the MMA:  D[v, r] = sum_h W_lm[v, h] * hidden[r, h].  A pair owns 256 vocabulary rows per
-//       tile; each CTA streams its 128 rows of W_lm and HALF of the hidden rows per K block with TMA, and one
+//       dimension of the MMA:  D[v, r] = sum_h W_lm[v, h] * hidden[r, h].  A pair owns up to 256 vocabulary rows
+//       per tile; each CTA streams its (up to 128) rows of W_lm and HALF of the hidden rows per K block with TMA, and one
 //       thread of the leader CTA issues tcgen05.mma.cta_group::2 (bf16 x bf16 -> fp32 in tensor memory) that reads
 //       both halves.  Drain warps copy finished accumulators to the fp32 logits buffer; statistics warps re-read
 //       that tile row-wise (it is still in L2) and keep, per verify position, the running softmax statistics
@@ -73,6 +73,7 @@ struct K1Params {
   int rows;       // rows of this pass (<= n_sub * N)
   int V, n_ptiles, n_kblocks, stages, nbuf;
   int n_sub, N;   // MMAs per K step and their N (verify rows each; multiple of 16)
+  int tile_rows;  // vocabulary rows per CTA per tile (<= 128, multiple of 4): balances the tiles over the pairs
   int ldl;        // row pitch of the logits buffer, in floats
   int vec_ok;     // 16-byte loads of the logits buffer allowed (pitch and base aligned)
   float* logits;
@@ -355,6 +356,8 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
   const int half_n = p.N >> 1;                           // hidden rows this CTA supplies per MMA
   const uint32_t hid_block_bytes = static_cast<uint32_t>(half_n) * 128u;
   const uint32_t stage_bytes = kWBlockBytes + p.n_sub * hid_block_bytes;
+  const uint32_t tx_bytes = static_cast<uint32_t>(p.tile_rows) * 128u + p.n_sub * hid_block_bytes;   // per CTA and slot
+  const int pair_rows = 2 * p.tile_rows;                 // vocabulary rows of a pair's tile
   const uint32_t bar_base = base + p.stages * stage_bytes;
   const uint32_t full_bar = bar_base, empty_bar = bar_base + 96, tfull_bar = bar_base + 192,
                  tempty_bar = bar_base + 208, lready_bar = bar_base + 224, sfree_bar = bar_base + 240;
@@ -399,13 +402,13 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
       uint32_t phase = 0;
       bool ok = true;
       for (int t = 0; t < my_tiles && ok; ++t) {
-        const int v0 = (pair + t * npairs) * kPairTile + static_cast<int>(rank) * kLanes;
+        const int v0 = (pair + t * npairs) * pair_rows + static_cast<int>(rank) * p.tile_rows;
         int kx = 0;                                      // K coordinate of the block, in elements
         for (int kb = 0; kb < p.n_kblocks; ++kb, kx += kBlockK) {
           if (!mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
           const uint32_t sa = base + stage * stage_bytes;
           const uint32_t fb = leader_full + 8 * stage;
-          mbar_expect_tx_cluster(fb, stage_bytes);
+          mbar_expect_tx_cluster(fb, tx_bytes);
           tma_load_2d(sa, &tmap_w, fb, kx, v0, pol_w);
           for (int s = 0; s < p.n_sub; ++s)
             tma_load_2d(sa + kWBlockBytes + s * hid_block_bytes, &tmap_hidden, fb, kx,
@@ -470,8 +473,9 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
       const int par = t & 1;
       if (!mbar_wait_warp(tfull_bar + 8 * buf, acc_phase, abort_flag, p.status)) { ok = false; break; }
       tc_fence_after();
-      const int vocab = (pair + t * npairs) * kPairTile + static_cast<int>(rank) * kLanes + quarter * 32 + lane;
-      const bool vocab_ok = vocab < p.V;
+      const int tile_lane = quarter * 32 + lane;         // lanes at or beyond tile_rows hold nothing
+      const int vocab = (pair + t * npairs) * pair_rows + static_cast<int>(rank) * p.tile_rows + tile_lane;
+      const bool vocab_ok = tile_lane < p.tile_rows && vocab < p.V;
       const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * 256;
       for (int ch = group; ch < n_chunks; ch += 2) {
         const int s = ch / sub_chunks, j = ch - s * sub_chunks;
@@ -518,8 +522,8 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
     for (int t = 0; t < my_tiles && ok; ++t) {
       const int par = t & 1;
       if (!mbar_wait_warp(lready_bar + 8 * par, static_cast<uint32_t>(t >> 1) & 1u, abort_flag, p.status)) { ok = false; break; }
-      const int vbase = (pair + t * npairs) * kPairTile + static_cast<int>(rank) * kLanes;
-      const int lim = p.V - vbase;                       // logits of this tile inside the vocabulary
+      const int vbase = (pair + t * npairs) * pair_rows + static_cast<int>(rank) * p.tile_rows;
+      const int lim = min(p.tile_rows, p.V - vbase);     // logits of this tile that exist
       if (lim > 0) {
 #pragma unroll
         for (int i = 0; i < kStatsRowsPerThread; ++i) {
@@ -527,24 +531,25 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
           if (r < p.rows) {
             const float* src = p.logits + static_cast<size_t>(p.row0 + r) * p.ldl + vbase;
             float v[32];
-            if (p.vec_ok && lim >= kLanes) {
+            int n = 0;                                   // this thread's columns ascend with the index: a prefix is valid
 #pragma unroll
-              for (int it = 0; it < 8; ++it) {
-                const float4 x = __ldcg(reinterpret_cast<const float4*>(src + 16 * it + 4 * part));
+            for (int it = 0; it < 8; ++it) {
+              const int col = 16 * it + 4 * part;
+              if (p.vec_ok && col + 4 <= lim) {
+                const float4 x = __ldcg(reinterpret_cast<const float4*>(src + col));
                 v[4 * it] = x.x; v[4 * it + 1] = x.y; v[4 * it + 2] = x.z; v[4 * it + 3] = x.w;
-              }
-              stats_fold<true>(v, 32, st[i]);
-            } else {
-              int n = 0;                                 // this thread's columns ascend with the index: a prefix is valid
+                n = 4 * it + 4;
+              } else {
 #pragma unroll
-              for (int idx = 0; idx < 32; ++idx) {
-                const int col = 16 * (idx >> 2) + 4 * part + (idx & 3);
-                const bool in = col < lim;
-                v[idx] = in ? __ldcg(src + col) : 0.f;
-                n += in ? 1 : 0;
+                for (int j = 0; j < 4; ++j) {
+                  const bool in = col + j < lim;
+                  v[4 * it + j] = in ? __ldcg(src + col + j) : 0.f;
+                  n += in ? 1 : 0;
+                }
               }
-              if (n > 0) stats_fold<false>(v, n, st[i]);
             }
+            if (n == 32) stats_fold<true>(v, 32, st[i]);
+            else if (n > 0) stats_fold<false>(v, n, st[i]);
           }
         }
       }
@@ -881,7 +886,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 struct Plan {
-  int n_sub, N, rows_per_pass, passes, grid, stages, nbuf, n_ptiles, n_kblocks, smem_bytes;
+  int n_sub, N, rows_per_pass, passes, grid, stages, nbuf, n_ptiles, n_kblocks, smem_bytes, tile_rows;
 };
 
 }  // namespace
@@ -969,8 +974,16 @@ Plan make_plan(const hola_ctx* ctx, int M) {
   if (ctx->force_stages && ctx->force_stages < stages) stages = ctx->force_stages;
   best.stages = stages;
   best.nbuf = best.n_sub == 1 ? 2 : 1;
-  best.n_ptiles = (ctx->V + kPairTile - 1) / kPairTile;
+  // Vocabulary rows per CTA per tile: the smallest multiple of 4 that covers V in the fewest whole rounds over
+  // all pairs, so that every pair streams the same number of bytes (V = 32000 on 74 pairs: 2 rounds of 112 + 112
+  // rows instead of 1.69 rounds of 128 + 128).
   const int pairs = ctx->num_sms / 2 > 0 ? ctx->num_sms / 2 : 1;
+  const int rounds = (ctx->V + pairs * kPairTile - 1) / (pairs * kPairTile);
+  int tile_rows = round_up((ctx->V + 2 * pairs * rounds - 1) / (2 * pairs * rounds), 4);
+  if (tile_rows < 8) tile_rows = 8;
+  if (tile_rows > kLanes) tile_rows = kLanes;
+  best.tile_rows = tile_rows;
+  best.n_ptiles = (ctx->V + 2 * tile_rows - 1) / (2 * tile_rows);
   best.grid = 2 * (best.n_ptiles < pairs ? best.n_ptiles : pairs);
   best.n_kblocks = (ctx->H + kBlockK - 1) / kBlockK;
   best.smem_bytes = stages * stage_bytes + kBarrierBytes + 1024;
@@ -1011,11 +1024,12 @@ hola_status run_lm_head(hola_ctx* ctx, const hola_verify_args* a, float* logits,
   hola_status s = encode_map(ctx, &th, a->hidden, static_cast<uint64_t>(M), static_cast<uint64_t>(a->H),
                              static_cast<uint32_t>(pl.N / 2));
   if (s != HOLA_OK) return s;
-  s = encode_map(ctx, &tw, a->W_lm, static_cast<uint64_t>(a->V), static_cast<uint64_t>(a->H), kLanes);
+  s = encode_map(ctx, &tw, a->W_lm, static_cast<uint64_t>(a->V), static_cast<uint64_t>(a->H),
+                 static_cast<uint32_t>(pl.tile_rows));
   if (s != HOLA_OK) return s;
   K1Params kp;
   kp.M = M; kp.V = a->V; kp.n_ptiles = pl.n_ptiles; kp.n_kblocks = pl.n_kblocks;
-  kp.stages = pl.stages; kp.nbuf = pl.nbuf; kp.n_sub = pl.n_sub; kp.N = pl.N; kp.ldl = ldl;
+  kp.stages = pl.stages; kp.nbuf = pl.nbuf; kp.n_sub = pl.n_sub; kp.N = pl.N; kp.tile_rows = pl.tile_rows; kp.ldl = ldl;
   kp.vec_ok = (ldl % 4 == 0 && aligned16(logits)) ? 1 : 0;
   kp.logits = logits; kp.partials = ctx->partials; kp.part_stride = ctx->max_rows;
   kp.status = a->status_word ? a->status_word : ctx->status;
@@ -1189,7 +1203,7 @@ hola_status hola_plan(const hola_ctx* ctx, int B, int k, hola_plan_info* out) {
   if (!ctx || !out || B < 0 || k < 0) return HOLA_ERR_INVALID_ARG;
   if (B > ctx->maxB || k > ctx->maxK) return HOLA_ERR_UNSUPPORTED_SHAPE;
   const Plan pl = make_plan(ctx, B * (k + 1));
-  out->tile_v = kPairTile; out->grid = pl.grid; out->stages = pl.stages; out->rows_per_pass = pl.rows_per_pass;
+  out->tile_v = 2 * pl.tile_rows; out->grid = pl.grid; out->stages = pl.stages; out->rows_per_pass = pl.rows_per_pass;
   out->passes = pl.passes; out->kernels_per_call = pl.passes + 1;
   return HOLA_OK;
 }
