@@ -33,9 +33,17 @@ METRIC = "verify_positions_per_s"
 UNIT = "positions/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of lm_head_entropy_kernel, from the ncu captures
-# summarised under profiles/ (None: not captured for that workload).
-NCU_TRAFFIC_BYTES = {}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of lm_head_entropy_kernel, from the ncu capture summarised
+# in profiles/lm_head_entropy_kernel__batched__ncu_full.md (workload "batched": B=64 k=5 H=4096 V=32000).  The
+# traffic is W_lm + hidden + logits write-back, all proportional to V at fixed B, k, H, so a workload with the same
+# B, k, H gets the captured figure scaled by V; any other workload reports null.
+NCU_TRAFFIC = {"shape": (64, 5, 4096), "V": 32000, "bytes": 265913856 + 11264256}
+
+
+def ncu_traffic_bytes(w):
+    if (w.B, w.k, w.H) != NCU_TRAFFIC["shape"]:
+        return None
+    return NCU_TRAFFIC["bytes"] * w.V / NCU_TRAFFIC["V"]
 
 
 def load_peaks():
@@ -291,7 +299,7 @@ def main():
             roof = {"bound": "hbm", "achieved": work["gemm_bytes"] / t_k1 / 1e9, "peak": peaks["hbm_gbs"],
                     "unit": "GB/s"}
         roof["frac"] = roof["achieved"] / roof["peak"]
-        roof["traffic"] = NCU_TRAFFIC_BYTES.get(w.name)
+        roof["traffic"] = ncu_traffic_bytes(w)
         roof.update({"kernel": "lm_head_entropy_kernel", "kernel_ms": k1_ms, "launches_per_step": plan["passes"],
                      "peak_source": f"of {peak_kind}", "hbm_gbs_achieved": work["gemm_bytes"] / t_k1 / 1e9,
                      "hbm_frac": work["gemm_bytes"] / t_k1 / 1e9 / peaks["hbm_gbs"],
