@@ -64,6 +64,10 @@ constexpr int kK3Warps = kK3Threads / 32;
 constexpr int kChunk = 128;                      // vocabulary entries per warp step (32 lanes x 4)
 constexpr int kMaxChunks = 4096;                 // => V <= 524288
 constexpr int kMaxK1 = 64;                       // k + 1 <= 64
+#ifndef K3_UNROLL
+#define K3_UNROLL 4
+#endif
+constexpr int kK3Unroll = K3_UNROLL;             // vocabulary chunks a warp has in flight per step
 
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -628,12 +632,14 @@ __device__ __forceinline__ double warp_sum_f64(double x) {
   return x;
 }
 
-// The four residual masses of vocabulary entries base..base+3 of one row.
-// residual = true:  r = max(0, p - q);  false: r = p.   Entries at or beyond V give 0.
+// Logits and draft probabilities of vocabulary entries base..base+3 of one row (q = 0 when the row is drawn
+// from p itself; entries at or beyond V get l = -inf, q = 0 and so no mass).  Loads only: a caller can issue
+// several of these before using any, which keeps more requests in flight.
 template <bool kVec>
-__device__ __forceinline__ void load_r4(const float* lrow, const void* qrow, int q_dtype, bool residual, int base,
-                                        int V, float logZ, float r[4]) {
-  float l[4], q[4] = {0.f, 0.f, 0.f, 0.f};
+__device__ __forceinline__ void fetch4(const float* lrow, const void* qrow, int q_dtype, bool residual, int base,
+                                       int V, float l[4], float q[4]) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) q[i] = 0.f;
   if (kVec && base + 3 < V) {
     const float4 l4 = *reinterpret_cast<const float4*>(lrow + base);
     l[0] = l4.x; l[1] = l4.y; l[2] = l4.z; l[3] = l4.w;
@@ -647,23 +653,33 @@ __device__ __forceinline__ void load_r4(const float* lrow, const void* qrow, int
         q[0] = q4.x; q[1] = q4.y; q[2] = q4.z; q[3] = q4.w;
       }
     }
-#pragma unroll
-    for (int i = 0; i < 4; ++i) r[i] = fmaxf(0.f, expf(l[i] - logZ) - q[i]);
   } else {
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const int v = base + i;
+      l[i] = -CUDART_INF_F;
       if (v < V) {
-        float qq = 0.f;
+        l[i] = lrow[v];
         if (residual)
-          qq = (q_dtype == HOLA_Q_BF16) ? __bfloat162float(static_cast<const __nv_bfloat16*>(qrow)[v])
-                                        : static_cast<const float*>(qrow)[v];
-        r[i] = fmaxf(0.f, expf(lrow[v] - logZ) - qq);
-      } else {
-        r[i] = 0.f;
+          q[i] = (q_dtype == HOLA_Q_BF16) ? __bfloat162float(static_cast<const __nv_bfloat16*>(qrow)[v])
+                                          : static_cast<const float*>(qrow)[v];
       }
     }
   }
+}
+
+// The four residual masses  r = max(0, p - q)  with  p = e^(l - logZ)  (q = 0: r = p).
+__device__ __forceinline__ void resid4(const float l[4], const float q[4], float logZ, float r[4]) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) r[i] = fmaxf(0.f, expf(l[i] - logZ) - q[i]);
+}
+
+template <bool kVec>
+__device__ __forceinline__ void load_r4(const float* lrow, const void* qrow, int q_dtype, bool residual, int base,
+                                        int V, float logZ, float r[4]) {
+  float l[4], q[4];
+  fetch4<kVec>(lrow, qrow, q_dtype, residual, base, V, l, q);
+  resid4(l, q, logZ, r);
 }
 
 __device__ __forceinline__ float clamp_uniform(float u, unsigned& flags) {
@@ -762,19 +778,20 @@ __global__ void __launch_bounds__(kK3Threads) accept_sample_kernel(const K3Param
   bool residual = n < k;
 
   for (int attempt = 0; attempt < 2; ++attempt) {
-    for (int c0 = warp; c0 < mine; c0 += 4 * kK3Warps) {
-      float r[4][4];
+    for (int c0 = warp; c0 < mine; c0 += kK3Unroll * kK3Warps) {
+      float l[kK3Unroll][4], q[kK3Unroll][4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
+      for (int i = 0; i < kK3Unroll; ++i) {              // all loads of this step first
         const int c = c0 + i * kK3Warps;
-        if (c < mine)
-          load_r4<kVec>(lrow, qrow, p.q_dtype, residual, (c_first + c) * kChunk + lane * 4, V, logZ, r[i]);
+        if (c < mine) fetch4<kVec>(lrow, qrow, p.q_dtype, residual, (c_first + c) * kChunk + lane * 4, V, l[i], q[i]);
       }
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
+      for (int i = 0; i < kK3Unroll; ++i) {
         const int c = c0 + i * kK3Warps;
         if (c < mine) {
-          const double sum = warp_sum_f64(((static_cast<double>(r[i][0]) + r[i][1]) + r[i][2]) + r[i][3]);
+          float r[4];
+          resid4(l[i], q[i], logZ, r);
+          const double sum = warp_sum_f64(((static_cast<double>(r[0]) + r[1]) + r[2]) + r[3]);
           if (lane == 0) csum[c] = sum;
         }
       }
