@@ -6,7 +6,9 @@ The comparison rule:
   * accept_len: equal, except where the oracle's own decision margin at a position that decided the outcome,
     |H - tau| or |u - min(1, p/q)|, is below 1e-4 - such cases are counted, not failed;
   * next_tok: compared only where accept_len agrees; equal, except where the supplied uniform lies within 1e-4
-    (in probability mass) of the oracle's CDF interval of the token under test - counted separately.
+    (in probability mass) of the oracle's CDF interval of the token under test - counted separately;
+  * greedy verifier: the accept decision's margin is the gap between the two largest logits of that row, and a
+    next_tok mismatch is a margin case only where that gap is below 1e-4.
 Nothing here is used by the product path.
 """
 from __future__ import annotations
@@ -31,11 +33,12 @@ def torch_to_numpy(t):
     return t.numpy()
 
 
-def run_oracle(w, keep_logits: bool = True, nthreads: int = 0) -> ref.RefResult:
+def run_oracle(w, keep_logits: bool = True, nthreads: int = 0, gate_source: int = 0,
+               fallback: int = 0) -> ref.RefResult:
     """Runs the oracle on a workload object with torch tensors hidden, W_lm, draft_tok, draft_q, uniforms, tau."""
     return ref.verify(torch_to_numpy(w.hidden), torch_to_numpy(w.W_lm), torch_to_numpy(w.draft_tok),
                       torch_to_numpy(w.draft_q), torch_to_numpy(w.uniforms), w.tau, keep_logits=keep_logits,
-                      nthreads=nthreads)
+                      nthreads=nthreads, gate_source=gate_source, fallback=fallback)
 
 
 @dataclass
@@ -102,7 +105,11 @@ def compare(oracle: ref.RefResult, q_np: np.ndarray, uniforms: np.ndarray, accep
             rep.token_exact += 1
             continue
         ok = False
-        if oracle.logits is not None and 0 <= t_got < oracle.logits.shape[2]:
+        if oracle.fallback == ref.FALLBACK_GREEDY:
+            # greedy verifier: the two sides may differ only where the top two logits of that row nearly tie
+            ok = 0 <= t_got < (oracle.logits.shape[2] if oracle.logits is not None else 1 << 30) and \
+                oracle.margin_argmax[b, n_ref] < MARGIN
+        elif oracle.logits is not None and 0 <= t_got < oracle.logits.shape[2]:
             p = np.exp(oracle.logits[b, n_ref] - oracle.logZ[b, n_ref])
             r = np.maximum(0.0, p - _q_row_f64(q_np, b, n_ref)) if n_ref < k else p
             R = r.sum()

@@ -25,6 +25,14 @@
 //      If R <= 0 then r = p_n.  next_tok = smallest v whose running sum c(v) = sum_{w<=v} r(w) exceeds u_k * R.
 //   6. decision margins, so that a comparison can tell a near-tie from an error.
 //
+// Two variants of steps 4-5, selected by arguments (defaults reproduce the steps above):
+//   gate_source = 1: the gate looks at the entropy of the DRAFT distribution, H^q_j = -sum_v q_j(v) ln q_j(v), which
+//      is what the HSD section literally says ("uncertainty in the draft distribution"); q is used as given, terms
+//      with q = 0 contribute 0, the result is clamped at >= 0.  The target entropy is still computed and returned.
+//   fallback = 1: the verifier decides greedily (Eq. 1 read as "take the verifier's own token"): at a position
+//      where the gate is off the draft token is kept iff it equals argmax_v p_j(v) (lowest token id on ties);
+//      the token that follows the accepted run is argmax p_n.  No uniform is consumed.
+//
 // Parity pins live in tests/test_oracle_pins.py (closed forms, invariants, exact-integer products, brute-force
 // marginals on 8- and 16-token vocabularies).  The choice of verifier rule itself (step 4/5) has no counterpart
 // in the authors' code to compare with: "parity unpinned" for that choice, pinned for its arithmetic.
@@ -83,9 +91,11 @@ void softmax_entropy_row(const double* l, int V, double* logZ_out, double* H_out
 // Steps 2-6 for one sequence, given its (k+1) rows of fp64 logits.
 void verify_one_sequence(int k, int V, const double* logits /*[k+1][V]*/, const int32_t* tok /*[k]*/,
                          const void* q /*[k][V]*/, int q_dtype, const float* u /*[k+1]*/, double tau,
+                         int gate_source, int fallback,
                          int32_t* accept_len, int32_t* next_tok, double* entropy /*[k+1]*/,
                          double* logZ /*[k+1]*/, double* margin_accept /*[k] or null*/,
                          double* margin_gate /*[k] or null*/, double* margin_cdf /*[1] or null*/,
+                         double* draft_entropy /*[k] or null*/, double* margin_argmax /*[k+1] or null*/,
                          uint32_t* flags) {
   for (int j = 0; j <= k; ++j)
     softmax_entropy_row(logits + static_cast<size_t>(j) * V, V, &logZ[j], &entropy[j]);
@@ -94,7 +104,39 @@ void verify_one_sequence(int k, int V, const double* logits /*[k+1][V]*/, const 
     if (margin_gate) margin_gate[j] = kInf;
   }
 
-  // Step 4: gate, then ratio test, in draft order.
+  // Entropy of each draft row (gate_source = 1), by the definition, term by term.
+  std::vector<double> Hq(static_cast<size_t>(k), 0.0);
+  if (gate_source == 1 || draft_entropy) {
+    for (int j = 0; j < k; ++j) {
+      double h = 0.0;
+      for (int v = 0; v < V; ++v) {
+        const double qv = load_as_double(q, q_dtype, static_cast<size_t>(j) * V + v);
+        if (qv > 0.0) h -= qv * std::log(qv);
+      }
+      if (h < 0.0) h = 0.0;
+      Hq[j] = h;
+      if (draft_entropy) draft_entropy[j] = h;
+    }
+  }
+
+  // Greedy verifier (fallback = 1): the verifier's own token at every position, lowest id on ties, and the gap
+  // to the runner-up as the decision margin.
+  std::vector<int32_t> amax(static_cast<size_t>(k) + 1, 0);
+  std::vector<double> gap(static_cast<size_t>(k) + 1, kInf);
+  if (fallback == 1) {
+    for (int j = 0; j <= k; ++j) {
+      const double* lj = logits + static_cast<size_t>(j) * V;
+      int best = 0;
+      for (int v = 1; v < V; ++v) if (lj[v] > lj[best]) best = v;
+      double second = -kInf;
+      for (int v = 0; v < V; ++v) if (v != best && lj[v] > second) second = lj[v];
+      amax[j] = best;
+      gap[j] = lj[best] - second;
+      if (margin_argmax) margin_argmax[j] = gap[j];
+    }
+  }
+
+  // Step 4: gate, then the verifier's test, in draft order.
   int n = k;
   for (int j = 0; j < k; ++j) {
     const int32_t x = tok[j];
@@ -103,8 +145,14 @@ void verify_one_sequence(int k, int V, const double* logits /*[k+1][V]*/, const 
       n = j;
       break;
     }
-    if (margin_gate) margin_gate[j] = std::fabs(entropy[j] - tau);
-    if (entropy[j] < tau) continue;                       // fast path: gate fired
+    const double gate_value = gate_source == 1 ? Hq[j] : entropy[j];
+    if (margin_gate) margin_gate[j] = std::fabs(gate_value - tau);
+    if (gate_value < tau) continue;                       // fast path: gate fired
+    if (fallback == 1) {
+      if (margin_accept) margin_accept[j] = gap[j];
+      if (x != amax[j]) { n = j; break; }
+      continue;
+    }
     double uj = static_cast<double>(u[j]);
     if (!(uj >= 0.0)) { uj = 0.0; *flags |= 2u; }
     if (uj >= 1.0) { uj = static_cast<double>(std::nextafter(1.0f, 0.0f)); *flags |= 2u; }
@@ -117,6 +165,11 @@ void verify_one_sequence(int k, int V, const double* logits /*[k+1][V]*/, const 
     if (!(uj < ratio)) { n = j; break; }
   }
   *accept_len = n;
+  if (fallback == 1) {              // greedy: the verifier's own token follows the accepted run
+    *next_tok = amax[n];
+    if (margin_cdf) *margin_cdf = kInf;
+    return;
+  }
 
   // Step 5: residual (or the verifier's own distribution at the bonus position) and inverse-CDF draw.
   const double* ln = logits + static_cast<size_t>(n) * V;
@@ -198,46 +251,74 @@ int hola_ref_softmax_entropy(int M, int V, const double* logits64, double* logZ,
 
 // Steps 2-6 from given fp64 logits [B][k+1][V].  q is [B][k][V] in q_dtype.  Margin pointers may be null.
 // flags_out (optional, [B]): bit0 bad token, bit1 uniform outside [0,1), bit3 residual mass was zero.
-int hola_verify_from_logits_ref(int B, int k, int V, const double* logits64, const int32_t* draft_tok,
-                                const void* draft_q, int q_dtype, const float* uniforms, double tau,
-                                int32_t* accept_len, int32_t* next_tok, double* entropy, double* logZ,
-                                double* margin_accept, double* margin_gate, double* margin_cdf,
-                                uint32_t* flags_out) {
+// gate_source / fallback select the variants described at the top; draft_entropy ([B][k]) and margin_argmax
+// ([B][k+1]) are optional outputs.
+int hola_verify_from_logits_ref_ex(int B, int k, int V, const double* logits64, const int32_t* draft_tok,
+                                   const void* draft_q, int q_dtype, const float* uniforms, double tau,
+                                   int gate_source, int fallback,
+                                   int32_t* accept_len, int32_t* next_tok, double* entropy, double* logZ,
+                                   double* margin_accept, double* margin_gate, double* margin_cdf,
+                                   double* draft_entropy, double* margin_argmax, uint32_t* flags_out) {
   if (B < 0 || k < 0 || V <= 0 || !logits64 || !uniforms || !accept_len || !next_tok || !entropy || !logZ)
     return 1;
   if (k > 0 && (!draft_tok || !draft_q)) return 1;
+  if (gate_source < 0 || gate_source > 1 || fallback < 0 || fallback > 1) return 1;
   const size_t qElem = (q_dtype == REF_BF16) ? 2 : (q_dtype == REF_F32 ? 4 : 8);
   for (int b = 0; b < B; ++b) {
     uint32_t flags = 0;
     const char* qb = static_cast<const char*>(draft_q) + static_cast<size_t>(b) * k * V * qElem;
     verify_one_sequence(k, V, logits64 + static_cast<size_t>(b) * (k + 1) * V,
                         draft_tok ? draft_tok + static_cast<size_t>(b) * k : nullptr, qb, q_dtype,
-                        uniforms + static_cast<size_t>(b) * (k + 1), tau, &accept_len[b], &next_tok[b],
-                        entropy + static_cast<size_t>(b) * (k + 1), logZ + static_cast<size_t>(b) * (k + 1),
+                        uniforms + static_cast<size_t>(b) * (k + 1), tau, gate_source, fallback, &accept_len[b],
+                        &next_tok[b], entropy + static_cast<size_t>(b) * (k + 1),
+                        logZ + static_cast<size_t>(b) * (k + 1),
                         margin_accept ? margin_accept + static_cast<size_t>(b) * k : nullptr,
                         margin_gate ? margin_gate + static_cast<size_t>(b) * k : nullptr,
-                        margin_cdf ? margin_cdf + b : nullptr, &flags);
+                        margin_cdf ? margin_cdf + b : nullptr,
+                        draft_entropy ? draft_entropy + static_cast<size_t>(b) * k : nullptr,
+                        margin_argmax ? margin_argmax + static_cast<size_t>(b) * (k + 1) : nullptr, &flags);
     if (flags_out) flags_out[b] = flags;
   }
   return 0;
 }
 
+int hola_verify_from_logits_ref(int B, int k, int V, const double* logits64, const int32_t* draft_tok,
+                                const void* draft_q, int q_dtype, const float* uniforms, double tau,
+                                int32_t* accept_len, int32_t* next_tok, double* entropy, double* logZ,
+                                double* margin_accept, double* margin_gate, double* margin_cdf,
+                                uint32_t* flags_out) {
+  return hola_verify_from_logits_ref_ex(B, k, V, logits64, draft_tok, draft_q, q_dtype, uniforms, tau, 0, 0,
+                                        accept_len, next_tok, entropy, logZ, margin_accept, margin_gate,
+                                        margin_cdf, nullptr, nullptr, flags_out);
+}
+
 // The whole verify step.  hidden [B][k+1][H] and W [V][H] in in_dtype; logits64 is optional output/scratch
 // ([B][k+1][V]; allocated internally when null).
-int hola_verify_ref(int B, int k, int H, int V, const void* hidden, const void* W, int in_dtype,
-                    const int32_t* draft_tok, const void* draft_q, int q_dtype, const float* uniforms,
-                    double tau, int32_t* accept_len, int32_t* next_tok, double* entropy, double* logZ,
-                    double* margin_accept, double* margin_gate, double* margin_cdf, double* logits64,
-                    uint32_t* flags_out, int nthreads) {
+int hola_verify_ref_ex(int B, int k, int H, int V, const void* hidden, const void* W, int in_dtype,
+                       const int32_t* draft_tok, const void* draft_q, int q_dtype, const float* uniforms,
+                       double tau, int gate_source, int fallback, int32_t* accept_len, int32_t* next_tok,
+                       double* entropy, double* logZ, double* margin_accept, double* margin_gate,
+                       double* margin_cdf, double* draft_entropy, double* margin_argmax, double* logits64,
+                       uint32_t* flags_out, int nthreads) {
   if (B < 0 || k < 0 || H <= 0 || V <= 0) return 1;
   const size_t M = static_cast<size_t>(B) * (k + 1);
   std::vector<double> own;
   if (!logits64) { own.resize(M * V); logits64 = own.data(); }
   int rc = hola_ref_logits(static_cast<int>(M), H, V, hidden, W, in_dtype, logits64, nthreads);
   if (rc) return rc;
-  return hola_verify_from_logits_ref(B, k, V, logits64, draft_tok, draft_q, q_dtype, uniforms, tau,
-                                     accept_len, next_tok, entropy, logZ, margin_accept, margin_gate,
-                                     margin_cdf, flags_out);
+  return hola_verify_from_logits_ref_ex(B, k, V, logits64, draft_tok, draft_q, q_dtype, uniforms, tau, gate_source,
+                                        fallback, accept_len, next_tok, entropy, logZ, margin_accept, margin_gate,
+                                        margin_cdf, draft_entropy, margin_argmax, flags_out);
+}
+
+int hola_verify_ref(int B, int k, int H, int V, const void* hidden, const void* W, int in_dtype,
+                    const int32_t* draft_tok, const void* draft_q, int q_dtype, const float* uniforms,
+                    double tau, int32_t* accept_len, int32_t* next_tok, double* entropy, double* logZ,
+                    double* margin_accept, double* margin_gate, double* margin_cdf, double* logits64,
+                    uint32_t* flags_out, int nthreads) {
+  return hola_verify_ref_ex(B, k, H, V, hidden, W, in_dtype, draft_tok, draft_q, q_dtype, uniforms, tau, 0, 0,
+                            accept_len, next_tok, entropy, logZ, margin_accept, margin_gate, margin_cdf, nullptr,
+                            nullptr, logits64, flags_out, nthreads);
 }
 
 int hola_ref_max_threads(void) {

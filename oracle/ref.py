@@ -81,6 +81,10 @@ class RefResult:
     margin_cdf: np.ndarray      # float64 [B]
     flags: np.ndarray           # uint32 [B]
     logits: np.ndarray | None   # float64 [B, k+1, V]
+    draft_entropy: np.ndarray | None = None    # float64 [B, k]: entropy of each draft row
+    margin_argmax: np.ndarray | None = None    # float64 [B, k+1]: top-1 minus top-2 logit (greedy verifier only)
+    gate_source: int = 0        # 0: entropy of the target distribution gates; 1: entropy of the draft distribution
+    fallback: int = 0           # 0: speculative-sampling test and residual draw; 1: greedy verifier
 
 
 def logits(hidden: np.ndarray, W: np.ndarray, nthreads: int = 0) -> np.ndarray:
@@ -110,15 +114,20 @@ def softmax_entropy(logits64: np.ndarray):
     return logZ, H
 
 
+GATE_TARGET, GATE_DRAFT = 0, 1
+FALLBACK_SAMPLE, FALLBACK_GREEDY = 0, 1
+
+
 def _outputs(B, k):
     return dict(
         accept_len=np.empty(B, dtype=np.int32), next_tok=np.empty(B, dtype=np.int32),
         entropy=np.empty((B, k + 1)), logZ=np.empty((B, k + 1)),
         margin_accept=np.empty((B, k)), margin_gate=np.empty((B, k)), margin_cdf=np.empty(B),
-        flags=np.zeros(B, dtype=np.uint32))
+        flags=np.zeros(B, dtype=np.uint32), draft_entropy=np.zeros((B, k)), margin_argmax=np.full((B, k + 1), np.inf))
 
 
-def verify_from_logits(logits64, draft_tok, draft_q, uniforms, tau) -> RefResult:
+def verify_from_logits(logits64, draft_tok, draft_q, uniforms, tau, gate_source: int = 0,
+                       fallback: int = 0) -> RefResult:
     """Steps 2-6 from fp64 logits [B, k+1, V]; draft_q [B, k, V] (uint16 bf16 bits, float32 or float64)."""
     logits64 = np.ascontiguousarray(logits64, dtype=np.float64)
     B, k1, V = logits64.shape
@@ -127,17 +136,18 @@ def verify_from_logits(logits64, draft_tok, draft_q, uniforms, tau) -> RefResult
     draft_q = np.ascontiguousarray(draft_q).reshape(B, k, V)
     uniforms = np.ascontiguousarray(uniforms, dtype=np.float32).reshape(B, k + 1)
     o = _outputs(B, k)
-    rc = lib().hola_verify_from_logits_ref(
+    rc = lib().hola_verify_from_logits_ref_ex(
         B, k, V, _ptr(logits64), _ptr(draft_tok), _ptr(draft_q), _dtype_code(draft_q), _ptr(uniforms),
-        ctypes.c_double(float(tau)), _ptr(o["accept_len"]), _ptr(o["next_tok"]), _ptr(o["entropy"]),
-        _ptr(o["logZ"]), _ptr(o["margin_accept"]), _ptr(o["margin_gate"]), _ptr(o["margin_cdf"]),
-        _ptr(o["flags"]))
+        ctypes.c_double(float(tau)), int(gate_source), int(fallback), _ptr(o["accept_len"]), _ptr(o["next_tok"]),
+        _ptr(o["entropy"]), _ptr(o["logZ"]), _ptr(o["margin_accept"]), _ptr(o["margin_gate"]), _ptr(o["margin_cdf"]),
+        _ptr(o["draft_entropy"]), _ptr(o["margin_argmax"]), _ptr(o["flags"]))
     if rc:
-        raise ValueError("hola_verify_from_logits_ref rejected its arguments")
-    return RefResult(logits=logits64, **o)
+        raise ValueError("hola_verify_from_logits_ref_ex rejected its arguments")
+    return RefResult(logits=logits64, gate_source=int(gate_source), fallback=int(fallback), **o)
 
 
-def verify(hidden, W, draft_tok, draft_q, uniforms, tau, keep_logits: bool = False, nthreads: int = 0) -> RefResult:
+def verify(hidden, W, draft_tok, draft_q, uniforms, tau, keep_logits: bool = False, nthreads: int = 0,
+           gate_source: int = 0, fallback: int = 0) -> RefResult:
     """The whole verify step.  hidden [B, k+1, H] and W [V, H] share a dtype (uint16 bf16 bits / f32 / f64)."""
     hidden = np.ascontiguousarray(hidden)
     W = np.ascontiguousarray(W)
@@ -151,11 +161,12 @@ def verify(hidden, W, draft_tok, draft_q, uniforms, tau, keep_logits: bool = Fal
     uniforms = np.ascontiguousarray(uniforms, dtype=np.float32).reshape(B, k + 1)
     o = _outputs(B, k)
     lg = np.empty((B, k + 1, V)) if keep_logits else None
-    rc = lib().hola_verify_ref(
+    rc = lib().hola_verify_ref_ex(
         B, k, H, V, _ptr(hidden), _ptr(W), code, _ptr(draft_tok), _ptr(draft_q), _dtype_code(draft_q),
-        _ptr(uniforms), ctypes.c_double(float(tau)), _ptr(o["accept_len"]), _ptr(o["next_tok"]),
-        _ptr(o["entropy"]), _ptr(o["logZ"]), _ptr(o["margin_accept"]), _ptr(o["margin_gate"]),
-        _ptr(o["margin_cdf"]), _ptr(lg), _ptr(o["flags"]), nthreads)
+        _ptr(uniforms), ctypes.c_double(float(tau)), int(gate_source), int(fallback), _ptr(o["accept_len"]),
+        _ptr(o["next_tok"]), _ptr(o["entropy"]), _ptr(o["logZ"]), _ptr(o["margin_accept"]), _ptr(o["margin_gate"]),
+        _ptr(o["margin_cdf"]), _ptr(o["draft_entropy"]), _ptr(o["margin_argmax"]), _ptr(lg), _ptr(o["flags"]),
+        nthreads)
     if rc:
-        raise ValueError("hola_verify_ref rejected its arguments")
-    return RefResult(logits=lg, **o)
+        raise ValueError("hola_verify_ref_ex rejected its arguments")
+    return RefResult(logits=lg, gate_source=int(gate_source), fallback=int(fallback), **o)

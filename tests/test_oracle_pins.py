@@ -428,3 +428,93 @@ def test_full_entry_matches_from_logits_composition_on_bf16_inputs():
     part = ref.verify_from_logits(full.logits, tok, ref.bf16_bits_to_f64(qb), u, 1.5)
     assert np.array_equal(full.accept_len, part.accept_len) and np.array_equal(full.next_tok, part.next_tok)
     assert np.array_equal(full.entropy, part.entropy)
+
+
+# ------------------------------------------------------------------ variants: draft-entropy gate, greedy verifier
+def test_draft_entropy_matches_scipy_and_closed_forms():
+    # H(q) = -sum q ln q: library routine on random rows, ln V on a uniform row, 0 on a one-hot row, and the
+    # two-level closed form; bf16-stored rows are used as stored (no renormalisation).
+    rng = np.random.default_rng(500)
+    V, k = 37, 4
+    q = rng.dirichlet(np.ones(V) * 0.3, size=k)
+    q[1] = 1.0 / V
+    q[2] = 0.0; q[2, 5] = 1.0
+    q[3] = 0.25 / (V - 1); q[3, 9] = 0.75
+    l = rng.normal(size=(1, k + 1, V))
+    got = ref.verify_from_logits(l, [[0] * k], q[None], np.full((1, k + 1), 0.5, np.float32), 0.0,
+                                 gate_source=ref.GATE_DRAFT)
+    want = [scipy.stats.entropy(q[0]), math.log(V), 0.0, -0.75 * math.log(0.75) - 0.25 * math.log(0.25 / (V - 1))]
+    np.testing.assert_allclose(got.draft_entropy[0], want, rtol=0, atol=1e-12)
+    qb = ref.f32_to_bf16_bits(q.astype(np.float32))
+    got_b = ref.verify_from_logits(l, [[0] * k], qb[None], np.full((1, k + 1), 0.5, np.float32), 0.0,
+                                   gate_source=ref.GATE_DRAFT)
+    qs = ref.bf16_bits_to_f64(qb)
+    want_b = [-(r[r > 0] * np.log(r[r > 0])).sum() for r in qs]      # sum q != 1 after rounding: not scipy's normalised form
+    np.testing.assert_allclose(got_b.draft_entropy[0], want_b, rtol=0, atol=1e-12)
+
+
+def test_draft_entropy_gate_uses_q_not_p():
+    # a peaked draft row under a flat target: gated only when the gate looks at the draft, and vice versa
+    V = 16
+    flat = np.zeros(V)
+    peaked = np.zeros(V); peaked[3] = 12.0
+    q_peaked = np.exp(peaked) / np.exp(peaked).sum()
+    q_flat = np.full(V, 1.0 / V)
+    u = np.array([[0.999999, 0.5]], np.float32)
+    x = 7                                                   # p(7)/q(7) is tiny under the peaked draft: ratio test rejects
+    # target flat (H = ln 16 = 2.77), draft peaked (H ~ 0.001), tau = 1.5
+    a = ref.verify_from_logits(np.stack([flat, flat])[None], [[3]], q_peaked[None, None], u, 1.5)
+    b = ref.verify_from_logits(np.stack([flat, flat])[None], [[3]], q_peaked[None, None], u, 1.5, gate_source=ref.GATE_DRAFT)
+    assert a.accept_len[0] == 0 and b.accept_len[0] == 1   # p(3)/q(3) = (1/16)/0.9999 < u: only the draft gate accepts
+    assert abs(b.margin_gate[0, 0] - abs(b.draft_entropy[0, 0] - 1.5)) < 1e-12
+    # target peaked (H ~ 0), draft flat: only the target gate accepts the (wrong) draft token
+    c = ref.verify_from_logits(np.stack([peaked, flat])[None], [[x]], q_flat[None, None], u, 1.5)
+    d = ref.verify_from_logits(np.stack([peaked, flat])[None], [[x]], q_flat[None, None], u, 1.5, gate_source=ref.GATE_DRAFT)
+    assert c.accept_len[0] == 1 and d.accept_len[0] == 0
+    # the target entropy that is returned does not depend on which one gates
+    np.testing.assert_array_equal(c.entropy, d.entropy)
+
+
+def test_greedy_verifier_is_numpy_argmax():
+    # gate off: a draft token survives iff it is the verifier's argmax; the next token is the argmax of the first
+    # row that broke (or of row k).  Checked against numpy.argmax on random fp64 logits, ties included.
+    rng = np.random.default_rng(501)
+    B, k, V = 40, 4, 23
+    l = rng.normal(size=(B, k + 1, V)).round(1)            # rounding makes exact ties appear
+    am = l.argmax(-1)                                       # numpy: first maximal index = lowest token id
+    tok = am[:, :k].copy()
+    wrong = rng.random((B, k)) < 0.3
+    tok[wrong] = (tok[wrong] + 1 + rng.integers(0, V - 1, wrong.sum())) % V
+    q = rng.dirichlet(np.ones(V), size=(B, k))
+    u = rng.random((B, k + 1)).astype(np.float32)
+    got = ref.verify_from_logits(l, tok, q, u, 0.0, fallback=ref.FALLBACK_GREEDY)
+    for b in range(B):
+        n = next((j for j in range(k) if tok[b, j] != am[b, j]), k)
+        assert got.accept_len[b] == n and got.next_tok[b] == am[b, n]
+    assert 0 < got.accept_len.mean() < k
+    top2 = np.sort(l, -1)[..., -2:]
+    np.testing.assert_allclose(got.margin_argmax, top2[..., 1] - top2[..., 0], atol=1e-12)
+    # uniforms play no part
+    got2 = ref.verify_from_logits(l, tok, q, 1.0 - u, 0.0, fallback=ref.FALLBACK_GREEDY)
+    assert np.array_equal(got.accept_len, got2.accept_len) and np.array_equal(got.next_tok, got2.next_tok)
+
+
+def test_greedy_verifier_with_gate_keeps_gated_drafts():
+    # tau = +inf gates everything: all k drafts kept whatever they are, next token = argmax p_k
+    rng = np.random.default_rng(502)
+    l = rng.normal(size=(3, 3, 11))
+    tok = rng.integers(0, 11, (3, 2))
+    q = rng.dirichlet(np.ones(11), size=(3, 2))
+    got = ref.verify_from_logits(l, tok, q, np.zeros((3, 3), np.float32), INF, fallback=ref.FALLBACK_GREEDY)
+    assert np.all(got.accept_len == 2) and np.array_equal(got.next_tok, l[:, 2].argmax(-1))
+    # both variants together through the full entry point on bf16 inputs: same answers as the composition
+    H, V, k = 24, 50, 3
+    hid = ref.f32_to_bf16_bits(rng.normal(size=(2, k + 1, H)).astype(np.float32))
+    W = ref.f32_to_bf16_bits((rng.normal(size=(V, H)) * 0.3).astype(np.float32))
+    q = rng.dirichlet(np.ones(V) * 0.2, size=(2, k)).astype(np.float32)
+    tok = rng.integers(0, V, (2, k))
+    u = rng.random((2, k + 1)).astype(np.float32)
+    full = ref.verify(hid, W, tok, q, u, 2.0, keep_logits=True, gate_source=ref.GATE_DRAFT, fallback=ref.FALLBACK_GREEDY)
+    comp = ref.verify_from_logits(full.logits, tok, q, u, 2.0, gate_source=ref.GATE_DRAFT, fallback=ref.FALLBACK_GREEDY)
+    assert np.array_equal(full.accept_len, comp.accept_len) and np.array_equal(full.next_tok, comp.next_tok)
+    np.testing.assert_array_equal(full.draft_entropy, comp.draft_entropy)
