@@ -187,6 +187,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default="large_vocab", choices=sorted(workloads.CONFIG_SHAPES))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--gate", default="target", choices=["target", "draft"],
+                    help="which entropy feeds the gate: the verifier's softmax (default) or the draft row")
+    ap.add_argument("--fallback", default="sample", choices=["sample", "greedy"],
+                    help="what the gate-off branch does: speculative-sampling test (default) or greedy verifier")
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--cpu-budget-s", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -214,10 +218,14 @@ def main():
     if w.V * w.H * 2 <= 200e6:
         flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
 
+    gate_source = 1 if args.gate == "draft" else 0
+    fallback = 1 if args.fallback == "greedy" else 0
+
     def step():
         if flush is not None:
             flush.zero_()
-        ctx.hola_verify(w.hidden, w.W_lm, w.draft_tok, w.draft_q, w.uniforms, w.tau, out=out)
+        ctx.hola_verify(w.hidden, w.W_lm, w.draft_tok, w.draft_q, w.uniforms, w.tau, out=out,
+                        gate_source=gate_source, fallback=fallback)
 
     sampler = ClockSampler(local)
     sampler.start()
@@ -268,7 +276,7 @@ def main():
 
     def e2e_step():
         ctx.hola_verify_host(host["hidden"], w.W_lm, host["draft_tok"], host["draft_q"], host["uniforms"], w.tau,
-                             out=hout)
+                             out=hout, gate_source=gate_source, fallback=fallback)
 
     for _ in range(3):
         e2e_step()
@@ -309,10 +317,11 @@ def main():
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms_max / args.steps, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-                "config": config_block(w, {"plan": plan, "parallelism": f"replicas x{world}"}),
+                "config": config_block(w, {"plan": plan, "parallelism": f"replicas x{world}", "gate": args.gate,
+                                           "fallback": args.fallback}),
                 "clocks": clocks,
                 "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-                "gpu_launches": plan["kernels_per_call"] * args.steps,
+                "gpu_launches": (plan["kernels_per_call"] + (1 if gate_source and w.k > 0 else 0)) * args.steps,
                 "accepted_tokens_per_s": accepted_all * args.steps / (ms_max * 1e-3),
                 "roofline": roof}
         if world == 1 and not args.no_cpu_baseline:

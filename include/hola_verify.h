@@ -41,6 +41,19 @@ typedef enum {
 
 typedef enum { HOLA_Q_BF16 = 0, HOLA_Q_F32 = 1 } hola_q_dtype;
 
+/* Which distribution's entropy feeds the gate g(t) = 1[H < tau].  The HSD section calls H "uncertainty in the draft
+ * distribution" but writes it with the verifier's symbol p; both readings are available. */
+typedef enum {
+  HOLA_GATE_TARGET_ENTROPY = 0, /* H of the verifier's softmax at the position (default) */
+  HOLA_GATE_DRAFT_ENTROPY = 1   /* H(q_j) = -sum_v q_j(v) ln q_j(v) of the draft row, q used as given */
+} hola_gate_source;
+
+/* What the "otherwise" branch of Eq. (1), y_t = f_ver(...), does where the gate is off. */
+typedef enum {
+  HOLA_FALLBACK_SAMPLE = 0,     /* speculative-sampling test u q(x) < p(x), residual draw at the first rejection (default) */
+  HOLA_FALLBACK_GREEDY = 1      /* greedy verifier: keep x iff x = argmax_v p(v) (lowest id on ties); next_tok = argmax p_n */
+} hola_fallback;
+
 /* Bits of the device status word (OR-ed by the kernels; the caller clears it). */
 #define HOLA_FLAG_BAD_TOKEN 1u   /* a draft token outside [0,V): treated as a rejection at that position    */
 #define HOLA_FLAG_BAD_UNIFORM 2u /* a uniform outside [0,1): clamped into [0, 1 - 2^-24]                     */
@@ -65,6 +78,9 @@ typedef struct {
   float* logZ;             /* out fp32 [B][k+1], log-sum-exp of the logits                                     */
   float* logits_out;       /* out fp32 [B][k+1][V], optional (NULL: the context's own scratch is used)         */
   uint32_t* status_word;   /* in/out uint32 [1], optional: HOLA_FLAG_* bits are OR-ed in                       */
+  int32_t gate_source;     /* hola_gate_source; 0 (zero-initialised struct) = target entropy                   */
+  int32_t fallback;        /* hola_fallback; 0 = speculative sampling.  With GREEDY the uniforms are not read  */
+  float* draft_entropy;    /* out fp32 [B][k], optional: H(q_j), written when gate_source = DRAFT_ENTROPY       */
 } hola_verify_args;
 
 /* Creates a context on `device` able to serve calls with B <= maxB, k <= maxK and exactly this H and V.
@@ -90,7 +106,8 @@ hola_status hola_verify_host(hola_ctx* ctx, const hola_verify_args* args, void* 
 /* Partial entry points, the steps of the path exposed one by one (same argument struct).
  * hola_lm_head_entropy: steps 1-2 only; fills logits (logits_out or scratch), entropy, logZ.
  * hola_accept_sample:   steps 3-5 only, from fp32 logits in args->logits_out (required) and the entropy / logZ
- *                       arrays already present in args->entropy / args->logZ (inputs here). */
+ *                       arrays already present in args->entropy / args->logZ (inputs here).  The greedy fallback
+ *                       needs the arg-max found by step 2 and is only available through hola_verify. */
 hola_status hola_lm_head_entropy(hola_ctx* ctx, const hola_verify_args* args, void* cuda_stream);
 hola_status hola_accept_sample(hola_ctx* ctx, const hola_verify_args* args, void* cuda_stream);
 

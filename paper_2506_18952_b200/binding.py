@@ -15,6 +15,8 @@ from . import build as _build
 
 HOLA_OK = 0
 HOLA_Q_BF16, HOLA_Q_F32 = 0, 1
+HOLA_GATE_TARGET_ENTROPY, HOLA_GATE_DRAFT_ENTROPY = 0, 1
+HOLA_FALLBACK_SAMPLE, HOLA_FALLBACK_GREEDY = 0, 1
 FLAG_BAD_TOKEN, FLAG_BAD_UNIFORM, FLAG_TIMEOUT, FLAG_R_ZERO = 1, 2, 4, 8
 
 EXPORTS = ["hola_create", "hola_destroy", "hola_workspace_bytes", "hola_verify", "hola_verify_host",
@@ -32,7 +34,8 @@ class hola_verify_args(ctypes.Structure):
                 ("draft_q", ctypes.c_void_p), ("q_dtype", ctypes.c_int32), ("uniforms", ctypes.c_void_p),
                 ("tau", ctypes.c_float), ("accept_len", ctypes.c_void_p), ("next_tok", ctypes.c_void_p),
                 ("entropy", ctypes.c_void_p), ("logZ", ctypes.c_void_p), ("logits_out", ctypes.c_void_p),
-                ("status_word", ctypes.c_void_p)]
+                ("status_word", ctypes.c_void_p), ("gate_source", ctypes.c_int32), ("fallback", ctypes.c_int32),
+                ("draft_entropy", ctypes.c_void_p)]
 
 
 class hola_plan_info(ctypes.Structure):
@@ -123,6 +126,7 @@ class VerifyOutputs:
     logZ: torch.Tensor         # fp32 [B, k+1]
     logits: torch.Tensor | None
     status: torch.Tensor       # uint32 as int32 [1]
+    draft_entropy: torch.Tensor | None = None   # fp32 [B, k], filled when the gate looks at the draft rows
 
 
 class HolaVerify:
@@ -170,7 +174,8 @@ class HolaVerify:
         _check(self.lib, self._ctx, st, "hola_profile_end")
         return {"lm_head_ms": a.value, "accept_sample_ms": b.value, "calls": n.value}
 
-    def _args(self, hidden, W_lm, draft_tok, draft_q, uniforms, tau, out: VerifyOutputs, B, k):
+    def _args(self, hidden, W_lm, draft_tok, draft_q, uniforms, tau, out: VerifyOutputs, B, k,
+              gate_source: int = HOLA_GATE_TARGET_ENTROPY, fallback: int = HOLA_FALLBACK_SAMPLE):
         if hidden.dtype != torch.bfloat16 or W_lm.dtype != torch.bfloat16:
             raise HolaError("hidden and W_lm must be bfloat16")
         if draft_q is not None and draft_q.dtype not in (torch.bfloat16, torch.float32):
@@ -190,6 +195,8 @@ class HolaVerify:
         a.entropy, a.logZ = _dptr(out.entropy), _dptr(out.logZ)
         a.logits_out = _dptr(out.logits)
         a.status_word = _dptr(out.status)
+        a.gate_source, a.fallback = int(gate_source), int(fallback)
+        a.draft_entropy = _dptr(out.draft_entropy)
         return a
 
     def alloc_outputs(self, B: int, k: int, want_logits: bool = False, device=None) -> VerifyOutputs:
@@ -200,14 +207,16 @@ class HolaVerify:
             entropy=torch.empty((B, k + 1), dtype=torch.float32, device=dev),
             logZ=torch.empty((B, k + 1), dtype=torch.float32, device=dev),
             logits=torch.empty((B, k + 1, self.V), dtype=torch.float32, device=dev) if want_logits else None,
-            status=torch.zeros(1, dtype=torch.int32, device=dev))
+            status=torch.zeros(1, dtype=torch.int32, device=dev),
+            draft_entropy=torch.zeros((B, k), dtype=torch.float32, device=dev))
 
     def hola_verify(self, hidden, W_lm, draft_tok, draft_q, uniforms, tau, out: VerifyOutputs | None = None,
-                    want_logits: bool = False, stream=None) -> VerifyOutputs:
+                    want_logits: bool = False, stream=None, gate_source: int = HOLA_GATE_TARGET_ENTROPY,
+                    fallback: int = HOLA_FALLBACK_SAMPLE) -> VerifyOutputs:
         """The whole verify step on device tensors, asynchronous on the stream."""
         B, k = hidden.shape[0], hidden.shape[1] - 1
         out = out or self.alloc_outputs(B, k, want_logits)
-        a = self._args(hidden, W_lm, draft_tok, draft_q, uniforms, tau, out, B, k)
+        a = self._args(hidden, W_lm, draft_tok, draft_q, uniforms, tau, out, B, k, gate_source, fallback)
         _check(self.lib, self._ctx, self.lib.hola_verify(self._ctx, ctypes.byref(a), _stream_ptr(stream)), "hola_verify")
         return out
 
@@ -240,7 +249,8 @@ class HolaVerify:
         return out
 
     def hola_verify_host(self, hidden, W_lm, draft_tok, draft_q, uniforms, tau, out: VerifyOutputs | None = None,
-                         stream=None) -> VerifyOutputs:
+                         stream=None, gate_source: int = HOLA_GATE_TARGET_ENTROPY,
+                         fallback: int = HOLA_FALLBACK_SAMPLE) -> VerifyOutputs:
         """End-to-end form: per-step inputs and all outputs are HOST tensors (pinned for async copies);
         W_lm is the resident device weight.  Returns after the stream has been synchronised."""
         B, k = hidden.shape[0], hidden.shape[1] - 1
@@ -250,7 +260,7 @@ class HolaVerify:
             if t is not None and t.device.type != "cpu":
                 raise HolaError("hola_verify_host takes host tensors for the per-step inputs")
         out = out or self.alloc_outputs(B, k, False, device=torch.device("cpu"))
-        a = self._args(hidden, W_lm, draft_tok, draft_q, uniforms, tau, out, B, k)
+        a = self._args(hidden, W_lm, draft_tok, draft_q, uniforms, tau, out, B, k, gate_source, fallback)
         a.logits_out = None
         _check(self.lib, self._ctx, self.lib.hola_verify_host(self._ctx, ctypes.byref(a), _stream_ptr(stream)),
                "hola_verify_host")

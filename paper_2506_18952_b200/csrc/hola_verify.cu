@@ -96,6 +96,9 @@ struct K3Params {
   int q_dtype;
   const float* u;
   float tau;
+  int gate_source;          // hola_gate_source
+  int fallback;             // hola_fallback
+  const float* draft_entropy;   // [B][k], read when gate_source == HOLA_GATE_DRAFT_ENTROPY
   int* accept_len;
   int* next_tok;
   float* entropy;
@@ -287,8 +290,9 @@ __device__ __forceinline__ uint32_t make_idesc_bf16_m256(uint32_t n) {
 // logZ = m + ln s;  H = -sum p ln p = ln s - t/s.
 struct Stats {
   float m, s, t;
+  int arg;        // vocabulary index of the maximum (lowest index among equals): the greedy verifier's token
 };
-__device__ __forceinline__ Stats stats_empty() { return Stats{-CUDART_INF_F, 0.f, 0.f}; }
+__device__ __forceinline__ Stats stats_empty() { return Stats{-CUDART_INF_F, 0.f, 0.f, 0x7fffffff}; }
 
 __device__ __forceinline__ Stats stats_merge(Stats a, Stats b) {
   if (b.m == -CUDART_INF_F) return a;
@@ -300,12 +304,14 @@ __device__ __forceinline__ Stats stats_merge(Stats a, Stats b) {
   r.m = m;
   r.s = ea * a.s + eb * b.s;
   r.t = ea * (a.t + da * a.s) + eb * (b.t + db * b.s);
+  r.arg = a.m > b.m ? a.arg : (b.m > a.m ? b.arg : min(a.arg, b.arg));
   return r;
 }
 
-// Fold `n` (1..32) logits into the running statistics.
+// Fold `n` (1..32) logits into the running statistics.  Element i is vocabulary entry
+// vocab0 + 16 * (i / 4) + (i % 4): the statistics threads' interleaved share of a row (ascending in i).
 template <bool kFull>
-__device__ __forceinline__ void stats_fold(const float* v, int n, Stats& st) {
+__device__ __forceinline__ void stats_fold(const float* v, int n, int vocab0, Stats& st) {
   float cmax = v[0];
 #pragma unroll
   for (int i = 1; i < 32; ++i)
@@ -318,6 +324,12 @@ __device__ __forceinline__ void stats_fold(const float* v, int n, Stats& st) {
       st.s *= sc;
     }
     st.m = cmax;
+    int first = 0;
+#pragma unroll
+    for (int i = 31; i > 0; --i)
+      if ((kFull || i < n) && v[i] == cmax) first = i;
+    if (v[0] == cmax) first = 0;
+    st.arg = vocab0 + 16 * (first >> 2) + (first & 3);
   }
   const float m = st.m;
   const float mneg2 = -m * kLog2e;
@@ -552,8 +564,8 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
                 }
               }
             }
-            if (n == 32) stats_fold<true>(v, 32, st[i]);
-            else if (n > 0) stats_fold<false>(v, n, st[i]);
+            if (n == 32) stats_fold<true>(v, 32, vbase + 4 * part, st[i]);
+            else if (n > 0) stats_fold<false>(v, n, vbase + 4 * part, st[i]);
           }
         }
       }
@@ -570,11 +582,13 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
           o.m = __shfl_xor_sync(0xffffffffu, a.m, off);
           o.s = __shfl_xor_sync(0xffffffffu, a.s, off);
           o.t = __shfl_xor_sync(0xffffffffu, a.t, off);
+          o.arg = __shfl_xor_sync(0xffffffffu, a.arg, off);
           a = ((lane & off) == 0) ? stats_merge(a, o) : stats_merge(o, a);
         }
         const int r = rsub + (kStatsThreads / 4) * i;
         if (part == 0 && r < p.rows)
-          p.partials[static_cast<size_t>(blockIdx.x) * p.part_stride + p.row0 + r] = make_float4(a.m, a.s, a.t, 0.f);
+          p.partials[static_cast<size_t>(blockIdx.x) * p.part_stride + p.row0 + r] =
+              make_float4(a.m, a.s, a.t, __int_as_float(a.arg));
       }
     }
   }
@@ -596,7 +610,7 @@ __device__ __forceinline__ Stats warp_merge_partials(const float4* partials, int
   Stats st = stats_empty();
   for (int i = lane; i < nparts; i += 32) {
     const float4 x = partials[static_cast<size_t>(i) * part_stride + row];
-    st = stats_merge(st, Stats{x.x, x.y, x.z});
+    st = stats_merge(st, Stats{x.x, x.y, x.z, __float_as_int(x.w)});
   }
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) {
@@ -604,6 +618,7 @@ __device__ __forceinline__ Stats warp_merge_partials(const float4* partials, int
     o.m = __shfl_xor_sync(0xffffffffu, st.m, off);
     o.s = __shfl_xor_sync(0xffffffffu, st.s, off);
     o.t = __shfl_xor_sync(0xffffffffu, st.t, off);
+    o.arg = __shfl_xor_sync(0xffffffffu, st.arg, off);
     // merge in a fixed (lower lane first) order so that every lane holds bit-identical results
     st = ((lane & off) == 0) ? stats_merge(st, o) : stats_merge(o, st);
   }
@@ -696,8 +711,8 @@ template <bool kVec>
 __global__ void __launch_bounds__(kK3Threads) accept_sample_kernel(const K3Params p) {
   extern __shared__ double csum[];                       // per-chunk residual mass of this CTA's slice
   __shared__ double sh_tot[2][8];                        // slice totals of the whole cluster, per attempt
-  __shared__ float sh_logZ[kMaxK1], sh_H[kMaxK1], sh_lx[kMaxK1], sh_qx[kMaxK1], sh_u[kMaxK1];
-  __shared__ int sh_x[kMaxK1];
+  __shared__ float sh_logZ[kMaxK1], sh_H[kMaxK1], sh_lx[kMaxK1], sh_qx[kMaxK1], sh_u[kMaxK1], sh_Hq[kMaxK1];
+  __shared__ int sh_x[kMaxK1], sh_amax[kMaxK1];
   __shared__ int sh_n;
   __shared__ unsigned sh_flags;
 
@@ -722,6 +737,7 @@ __global__ void __launch_bounds__(kK3Threads) accept_sample_kernel(const K3Param
                                       : static_cast<const float*>(p.q)[qi];
     }
     sh_lx[j] = lx; sh_qx[j] = qx;
+    sh_Hq[j] = p.gate_source == HOLA_GATE_DRAFT_ENTROPY ? p.draft_entropy[b * k + j] : 0.f;
   }
   // ---- softmax statistics of this sequence's k+1 positions
   if (p.combine) {
@@ -730,7 +746,7 @@ __global__ void __launch_bounds__(kK3Threads) accept_sample_kernel(const K3Param
       if (lane == 0) {
         float lz, h;
         stats_to_outputs(st, &lz, &h);
-        sh_logZ[j] = lz; sh_H[j] = h;
+        sh_logZ[j] = lz; sh_H[j] = h; sh_amax[j] = st.arg;
         if (rank == 0) { p.logZ[row_first + j] = lz; p.entropy[row_first + j] = h; }
       }
     }
@@ -749,7 +765,12 @@ __global__ void __launch_bounds__(kK3Threads) accept_sample_kernel(const K3Param
     for (int j = 0; j < k; ++j) {
       const int x = sh_x[j];
       if (x < 0 || x >= V) { flags |= HOLA_FLAG_BAD_TOKEN; n = j; break; }
-      if (sh_H[j] < p.tau) continue;                     // entropy gate: fast path keeps the draft token
+      const float gate_value = p.gate_source == HOLA_GATE_DRAFT_ENTROPY ? sh_Hq[j] : sh_H[j];
+      if (gate_value < p.tau) continue;                  // entropy gate: fast path keeps the draft token
+      if (p.fallback == HOLA_FALLBACK_GREEDY) {          // the verifier's own token, or the run ends here
+        if (x != sh_amax[j]) { n = j; break; }
+        continue;
+      }
       const float u = clamp_uniform(sh_u[j], flags);
       const float px = expf(sh_lx[j] - sh_logZ[j]);
       const float qx = sh_qx[j];
@@ -758,9 +779,16 @@ __global__ void __launch_bounds__(kK3Threads) accept_sample_kernel(const K3Param
     }
     sh_n = n;
     sh_flags = flags;
-    if (rank == 0) p.accept_len[b] = n;
+    if (rank == 0) {
+      p.accept_len[b] = n;
+      if (p.fallback == HOLA_FALLBACK_GREEDY) {          // greedy: argmax p_n follows the accepted run; no draw
+        p.next_tok[b] = min(max(sh_amax[n], 0), V - 1);
+        if (flags && p.status) atomicOr(p.status, flags);
+      }
+    }
   }
   __syncthreads();
+  if (p.fallback == HOLA_FALLBACK_GREEDY) return;        // same decision in every CTA of the cluster
 
   // ---- this CTA's slice of row n: per-chunk residual mass
   const int n = sh_n;
@@ -897,6 +925,61 @@ __global__ void __launch_bounds__(kK3Threads) accept_sample_kernel(const K3Param
   }
 }
 
+// ------------------------------------------------------------------------------------------------ draft entropy
+// H(q) = -sum_v q ln q of each draft row (one CTA per row): the gate value when the gate looks at the draft
+// distribution, as the HSD section words it.  q is used as stored; entries with q <= 0 contribute nothing.
+__global__ void __launch_bounds__(256) draft_entropy_kernel(const void* q, int q_dtype, int V, float* out) {
+  __shared__ double sh_part[8];
+  const size_t row = blockIdx.x;
+  double acc = 0.0;
+  if (q_dtype == HOLA_Q_BF16) {
+    const __nv_bfloat16* qr = static_cast<const __nv_bfloat16*>(q) + row * V;
+    const bool vec = (reinterpret_cast<uintptr_t>(qr) & 15u) == 0;
+    const int nvec = vec ? V / 8 : 0;
+    for (int i = threadIdx.x; i < nvec; i += 256) {
+      const uint4 raw = reinterpret_cast<const uint4*>(qr)[i];
+      const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+      float part = 0.f;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float a = __uint_as_float(w[j] << 16), c = __uint_as_float(w[j] & 0xFFFF0000u);
+        if (a > 0.f) part = fmaf(a, logf(a), part);
+        if (c > 0.f) part = fmaf(c, logf(c), part);
+      }
+      acc += part;
+    }
+    for (int v = nvec * 8 + threadIdx.x; v < V; v += 256) {
+      const float a = __bfloat162float(qr[v]);
+      if (a > 0.f) acc += a * logf(a);
+    }
+  } else {
+    const float* qr = static_cast<const float*>(q) + row * V;
+    const bool vec = (reinterpret_cast<uintptr_t>(qr) & 15u) == 0;
+    const int nvec = vec ? V / 4 : 0;
+    for (int i = threadIdx.x; i < nvec; i += 256) {
+      const float4 x = reinterpret_cast<const float4*>(qr)[i];
+      const float e[4] = {x.x, x.y, x.z, x.w};
+      float part = 0.f;
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if (e[j] > 0.f) part = fmaf(e[j], logf(e[j]), part);
+      acc += part;
+    }
+    for (int v = nvec * 4 + threadIdx.x; v < V; v += 256) {
+      const float a = qr[v];
+      if (a > 0.f) acc += a * logf(a);
+    }
+  }
+  acc = warp_sum_f64(acc);
+  if ((threadIdx.x & 31) == 0) sh_part[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double tot = 0.0;
+    for (int i = 0; i < 8; ++i) tot += sh_part[i];
+    out[row] = fmaxf(0.f, static_cast<float>(-tot));
+  }
+}
+
 // ------------------------------------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -916,6 +999,7 @@ struct hola_ctx {
   float* logits;            // [max_rows][ldl]
   float4* partials;         // [num_sms][max_rows]
   unsigned* status;         // [1]
+  float* hq;                // [max_rows] draft-row entropies when the caller does not ask for them
   // staging for hola_verify_host
   void* st_hidden; int* st_tok; void* st_q; float* st_u;
   int* st_accept; int* st_next; float* st_entropy; float* st_logZ;
@@ -931,7 +1015,7 @@ namespace {
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WsLayout {
-  size_t logits, partials, status, st_hidden, st_tok, st_q, st_u, st_accept, st_next, st_entropy, st_logZ, total;
+  size_t logits, partials, status, hq, st_hidden, st_tok, st_q, st_u, st_accept, st_next, st_entropy, st_logZ, total;
 };
 
 WsLayout ws_layout(int maxB, int maxK, int H, int V, int num_sms) {
@@ -943,6 +1027,7 @@ WsLayout ws_layout(int maxB, int maxK, int H, int V, int num_sms) {
   w.logits = take(rows * ldl * 4);
   w.partials = take(static_cast<size_t>(num_sms) * rows * 16);
   w.status = take(4);
+  w.hq = take(rows * 4);
   w.st_hidden = take(rows * H * 2);
   w.st_tok = take(static_cast<size_t>(maxB) * maxK * 4);
   w.st_q = take(static_cast<size_t>(maxB) * maxK * V * 4);
@@ -1028,6 +1113,9 @@ hola_status check_common(const hola_ctx* ctx, const hola_verify_args* a) {
   if (a->B < 0 || a->k < 0 || a->H <= 0 || a->V <= 0) return HOLA_ERR_INVALID_ARG;
   if (a->H != ctx->H || a->V != ctx->V || a->B > ctx->maxB || a->k > ctx->maxK) return HOLA_ERR_UNSUPPORTED_SHAPE;
   if (a->q_dtype != HOLA_Q_BF16 && a->q_dtype != HOLA_Q_F32) return HOLA_ERR_INVALID_ARG;
+  if (a->gate_source != HOLA_GATE_TARGET_ENTROPY && a->gate_source != HOLA_GATE_DRAFT_ENTROPY)
+    return HOLA_ERR_INVALID_ARG;
+  if (a->fallback != HOLA_FALLBACK_SAMPLE && a->fallback != HOLA_FALLBACK_GREEDY) return HOLA_ERR_INVALID_ARG;
   return HOLA_OK;
 }
 
@@ -1081,6 +1169,15 @@ hola_status run_accept_sample(hola_ctx* ctx, const hola_verify_args* a, const fl
   kp.B = a->B; kp.k = a->k; kp.V = a->V; kp.ldl = ldl; kp.logits = logits;
   kp.partials = ctx->partials; kp.nparts = nparts; kp.part_stride = ctx->max_rows; kp.combine = combine;
   kp.tok = a->draft_tok; kp.q = a->draft_q; kp.q_dtype = a->q_dtype; kp.u = a->uniforms; kp.tau = a->tau;
+  kp.gate_source = a->gate_source; kp.fallback = a->fallback; kp.draft_entropy = nullptr;
+  if (a->gate_source == HOLA_GATE_DRAFT_ENTROPY && a->k > 0) {
+    // one more pass over the draft rows: H(q_j) for every (sequence, draft position)
+    float* hq = a->draft_entropy ? a->draft_entropy : ctx->hq;
+    draft_entropy_kernel<<<a->B * a->k, 256, 0, stream>>>(a->draft_q, a->q_dtype, a->V, hq);
+    const cudaError_t e0 = cudaGetLastError();
+    if (e0 != cudaSuccess) { set_error(ctx, "launch draft_entropy_kernel", e0); return HOLA_ERR_CUDA; }
+    kp.draft_entropy = hq;
+  }
   kp.accept_len = a->accept_len; kp.next_tok = a->next_tok; kp.entropy = a->entropy; kp.logZ = a->logZ;
   kp.status = a->status_word ? a->status_word : ctx->status;
   const bool vec = (a->V % 4 == 0) && (ldl % 4 == 0) && aligned16(logits) && (a->k == 0 || aligned16(a->draft_q));
@@ -1195,6 +1292,7 @@ hola_status hola_create(hola_ctx** out, int device, int maxB, int maxK, int H, i
   ctx->logits = reinterpret_cast<float*>(ctx->ws + w.logits);
   ctx->partials = reinterpret_cast<float4*>(ctx->ws + w.partials);
   ctx->status = reinterpret_cast<unsigned*>(ctx->ws + w.status);
+  ctx->hq = reinterpret_cast<float*>(ctx->ws + w.hq);
   ctx->st_hidden = ctx->ws + w.st_hidden; ctx->st_tok = reinterpret_cast<int*>(ctx->ws + w.st_tok);
   ctx->st_q = ctx->ws + w.st_q; ctx->st_u = reinterpret_cast<float*>(ctx->ws + w.st_u);
   ctx->st_accept = reinterpret_cast<int*>(ctx->ws + w.st_accept);
@@ -1250,6 +1348,7 @@ hola_status hola_accept_sample(hola_ctx* ctx, const hola_verify_args* a, void* c
   if (a->B == 0) return HOLA_OK;
   if ((s = check_sample_args(a)) != HOLA_OK) return s;
   if (!a->logits_out) return HOLA_ERR_INVALID_ARG;
+  if (a->fallback == HOLA_FALLBACK_GREEDY) return HOLA_ERR_INVALID_ARG;   // needs the arg-max of the fused path
   DeviceGuard guard(ctx->device);
   return run_accept_sample(ctx, a, a->logits_out, a->V, 0, 0, static_cast<cudaStream_t>(cuda_stream));
 }
@@ -1340,13 +1439,15 @@ hola_status hola_verify_host(hola_ctx* ctx, const hola_verify_args* a, void* cud
   hola_verify_args d = *a;
   d.hidden = ctx->st_hidden; d.draft_tok = ctx->st_tok; d.draft_q = ctx->st_q; d.uniforms = ctx->st_u;
   d.accept_len = ctx->st_accept; d.next_tok = ctx->st_next; d.entropy = ctx->st_entropy; d.logZ = ctx->st_logZ;
-  d.logits_out = nullptr; d.status_word = ctx->status;
+  d.logits_out = nullptr; d.status_word = ctx->status; d.draft_entropy = nullptr;
   if ((s = hola_verify(ctx, &d, cuda_stream)) != HOLA_OK) return s;
   d2h(a->accept_len, ctx->st_accept, static_cast<size_t>(a->B) * 4);
   d2h(a->next_tok, ctx->st_next, static_cast<size_t>(a->B) * 4);
   d2h(a->entropy, ctx->st_entropy, rows * 4);
   d2h(a->logZ, ctx->st_logZ, rows * 4);
   if (a->status_word) d2h(a->status_word, ctx->status, 4);
+  if (a->draft_entropy && a->gate_source == HOLA_GATE_DRAFT_ENTROPY)
+    d2h(a->draft_entropy, ctx->hq, static_cast<size_t>(a->B) * a->k * 4);
   if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
   if (e != cudaSuccess) { set_error(ctx, "device-to-host copy", e); return HOLA_ERR_CUDA; }
   return HOLA_OK;

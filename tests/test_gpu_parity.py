@@ -24,12 +24,12 @@ def _np(t):
     return compare.torch_to_numpy(t)
 
 
-def run_gpu(binding, w, want_logits=False, tau=None, ctx=None):
+def run_gpu(binding, w, want_logits=False, tau=None, ctx=None, gate_source=0, fallback=0):
     own = ctx is None
     ctx = ctx or binding.HolaVerify(max(w.B, 1), w.k, w.H, w.V)
     try:
         out = ctx.hola_verify(w.hidden, w.W_lm, w.draft_tok, w.draft_q, w.uniforms, w.tau if tau is None else tau,
-                              want_logits=want_logits)
+                              want_logits=want_logits, gate_source=gate_source, fallback=fallback)
         torch.cuda.synchronize()
     finally:
         if own:
@@ -37,16 +37,18 @@ def run_gpu(binding, w, want_logits=False, tau=None, ctx=None):
     return out
 
 
-def check_against_oracle(binding, w, seqs=None, want_logits=True, tau=None, out=None):
+def check_against_oracle(binding, w, seqs=None, want_logits=True, tau=None, out=None, gate_source=0, fallback=0):
     """Runs the GPU path on the whole workload and the oracle on `seqs` (all sequences when None)."""
     tau = w.tau if tau is None else tau
-    out = out or run_gpu(binding, w, want_logits=want_logits, tau=tau)
+    out = out or run_gpu(binding, w, want_logits=want_logits, tau=tau, gate_source=gate_source, fallback=fallback)
     status = int(out.status.item())
     assert status & binding.FLAG_TIMEOUT == 0, "a device-side wait timed out"
     sub = w if seqs is None else w.slice(seqs)
     idx = np.arange(w.B) if seqs is None else np.asarray(list(seqs))
     sub.tau = tau
-    orc = compare.run_oracle(sub, keep_logits=True)
+    orc = compare.run_oracle(sub, keep_logits=True, gate_source=gate_source, fallback=fallback)
+    if gate_source == 1 and w.k > 0:
+        assert np.max(np.abs(_np(out.draft_entropy)[idx] - orc.draft_entropy)) <= compare.ENTROPY_ATOL
     rep = compare.compare(orc, _np(sub.draft_q), _np(sub.uniforms), _np(out.accept_len)[idx], _np(out.next_tok)[idx],
                           _np(out.entropy)[idx], _np(out.logZ)[idx],
                           _np(out.logits)[idx] if out.logits is not None else None)
@@ -192,6 +194,52 @@ def test_accept_sample_entry_from_oracle_logits(binding):
                           Hn.reshape(w.B, -1), lz.reshape(w.B, -1))
     assert rep.ok and rep.accept_exact >= w.B - 1, rep.summary()
     assert 0 < _np(out.accept_len).mean() < w.k       # both branches taken
+
+
+# ------------------------------------------------------------------------------------------ gate / verifier variants
+@pytest.mark.parametrize("gate_source,fallback", [(1, 0), (0, 1), (1, 1)])
+@pytest.mark.parametrize("B,k,H,V,qd", [(41, 5, 128, 3001, torch.bfloat16), (9, 3, 64, 1000, torch.float32)])
+def test_draft_entropy_gate_and_greedy_verifier(binding, gate_source, fallback, B, k, H, V, qd):
+    # w_std large enough that target rows are peaked sometimes (greedy accepts happen), draft noise small in the
+    # first half; tau in the middle of the draft entropies so that both gate branches are taken.
+    w = workloads.gaussian_head("variants", B, k, H, V, seed=31 * B + V, device=DEV, w_std=0.6, sigma=0.3, q_dtype=qd,
+                                tau=0.0, sigma_far=1.5)
+    probe = compare.run_oracle(w, keep_logits=False, gate_source=1)
+    w.tau = float(np.median(probe.draft_entropy if gate_source == 1 else probe.entropy[:, :k]))
+    if fallback == 1:                                    # let half of the draft tokens be the verifier's own choice
+        am = torch.from_numpy(compare.run_oracle(w, keep_logits=True).logits.argmax(-1)[:, :k].astype(np.int32)).to(DEV)
+        take = torch.rand((B, k), device=DEV, generator=torch.Generator(device=DEV).manual_seed(5)) < 0.6
+        w.draft_tok = torch.where(take, am, w.draft_tok).contiguous()
+    out, orc, rep = check_against_oracle(binding, w, gate_source=gate_source, fallback=fallback)
+    check_ranges(w, out)
+    acc = _np(out.accept_len)
+    assert 0 < acc.mean() < k                            # some runs break, some survive
+    gated = (orc.margin_gate < np.inf) & ((orc.draft_entropy if gate_source == 1 else orc.entropy[:, :k]) < w.tau)
+    assert gated.any() and (~gated).any()                # both branches of the gate were evaluated
+    if fallback == 1:                                    # the emitted token is always the verifier's arg-max
+        lg = _np(out.logits)
+        nxt = _np(out.next_tok)
+        assert np.array_equal(nxt, lg[np.arange(B), acc].argmax(-1))
+
+
+def test_greedy_verifier_on_the_large_vocabulary_shape(binding):
+    w = workloads.make_config("large_vocab", DEV)
+    out, _, _ = check_against_oracle(binding, w, seqs=[3, 30, 59], gate_source=1, fallback=1, want_logits=False)
+    check_ranges(w, out)
+
+
+def test_variant_arguments_are_validated(binding):
+    w = workloads.gaussian_head("v", 2, 2, 64, 100, seed=1, device=DEV)
+    with binding.HolaVerify(2, 2, 64, 100) as ctx:
+        with pytest.raises(binding.HolaError, match="invalid argument"):
+            ctx.hola_verify(w.hidden, w.W_lm, w.draft_tok, w.draft_q, w.uniforms, 1.5, gate_source=2)
+        with pytest.raises(binding.HolaError, match="invalid argument"):
+            ctx.hola_verify(w.hidden, w.W_lm, w.draft_tok, w.draft_q, w.uniforms, 1.5, fallback=-1)
+        # a bad token still ends the run under the greedy verifier, and is flagged
+        w.draft_tok[1, 0] = 100
+        out = ctx.hola_verify(w.hidden, w.W_lm, w.draft_tok, w.draft_q, w.uniforms, 0.0, fallback=1)
+        torch.cuda.synchronize()
+        assert int(out.accept_len[1]) == 0 and int(out.status.item()) & binding.FLAG_BAD_TOKEN
 
 
 # ------------------------------------------------------------------------------------------ degenerate inputs
