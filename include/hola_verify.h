@@ -13,6 +13,10 @@
  *      or from p at position k when every draft was accepted, by inverse CDF with the supplied uniform
  *      (ascending token id, first token whose cumulative mass exceeds u * total).
  *
+ * Two switches select the other readings of the paper's text: gate_source (entropy of the draft row instead of the
+ * verifier's softmax, the HSD section's "uncertainty in the draft distribution") and fallback (a greedy verifier,
+ * y = argmax p, instead of the speculative-sampling test).  A zero-initialised struct gives steps 1-5 as listed.
+ *
  * All pointers in hola_verify_args are DEVICE pointers unless a field says otherwise.  Every buffer is owned by
  * the caller.  The library allocates device memory only inside hola_create and frees it in hola_destroy.
  * No function throws, aborts or exits; each returns a hola_status.

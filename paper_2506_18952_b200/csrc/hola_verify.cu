@@ -69,6 +69,8 @@ constexpr int kMaxK1 = 64;                       // k + 1 <= 64
 #endif
 constexpr int kK3Unroll = K3_UNROLL;             // vocabulary chunks a warp has in flight per step
 
+constexpr int kHqSlices = 8;                     // CTAs that share one draft row in draft_entropy_kernel
+
 constexpr float kLog2e = 1.4426950408889634f;
 
 struct K1Params {
@@ -98,7 +100,8 @@ struct K3Params {
   float tau;
   int gate_source;          // hola_gate_source
   int fallback;             // hola_fallback
-  const float* draft_entropy;   // [B][k], read when gate_source == HOLA_GATE_DRAFT_ENTROPY
+  const double* hq_part;        // [B][k][kHqSlices] slice sums of q ln q, read when the draft entropy gates
+  float* draft_entropy;         // [B][k] optional output of H(q_j)
   int* accept_len;
   int* next_tok;
   float* entropy;
@@ -737,7 +740,14 @@ __global__ void __launch_bounds__(kK3Threads) accept_sample_kernel(const K3Param
                                       : static_cast<const float*>(p.q)[qi];
     }
     sh_lx[j] = lx; sh_qx[j] = qx;
-    sh_Hq[j] = p.gate_source == HOLA_GATE_DRAFT_ENTROPY ? p.draft_entropy[b * k + j] : 0.f;
+    float hq = 0.f;
+    if (p.gate_source == HOLA_GATE_DRAFT_ENTROPY) {
+      double tot = 0.0;
+      for (int sl = 0; sl < kHqSlices; ++sl) tot += p.hq_part[(static_cast<size_t>(b) * k + j) * kHqSlices + sl];
+      hq = fmaxf(0.f, static_cast<float>(-tot));
+      if (rank == 0 && p.draft_entropy) p.draft_entropy[b * k + j] = hq;
+    }
+    sh_Hq[j] = hq;
   }
   // ---- softmax statistics of this sequence's k+1 positions
   if (p.combine) {
@@ -928,46 +938,61 @@ __global__ void __launch_bounds__(kK3Threads) accept_sample_kernel(const K3Param
 // ------------------------------------------------------------------------------------------------ draft entropy
 // H(q) = -sum_v q ln q of each draft row (one CTA per row): the gate value when the gate looks at the draft
 // distribution, as the HSD section words it.  q is used as stored; entries with q <= 0 contribute nothing.
-__global__ void __launch_bounds__(256) draft_entropy_kernel(const void* q, int q_dtype, int V, float* out) {
+// q ln q for q > 0, else 0.  The fast logarithm (absolute error about 2^-21 near 1, a few ulp elsewhere) is
+// ample here: every term is weighted by q <= 1 and the sum is compared at 1e-4.
+__device__ __forceinline__ float qlnq(float a) { return a > 0.f ? a * __logf(a) : 0.f; }
+__device__ __forceinline__ float qlnq8(const uint4 raw) {     // sum over eight bf16 values
+  const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+  float part = 0.f;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) part += qlnq(__uint_as_float(w[j] << 16)) + qlnq(__uint_as_float(w[j] & 0xFFFF0000u));
+  return part;
+}
+__device__ __forceinline__ float qlnq4(const float4 x) { return (qlnq(x.x) + qlnq(x.y)) + (qlnq(x.z) + qlnq(x.w)); }
+
+// Grid (rows, kHqSlices): CTA (r, s) sums slice s of row r and leaves the partial sum in part[r][s]; the
+// accept/sample kernel adds the slices in index order.
+__global__ void __launch_bounds__(256) draft_entropy_kernel(const void* q, int q_dtype, int V, double* part) {
   __shared__ double sh_part[8];
   const size_t row = blockIdx.x;
+  const int slice = blockIdx.y;
   double acc = 0.0;
+  constexpr int kInFlight = 4;                           // independent 16-byte loads per thread and step
   if (q_dtype == HOLA_Q_BF16) {
     const __nv_bfloat16* qr = static_cast<const __nv_bfloat16*>(q) + row * V;
     const bool vec = (reinterpret_cast<uintptr_t>(qr) & 15u) == 0;
     const int nvec = vec ? V / 8 : 0;
-    for (int i = threadIdx.x; i < nvec; i += 256) {
-      const uint4 raw = reinterpret_cast<const uint4*>(qr)[i];
-      const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-      float part = 0.f;
+    const uint4* q16 = reinterpret_cast<const uint4*>(qr);
+    const int per = (nvec + kHqSlices - 1) / kHqSlices, end = min(nvec, (slice + 1) * per);
+    int i = slice * per + threadIdx.x;
+    for (; i + (kInFlight - 1) * 256 < end; i += kInFlight * 256) {
+      uint4 raw[kInFlight];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const float a = __uint_as_float(w[j] << 16), c = __uint_as_float(w[j] & 0xFFFF0000u);
-        if (a > 0.f) part = fmaf(a, logf(a), part);
-        if (c > 0.f) part = fmaf(c, logf(c), part);
-      }
-      acc += part;
+      for (int u = 0; u < kInFlight; ++u) raw[u] = q16[i + u * 256];
+#pragma unroll
+      for (int u = 0; u < kInFlight; ++u) acc += qlnq8(raw[u]);
     }
-    for (int v = nvec * 8 + threadIdx.x; v < V; v += 256) {
-      const float a = __bfloat162float(qr[v]);
-      if (a > 0.f) acc += a * logf(a);
+    for (; i < end; i += 256) acc += qlnq8(q16[i]);
+    for (int v = nvec * 8 + threadIdx.x; slice == 0 && v < V; v += 256) {    // scalar tail (or whole row): slice 0
+      acc += qlnq(__bfloat162float(qr[v]));
     }
   } else {
     const float* qr = static_cast<const float*>(q) + row * V;
     const bool vec = (reinterpret_cast<uintptr_t>(qr) & 15u) == 0;
     const int nvec = vec ? V / 4 : 0;
-    for (int i = threadIdx.x; i < nvec; i += 256) {
-      const float4 x = reinterpret_cast<const float4*>(qr)[i];
-      const float e[4] = {x.x, x.y, x.z, x.w};
-      float part = 0.f;
+    const float4* q16 = reinterpret_cast<const float4*>(qr);
+    const int per = (nvec + kHqSlices - 1) / kHqSlices, end = min(nvec, (slice + 1) * per);
+    int i = slice * per + threadIdx.x;
+    for (; i + (kInFlight - 1) * 256 < end; i += kInFlight * 256) {
+      float4 raw[kInFlight];
 #pragma unroll
-      for (int j = 0; j < 4; ++j)
-        if (e[j] > 0.f) part = fmaf(e[j], logf(e[j]), part);
-      acc += part;
+      for (int u = 0; u < kInFlight; ++u) raw[u] = q16[i + u * 256];
+#pragma unroll
+      for (int u = 0; u < kInFlight; ++u) acc += qlnq4(raw[u]);
     }
-    for (int v = nvec * 4 + threadIdx.x; v < V; v += 256) {
-      const float a = qr[v];
-      if (a > 0.f) acc += a * logf(a);
+    for (; i < end; i += 256) acc += qlnq4(q16[i]);
+    for (int v = nvec * 4 + threadIdx.x; slice == 0 && v < V; v += 256) {
+      acc += qlnq(qr[v]);
     }
   }
   acc = warp_sum_f64(acc);
@@ -976,7 +1001,7 @@ __global__ void __launch_bounds__(256) draft_entropy_kernel(const void* q, int q
   if (threadIdx.x == 0) {
     double tot = 0.0;
     for (int i = 0; i < 8; ++i) tot += sh_part[i];
-    out[row] = fmaxf(0.f, static_cast<float>(-tot));
+    part[row * kHqSlices + slice] = tot;
   }
 }
 
@@ -999,7 +1024,7 @@ struct hola_ctx {
   float* logits;            // [max_rows][ldl]
   float4* partials;         // [num_sms][max_rows]
   unsigned* status;         // [1]
-  float* hq;                // [max_rows] draft-row entropies when the caller does not ask for them
+  double* hq;               // [max_rows][kHqSlices] slice sums of q ln q over the draft rows
   // staging for hola_verify_host
   void* st_hidden; int* st_tok; void* st_q; float* st_u;
   int* st_accept; int* st_next; float* st_entropy; float* st_logZ;
@@ -1027,14 +1052,14 @@ WsLayout ws_layout(int maxB, int maxK, int H, int V, int num_sms) {
   w.logits = take(rows * ldl * 4);
   w.partials = take(static_cast<size_t>(num_sms) * rows * 16);
   w.status = take(4);
-  w.hq = take(rows * 4);
+  w.hq = take(rows * kHqSlices * 8);
   w.st_hidden = take(rows * H * 2);
   w.st_tok = take(static_cast<size_t>(maxB) * maxK * 4);
   w.st_q = take(static_cast<size_t>(maxB) * maxK * V * 4);
   w.st_u = take(rows * 4);
   w.st_accept = take(static_cast<size_t>(maxB) * 4);
   w.st_next = take(static_cast<size_t>(maxB) * 4);
-  w.st_entropy = take(rows * 4);
+  w.st_entropy = take(rows * 8);                         // target entropies, then the draft-row entropies
   w.st_logZ = take(rows * 4);
   w.total = off;
   return w;
@@ -1169,14 +1194,14 @@ hola_status run_accept_sample(hola_ctx* ctx, const hola_verify_args* a, const fl
   kp.B = a->B; kp.k = a->k; kp.V = a->V; kp.ldl = ldl; kp.logits = logits;
   kp.partials = ctx->partials; kp.nparts = nparts; kp.part_stride = ctx->max_rows; kp.combine = combine;
   kp.tok = a->draft_tok; kp.q = a->draft_q; kp.q_dtype = a->q_dtype; kp.u = a->uniforms; kp.tau = a->tau;
-  kp.gate_source = a->gate_source; kp.fallback = a->fallback; kp.draft_entropy = nullptr;
+  kp.gate_source = a->gate_source; kp.fallback = a->fallback; kp.hq_part = nullptr; kp.draft_entropy = a->draft_entropy;
   if (a->gate_source == HOLA_GATE_DRAFT_ENTROPY && a->k > 0) {
     // one more pass over the draft rows: H(q_j) for every (sequence, draft position)
-    float* hq = a->draft_entropy ? a->draft_entropy : ctx->hq;
-    draft_entropy_kernel<<<a->B * a->k, 256, 0, stream>>>(a->draft_q, a->q_dtype, a->V, hq);
+    draft_entropy_kernel<<<dim3(static_cast<unsigned>(a->B * a->k), kHqSlices), 256, 0, stream>>>(
+        a->draft_q, a->q_dtype, a->V, ctx->hq);
     const cudaError_t e0 = cudaGetLastError();
     if (e0 != cudaSuccess) { set_error(ctx, "launch draft_entropy_kernel", e0); return HOLA_ERR_CUDA; }
-    kp.draft_entropy = hq;
+    kp.hq_part = ctx->hq;
   }
   kp.accept_len = a->accept_len; kp.next_tok = a->next_tok; kp.entropy = a->entropy; kp.logZ = a->logZ;
   kp.status = a->status_word ? a->status_word : ctx->status;
@@ -1292,7 +1317,7 @@ hola_status hola_create(hola_ctx** out, int device, int maxB, int maxK, int H, i
   ctx->logits = reinterpret_cast<float*>(ctx->ws + w.logits);
   ctx->partials = reinterpret_cast<float4*>(ctx->ws + w.partials);
   ctx->status = reinterpret_cast<unsigned*>(ctx->ws + w.status);
-  ctx->hq = reinterpret_cast<float*>(ctx->ws + w.hq);
+  ctx->hq = reinterpret_cast<double*>(ctx->ws + w.hq);
   ctx->st_hidden = ctx->ws + w.st_hidden; ctx->st_tok = reinterpret_cast<int*>(ctx->ws + w.st_tok);
   ctx->st_q = ctx->ws + w.st_q; ctx->st_u = reinterpret_cast<float*>(ctx->ws + w.st_u);
   ctx->st_accept = reinterpret_cast<int*>(ctx->ws + w.st_accept);
@@ -1439,7 +1464,8 @@ hola_status hola_verify_host(hola_ctx* ctx, const hola_verify_args* a, void* cud
   hola_verify_args d = *a;
   d.hidden = ctx->st_hidden; d.draft_tok = ctx->st_tok; d.draft_q = ctx->st_q; d.uniforms = ctx->st_u;
   d.accept_len = ctx->st_accept; d.next_tok = ctx->st_next; d.entropy = ctx->st_entropy; d.logZ = ctx->st_logZ;
-  d.logits_out = nullptr; d.status_word = ctx->status; d.draft_entropy = nullptr;
+  d.logits_out = nullptr; d.status_word = ctx->status;
+  d.draft_entropy = a->draft_entropy ? ctx->st_entropy + rows : nullptr;   // staged after the entropies
   if ((s = hola_verify(ctx, &d, cuda_stream)) != HOLA_OK) return s;
   d2h(a->accept_len, ctx->st_accept, static_cast<size_t>(a->B) * 4);
   d2h(a->next_tok, ctx->st_next, static_cast<size_t>(a->B) * 4);
@@ -1447,7 +1473,7 @@ hola_status hola_verify_host(hola_ctx* ctx, const hola_verify_args* a, void* cud
   d2h(a->logZ, ctx->st_logZ, rows * 4);
   if (a->status_word) d2h(a->status_word, ctx->status, 4);
   if (a->draft_entropy && a->gate_source == HOLA_GATE_DRAFT_ENTROPY)
-    d2h(a->draft_entropy, ctx->hq, static_cast<size_t>(a->B) * a->k * 4);
+    d2h(a->draft_entropy, ctx->st_entropy + rows, static_cast<size_t>(a->B) * a->k * 4);
   if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
   if (e != cudaSuccess) { set_error(ctx, "device-to-host copy", e); return HOLA_ERR_CUDA; }
   return HOLA_OK;
