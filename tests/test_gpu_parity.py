@@ -334,6 +334,35 @@ def test_host_entry_equals_device_entry(binding):
     assert torch.equal(h.entropy, d.entropy.cpu()) and torch.equal(h.logZ, d.logZ.cpu())
 
 
+# ------------------------------------------------------------------------------------------ multi-round decode loop
+@pytest.mark.parametrize("gate_source,fallback", [(0, 0), (1, 1)])
+def test_multi_round_decode_loop(binding, gate_source, fallback):
+    # Algorithm 1 as a loop: every round's verify call agrees with the oracle on that round's arrays, and the
+    # context grows by exactly the accepted drafts plus the verifier's token.
+    from paper_2506_18952_b200 import driver
+    B, k, H, V, rounds = 6, 3, 128, 2000, 5
+    models = driver.SyntheticPair(V, H, seed=77, device=torch.device(DEV))
+    prompt = torch.randint(0, V, (B, 2), device=DEV, generator=torch.Generator(device=DEV).manual_seed(3))
+    with binding.HolaVerify(B, k, H, V) as ctx:
+        res = driver.hsd_decode(ctx, models, prompt, k, 1.5, rounds, seed=11, gate_source=gate_source,
+                                fallback=fallback, keep_records=True)
+    want = [list(map(int, prompt[b])) for b in range(B)]
+    gated = 0
+    for rec in res.records:
+        w = workloads.VerifyInputs("round", B, k, H, V, 1.5, rec.hidden, models.W_lm, rec.draft_tok, rec.draft_q,
+                                   rec.uniforms)
+        check_against_oracle(binding, w, out=rec.out, gate_source=gate_source, fallback=fallback)
+        gated += int((rec.out.entropy[:, :k] < 1.5).sum())
+        for b in range(B):
+            n = int(rec.out.accept_len[b])
+            want[b] += list(map(int, rec.draft_tok[b, :n])) + [int(rec.out.next_tok[b])]
+    for b in range(B):
+        assert int(res.lengths[b]) == len(want[b]) and list(map(int, res.tokens[b, :len(want[b])])) == want[b]
+    emitted = int((res.lengths - 2).sum())
+    assert B * rounds <= emitted <= B * rounds * (k + 1) and emitted > B * rounds     # more than one token per call
+    assert res.verify_ms > 0 and res.total_ms >= res.verify_ms
+
+
 # ------------------------------------------------------------------------------------------ the named workloads
 def test_edge_decode_config_full(binding):
     w = workloads.make_config("edge", DEV)
