@@ -104,7 +104,8 @@ hola_status hola_verify(hola_ctx* ctx, const hola_verify_args* args, void* cuda_
 /* End-to-end form for callers whose per-step data lives in host memory.  Same computation as hola_verify, but
  * hidden, draft_tok, draft_q, uniforms are HOST pointers (pinned memory makes the copies asynchronous) and
  * accept_len, next_tok, entropy, logZ, status_word are HOST outputs; logits_out is ignored.  W_lm stays a
- * DEVICE pointer: weights are resident.  Copies in, runs, copies out and synchronises the stream. */
+ * DEVICE pointer: weights are resident.  Copies in, runs, copies out and synchronises the stream.  The draft
+ * tensor, the largest input, is copied on a stream owned by the context while the LM-head GEMM already runs. */
 hola_status hola_verify_host(hola_ctx* ctx, const hola_verify_args* args, void* cuda_stream);
 
 /* Partial entry points, the steps of the path exposed one by one (same argument struct).

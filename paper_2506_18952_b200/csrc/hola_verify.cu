@@ -1029,6 +1029,9 @@ struct hola_ctx {
   void* st_hidden; int* st_tok; void* st_q; float* st_u;
   int* st_accept; int* st_next; float* st_entropy; float* st_logZ;
   int force_stages;
+  cudaStream_t copy_stream;   // hola_verify_host: the draft tensor travels here while the GEMM runs
+  cudaEvent_t copy_done;
+  int host_overlap;           // 1: copy the draft tensor on copy_stream while the GEMM runs
   // optional per-kernel timing (hola_profile_begin / hola_profile_end)
   cudaEvent_t* prof_ev;     // 3 events per recorded call: before the GEMM, after it, after accept/sample
   int prof_cap, prof_n, prof_on;
@@ -1306,6 +1309,8 @@ hola_status hola_create(hola_ctx** out, int device, int maxB, int maxK, int H, i
   ctx->H = H; ctx->V = V; ctx->ldl = static_cast<int>(align_up(static_cast<size_t>(V), 4));
   ctx->max_rows = maxB * (maxK + 1);
   ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
+  ctx->host_overlap = 1;
+  if (const char* e = getenv("HOLA_HOST_OVERLAP")) ctx->host_overlap = atoi(e) != 0;   // tuning override
   if (const char* e = getenv("HOLA_STAGES")) {           // tuning override for sweeps: fewer ring slots
     const int st = atoi(e);
     if (st >= 2 && st <= kMaxStages) ctx->force_stages = st;
@@ -1325,6 +1330,13 @@ hola_status hola_create(hola_ctx** out, int device, int maxB, int maxK, int H, i
   ctx->st_entropy = reinterpret_cast<float*>(ctx->ws + w.st_entropy);
   ctx->st_logZ = reinterpret_cast<float*>(ctx->ws + w.st_logZ);
   cudaMemset(ctx->status, 0, 4);
+  if (cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) != cudaSuccess ||
+      cudaEventCreateWithFlags(&ctx->copy_done, cudaEventDisableTiming) != cudaSuccess) {
+    if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
+    cudaFree(ctx->ws);
+    free(ctx);
+    return HOLA_ERR_CUDA;
+  }
   *out = ctx;
   return HOLA_OK;
 }
@@ -1334,6 +1346,8 @@ hola_status hola_destroy(hola_ctx* ctx) {
   DeviceGuard guard(ctx->device);
   for (int i = 0; i < 3 * ctx->prof_cap; ++i) cudaEventDestroy(ctx->prof_ev[i]);
   free(ctx->prof_ev);
+  if (ctx->copy_done) cudaEventDestroy(ctx->copy_done);
+  if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
   cudaFree(ctx->ws);
   free(ctx);
   return HOLA_OK;
@@ -1378,6 +1392,32 @@ hola_status hola_accept_sample(hola_ctx* ctx, const hola_verify_args* a, void* c
   return run_accept_sample(ctx, a, a->logits_out, a->V, 0, 0, static_cast<cudaStream_t>(cuda_stream));
 }
 
+}  // extern "C"
+
+namespace {
+
+// The whole step on device buffers.  `before_sample`, when given, is an event the accept/sample part waits for
+// (the draft tensor still being copied in by hola_verify_host).
+hola_status verify_device(hola_ctx* ctx, const hola_verify_args* a, cudaStream_t stream, cudaEvent_t before_sample) {
+  const Plan pl = make_plan(ctx, a->B * (a->k + 1));
+  float* logits = a->logits_out ? a->logits_out : ctx->logits;
+  const int ldl = a->logits_out ? a->V : ctx->ldl;
+  const bool prof = ctx->prof_on && ctx->prof_n < ctx->prof_cap;
+  cudaEvent_t* ev = prof ? ctx->prof_ev + 3 * ctx->prof_n : nullptr;
+  if (prof) cudaEventRecord(ev[0], stream);
+  hola_status s = run_lm_head(ctx, a, logits, ldl, pl, stream);
+  if (s != HOLA_OK) return s;
+  if (prof) cudaEventRecord(ev[1], stream);
+  if (before_sample && cudaStreamWaitEvent(stream, before_sample, 0) != cudaSuccess) return HOLA_ERR_CUDA;
+  s = run_accept_sample(ctx, a, logits, ldl, 1, pl.grid, stream);
+  if (prof) { cudaEventRecord(ev[2], stream); ctx->prof_n++; }
+  return s;
+}
+
+}  // namespace
+
+extern "C" {
+
 hola_status hola_verify(hola_ctx* ctx, const hola_verify_args* a, void* cuda_stream) {
   hola_status s = check_common(ctx, a);
   if (s != HOLA_OK) return s;
@@ -1385,18 +1425,7 @@ hola_status hola_verify(hola_ctx* ctx, const hola_verify_args* a, void* cuda_str
   if ((s = check_lm_head_args(ctx, a)) != HOLA_OK) return s;
   if ((s = check_sample_args(a)) != HOLA_OK) return s;
   DeviceGuard guard(ctx->device);
-  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  const Plan pl = make_plan(ctx, a->B * (a->k + 1));
-  float* logits = a->logits_out ? a->logits_out : ctx->logits;
-  const int ldl = a->logits_out ? a->V : ctx->ldl;
-  const bool prof = ctx->prof_on && ctx->prof_n < ctx->prof_cap;
-  cudaEvent_t* ev = prof ? ctx->prof_ev + 3 * ctx->prof_n : nullptr;
-  if (prof) cudaEventRecord(ev[0], stream);
-  if ((s = run_lm_head(ctx, a, logits, ldl, pl, stream)) != HOLA_OK) return s;
-  if (prof) cudaEventRecord(ev[1], stream);
-  s = run_accept_sample(ctx, a, logits, ldl, 1, pl.grid, stream);
-  if (prof) { cudaEventRecord(ev[2], stream); ctx->prof_n++; }
-  return s;
+  return verify_device(ctx, a, static_cast<cudaStream_t>(cuda_stream), nullptr);
 }
 
 hola_status hola_profile_begin(hola_ctx* ctx, int max_calls) {
@@ -1455,10 +1484,20 @@ hola_status hola_verify_host(hola_ctx* ctx, const hola_verify_args* a, void* cud
   auto d2h = [&](void* dst, const void* src, size_t bytes) {
     if (e == cudaSuccess && bytes) e = cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToHost, stream);
   };
+  // The small inputs go first (copies queue on the DMA engine in issue order).  The draft tensor is by far the
+  // largest input and only the accept/sample part reads it: it travels on the context's own stream while the
+  // GEMM runs on the caller's.  (The previous call synchronised before returning, so the staging is free.)
   h2d(ctx->st_hidden, a->hidden, rows * a->H * 2);
   h2d(ctx->st_tok, a->draft_tok, static_cast<size_t>(a->B) * a->k * 4);
-  h2d(ctx->st_q, a->draft_q, static_cast<size_t>(a->B) * a->k * a->V * q_elem);
   h2d(ctx->st_u, a->uniforms, rows * 4);
+  const size_t q_bytes = static_cast<size_t>(a->B) * a->k * a->V * q_elem;
+  const bool overlap = q_bytes && ctx->host_overlap;
+  if (overlap) {
+    if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->st_q, a->draft_q, q_bytes, cudaMemcpyHostToDevice, ctx->copy_stream);
+    if (e == cudaSuccess) e = cudaEventRecord(ctx->copy_done, ctx->copy_stream);
+  } else {
+    h2d(ctx->st_q, a->draft_q, q_bytes);
+  }
   if (e == cudaSuccess) e = cudaMemsetAsync(ctx->status, 0, 4, stream);
   if (e != cudaSuccess) { set_error(ctx, "host-to-device copy", e); return HOLA_ERR_CUDA; }
   hola_verify_args d = *a;
@@ -1466,7 +1505,8 @@ hola_status hola_verify_host(hola_ctx* ctx, const hola_verify_args* a, void* cud
   d.accept_len = ctx->st_accept; d.next_tok = ctx->st_next; d.entropy = ctx->st_entropy; d.logZ = ctx->st_logZ;
   d.logits_out = nullptr; d.status_word = ctx->status;
   d.draft_entropy = a->draft_entropy ? ctx->st_entropy + rows : nullptr;   // staged after the entropies
-  if ((s = hola_verify(ctx, &d, cuda_stream)) != HOLA_OK) return s;
+  if ((s = check_lm_head_args(ctx, &d)) != HOLA_OK) return s;
+  if ((s = verify_device(ctx, &d, stream, overlap ? ctx->copy_done : nullptr)) != HOLA_OK) return s;
   d2h(a->accept_len, ctx->st_accept, static_cast<size_t>(a->B) * 4);
   d2h(a->next_tok, ctx->st_next, static_cast<size_t>(a->B) * 4);
   d2h(a->entropy, ctx->st_entropy, rows * 4);
