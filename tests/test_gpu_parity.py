@@ -196,6 +196,22 @@ def test_accept_sample_entry_from_oracle_logits(binding):
     assert 0 < _np(out.accept_len).mean() < w.k       # both branches taken
 
 
+def test_maximum_sizes(binding):
+    # the largest k the library takes (k + 1 = 64 positions per sequence) and the largest vocabulary (524288):
+    # 2115 vocabulary tiles per launch, 4096 chunks in the accept/sample pass
+    w = workloads.gaussian_head("max-k", 3, 63, 64, 300, seed=63, device=DEV, w_std=0.4, sigma=0.3, tau=3.0)
+    out, _, _ = check_against_oracle(binding, w)
+    check_ranges(w, out)
+    assert _np(out.accept_len).max() > 5
+    w = workloads.gaussian_head("max-v", 2, 1, 64, 524288, seed=64, device=DEV, w_std=0.3, sigma=1.0, tau=1.5)
+    out, _, _ = check_against_oracle(binding, w)
+    check_ranges(w, out)
+    lib = binding.load_library()
+    import ctypes
+    ctx = ctypes.c_void_p()
+    assert lib.hola_create(ctypes.byref(ctx), 0, 1, 1, 64, 524289) == 2      # one past the largest vocabulary
+
+
 # ------------------------------------------------------------------------------------------ gate / verifier variants
 @pytest.mark.parametrize("gate_source,fallback", [(1, 0), (0, 1), (1, 1)])
 @pytest.mark.parametrize("B,k,H,V,qd", [(41, 5, 128, 3001, torch.bfloat16), (9, 3, 64, 1000, torch.float32)])
