@@ -58,6 +58,12 @@ typedef enum {
   HOLA_FALLBACK_GREEDY = 1      /* greedy verifier: keep x iff x = argmax_v p(v) (lowest id on ties); next_tok = argmax p_n */
 } hola_fallback;
 
+/* Storage of W_lm.  HOLA_W_INT8 is the 8-bit case of the Lo-Bi quantiser applied to the LM head (Lo-Bi Optimization
+ * section; the paper leaves the quantiser's format open): int8 [V][H] plus one fp32 scale per vocabulary row,
+ * W8[v][h] = w_scale[v] * q[v][h].  The weights are streamed at half the bytes, expanded exactly to bf16 on chip, and
+ * the scale multiplies the fp32 accumulators.  At most 256 verify rows go into one pass over W_lm in this mode. */
+typedef enum { HOLA_W_BF16 = 0, HOLA_W_INT8 = 1 } hola_w_dtype;
+
 /* Bits of the device status word (OR-ed by the kernels; the caller clears it). */
 #define HOLA_FLAG_BAD_TOKEN 1u   /* a draft token outside [0,V): treated as a rejection at that position    */
 #define HOLA_FLAG_BAD_UNIFORM 2u /* a uniform outside [0,1): clamped into [0, 1 - 2^-24]                     */
@@ -85,6 +91,9 @@ typedef struct {
   int32_t gate_source;     /* hola_gate_source; 0 (zero-initialised struct) = target entropy                   */
   int32_t fallback;        /* hola_fallback; 0 = speculative sampling.  With GREEDY the uniforms are not read  */
   float* draft_entropy;    /* out fp32 [B][k], optional: H(q_j), written when gate_source = DRAFT_ENTROPY       */
+  int32_t w_dtype;         /* hola_w_dtype; 0 = W_lm is bf16.  INT8: W_lm is int8 [V][H], H % 16 == 0             */
+  int32_t reserved_;       /* must be 0                                                                        */
+  const float* w_scale;    /* fp32 [V], required with HOLA_W_INT8: scale of each vocabulary row                */
 } hola_verify_args;
 
 /* Creates a context on `device` able to serve calls with B <= maxB, k <= maxK and exactly this H and V.
@@ -134,6 +143,12 @@ hola_status hola_accept_sample(hola_ctx* ctx, const hola_verify_args* args, void
  * are safe, but two calls that overlap on the GPU (issued on different streams, say) race on it and give
  * wrong entropy / logZ.  Serialise them. */
 hola_status hola_lm_head_entropy_static(const hola_verify_args* args, void* cuda_stream);
+
+/* Quantises a bf16 W_lm [V][H] (device) to the HOLA_W_INT8 form, on the current device, asynchronously on the
+ * stream: scale[v] = max_h |W[v][h]| / 127 (1 for an all-zero row), q = clip(rint(W / scale), -127, 127), evaluated in
+ * fp32 with ties to even.  q_out is int8 [V][H], scale_out fp32 [V], both device buffers of the caller.  Allocates
+ * nothing and needs no context. */
+hola_status hola_quantize_w8(const void* W_bf16, int V, int H, void* q_out, float* scale_out, void* cuda_stream);
 
 /* Launch geometry chosen for a shape (for reports): vocabulary rows per tile of a CTA pair, grid size (CTAs),
  * shared-memory ring slots, verify rows per pass, passes over W_lm, kernel launches per hola_verify call. */

@@ -17,10 +17,11 @@ HOLA_OK = 0
 HOLA_Q_BF16, HOLA_Q_F32 = 0, 1
 HOLA_GATE_TARGET_ENTROPY, HOLA_GATE_DRAFT_ENTROPY = 0, 1
 HOLA_FALLBACK_SAMPLE, HOLA_FALLBACK_GREEDY = 0, 1
+HOLA_W_BF16, HOLA_W_INT8 = 0, 1
 FLAG_BAD_TOKEN, FLAG_BAD_UNIFORM, FLAG_TIMEOUT, FLAG_R_ZERO = 1, 2, 4, 8
 
 EXPORTS = ["hola_create", "hola_destroy", "hola_workspace_bytes", "hola_verify", "hola_verify_host",
-           "hola_lm_head_entropy", "hola_accept_sample", "hola_lm_head_entropy_static", "hola_plan", "hola_profile_begin", "hola_profile_end", "hola_strerror", "hola_last_cuda_error",
+           "hola_lm_head_entropy", "hola_accept_sample", "hola_lm_head_entropy_static", "hola_quantize_w8", "hola_plan", "hola_profile_begin", "hola_profile_end", "hola_strerror", "hola_last_cuda_error",
            "hola_version"]
 
 
@@ -35,7 +36,8 @@ class hola_verify_args(ctypes.Structure):
                 ("tau", ctypes.c_float), ("accept_len", ctypes.c_void_p), ("next_tok", ctypes.c_void_p),
                 ("entropy", ctypes.c_void_p), ("logZ", ctypes.c_void_p), ("logits_out", ctypes.c_void_p),
                 ("status_word", ctypes.c_void_p), ("gate_source", ctypes.c_int32), ("fallback", ctypes.c_int32),
-                ("draft_entropy", ctypes.c_void_p)]
+                ("draft_entropy", ctypes.c_void_p), ("w_dtype", ctypes.c_int32), ("reserved_", ctypes.c_int32),
+                ("w_scale", ctypes.c_void_p)]
 
 
 class hola_plan_info(ctypes.Structure):
@@ -65,6 +67,9 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
         fn.argtypes = [ctypes.c_void_p, ctypes.POINTER(hola_verify_args), ctypes.c_void_p]
     lib.hola_lm_head_entropy_static.restype = ctypes.c_int
     lib.hola_lm_head_entropy_static.argtypes = [ctypes.POINTER(hola_verify_args), ctypes.c_void_p]
+    lib.hola_quantize_w8.restype = ctypes.c_int
+    lib.hola_quantize_w8.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p,
+                                     ctypes.c_void_p]
     lib.hola_plan.restype = ctypes.c_int
     lib.hola_plan.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.POINTER(hola_plan_info)]
     lib.hola_profile_begin.restype = ctypes.c_int
@@ -96,6 +101,21 @@ def _dptr(t: torch.Tensor | None):
 def _stream_ptr(stream) -> ctypes.c_void_p:
     s = torch.cuda.current_stream() if stream is None else stream
     return ctypes.c_void_p(s.cuda_stream)
+
+
+def hola_quantize_w8(W_lm: torch.Tensor, stream=None):
+    """8-bit form of a bf16 W_lm [V, H] on the device: returns (q int8 [V, H], scale fp32 [V]).  The integers and the
+    scales are computed by the library's kernel; torch only provides the two output buffers."""
+    if W_lm.dtype != torch.bfloat16 or not W_lm.is_cuda or not W_lm.is_contiguous():
+        raise HolaError("hola_quantize_w8 takes a contiguous bfloat16 device tensor")
+    lib = load_library()
+    V, H = W_lm.shape
+    q = torch.empty((V, H), dtype=torch.int8, device=W_lm.device)
+    scale = torch.empty((V,), dtype=torch.float32, device=W_lm.device)
+    with torch.cuda.device(W_lm.device):
+        _check(lib, None, lib.hola_quantize_w8(_dptr(W_lm), V, H, _dptr(q), _dptr(scale), _stream_ptr(stream)),
+               "hola_quantize_w8")
+    return q, scale
 
 
 def hola_lm_head_entropy_static(hidden, W_lm, logits, entropy, logZ, stream=None) -> None:
@@ -175,9 +195,11 @@ class HolaVerify:
         return {"lm_head_ms": a.value, "accept_sample_ms": b.value, "calls": n.value}
 
     def _args(self, hidden, W_lm, draft_tok, draft_q, uniforms, tau, out: VerifyOutputs, B, k,
-              gate_source: int = HOLA_GATE_TARGET_ENTROPY, fallback: int = HOLA_FALLBACK_SAMPLE):
-        if hidden.dtype != torch.bfloat16 or W_lm.dtype != torch.bfloat16:
-            raise HolaError("hidden and W_lm must be bfloat16")
+              gate_source: int = HOLA_GATE_TARGET_ENTROPY, fallback: int = HOLA_FALLBACK_SAMPLE, w_scale=None):
+        if hidden.dtype != torch.bfloat16 or W_lm.dtype not in (torch.bfloat16, torch.int8):
+            raise HolaError("hidden must be bfloat16, W_lm bfloat16 or int8")
+        if (W_lm.dtype == torch.int8) != (w_scale is not None):
+            raise HolaError("an int8 W_lm goes with w_scale (fp32 per vocabulary row), a bfloat16 one without")
         if draft_q is not None and draft_q.dtype not in (torch.bfloat16, torch.float32):
             raise HolaError("draft_q must be bfloat16 or float32")
         for t in (hidden, W_lm, draft_tok, draft_q, uniforms):
@@ -197,6 +219,8 @@ class HolaVerify:
         a.status_word = _dptr(out.status)
         a.gate_source, a.fallback = int(gate_source), int(fallback)
         a.draft_entropy = _dptr(out.draft_entropy)
+        a.w_dtype = HOLA_W_INT8 if w_scale is not None else HOLA_W_BF16
+        a.w_scale = _dptr(w_scale)
         return a
 
     def alloc_outputs(self, B: int, k: int, want_logits: bool = False, device=None) -> VerifyOutputs:
@@ -212,19 +236,20 @@ class HolaVerify:
 
     def hola_verify(self, hidden, W_lm, draft_tok, draft_q, uniforms, tau, out: VerifyOutputs | None = None,
                     want_logits: bool = False, stream=None, gate_source: int = HOLA_GATE_TARGET_ENTROPY,
-                    fallback: int = HOLA_FALLBACK_SAMPLE) -> VerifyOutputs:
-        """The whole verify step on device tensors, asynchronous on the stream."""
+                    fallback: int = HOLA_FALLBACK_SAMPLE, w_scale=None) -> VerifyOutputs:
+        """The whole verify step on device tensors, asynchronous on the stream.  With w_scale, W_lm is the int8 form
+        made by hola_quantize_w8."""
         B, k = hidden.shape[0], hidden.shape[1] - 1
         out = out or self.alloc_outputs(B, k, want_logits)
-        a = self._args(hidden, W_lm, draft_tok, draft_q, uniforms, tau, out, B, k, gate_source, fallback)
+        a = self._args(hidden, W_lm, draft_tok, draft_q, uniforms, tau, out, B, k, gate_source, fallback, w_scale)
         _check(self.lib, self._ctx, self.lib.hola_verify(self._ctx, ctypes.byref(a), _stream_ptr(stream)), "hola_verify")
         return out
 
     def hola_lm_head_entropy(self, hidden, W_lm, out: VerifyOutputs | None = None, want_logits: bool = True,
-                             stream=None) -> VerifyOutputs:
+                             stream=None, w_scale=None) -> VerifyOutputs:
         B, k = hidden.shape[0], hidden.shape[1] - 1
         out = out or self.alloc_outputs(B, k, want_logits)
-        a = self._args(hidden, W_lm, None, None, None, 0.0, out, B, k)
+        a = self._args(hidden, W_lm, None, None, None, 0.0, out, B, k, w_scale=w_scale)
         _check(self.lib, self._ctx, self.lib.hola_lm_head_entropy(self._ctx, ctypes.byref(a), _stream_ptr(stream)),
                "hola_lm_head_entropy")
         return out
@@ -250,7 +275,7 @@ class HolaVerify:
 
     def hola_verify_host(self, hidden, W_lm, draft_tok, draft_q, uniforms, tau, out: VerifyOutputs | None = None,
                          stream=None, gate_source: int = HOLA_GATE_TARGET_ENTROPY,
-                         fallback: int = HOLA_FALLBACK_SAMPLE) -> VerifyOutputs:
+                         fallback: int = HOLA_FALLBACK_SAMPLE, w_scale=None) -> VerifyOutputs:
         """End-to-end form: per-step inputs and all outputs are HOST tensors (pinned for async copies);
         W_lm is the resident device weight.  Returns after the stream has been synchronised."""
         B, k = hidden.shape[0], hidden.shape[1] - 1
@@ -260,7 +285,7 @@ class HolaVerify:
             if t is not None and t.device.type != "cpu":
                 raise HolaError("hola_verify_host takes host tensors for the per-step inputs")
         out = out or self.alloc_outputs(B, k, False, device=torch.device("cpu"))
-        a = self._args(hidden, W_lm, draft_tok, draft_q, uniforms, tau, out, B, k, gate_source, fallback)
+        a = self._args(hidden, W_lm, draft_tok, draft_q, uniforms, tau, out, B, k, gate_source, fallback, w_scale)
         a.logits_out = None
         _check(self.lib, self._ctx, self.lib.hola_verify_host(self._ctx, ctypes.byref(a), _stream_ptr(stream)),
                "hola_verify_host")

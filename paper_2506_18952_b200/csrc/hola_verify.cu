@@ -53,6 +53,13 @@ constexpr int kStatsThreads = kStatsWarps * 32;
 constexpr int kK1Warps = 2 + kDrainWarps + kStatsWarps;   // warp 0 TMA, warp 1 MMA + tensor-memory owner
 constexpr int kK1Threads = kK1Warps * 32;
 constexpr int kStatsRowsPerThread = kMaxRowsPerPass * 4 / kStatsThreads;   // four threads share a row
+// 8-bit W_lm: the int8 tile lands in a raw block, converter warps expand it to the bf16 tile the MMA reads.
+// The kernel then runs 4 statistics warps (at most 256 rows per pass), 1 warp loading hidden and 3 converters.
+constexpr int kRawBlockBytes = kLanes * kBlockK;  // int8 [128][64]
+constexpr int kW8StatsWarps = 4;
+constexpr int kW8HiddenWarp = 2 + kDrainWarps + kW8StatsWarps;     // warp 14
+constexpr int kConvWarps = kK1Warps - kW8HiddenWarp - 1;           // warps 15..17
+constexpr int kConvThreads = kConvWarps * 32;
 constexpr int kTmemCols = 512;
 constexpr int kMaxStages = 12;
 constexpr int kSmemBudget = 227 * 1024;          // dynamic shared memory per CTA on sm_100
@@ -82,8 +89,9 @@ struct K1Params {
   int tile_rows;  // vocabulary rows per CTA per tile (<= 128, multiple of 4): balances the tiles over the pairs
   int ldl;        // row pitch of the logits buffer, in floats
   int vec_ok;     // 16-byte loads of the logits buffer allowed (pitch and base aligned)
+  const float* w_scale;   // 8-bit W_lm: fp32 scale per vocabulary row, applied to the accumulators
   float* logits;
-  float4* partials;   // [grid][part_stride] (m, s, t, unused)
+  float4* partials;   // [grid][part_stride] (m, s, t, arg-max index)
   int part_stride;
   unsigned* status;
 };
@@ -359,6 +367,9 @@ __device__ __forceinline__ void stats_fold(const float* v, int n, int vocab0, St
 //   lready[2]  @224  per CTA: the 8 drain warps have stored the tile's logits (by tile parity)
 //   sfree[2]   @240  per CTA: the 8 statistics warps are done with that tile (keeps lready from lapping)
 //   tensor-memory base @256, abort flag @260
+//   8-bit W_lm only: rawfull[12] @272 per CTA: the int8 tile of the slot has landed; rawempty[12] @368 per CTA: the
+//   converter warps have expanded it.  full[] then collects, besides the hidden bytes, one arrival per converter warp.
+template <bool kW8>
 __global__ void __launch_bounds__(kK1Threads, 1)
 lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __grid_constant__ CUtensorMap tmap_w,
                        const K1Params p) {
@@ -374,25 +385,33 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
   const int npairs = gridDim.x >> 1;
   const int half_n = p.N >> 1;                           // hidden rows this CTA supplies per MMA
   const uint32_t hid_block_bytes = static_cast<uint32_t>(half_n) * 128u;
-  const uint32_t stage_bytes = kWBlockBytes + p.n_sub * hid_block_bytes;
-  const uint32_t tx_bytes = static_cast<uint32_t>(p.tile_rows) * 128u + p.n_sub * hid_block_bytes;   // per CTA and slot
+  const uint32_t raw_off = kWBlockBytes + p.n_sub * hid_block_bytes;     // int8 block of the slot (8-bit W_lm only)
+  const uint32_t stage_bytes = raw_off + (kW8 ? kRawBlockBytes : 0);
+  const uint32_t hid_tx_bytes = p.n_sub * hid_block_bytes;
+  const uint32_t tx_bytes = static_cast<uint32_t>(p.tile_rows) * 128u + hid_tx_bytes;   // bf16 W_lm: per CTA and slot
+  const uint32_t raw_tx_bytes = static_cast<uint32_t>(p.tile_rows) * 64u;
   const int pair_rows = 2 * p.tile_rows;                 // vocabulary rows of a pair's tile
   const uint32_t bar_base = base + p.stages * stage_bytes;
   const uint32_t full_bar = bar_base, empty_bar = bar_base + 96, tfull_bar = bar_base + 192,
-                 tempty_bar = bar_base + 208, lready_bar = bar_base + 224, sfree_bar = bar_base + 240;
+                 tempty_bar = bar_base + 208, lready_bar = bar_base + 224, sfree_bar = bar_base + 240,
+                 rawfull_bar = bar_base + 272, rawempty_bar = bar_base + 368;
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + p.stages * stage_bytes + 256);
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + p.stages * stage_bytes + 260);
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < p.stages; ++i) {
-      mbar_init(full_bar + 8 * i, 2);
+      mbar_init(full_bar + 8 * i, kW8 ? 2 + 2 * kConvWarps : 2);
       mbar_init(empty_bar + 8 * i, 1);
+      if (kW8) {
+        mbar_init(rawfull_bar + 8 * i, 1);
+        mbar_init(rawempty_bar + 8 * i, kConvWarps);
+      }
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(tfull_bar + 8 * i, 1);
       mbar_init(tempty_bar + 8 * i, 2 * kDrainWarps);
       mbar_init(lready_bar + 8 * i, kDrainWarps);
-      mbar_init(sfree_bar + 8 * i, kStatsWarps);
+      mbar_init(sfree_bar + 8 * i, kW8 ? kW8StatsWarps : kStatsWarps);
     }
     *abort_flag = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -417,6 +436,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
       const uint64_t pol_w = l2_policy_evict_first();    // W_lm is streamed once
       const uint64_t pol_h = l2_policy_evict_last();     // hidden is re-read for every tile
       const uint32_t leader_full = map_to_cta(full_bar, 0);
+      const uint32_t own_rawfull = map_to_cta(rawfull_bar, rank);
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
@@ -424,14 +444,22 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
         const int v0 = (pair + t * npairs) * pair_rows + static_cast<int>(rank) * p.tile_rows;
         int kx = 0;                                      // K coordinate of the block, in elements
         for (int kb = 0; kb < p.n_kblocks; ++kb, kx += kBlockK) {
-          if (!mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
           const uint32_t sa = base + stage * stage_bytes;
-          const uint32_t fb = leader_full + 8 * stage;
-          mbar_expect_tx_cluster(fb, tx_bytes);
-          tma_load_2d(sa, &tmap_w, fb, kx, v0, pol_w);
-          for (int s = 0; s < p.n_sub; ++s)
-            tma_load_2d(sa + kWBlockBytes + s * hid_block_bytes, &tmap_hidden, fb, kx,
-                        p.row0 + s * p.N + static_cast<int>(rank) * half_n, pol_h);
+          if (kW8) {
+            // only the int8 tile: its slot is free again as soon as the converters have read it
+            if (!mbar_wait(rawempty_bar + 8 * stage, phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
+            const uint32_t rb = own_rawfull + 8 * stage;
+            mbar_expect_tx_cluster(rb, raw_tx_bytes);
+            tma_load_2d(sa + raw_off, &tmap_w, rb, kx, v0, pol_w);
+          } else {
+            if (!mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
+            const uint32_t fb = leader_full + 8 * stage;
+            mbar_expect_tx_cluster(fb, tx_bytes);
+            tma_load_2d(sa, &tmap_w, fb, kx, v0, pol_w);
+            for (int s = 0; s < p.n_sub; ++s)
+              tma_load_2d(sa + kWBlockBytes + s * hid_block_bytes, &tmap_hidden, fb, kx,
+                          p.row0 + s * p.N + static_cast<int>(rank) * half_n, pol_h);
+          }
           if (++stage == p.stages) { stage = 0; phase ^= 1u; }
         }
       }
@@ -495,6 +523,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
       const int tile_lane = quarter * 32 + lane;         // lanes at or beyond tile_rows hold nothing
       const int vocab = (pair + t * npairs) * pair_rows + static_cast<int>(rank) * p.tile_rows + tile_lane;
       const bool vocab_ok = tile_lane < p.tile_rows && vocab < p.V;
+      const float w_scale = (kW8 && vocab_ok) ? p.w_scale[vocab] : 1.f;    // 8-bit W_lm: the row's scale
       const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * 256;
       for (int ch = group; ch < n_chunks; ch += 2) {
         const int s = ch / sub_chunks, j = ch - s * sub_chunks;
@@ -509,11 +538,11 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
           float* dst = p.logits + static_cast<size_t>(r0) * p.ldl + vocab;
           if (n_ok == 32) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) dst[static_cast<size_t>(i) * p.ldl] = v[i];
+            for (int i = 0; i < 32; ++i) dst[static_cast<size_t>(i) * p.ldl] = kW8 ? v[i] * w_scale : v[i];
           } else {
 #pragma unroll
             for (int i = 0; i < 32; ++i)
-              if (i < n_ok) dst[static_cast<size_t>(i) * p.ldl] = v[i];
+              if (i < n_ok) dst[static_cast<size_t>(i) * p.ldl] = kW8 ? v[i] * w_scale : v[i];
           }
         }
       }
@@ -528,10 +557,11 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
       __syncwarp();
       if (lane == 0) mbar_arrive(lready_bar + 8 * par);  // release: this warp's stores are visible to the CTA
     }
-  } else {
+  } else if (!kW8 || warp < kW8HiddenWarp) {
     // ------------------------------------------------------------------ statistics warps
     // Four threads share a verify row: thread `part` takes floats 16*it + 4*part .. +3 (it = 0..7) of the row's 128
     // logits of this tile, so a warp's load covers 8 rows x 64 contiguous bytes.
+    constexpr int kRowStep = (kW8 ? kW8StatsWarps : kStatsWarps) * 32 / 4;    // rows covered per step of the warps
     const int ts = threadIdx.x - (2 + kDrainWarps) * 32;
     const int part = ts & 3, rsub = ts >> 2;
     Stats st[kStatsRowsPerThread];
@@ -546,7 +576,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
       if (lim > 0) {
 #pragma unroll
         for (int i = 0; i < kStatsRowsPerThread; ++i) {
-          const int r = rsub + (kStatsThreads / 4) * i;
+          const int r = rsub + kRowStep * i;
           if (r < p.rows) {
             const float* src = p.logits + static_cast<size_t>(p.row0 + r) * p.ldl + vbase;
             float v[32];
@@ -588,10 +618,76 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
           o.arg = __shfl_xor_sync(0xffffffffu, a.arg, off);
           a = ((lane & off) == 0) ? stats_merge(a, o) : stats_merge(o, a);
         }
-        const int r = rsub + (kStatsThreads / 4) * i;
+        const int r = rsub + kRowStep * i;
         if (part == 0 && r < p.rows)
           p.partials[static_cast<size_t>(blockIdx.x) * p.part_stride + p.row0 + r] =
               make_float4(a.m, a.s, a.t, __int_as_float(a.arg));
+      }
+    }
+  } else if (warp == kW8HiddenWarp) {
+    // ------------------------------------------------------------------ 8-bit W_lm: TMA producer of the hidden blocks
+    if (elect_one()) {
+      const uint64_t pol_h = l2_policy_evict_last();
+      const uint32_t leader_full = map_to_cta(full_bar, 0);
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int t = 0; t < my_tiles && ok; ++t) {
+        int kx = 0;
+        for (int kb = 0; kb < p.n_kblocks; ++kb, kx += kBlockK) {
+          if (!mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
+          const uint32_t sa = base + stage * stage_bytes;
+          const uint32_t fb = leader_full + 8 * stage;
+          mbar_expect_tx_cluster(fb, hid_tx_bytes);
+          for (int s = 0; s < p.n_sub; ++s)
+            tma_load_2d(sa + kWBlockBytes + s * hid_block_bytes, &tmap_hidden, fb, kx,
+                        p.row0 + s * p.N + static_cast<int>(rank) * half_n, pol_h);
+          if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ 8-bit W_lm: converter warps
+    // int8 [tile_rows][64] (row pitch 64 bytes) -> bf16 [tile_rows][64] in the 128-byte-swizzled K-major layout the
+    // MMA reads: 16-byte chunk c of row r sits at chunk position c ^ (r % 8) of its 128-byte row.  Every int8 value is
+    // exact in bf16; the row's scale is applied to the accumulators by the drain warps.
+    const int ct = threadIdx.x - (kW8HiddenWarp + 1) * 32;
+    const uint32_t leader_full = map_to_cta(full_bar, 0);
+    const int units = p.tile_rows * 4;                   // 16-byte pieces of the int8 tile
+    int stage = 0;
+    uint32_t phase = 0;
+    bool ok = true;
+    for (int t = 0; t < my_tiles && ok; ++t) {
+      for (int kb = 0; kb < p.n_kblocks; ++kb) {
+        if (!mbar_wait_warp(rawfull_bar + 8 * stage, phase, abort_flag, p.status) ||
+            !mbar_wait_warp(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
+        uint8_t* slot = smem + stage * stage_bytes;
+        for (int u = ct; u < units; u += kConvThreads) {
+          const int row = u >> 2, c = u & 3;
+          const uint4 x = *reinterpret_cast<const uint4*>(slot + raw_off + row * 64 + c * 16);
+          const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+          uint32_t o[8];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const float f0 = static_cast<float>(static_cast<int>(static_cast<signed char>(w[j] & 0xFFu)));
+            const float f1 = static_cast<float>(static_cast<int>(static_cast<signed char>((w[j] >> 8) & 0xFFu)));
+            const float f2 = static_cast<float>(static_cast<int>(static_cast<signed char>((w[j] >> 16) & 0xFFu)));
+            const float f3 = static_cast<float>(static_cast<int>(static_cast<signed char>(w[j] >> 24)));
+            const __nv_bfloat162 a = __floats2bfloat162_rn(f0, f1), b = __floats2bfloat162_rn(f2, f3);
+            o[2 * j] = *reinterpret_cast<const uint32_t*>(&a);
+            o[2 * j + 1] = *reinterpret_cast<const uint32_t*>(&b);
+          }
+          uint8_t* drow = slot + (row >> 3) * 1024 + (row & 7) * 128;
+          *reinterpret_cast<uint4*>(drow + (((2 * c) ^ (row & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+          *reinterpret_cast<uint4*>(drow + (((2 * c + 1) ^ (row & 7)) << 4)) = make_uint4(o[4], o[5], o[6], o[7]);
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // generic-proxy writes, read by the MMA
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive_cluster(leader_full + 8 * stage);  // this warp's share of the bf16 tile is in place
+          mbar_arrive(rawempty_bar + 8 * stage);         // and the int8 block may be refilled
+        }
+        if (++stage == p.stages) { stage = 0; phase ^= 1u; }
       }
     }
   }
@@ -935,6 +1031,38 @@ __global__ void __launch_bounds__(kK3Threads) accept_sample_kernel(const K3Param
   }
 }
 
+// ------------------------------------------------------------------------------------------------ 8-bit quantiser
+// The 8-bit case of the Lo-Bi quantiser on the LM head (Lo-Bi Optimization section; the quantiser itself is not
+// spelled out there): one vocabulary row per sub-block, symmetric integers in [-127, 127], one fp32 scale per row,
+//   scale = max|w| / 127 (1 for an all-zero row),  q = clip(rint(w / scale)),  all in fp32, ties to even.
+// One CTA per row.
+__global__ void __launch_bounds__(256) quantize_rows_int8_kernel(const __nv_bfloat16* W, int H, signed char* q,
+                                                                 float* scale) {
+  __shared__ float sh_max[8];
+  __shared__ float sh_scale;
+  const size_t row = blockIdx.x;
+  const __nv_bfloat16* wr = W + row * H;
+  float amax = 0.f;
+  for (int h = threadIdx.x; h < H; h += 256) amax = fmaxf(amax, fabsf(__bfloat162float(wr[h])));
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, off));
+  if ((threadIdx.x & 31) == 0) sh_max[threadIdx.x >> 5] = amax;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float m = 0.f;
+    for (int i = 0; i < 8; ++i) m = fmaxf(m, sh_max[i]);
+    const float sc = m > 0.f ? __fdiv_rn(m, 127.f) : 1.f;
+    sh_scale = sc;
+    scale[row] = sc;
+  }
+  __syncthreads();
+  const float sc = sh_scale;
+  for (int h = threadIdx.x; h < H; h += 256) {
+    const float r = rintf(__fdiv_rn(__bfloat162float(wr[h]), sc));
+    q[row * H + h] = static_cast<signed char>(fminf(127.f, fmaxf(-127.f, r)));
+  }
+}
+
 // ------------------------------------------------------------------------------------------------ draft entropy
 // H(q) = -sum_v q ln q of each draft row (one CTA per row): the gate value when the gate looks at the draft
 // distribution, as the HSD section words it.  q is used as stored; entries with q <= 0 contribute nothing.
@@ -1079,12 +1207,14 @@ int round_up(int x, int a) { return (x + a - 1) / a * a; }
 // Splits M verify rows into passes over W_lm and each pass into one or two MMAs per K step.
 // A pass holds at most 512 rows (two MMAs of N <= 256 fill the tensor memory); N is a multiple of 16.
 // Cost per pass: the slower of streaming W_lm once and the padded rows' tensor time, plus a fixed launch cost.
-Plan make_plan(const hola_ctx* ctx, int M) {
+Plan make_plan(const hola_ctx* ctx, int M, bool w8 = false) {
   Plan best{};
   double best_cost = 1e300;
   const int rows = M > 0 ? M : 1;
-  const int p_min = (rows + kMaxRowsPerPass - 1) / kMaxRowsPerPass;
-  const double t_hbm = 2.0 * ctx->V * static_cast<double>(ctx->H) / 6.4e12;
+  // 8-bit W_lm: one MMA per K step (at most 256 rows per pass), and the slot also holds the int8 block
+  const int max_rows_per_pass = w8 ? kMaxN : kMaxRowsPerPass;
+  const int p_min = (rows + max_rows_per_pass - 1) / max_rows_per_pass;
+  const double t_hbm = (w8 ? 1.0 : 2.0) * ctx->V * static_cast<double>(ctx->H) / 6.4e12;
   for (int passes = p_min; passes <= p_min + 3; ++passes) {
     const int r = (rows + passes - 1) / passes;
     const int n_sub = r > kMaxN ? 2 : 1;
@@ -1098,7 +1228,7 @@ Plan make_plan(const hola_ctx* ctx, int M) {
   }
   // a pass may end up empty when rows_per_pass * (passes - 1) already covers M
   best.passes = (rows + best.rows_per_pass - 1) / best.rows_per_pass;
-  const int stage_bytes = kWBlockBytes + best.n_sub * (best.N / 2) * 128;
+  const int stage_bytes = kWBlockBytes + best.n_sub * (best.N / 2) * 128 + (w8 ? kRawBlockBytes : 0);
   int stages = (kSmemBudget - 1024 - kBarrierBytes) / stage_bytes;
   if (stages > kMaxStages) stages = kMaxStages;
   if (ctx->force_stages && ctx->force_stages < stages) stages = ctx->force_stages;
@@ -1120,14 +1250,17 @@ Plan make_plan(const hola_ctx* ctx, int M) {
   return best;
 }
 
+// K-major 2-D tensor map with a box of 64 elements x box_rows.  bf16: 128-byte swizzle (the layout the MMA reads);
+// int8: plain rows of 64 bytes (the converter warps read them).
 hola_status encode_map(hola_ctx* ctx, CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols,
-                       uint32_t box_rows) {
+                       uint32_t box_rows, bool int8 = false) {
   const cuuint64_t dims[2] = {cols, rows};
-  const cuuint64_t strides[1] = {cols * 2};
+  const cuuint64_t strides[1] = {cols * (int8 ? 1u : 2u)};
   const cuuint32_t box[2] = {static_cast<cuuint32_t>(kBlockK), box_rows};
   const cuuint32_t estr[2] = {1, 1};
-  const CUresult r = ctx->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides,
-                                 box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+  const CUresult r = ctx->encode(map, int8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+                                 const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                 int8 ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
                                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
     snprintf(ctx->last_error, sizeof ctx->last_error, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
@@ -1157,8 +1290,9 @@ hola_status run_lm_head(hola_ctx* ctx, const hola_verify_args* a, float* logits,
   hola_status s = encode_map(ctx, &th, a->hidden, static_cast<uint64_t>(M), static_cast<uint64_t>(a->H),
                              static_cast<uint32_t>(pl.N / 2));
   if (s != HOLA_OK) return s;
+  const bool w8 = a->w_dtype == HOLA_W_INT8;
   s = encode_map(ctx, &tw, a->W_lm, static_cast<uint64_t>(a->V), static_cast<uint64_t>(a->H),
-                 static_cast<uint32_t>(pl.tile_rows));
+                 static_cast<uint32_t>(pl.tile_rows), w8);
   if (s != HOLA_OK) return s;
   K1Params kp;
   kp.M = M; kp.V = a->V; kp.n_ptiles = pl.n_ptiles; kp.n_kblocks = pl.n_kblocks;
@@ -1166,8 +1300,11 @@ hola_status run_lm_head(hola_ctx* ctx, const hola_verify_args* a, float* logits,
   kp.vec_ok = (ldl % 4 == 0 && aligned16(logits)) ? 1 : 0;
   kp.logits = logits; kp.partials = ctx->partials; kp.part_stride = ctx->max_rows;
   kp.status = a->status_word ? a->status_word : ctx->status;
-  cudaError_t e = cudaFuncSetAttribute(lm_head_entropy_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       pl.smem_bytes);
+  kp.w_scale = a->w_scale;
+  cudaError_t e = w8 ? cudaFuncSetAttribute(lm_head_entropy_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            pl.smem_bytes)
+                     : cudaFuncSetAttribute(lm_head_entropy_kernel<false>,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem_bytes);
   if (e != cudaSuccess) { set_error(ctx, "cudaFuncSetAttribute", e); return HOLA_ERR_CUDA; }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(static_cast<unsigned>(pl.grid));
@@ -1185,7 +1322,8 @@ hola_status run_lm_head(hola_ctx* ctx, const hola_verify_args* a, float* logits,
     kp.row0 = pass * pl.rows_per_pass;
     kp.rows = M - kp.row0 < pl.rows_per_pass ? M - kp.row0 : pl.rows_per_pass;
     if (kp.rows <= 0) break;
-    e = cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel, th, tw, kp);
+    e = w8 ? cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<true>, th, tw, kp)
+           : cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<false>, th, tw, kp);
     if (e != cudaSuccess) { set_error(ctx, "launch lm_head_entropy_kernel", e); return HOLA_ERR_CUDA; }
   }
   return HOLA_OK;
@@ -1236,6 +1374,11 @@ hola_status check_lm_head_args(const hola_ctx* ctx, const hola_verify_args* a) {
   if (!a->hidden || !a->W_lm) return HOLA_ERR_INVALID_ARG;
   if (!aligned16(a->hidden) || !aligned16(a->W_lm)) return HOLA_ERR_INVALID_ARG;
   if (a->H % 8 != 0) return HOLA_ERR_UNSUPPORTED_SHAPE;
+  if (a->w_dtype != HOLA_W_BF16 && a->w_dtype != HOLA_W_INT8) return HOLA_ERR_INVALID_ARG;
+  if (a->w_dtype == HOLA_W_INT8) {
+    if (!a->w_scale) return HOLA_ERR_INVALID_ARG;
+    if (a->H % 16 != 0) return HOLA_ERR_UNSUPPORTED_SHAPE;     // int8 row pitch must be a multiple of 16 bytes
+  }
   (void)ctx;
   return HOLA_OK;
 }
@@ -1371,7 +1514,7 @@ hola_status hola_lm_head_entropy(hola_ctx* ctx, const hola_verify_args* a, void*
   DeviceGuard guard(ctx->device);
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   const int M = a->B * (a->k + 1);
-  const Plan pl = make_plan(ctx, M);
+  const Plan pl = make_plan(ctx, M, a->w_dtype == HOLA_W_INT8);
   float* logits = a->logits_out ? a->logits_out : ctx->logits;
   const int ldl = a->logits_out ? a->V : ctx->ldl;
   if ((s = run_lm_head(ctx, a, logits, ldl, pl, stream)) != HOLA_OK) return s;
@@ -1399,7 +1542,7 @@ namespace {
 // The whole step on device buffers.  `before_sample`, when given, is an event the accept/sample part waits for
 // (the draft tensor still being copied in by hola_verify_host).
 hola_status verify_device(hola_ctx* ctx, const hola_verify_args* a, cudaStream_t stream, cudaEvent_t before_sample) {
-  const Plan pl = make_plan(ctx, a->B * (a->k + 1));
+  const Plan pl = make_plan(ctx, a->B * (a->k + 1), a->w_dtype == HOLA_W_INT8);
   float* logits = a->logits_out ? a->logits_out : ctx->logits;
   const int ldl = a->logits_out ? a->V : ctx->ldl;
   const bool prof = ctx->prof_on && ctx->prof_n < ctx->prof_cap;
@@ -1519,6 +1662,13 @@ hola_status hola_verify_host(hola_ctx* ctx, const hola_verify_args* a, void* cud
   return HOLA_OK;
 }
 
+hola_status hola_quantize_w8(const void* W_bf16, int V, int H, void* q_out, float* scale_out, void* cuda_stream) {
+  if (!W_bf16 || !q_out || !scale_out || V <= 0 || H <= 0) return HOLA_ERR_INVALID_ARG;
+  quantize_rows_int8_kernel<<<static_cast<unsigned>(V), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+      static_cast<const __nv_bfloat16*>(W_bf16), H, static_cast<signed char*>(q_out), scale_out);
+  return cudaGetLastError() == cudaSuccess ? HOLA_OK : HOLA_ERR_CUDA;
+}
+
 }  // extern "C"
 
 // ------------------------------------------------------------------------------------------------ no-allocation entry
@@ -1594,7 +1744,9 @@ extern "C" hola_status hola_lm_head_entropy_static(const hola_verify_args* a, vo
   if (s != HOLA_OK) return s;
   local.H = a->H; local.V = a->V; local.maxB = a->B; local.maxK = a->k;
   const int M = static_cast<int>(rows);
-  const Plan pl = make_plan(&local, M);
+  if (a->w_dtype != HOLA_W_BF16 && a->w_dtype != HOLA_W_INT8) return HOLA_ERR_INVALID_ARG;
+  if (a->w_dtype == HOLA_W_INT8 && (!a->w_scale || a->H % 16 != 0)) return HOLA_ERR_INVALID_ARG;
+  const Plan pl = make_plan(&local, M, a->w_dtype == HOLA_W_INT8);
   if (pl.grid > kStaticMaxCtas) return HOLA_ERR_STATIC_LIMIT;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   // The array keeps whatever the last call left.  The statistics slots are fully overwritten for the rows of this

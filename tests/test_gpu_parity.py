@@ -350,6 +350,87 @@ def test_host_entry_equals_device_entry(binding):
     assert torch.equal(h.entropy, d.entropy.cpu()) and torch.equal(h.logZ, d.logZ.cpu())
 
 
+# ------------------------------------------------------------------------------------------ 8-bit LM head
+def _w8_oracle(w, q8, scale, **kw):
+    """The oracle on the dequantised head: hidden widened to fp64, W8 = scale * q in fp64."""
+    from oracle import lobi
+    hid = ref.bf16_bits_to_f64(_np(w.hidden))
+    W8 = lobi.dequantize_rows(_np(q8), _np(scale))
+    return ref.verify(hid, W8, _np(w.draft_tok), _np(w.draft_q), _np(w.uniforms), w.tau, keep_logits=True, **kw)
+
+
+@pytest.mark.parametrize("V,H", [(1000, 64), (4099, 208), (32000, 128)])
+def test_quantiser_is_bit_exact(binding, V, H):
+    from oracle import lobi
+    g = torch.Generator(device=DEV).manual_seed(V)
+    W = (torch.randn((V, H), generator=g, device=DEV) * 0.02).bfloat16()
+    W[3] = 0
+    W[5, :4] = torch.tensor([1.0, 0.00390625, -0.01171875, 0.01953125], device=DEV).bfloat16()    # exact ties at 127 steps
+    W[5, 4:] = 0
+    q8, scale = binding.hola_quantize_w8(W)
+    torch.cuda.synchronize()
+    want_q, want_s = lobi.quantize_rows_int8(W.float().cpu().numpy())
+    assert np.array_equal(_np(scale), want_s)
+    assert np.array_equal(_np(q8), want_q)
+
+
+@pytest.mark.parametrize("B,k,H,V,qd", [
+    (1, 4, 64, 1000, torch.float32),       # the tiny shape
+    (37, 6, 256, 5000, torch.bfloat16),    # 259 rows: two passes of the 8-bit kernel, ragged vocabulary tail
+    (5, 2, 80, 1001, torch.bfloat16),      # K tail (H = 80), odd V
+    (70, 3, 128, 640, torch.float32),      # 280 rows
+])
+def test_int8_head_matches_oracle_on_dequantised_weights(binding, B, k, H, V, qd):
+    w = workloads.gaussian_head("w8", B, k, H, V, seed=B + V, device=DEV, w_std=0.3, sigma=1.0, q_dtype=qd,
+                                tau=1.5 + 0.1 * k, sigma_far=0.2)
+    q8, scale = binding.hola_quantize_w8(w.W_lm)
+    with binding.HolaVerify(B, k, H, V) as ctx:
+        out = ctx.hola_verify(w.hidden, q8, w.draft_tok, w.draft_q, w.uniforms, w.tau, want_logits=True, w_scale=scale)
+        torch.cuda.synchronize()
+    assert int(out.status.item()) & binding.FLAG_TIMEOUT == 0
+    orc = _w8_oracle(w, q8, scale)
+    rep = compare.compare(orc, _np(w.draft_q), _np(w.uniforms), _np(out.accept_len), _np(out.next_tok),
+                          _np(out.entropy), _np(out.logZ), _np(out.logits))
+    print(rep.summary())
+    assert rep.ok, rep.summary()
+    assert rep.accept_margin_cases <= max(1, B // 20) and rep.token_margin_cases <= max(1, B // 10)
+    check_ranges(w, out)
+    # and the quantised head stays close to the bf16 head it came from
+    full = compare.run_oracle(w, keep_logits=False)
+    assert np.max(np.abs(orc.entropy - full.entropy)) < 0.25
+
+
+def test_int8_head_small_integer_weights_are_bit_exact(binding):
+    # integer weights with row maximum 127: scale = 1, q = W, every product and sum exact
+    g = torch.Generator().manual_seed(9)
+    B, k, H, V = 40, 3, 192, 520
+    hidden = torch.randint(-4, 5, (B, k + 1, H), generator=g).float().bfloat16().to(DEV)
+    Wf = torch.randint(-5, 6, (V, H), generator=g).float()
+    Wf[:, 0] = 127.0
+    W = Wf.bfloat16().to(DEV)
+    q8, scale = binding.hola_quantize_w8(W)
+    assert torch.all(scale == 1.0) and torch.equal(q8.float(), W.float())
+    with binding.HolaVerify(B, k, H, V) as ctx:
+        out = ctx.hola_lm_head_entropy(hidden, q8, want_logits=True, w_scale=scale)
+        torch.cuda.synchronize()
+    want = ref.logits(_np(hidden).reshape(-1, H), _np(W)).reshape(B, k + 1, V)
+    assert np.array_equal(_np(out.logits).astype(np.float64), want)
+
+
+def test_int8_head_on_the_edge_shape(binding):
+    w = workloads.make_config("edge", DEV)
+    q8, scale = binding.hola_quantize_w8(w.W_lm)
+    with binding.HolaVerify(w.B, w.k, w.H, w.V) as ctx:
+        out = ctx.hola_verify(w.hidden, q8, w.draft_tok, w.draft_q, w.uniforms, w.tau, want_logits=True, w_scale=scale)
+        torch.cuda.synchronize()
+        with pytest.raises(binding.HolaError):
+            ctx.hola_verify(w.hidden, q8, w.draft_tok, w.draft_q, w.uniforms, w.tau)          # int8 without scales
+    orc = _w8_oracle(w, q8, scale)
+    rep = compare.compare(orc, _np(w.draft_q), _np(w.uniforms), _np(out.accept_len), _np(out.next_tok),
+                          _np(out.entropy), _np(out.logZ), _np(out.logits))
+    assert rep.ok and rep.max_logit_rel_err < 1e-3, rep.summary()
+
+
 # ------------------------------------------------------------------------------------------ multi-round decode loop
 @pytest.mark.parametrize("gate_source,fallback", [(0, 0), (1, 1)])
 def test_multi_round_decode_loop(binding, gate_source, fallback):
