@@ -112,11 +112,11 @@ class ClockSampler:
                 "reasons": seen, "samples": len(inside)}
 
 
-def algorithmic_work(w) -> dict:
+def algorithmic_work(w, w_bytes: int = 2) -> dict:
     """Strict algorithmic bytes and FLOPs of one step and of one launch of the dominant kernel."""
     M = w.M
     q_elem = w.draft_q.element_size()
-    gemm_bytes = w.V * w.H * 2 + M * w.H * 2                      # W_lm once + hidden once
+    gemm_bytes = w.V * w.H * w_bytes + (w.V * 4 if w_bytes == 1 else 0) + M * w.H * 2     # W_lm (+ scales) + hidden, once
     sample_bytes = w.B * w.V * q_elem + w.B * w.k * (4 + q_elem)  # one q row + k gathers per sequence
     out_bytes = w.B * 8 + M * 8
     flops = 2.0 * M * w.V * w.H
@@ -191,6 +191,8 @@ def main():
                     help="which entropy feeds the gate: the verifier's softmax (default) or the draft row")
     ap.add_argument("--fallback", default="sample", choices=["sample", "greedy"],
                     help="what the gate-off branch does: speculative-sampling test (default) or greedy verifier")
+    ap.add_argument("--weights", default="bf16", choices=["bf16", "int8"],
+                    help="storage of W_lm: bf16 (default) or the 8-bit form made by hola_quantize_w8")
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--cpu-budget-s", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -212,20 +214,24 @@ def main():
     from paper_2506_18952_b200 import binding
     w = workloads.make_config(args.workload, dev, seed_offset=hdist.rank_seed_offset(rank))
     ctx = binding.HolaVerify(w.B, w.k, w.H, w.V, device=local)
-    plan = ctx.hola_plan(w.B, w.k)
+    plan = ctx.hola_plan(w.B, w.k, binding.HOLA_W_INT8 if args.weights == "int8" else binding.HOLA_W_BF16)
     out = ctx.alloc_outputs(w.B, w.k, False)
     flush = None
     if w.V * w.H * 2 <= 200e6:
         flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
 
+    W_dev, w_scale = w.W_lm, None
+    if args.weights == "int8":
+        W_dev, w_scale = binding.hola_quantize_w8(w.W_lm)
+        torch.cuda.synchronize()
     gate_source = 1 if args.gate == "draft" else 0
     fallback = 1 if args.fallback == "greedy" else 0
 
     def step():
         if flush is not None:
             flush.zero_()
-        ctx.hola_verify(w.hidden, w.W_lm, w.draft_tok, w.draft_q, w.uniforms, w.tau, out=out,
-                        gate_source=gate_source, fallback=fallback)
+        ctx.hola_verify(w.hidden, W_dev, w.draft_tok, w.draft_q, w.uniforms, w.tau, out=out,
+                        gate_source=gate_source, fallback=fallback, w_scale=w_scale)
 
     sampler = ClockSampler(local)
     sampler.start()
@@ -275,8 +281,8 @@ def main():
         setattr(hout, f, getattr(hout, f).pin_memory())
 
     def e2e_step():
-        ctx.hola_verify_host(host["hidden"], w.W_lm, host["draft_tok"], host["draft_q"], host["uniforms"], w.tau,
-                             out=hout, gate_source=gate_source, fallback=fallback)
+        ctx.hola_verify_host(host["hidden"], W_dev, host["draft_tok"], host["draft_q"], host["uniforms"], w.tau,
+                             out=hout, gate_source=gate_source, fallback=fallback, w_scale=w_scale)
 
     for _ in range(3):
         e2e_step()
@@ -296,7 +302,7 @@ def main():
 
     if rank == 0:
         peaks, peak_kind = load_peaks()
-        work = algorithmic_work(w)
+        work = algorithmic_work(w, 1 if args.weights == "int8" else 2)
         t_mem = work["gemm_bytes"] / (peaks["hbm_gbs"] * 1e9)
         t_flop = work["flops"] / (peaks["bf16_tflops"] * 1e12)
         t_k1 = k1_ms * 1e-3 * plan["passes"]
@@ -307,7 +313,7 @@ def main():
             roof = {"bound": "hbm", "achieved": work["gemm_bytes"] / t_k1 / 1e9, "peak": peaks["hbm_gbs"],
                     "unit": "GB/s"}
         roof["frac"] = roof["achieved"] / roof["peak"]
-        roof["traffic"] = ncu_traffic_bytes(w)
+        roof["traffic"] = ncu_traffic_bytes(w) if args.weights == "bf16" else None
         roof.update({"kernel": "lm_head_entropy_kernel", "kernel_ms": k1_ms, "launches_per_step": plan["passes"],
                      "peak_source": f"of {peak_kind}", "hbm_gbs_achieved": work["gemm_bytes"] / t_k1 / 1e9,
                      "hbm_frac": work["gemm_bytes"] / t_k1 / 1e9 / peaks["hbm_gbs"],
@@ -318,7 +324,7 @@ def main():
                 "warmup": args.warmup, "ms_per_step": ms_max / args.steps, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
                 "config": config_block(w, {"plan": plan, "parallelism": f"replicas x{world}", "gate": args.gate,
-                                           "fallback": args.fallback}),
+                                           "fallback": args.fallback, "weights": args.weights}),
                 "clocks": clocks,
                 "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
                 "gpu_launches": (plan["kernels_per_call"] + (1 if gate_source and w.k > 0 else 0)) * args.steps,

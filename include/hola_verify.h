@@ -155,7 +155,8 @@ hola_status hola_quantize_w8(const void* W_bf16, int V, int H, void* q_out, floa
 typedef struct {
   int32_t tile_v, grid, stages, rows_per_pass, passes, kernels_per_call;
 } hola_plan_info;
-hola_status hola_plan(const hola_ctx* ctx, int B, int k, hola_plan_info* out);
+hola_status hola_plan(const hola_ctx* ctx, int B, int k, hola_plan_info* out);            /* bf16 W_lm */
+hola_status hola_plan_ex(const hola_ctx* ctx, int B, int k, int w_dtype, hola_plan_info* out);
 
 /* Per-kernel timing for reports.  Between hola_profile_begin and hola_profile_end every hola_verify call (at
  * most max_calls of them, max_calls <= 4096) records CUDA events on its stream around the LM-head GEMM launches

@@ -21,7 +21,7 @@ HOLA_W_BF16, HOLA_W_INT8 = 0, 1
 FLAG_BAD_TOKEN, FLAG_BAD_UNIFORM, FLAG_TIMEOUT, FLAG_R_ZERO = 1, 2, 4, 8
 
 EXPORTS = ["hola_create", "hola_destroy", "hola_workspace_bytes", "hola_verify", "hola_verify_host",
-           "hola_lm_head_entropy", "hola_accept_sample", "hola_lm_head_entropy_static", "hola_quantize_w8", "hola_plan", "hola_profile_begin", "hola_profile_end", "hola_strerror", "hola_last_cuda_error",
+           "hola_lm_head_entropy", "hola_accept_sample", "hola_lm_head_entropy_static", "hola_quantize_w8", "hola_plan", "hola_plan_ex", "hola_profile_begin", "hola_profile_end", "hola_strerror", "hola_last_cuda_error",
            "hola_version"]
 
 
@@ -72,6 +72,8 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
                                      ctypes.c_void_p]
     lib.hola_plan.restype = ctypes.c_int
     lib.hola_plan.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.POINTER(hola_plan_info)]
+    lib.hola_plan_ex.restype = ctypes.c_int
+    lib.hola_plan_ex.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.POINTER(hola_plan_info)]
     lib.hola_profile_begin.restype = ctypes.c_int
     lib.hola_profile_begin.argtypes = [ctypes.c_void_p, ctypes.c_int]
     lib.hola_profile_end.restype = ctypes.c_int
@@ -180,9 +182,9 @@ class HolaVerify:
         self.close()
 
     # -------------------------------------------------------------------------------------------------
-    def hola_plan(self, B: int, k: int) -> dict:
+    def hola_plan(self, B: int, k: int, w_dtype: int = HOLA_W_BF16) -> dict:
         info = hola_plan_info()
-        _check(self.lib, self._ctx, self.lib.hola_plan(self._ctx, B, k, ctypes.byref(info)), "hola_plan")
+        _check(self.lib, self._ctx, self.lib.hola_plan_ex(self._ctx, B, k, w_dtype, ctypes.byref(info)), "hola_plan_ex")
         return {n: getattr(info, n) for n, _ in info._fields_}
 
     def hola_profile_begin(self, max_calls: int):

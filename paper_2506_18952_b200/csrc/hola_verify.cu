@@ -54,11 +54,13 @@ constexpr int kK1Warps = 2 + kDrainWarps + kStatsWarps;   // warp 0 TMA, warp 1 
 constexpr int kK1Threads = kK1Warps * 32;
 constexpr int kStatsRowsPerThread = kMaxRowsPerPass * 4 / kStatsThreads;   // four threads share a row
 // 8-bit W_lm: the int8 tile lands in a raw block, converter warps expand it to the bf16 tile the MMA reads.
-// The kernel then runs 4 statistics warps (at most 256 rows per pass), 1 warp loading hidden and 3 converters.
+// That kernel takes at most 256 rows per pass, so 4 drain warps (2..5) and 4 statistics warps (10..13) are enough;
+// warp 14 loads the hidden blocks and warps 6..9 and 15..17 convert.
 constexpr int kRawBlockBytes = kLanes * kBlockK;  // int8 [128][64]
+constexpr int kW8DrainWarps = 4;
 constexpr int kW8StatsWarps = 4;
 constexpr int kW8HiddenWarp = 2 + kDrainWarps + kW8StatsWarps;     // warp 14
-constexpr int kConvWarps = kK1Warps - kW8HiddenWarp - 1;           // warps 15..17
+constexpr int kConvWarps = (kDrainWarps - kW8DrainWarps) + (kK1Warps - kW8HiddenWarp - 1);   // 4 + 3
 constexpr int kConvThreads = kConvWarps * 32;
 constexpr int kTmemCols = 512;
 constexpr int kMaxStages = 12;
@@ -357,6 +359,30 @@ __device__ __forceinline__ void stats_fold(const float* v, int n, int vocab0, St
   st.t = t;
 }
 
+// Sixteen int8 values (one 16-byte piece c of row `row` of the raw block) -> sixteen bf16 values at their place in
+// the 128-byte-swizzled K-major tile that starts at `tile`: chunk 2c and 2c+1 of the row, each XOR-ed with row % 8.
+__device__ __forceinline__ void expand_int8x16(const uint4 x, uint8_t* tile, int row, int c) {
+  const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+  uint32_t o[8];
+  // int8 -> float without conversion instructions: byte b + 128 placed in the low mantissa bits of 2^23 gives the
+  // float 2^23 + 128 + b exactly; one subtraction leaves b.  Two such floats pack into a bf16 pair (exact: |b| <= 128).
+  constexpr float kMagic = 8388608.f + 128.f;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const uint32_t u = w[j] ^ 0x80808080u;
+    const float f0 = __uint_as_float(__byte_perm(u, 0x4B000000u, 0x7650)) - kMagic;
+    const float f1 = __uint_as_float(__byte_perm(u, 0x4B000000u, 0x7651)) - kMagic;
+    const float f2 = __uint_as_float(__byte_perm(u, 0x4B000000u, 0x7652)) - kMagic;
+    const float f3 = __uint_as_float(__byte_perm(u, 0x4B000000u, 0x7653)) - kMagic;
+    const __nv_bfloat162 a = __floats2bfloat162_rn(f0, f1), b = __floats2bfloat162_rn(f2, f3);
+    o[2 * j] = *reinterpret_cast<const uint32_t*>(&a);
+    o[2 * j + 1] = *reinterpret_cast<const uint32_t*>(&b);
+  }
+  uint8_t* drow = tile + (row >> 3) * 1024 + (row & 7) * 128;
+  *reinterpret_cast<uint4*>(drow + (((2 * c) ^ (row & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+  *reinterpret_cast<uint4*>(drow + (((2 * c + 1) ^ (row & 7)) << 4)) = make_uint4(o[4], o[5], o[6], o[7]);
+}
+
 // ------------------------------------------------------------------------------------------------ K1
 // Shared memory: `stages` ring slots of [W_lm block 128 x 64 | hidden block(s) n_sub x (N/2) x 64], then the
 // barrier area.  Barriers (8 bytes each, offsets in the barrier area):
@@ -400,7 +426,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < p.stages; ++i) {
-      mbar_init(full_bar + 8 * i, kW8 ? 2 + 2 * kConvWarps : 2);
+      mbar_init(full_bar + 8 * i, kW8 ? 2 + 2 * kConvWarps : 2);   // + every converter warp of the pair with 8-bit W_lm
       mbar_init(empty_bar + 8 * i, 1);
       if (kW8) {
         mbar_init(rawfull_bar + 8 * i, 1);
@@ -409,8 +435,8 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(tfull_bar + 8 * i, 1);
-      mbar_init(tempty_bar + 8 * i, 2 * kDrainWarps);
-      mbar_init(lready_bar + 8 * i, kDrainWarps);
+      mbar_init(tempty_bar + 8 * i, 2 * (kW8 ? kW8DrainWarps : kDrainWarps));
+      mbar_init(lready_bar + 8 * i, kW8 ? kW8DrainWarps : kDrainWarps);
       mbar_init(sfree_bar + 8 * i, kW8 ? kW8StatsWarps : kStatsWarps);
     }
     *abort_flag = 0u;
@@ -507,10 +533,11 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
         if (ok) umma_commit_pair(tfull_bar + 8 * buf);   // accumulators of this tile are complete in both CTAs
       }
     }
-  } else if (warp < 2 + kDrainWarps) {
+  } else if (warp < 2 + (kW8 ? kW8DrainWarps : kDrainWarps)) {
     // ------------------------------------------------------------------ drain warps: tensor memory -> logits
     const int quarter = warp & 3;                        // tensor-memory lanes 32*quarter .. +31 (fixed by warp id)
     const int group = (warp - 2) >> 2;                   // the two warps of a quarter alternate over the chunks
+    constexpr int kChunkStep = kW8 ? 1 : 2;              // (one warp per quarter with 8-bit W_lm)
     const uint32_t leader_tempty = map_to_cta(tempty_bar, 0);
     const int n_chunks = p.n_sub * sub_chunks;
     bool ok = true;
@@ -525,7 +552,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
       const bool vocab_ok = tile_lane < p.tile_rows && vocab < p.V;
       const float w_scale = (kW8 && vocab_ok) ? p.w_scale[vocab] : 1.f;    // 8-bit W_lm: the row's scale
       const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * 256;
-      for (int ch = group; ch < n_chunks; ch += 2) {
+      for (int ch = group; ch < n_chunks; ch += kChunkStep) {
         const int s = ch / sub_chunks, j = ch - s * sub_chunks;
         float v[32];
         __syncwarp();                                    // tcgen05.ld is warp-collective: reconverge first
@@ -557,7 +584,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
       __syncwarp();
       if (lane == 0) mbar_arrive(lready_bar + 8 * par);  // release: this warp's stores are visible to the CTA
     }
-  } else if (!kW8 || warp < kW8HiddenWarp) {
+  } else if (!kW8 || (warp >= 2 + kDrainWarps && warp < kW8HiddenWarp)) {
     // ------------------------------------------------------------------ statistics warps
     // Four threads share a verify row: thread `part` takes floats 16*it + 4*part .. +3 (it = 0..7) of the row's 128
     // logits of this tile, so a warp's load covers 8 rows x 64 contiguous bytes.
@@ -651,7 +678,9 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
     // int8 [tile_rows][64] (row pitch 64 bytes) -> bf16 [tile_rows][64] in the 128-byte-swizzled K-major layout the
     // MMA reads: 16-byte chunk c of row r sits at chunk position c ^ (r % 8) of its 128-byte row.  Every int8 value is
     // exact in bf16; the row's scale is applied to the accumulators by the drain warps.
-    const int ct = threadIdx.x - (kW8HiddenWarp + 1) * 32;
+    // All converter warps share every K block (two independent 16-byte pieces per thread), in ring order.
+    const int cw = warp < 2 + kDrainWarps ? warp - (2 + kW8DrainWarps) : warp - (kW8HiddenWarp + 1) + (kDrainWarps - kW8DrainWarps);
+    const int ct = cw * 32 + lane;
     const uint32_t leader_full = map_to_cta(full_bar, 0);
     const int units = p.tile_rows * 4;                   // 16-byte pieces of the int8 tile
     int stage = 0;
@@ -662,24 +691,14 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
         if (!mbar_wait_warp(rawfull_bar + 8 * stage, phase, abort_flag, p.status) ||
             !mbar_wait_warp(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
         uint8_t* slot = smem + stage * stage_bytes;
-        for (int u = ct; u < units; u += kConvThreads) {
-          const int row = u >> 2, c = u & 3;
-          const uint4 x = *reinterpret_cast<const uint4*>(slot + raw_off + row * 64 + c * 16);
-          const uint32_t w[4] = {x.x, x.y, x.z, x.w};
-          uint32_t o[8];
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const float f0 = static_cast<float>(static_cast<int>(static_cast<signed char>(w[j] & 0xFFu)));
-            const float f1 = static_cast<float>(static_cast<int>(static_cast<signed char>((w[j] >> 8) & 0xFFu)));
-            const float f2 = static_cast<float>(static_cast<int>(static_cast<signed char>((w[j] >> 16) & 0xFFu)));
-            const float f3 = static_cast<float>(static_cast<int>(static_cast<signed char>(w[j] >> 24)));
-            const __nv_bfloat162 a = __floats2bfloat162_rn(f0, f1), b = __floats2bfloat162_rn(f2, f3);
-            o[2 * j] = *reinterpret_cast<const uint32_t*>(&a);
-            o[2 * j + 1] = *reinterpret_cast<const uint32_t*>(&b);
-          }
-          uint8_t* drow = slot + (row >> 3) * 1024 + (row & 7) * 128;
-          *reinterpret_cast<uint4*>(drow + (((2 * c) ^ (row & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
-          *reinterpret_cast<uint4*>(drow + (((2 * c + 1) ^ (row & 7)) << 4)) = make_uint4(o[4], o[5], o[6], o[7]);
+        for (int u0 = ct; u0 < units; u0 += 2 * kConvThreads) {
+          const int u1 = u0 + kConvThreads;
+          const bool has1 = u1 < units;
+          const uint4 x0 = *reinterpret_cast<const uint4*>(slot + raw_off + (u0 >> 2) * 64 + (u0 & 3) * 16);
+          uint4 x1 = make_uint4(0u, 0u, 0u, 0u);
+          if (has1) x1 = *reinterpret_cast<const uint4*>(slot + raw_off + (u1 >> 2) * 64 + (u1 & 3) * 16);
+          expand_int8x16(x0, slot, u0 >> 2, u0 & 3);
+          if (has1) expand_int8x16(x1, slot, u1 >> 2, u1 & 3);
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // generic-proxy writes, read by the MMA
         __syncwarp();
@@ -1496,13 +1515,18 @@ hola_status hola_destroy(hola_ctx* ctx) {
   return HOLA_OK;
 }
 
-hola_status hola_plan(const hola_ctx* ctx, int B, int k, hola_plan_info* out) {
+hola_status hola_plan_ex(const hola_ctx* ctx, int B, int k, int w_dtype, hola_plan_info* out) {
   if (!ctx || !out || B < 0 || k < 0) return HOLA_ERR_INVALID_ARG;
+  if (w_dtype != HOLA_W_BF16 && w_dtype != HOLA_W_INT8) return HOLA_ERR_INVALID_ARG;
   if (B > ctx->maxB || k > ctx->maxK) return HOLA_ERR_UNSUPPORTED_SHAPE;
-  const Plan pl = make_plan(ctx, B * (k + 1));
+  const Plan pl = make_plan(ctx, B * (k + 1), w_dtype == HOLA_W_INT8);
   out->tile_v = 2 * pl.tile_rows; out->grid = pl.grid; out->stages = pl.stages; out->rows_per_pass = pl.rows_per_pass;
   out->passes = pl.passes; out->kernels_per_call = pl.passes + 1;
   return HOLA_OK;
+}
+
+hola_status hola_plan(const hola_ctx* ctx, int B, int k, hola_plan_info* out) {
+  return hola_plan_ex(ctx, B, k, HOLA_W_BF16, out);
 }
 
 hola_status hola_lm_head_entropy(hola_ctx* ctx, const hola_verify_args* a, void* cuda_stream) {
