@@ -191,8 +191,9 @@ def main():
                     help="which entropy feeds the gate: the verifier's softmax (default) or the draft row")
     ap.add_argument("--fallback", default="sample", choices=["sample", "greedy"],
                     help="what the gate-off branch does: speculative-sampling test (default) or greedy verifier")
-    ap.add_argument("--weights", default="bf16", choices=["bf16", "int8"],
-                    help="storage of W_lm: bf16 (default) or the 8-bit form made by hola_quantize_w8")
+    ap.add_argument("--weights", default="bf16", choices=["bf16", "int8", "w8a8"],
+                    help="bf16 (default); int8: 8-bit W_lm from hola_quantize_w8, expanded exactly on chip; "
+                         "w8a8: 8-bit W_lm and hidden rows quantised on the fly, 8-bit tensor-core kind")
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--cpu-budget-s", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -214,14 +215,16 @@ def main():
     from paper_2506_18952_b200 import binding
     w = workloads.make_config(args.workload, dev, seed_offset=hdist.rank_seed_offset(rank))
     ctx = binding.HolaVerify(w.B, w.k, w.H, w.V, device=local)
-    plan = ctx.hola_plan(w.B, w.k, binding.HOLA_W_INT8 if args.weights == "int8" else binding.HOLA_W_BF16)
+    plan = ctx.hola_plan(w.B, w.k, {"bf16": binding.HOLA_W_BF16, "int8": binding.HOLA_W_INT8,
+                                    "w8a8": binding.HOLA_W8A8}[args.weights])
     out = ctx.alloc_outputs(w.B, w.k, False)
     flush = None
     if w.V * w.H * 2 <= 200e6:
         flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
 
     W_dev, w_scale = w.W_lm, None
-    if args.weights == "int8":
+    a8 = args.weights == "w8a8"
+    if args.weights != "bf16":
         W_dev, w_scale = binding.hola_quantize_w8(w.W_lm)
         torch.cuda.synchronize()
     gate_source = 1 if args.gate == "draft" else 0
@@ -231,7 +234,7 @@ def main():
         if flush is not None:
             flush.zero_()
         ctx.hola_verify(w.hidden, W_dev, w.draft_tok, w.draft_q, w.uniforms, w.tau, out=out,
-                        gate_source=gate_source, fallback=fallback, w_scale=w_scale)
+                        gate_source=gate_source, fallback=fallback, w_scale=w_scale, a8=a8)
 
     sampler = ClockSampler(local)
     sampler.start()
@@ -282,7 +285,7 @@ def main():
 
     def e2e_step():
         ctx.hola_verify_host(host["hidden"], W_dev, host["draft_tok"], host["draft_q"], host["uniforms"], w.tau,
-                             out=hout, gate_source=gate_source, fallback=fallback, w_scale=w_scale)
+                             out=hout, gate_source=gate_source, fallback=fallback, w_scale=w_scale, a8=a8)
 
     for _ in range(3):
         e2e_step()
@@ -302,12 +305,14 @@ def main():
 
     if rank == 0:
         peaks, peak_kind = load_peaks()
-        work = algorithmic_work(w, 1 if args.weights == "int8" else 2)
+        work = algorithmic_work(w, 2 if args.weights == "bf16" else 1)
         t_mem = work["gemm_bytes"] / (peaks["hbm_gbs"] * 1e9)
-        t_flop = work["flops"] / (peaks["bf16_tflops"] * 1e12)
+        # the 8-bit tensor-core kinds have twice the nominal rate of bf16: measured bf16 peak x 2 for --weights w8a8
+        tensor_peak = peaks["bf16_tflops"] * (2.0 if a8 else 1.0)
+        t_flop = work["flops"] / (tensor_peak * 1e12)
         t_k1 = k1_ms * 1e-3 * plan["passes"]
         if t_flop >= t_mem:
-            roof = {"bound": "tensor", "achieved": work["flops"] / t_k1 / 1e12, "peak": peaks["bf16_tflops"],
+            roof = {"bound": "tensor", "achieved": work["flops"] / t_k1 / 1e12, "peak": tensor_peak,
                     "unit": "TFLOP/s"}
         else:
             roof = {"bound": "hbm", "achieved": work["gemm_bytes"] / t_k1 / 1e9, "peak": peaks["hbm_gbs"],
@@ -322,12 +327,13 @@ def main():
                      "accept_sample_ms": k3_ms})
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms_max / args.steps, "higher_is_better": True,
-                "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "scaling": "weak", "vs_baseline": None, "dtype": "int8" if a8 else "bf16", "data": "synthetic",
                 "config": config_block(w, {"plan": plan, "parallelism": f"replicas x{world}", "gate": args.gate,
                                            "fallback": args.fallback, "weights": args.weights}),
                 "clocks": clocks,
                 "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-                "gpu_launches": (plan["kernels_per_call"] + (1 if gate_source and w.k > 0 else 0)) * args.steps,
+                "gpu_launches": (plan["kernels_per_call"] + (1 if gate_source and w.k > 0 else 0) + (1 if a8 else 0))
+                * args.steps,
                 "accepted_tokens_per_s": accepted_all * args.steps / (ms_max * 1e-3),
                 "roofline": roof}
         if world == 1 and not args.no_cpu_baseline:

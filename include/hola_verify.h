@@ -62,7 +62,13 @@ typedef enum {
  * section; the paper leaves the quantiser's format open): int8 [V][H] plus one fp32 scale per vocabulary row,
  * W8[v][h] = w_scale[v] * q[v][h].  The weights are streamed at half the bytes, expanded exactly to bf16 on chip, and
  * the scale multiplies the fp32 accumulators.  At most 256 verify rows go into one pass over W_lm in this mode. */
-typedef enum { HOLA_W_BF16 = 0, HOLA_W_INT8 = 1 } hola_w_dtype;
+typedef enum {
+  HOLA_W_BF16 = 0,
+  HOLA_W_INT8 = 1, /* int8 weights, bf16 activations: the weights are expanded exactly on chip (W8A16)             */
+  HOLA_W8A8 = 2    /* int8 weights AND the hidden rows quantised the same way (one fp32 scale per verify row) by the
+                    * library on the fly; products on the 8-bit tensor-core kind with exact int32 accumulation:
+                    * l[r][v] = w_scale[v] * h_scale[r] * sum_h q_hid[r][h] * q_w[v][h].  Needs a context. */
+} hola_w_dtype;
 
 /* Bits of the device status word (OR-ed by the kernels; the caller clears it). */
 #define HOLA_FLAG_BAD_TOKEN 1u   /* a draft token outside [0,V): treated as a rejection at that position    */
@@ -91,9 +97,9 @@ typedef struct {
   int32_t gate_source;     /* hola_gate_source; 0 (zero-initialised struct) = target entropy                   */
   int32_t fallback;        /* hola_fallback; 0 = speculative sampling.  With GREEDY the uniforms are not read  */
   float* draft_entropy;    /* out fp32 [B][k], optional: H(q_j), written when gate_source = DRAFT_ENTROPY       */
-  int32_t w_dtype;         /* hola_w_dtype; 0 = W_lm is bf16.  INT8: W_lm is int8 [V][H], H % 16 == 0             */
+  int32_t w_dtype;         /* hola_w_dtype; 0 = W_lm is bf16.  INT8 / W8A8: W_lm is int8 [V][H], H % 16 == 0      */
   int32_t reserved_;       /* must be 0                                                                        */
-  const float* w_scale;    /* fp32 [V], required with HOLA_W_INT8: scale of each vocabulary row                */
+  const float* w_scale;    /* fp32 [V], required with HOLA_W_INT8 / HOLA_W8A8: scale of each vocabulary row    */
 } hola_verify_args;
 
 /* Creates a context on `device` able to serve calls with B <= maxB, k <= maxK and exactly this H and V.

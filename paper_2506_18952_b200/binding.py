@@ -17,7 +17,7 @@ HOLA_OK = 0
 HOLA_Q_BF16, HOLA_Q_F32 = 0, 1
 HOLA_GATE_TARGET_ENTROPY, HOLA_GATE_DRAFT_ENTROPY = 0, 1
 HOLA_FALLBACK_SAMPLE, HOLA_FALLBACK_GREEDY = 0, 1
-HOLA_W_BF16, HOLA_W_INT8 = 0, 1
+HOLA_W_BF16, HOLA_W_INT8, HOLA_W8A8 = 0, 1, 2
 FLAG_BAD_TOKEN, FLAG_BAD_UNIFORM, FLAG_TIMEOUT, FLAG_R_ZERO = 1, 2, 4, 8
 
 EXPORTS = ["hola_create", "hola_destroy", "hola_workspace_bytes", "hola_verify", "hola_verify_host",
@@ -197,7 +197,8 @@ class HolaVerify:
         return {"lm_head_ms": a.value, "accept_sample_ms": b.value, "calls": n.value}
 
     def _args(self, hidden, W_lm, draft_tok, draft_q, uniforms, tau, out: VerifyOutputs, B, k,
-              gate_source: int = HOLA_GATE_TARGET_ENTROPY, fallback: int = HOLA_FALLBACK_SAMPLE, w_scale=None):
+              gate_source: int = HOLA_GATE_TARGET_ENTROPY, fallback: int = HOLA_FALLBACK_SAMPLE, w_scale=None,
+              a8: bool = False):
         if hidden.dtype != torch.bfloat16 or W_lm.dtype not in (torch.bfloat16, torch.int8):
             raise HolaError("hidden must be bfloat16, W_lm bfloat16 or int8")
         if (W_lm.dtype == torch.int8) != (w_scale is not None):
@@ -221,7 +222,9 @@ class HolaVerify:
         a.status_word = _dptr(out.status)
         a.gate_source, a.fallback = int(gate_source), int(fallback)
         a.draft_entropy = _dptr(out.draft_entropy)
-        a.w_dtype = HOLA_W_INT8 if w_scale is not None else HOLA_W_BF16
+        if a8 and w_scale is None:
+            raise HolaError("8-bit activations (a8) go with an int8 W_lm and its scales")
+        a.w_dtype = (HOLA_W8A8 if a8 else HOLA_W_INT8) if w_scale is not None else HOLA_W_BF16
         a.w_scale = _dptr(w_scale)
         return a
 
@@ -238,20 +241,21 @@ class HolaVerify:
 
     def hola_verify(self, hidden, W_lm, draft_tok, draft_q, uniforms, tau, out: VerifyOutputs | None = None,
                     want_logits: bool = False, stream=None, gate_source: int = HOLA_GATE_TARGET_ENTROPY,
-                    fallback: int = HOLA_FALLBACK_SAMPLE, w_scale=None) -> VerifyOutputs:
+                    fallback: int = HOLA_FALLBACK_SAMPLE, w_scale=None, a8: bool = False) -> VerifyOutputs:
         """The whole verify step on device tensors, asynchronous on the stream.  With w_scale, W_lm is the int8 form
-        made by hola_quantize_w8."""
+        made by hola_quantize_w8; with a8 as well, the hidden rows are quantised on the fly and the products run on
+        the 8-bit tensor-core kind."""
         B, k = hidden.shape[0], hidden.shape[1] - 1
         out = out or self.alloc_outputs(B, k, want_logits)
-        a = self._args(hidden, W_lm, draft_tok, draft_q, uniforms, tau, out, B, k, gate_source, fallback, w_scale)
+        a = self._args(hidden, W_lm, draft_tok, draft_q, uniforms, tau, out, B, k, gate_source, fallback, w_scale, a8)
         _check(self.lib, self._ctx, self.lib.hola_verify(self._ctx, ctypes.byref(a), _stream_ptr(stream)), "hola_verify")
         return out
 
     def hola_lm_head_entropy(self, hidden, W_lm, out: VerifyOutputs | None = None, want_logits: bool = True,
-                             stream=None, w_scale=None) -> VerifyOutputs:
+                             stream=None, w_scale=None, a8: bool = False) -> VerifyOutputs:
         B, k = hidden.shape[0], hidden.shape[1] - 1
         out = out or self.alloc_outputs(B, k, want_logits)
-        a = self._args(hidden, W_lm, None, None, None, 0.0, out, B, k, w_scale=w_scale)
+        a = self._args(hidden, W_lm, None, None, None, 0.0, out, B, k, w_scale=w_scale, a8=a8)
         _check(self.lib, self._ctx, self.lib.hola_lm_head_entropy(self._ctx, ctypes.byref(a), _stream_ptr(stream)),
                "hola_lm_head_entropy")
         return out
@@ -277,7 +281,7 @@ class HolaVerify:
 
     def hola_verify_host(self, hidden, W_lm, draft_tok, draft_q, uniforms, tau, out: VerifyOutputs | None = None,
                          stream=None, gate_source: int = HOLA_GATE_TARGET_ENTROPY,
-                         fallback: int = HOLA_FALLBACK_SAMPLE, w_scale=None) -> VerifyOutputs:
+                         fallback: int = HOLA_FALLBACK_SAMPLE, w_scale=None, a8: bool = False) -> VerifyOutputs:
         """End-to-end form: per-step inputs and all outputs are HOST tensors (pinned for async copies);
         W_lm is the resident device weight.  Returns after the stream has been synchronised."""
         B, k = hidden.shape[0], hidden.shape[1] - 1
@@ -287,7 +291,7 @@ class HolaVerify:
             if t is not None and t.device.type != "cpu":
                 raise HolaError("hola_verify_host takes host tensors for the per-step inputs")
         out = out or self.alloc_outputs(B, k, False, device=torch.device("cpu"))
-        a = self._args(hidden, W_lm, draft_tok, draft_q, uniforms, tau, out, B, k, gate_source, fallback, w_scale)
+        a = self._args(hidden, W_lm, draft_tok, draft_q, uniforms, tau, out, B, k, gate_source, fallback, w_scale, a8)
         a.logits_out = None
         _check(self.lib, self._ctx, self.lib.hola_verify_host(self._ctx, ctypes.byref(a), _stream_ptr(stream)),
                "hola_verify_host")

@@ -92,6 +92,7 @@ struct K1Params {
   int ldl;        // row pitch of the logits buffer, in floats
   int vec_ok;     // 16-byte loads of the logits buffer allowed (pitch and base aligned)
   const float* w_scale;   // 8-bit W_lm: fp32 scale per vocabulary row, applied to the accumulators
+  const float* h_scale;   // 8-bit activations (mode 2): fp32 scale per verify row
   float* logits;
   float4* partials;   // [grid][part_stride] (m, s, t, arg-max index)
   int part_stride;
@@ -238,15 +239,25 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
   asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
 }
 
-// D[tmem of both CTAs] (+)= A[smem of both CTAs] * B[smem of both CTAs]^T, bf16 inputs, fp32 accumulate.
+// D[tmem of both CTAs] (+)= A[smem of both CTAs] * B[smem of both CTAs]^T.  bf16 inputs with fp32 accumulation
+// (K = 16 per instruction) or, with kInt8, signed 8-bit inputs with int32 accumulation (K = 32 per instruction).
 // Issued by one thread of the pair's leader CTA; descriptors are shared-memory offsets valid in both CTAs.
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                          uint32_t accumulate) {
-  asm volatile(
-      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
-      " tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}"
-      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-      : "memory");
+template <bool kInt8>
+__device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                     uint32_t accumulate) {
+  if (kInt8) {
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+        " tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+  } else {
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+        " tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+  }
 }
 // The mbarrier at this shared-memory offset in BOTH CTAs of the pair gets one arrival once every MMA issued so far
 // by this thread has completed.
@@ -296,6 +307,10 @@ __device__ __forceinline__ uint64_t make_kmajor_sw128_desc(uint32_t smem_addr) {
 // Instruction descriptor, kind::f16: D fp32, A and B bf16, both K-major, M = 256 (the pair), N = n.
 __device__ __forceinline__ uint32_t make_idesc_bf16_m256(uint32_t n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((n >> 3) << 17) | ((256u >> 4) << 24);
+}
+// Instruction descriptor, kind::i8: D int32, A and B signed 8-bit, both K-major, M = 256, N = n (multiple of 32).
+__device__ __forceinline__ uint32_t make_idesc_s8_m256(uint32_t n) {
+  return (2u << 4) | (1u << 7) | (1u << 10) | ((n >> 3) << 17) | ((256u >> 4) << 24);
 }
 
 // ------------------------------------------------------------------------------------------------ softmax statistics
@@ -383,6 +398,16 @@ __device__ __forceinline__ void expand_int8x16(const uint4 x, uint8_t* tile, int
   *reinterpret_cast<uint4*>(drow + (((2 * c + 1) ^ (row & 7)) << 4)) = make_uint4(o[4], o[5], o[6], o[7]);
 }
 
+// One accumulator on its way to the logits buffer.  Mode 0: as is.  Mode 1: times the scale of the vocabulary row.
+// Mode 2: the accumulator is an int32 (bit pattern in `acc`); times the scales of the vocabulary row and of the
+// verify row.
+template <int kMode>
+__device__ __forceinline__ float scaled(float acc, float w_scale, const float* h_scale, int row) {
+  if (kMode == 1) return acc * w_scale;
+  if (kMode == 2) return static_cast<float>(__float_as_int(acc)) * (w_scale * h_scale[row]);
+  return acc;
+}
+
 // ------------------------------------------------------------------------------------------------ K1
 // Shared memory: `stages` ring slots of [W_lm block 128 x 64 | hidden block(s) n_sub x (N/2) x 64], then the
 // barrier area.  Barriers (8 bytes each, offsets in the barrier area):
@@ -395,10 +420,15 @@ __device__ __forceinline__ void expand_int8x16(const uint4 x, uint8_t* tile, int
 //   tensor-memory base @256, abort flag @260
 //   8-bit W_lm only: rawfull[12] @272 per CTA: the int8 tile of the slot has landed; rawempty[12] @368 per CTA: the
 //   converter warps have expanded it.  full[] then collects, besides the hidden bytes, one arrival per converter warp.
-template <bool kW8>
+// kMode: 0 bf16 x bf16; 1 int8 W_lm expanded to bf16 on chip (exact); 2 int8 W_lm x int8 hidden on the 8-bit MMA
+// kind (K blocks of 128 elements, so that a block is 128 bytes per row exactly as in mode 0; int32 accumulators).
+template <int kMode>
 __global__ void __launch_bounds__(kK1Threads, 1)
 lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __grid_constant__ CUtensorMap tmap_w,
                        const K1Params p) {
+  constexpr bool kW8 = kMode == 1;
+  constexpr bool kI8 = kMode == 2;
+  constexpr int kKStep = kI8 ? 2 * kBlockK : kBlockK;    // elements of K per ring slot
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;          // 128-byte swizzle wants 1024-byte aligned tiles
@@ -469,7 +499,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
       for (int t = 0; t < my_tiles && ok; ++t) {
         const int v0 = (pair + t * npairs) * pair_rows + static_cast<int>(rank) * p.tile_rows;
         int kx = 0;                                      // K coordinate of the block, in elements
-        for (int kb = 0; kb < p.n_kblocks; ++kb, kx += kBlockK) {
+        for (int kb = 0; kb < p.n_kblocks; ++kb, kx += kKStep) {
           const uint32_t sa = base + stage * stage_bytes;
           if (kW8) {
             // only the int8 tile: its slot is free again as soon as the converters have read it
@@ -493,7 +523,8 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (leader CTA only)
     if (rank == 0 && elect_one()) {
-      const uint32_t idesc = make_idesc_bf16_m256(static_cast<uint32_t>(p.N));
+      const uint32_t idesc = kI8 ? make_idesc_s8_m256(static_cast<uint32_t>(p.N))
+                                 : make_idesc_bf16_m256(static_cast<uint32_t>(p.N));
       const uint64_t desc0 = make_kmajor_sw128_desc(base);
       const bool two_mmas = p.n_sub == 2;
       int stage = 0;
@@ -515,17 +546,17 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
           // 16 bf16 = 32 bytes further along K inside the swizzled row: +2 in 16-byte address units
           if (two_mmas) {
             const uint64_t bdesc1 = bdesc0 + (hid_block_bytes >> 4);
-            umma_bf16(d0, adesc, bdesc0, idesc, acc);
-            umma_bf16(d0 + 256, adesc, bdesc1, idesc, acc);
+            umma<kI8>(d0, adesc, bdesc0, idesc, acc);
+            umma<kI8>(d0 + 256, adesc, bdesc1, idesc, acc);
 #pragma unroll
             for (int kk = 1; kk < kBlockK / 16; ++kk) {
-              umma_bf16(d0, adesc + 2 * kk, bdesc0 + 2 * kk, idesc, 1u);
-              umma_bf16(d0 + 256, adesc + 2 * kk, bdesc1 + 2 * kk, idesc, 1u);
+              umma<kI8>(d0, adesc + 2 * kk, bdesc0 + 2 * kk, idesc, 1u);
+              umma<kI8>(d0 + 256, adesc + 2 * kk, bdesc1 + 2 * kk, idesc, 1u);
             }
           } else {
-            umma_bf16(d0, adesc, bdesc0, idesc, acc);
+            umma<kI8>(d0, adesc, bdesc0, idesc, acc);
 #pragma unroll
-            for (int kk = 1; kk < kBlockK / 16; ++kk) umma_bf16(d0, adesc + 2 * kk, bdesc0 + 2 * kk, idesc, 1u);
+            for (int kk = 1; kk < kBlockK / 16; ++kk) umma<kI8>(d0, adesc + 2 * kk, bdesc0 + 2 * kk, idesc, 1u);
           }
           umma_commit_pair(empty_bar + 8 * stage);       // frees the slot in both CTAs once these MMAs have read it
           if (++stage == p.stages) { stage = 0; phase ^= 1u; }
@@ -550,7 +581,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
       const int tile_lane = quarter * 32 + lane;         // lanes at or beyond tile_rows hold nothing
       const int vocab = (pair + t * npairs) * pair_rows + static_cast<int>(rank) * p.tile_rows + tile_lane;
       const bool vocab_ok = tile_lane < p.tile_rows && vocab < p.V;
-      const float w_scale = (kW8 && vocab_ok) ? p.w_scale[vocab] : 1.f;    // 8-bit W_lm: the row's scale
+      const float w_scale = ((kW8 || kI8) && vocab_ok) ? p.w_scale[vocab] : 1.f;   // 8-bit W_lm: the row's scale
       const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * 256;
       for (int ch = group; ch < n_chunks; ch += kChunkStep) {
         const int s = ch / sub_chunks, j = ch - s * sub_chunks;
@@ -565,11 +596,11 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
           float* dst = p.logits + static_cast<size_t>(r0) * p.ldl + vocab;
           if (n_ok == 32) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) dst[static_cast<size_t>(i) * p.ldl] = kW8 ? v[i] * w_scale : v[i];
+            for (int i = 0; i < 32; ++i) dst[static_cast<size_t>(i) * p.ldl] = scaled<kMode>(v[i], w_scale, p.h_scale, r0 + i);
           } else {
 #pragma unroll
             for (int i = 0; i < 32; ++i)
-              if (i < n_ok) dst[static_cast<size_t>(i) * p.ldl] = kW8 ? v[i] * w_scale : v[i];
+              if (i < n_ok) dst[static_cast<size_t>(i) * p.ldl] = scaled<kMode>(v[i], w_scale, p.h_scale, r0 + i);
           }
         }
       }
@@ -661,7 +692,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
       bool ok = true;
       for (int t = 0; t < my_tiles && ok; ++t) {
         int kx = 0;
-        for (int kb = 0; kb < p.n_kblocks; ++kb, kx += kBlockK) {
+        for (int kb = 0; kb < p.n_kblocks; ++kb, kx += kKStep) {
           if (!mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
           const uint32_t sa = base + stage * stage_bytes;
           const uint32_t fb = leader_full + 8 * stage;
@@ -1172,6 +1203,8 @@ struct hola_ctx {
   float4* partials;         // [num_sms][max_rows]
   unsigned* status;         // [1]
   double* hq;               // [max_rows][kHqSlices] slice sums of q ln q over the draft rows
+  signed char* hid8;        // [max_rows][H] int8 hidden rows (8-bit activation mode)
+  float* hid_scale;         // [max_rows]
   // staging for hola_verify_host
   void* st_hidden; int* st_tok; void* st_q; float* st_u;
   int* st_accept; int* st_next; float* st_entropy; float* st_logZ;
@@ -1190,7 +1223,7 @@ namespace {
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WsLayout {
-  size_t logits, partials, status, hq, st_hidden, st_tok, st_q, st_u, st_accept, st_next, st_entropy, st_logZ, total;
+  size_t logits, partials, status, hq, hid8, hid_scale, st_hidden, st_tok, st_q, st_u, st_accept, st_next, st_entropy, st_logZ, total;
 };
 
 WsLayout ws_layout(int maxB, int maxK, int H, int V, int num_sms) {
@@ -1203,6 +1236,8 @@ WsLayout ws_layout(int maxB, int maxK, int H, int V, int num_sms) {
   w.partials = take(static_cast<size_t>(num_sms) * rows * 16);
   w.status = take(4);
   w.hq = take(rows * kHqSlices * 8);
+  w.hid8 = take(rows * static_cast<size_t>(H));
+  w.hid_scale = take(rows * 4);
   w.st_hidden = take(rows * H * 2);
   w.st_tok = take(static_cast<size_t>(maxB) * maxK * 4);
   w.st_q = take(static_cast<size_t>(maxB) * maxK * V * 4);
@@ -1226,19 +1261,21 @@ int round_up(int x, int a) { return (x + a - 1) / a * a; }
 // Splits M verify rows into passes over W_lm and each pass into one or two MMAs per K step.
 // A pass holds at most 512 rows (two MMAs of N <= 256 fill the tensor memory); N is a multiple of 16.
 // Cost per pass: the slower of streaming W_lm once and the padded rows' tensor time, plus a fixed launch cost.
-Plan make_plan(const hola_ctx* ctx, int M, bool w8 = false) {
+Plan make_plan(const hola_ctx* ctx, int M, int w_dtype = HOLA_W_BF16) {
+  const bool w8 = w_dtype == HOLA_W_INT8;        // int8 W_lm expanded on chip
+  const bool i8 = w_dtype == HOLA_W8A8;          // 8-bit MMA: N a multiple of 32, K blocks of 128, twice the rate
   Plan best{};
   double best_cost = 1e300;
   const int rows = M > 0 ? M : 1;
   // 8-bit W_lm: one MMA per K step (at most 256 rows per pass), and the slot also holds the int8 block
   const int max_rows_per_pass = w8 ? kMaxN : kMaxRowsPerPass;
   const int p_min = (rows + max_rows_per_pass - 1) / max_rows_per_pass;
-  const double t_hbm = (w8 ? 1.0 : 2.0) * ctx->V * static_cast<double>(ctx->H) / 6.4e12;
+  const double t_hbm = (w8 || i8 ? 1.0 : 2.0) * ctx->V * static_cast<double>(ctx->H) / 6.4e12;
   for (int passes = p_min; passes <= p_min + 3; ++passes) {
     const int r = (rows + passes - 1) / passes;
     const int n_sub = r > kMaxN ? 2 : 1;
-    const int N = round_up((r + n_sub - 1) / n_sub, 16);
-    const double t_mma = 2.0 * n_sub * N * static_cast<double>(ctx->V) * ctx->H / 1.4e15;
+    const int N = round_up((r + n_sub - 1) / n_sub, i8 ? 32 : 16);
+    const double t_mma = 2.0 * n_sub * N * static_cast<double>(ctx->V) * ctx->H / (i8 ? 2.8e15 : 1.4e15);
     const double cost = passes * ((t_mma > t_hbm ? t_mma : t_hbm) + 6e-6);
     if (cost < best_cost) {
       best_cost = cost;
@@ -1264,22 +1301,23 @@ Plan make_plan(const hola_ctx* ctx, int M, bool w8 = false) {
   best.tile_rows = tile_rows;
   best.n_ptiles = (ctx->V + 2 * tile_rows - 1) / (2 * tile_rows);
   best.grid = 2 * (best.n_ptiles < pairs ? best.n_ptiles : pairs);
-  best.n_kblocks = (ctx->H + kBlockK - 1) / kBlockK;
+  best.n_kblocks = i8 ? (ctx->H + 2 * kBlockK - 1) / (2 * kBlockK) : (ctx->H + kBlockK - 1) / kBlockK;
   best.smem_bytes = stages * stage_bytes + kBarrierBytes + 1024;
   return best;
 }
 
 // K-major 2-D tensor map with a box of 64 elements x box_rows.  bf16: 128-byte swizzle (the layout the MMA reads);
 // int8: plain rows of 64 bytes (the converter warps read them).
+// int8 with swizzle (8-bit MMA): box of 128 elements = 128 bytes, 128-byte swizzle, the same bytes as a bf16 block.
 hola_status encode_map(hola_ctx* ctx, CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols,
-                       uint32_t box_rows, bool int8 = false) {
+                       uint32_t box_rows, bool int8 = false, bool int8_swizzled = false) {
   const cuuint64_t dims[2] = {cols, rows};
   const cuuint64_t strides[1] = {cols * (int8 ? 1u : 2u)};
-  const cuuint32_t box[2] = {static_cast<cuuint32_t>(kBlockK), box_rows};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(int8_swizzled ? 2 * kBlockK : kBlockK), box_rows};
   const cuuint32_t estr[2] = {1, 1};
   const CUresult r = ctx->encode(map, int8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
                                  const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                                 int8 ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
+                                 (int8 && !int8_swizzled) ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
                                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
     snprintf(ctx->last_error, sizeof ctx->last_error, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
@@ -1305,13 +1343,24 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 hola_status run_lm_head(hola_ctx* ctx, const hola_verify_args* a, float* logits, int ldl, const Plan& pl,
                         cudaStream_t stream) {
   const int M = a->B * (a->k + 1);
+  const bool w8 = a->w_dtype == HOLA_W_INT8, i8 = a->w_dtype == HOLA_W8A8;
   CUtensorMap th, tw;
-  hola_status s = encode_map(ctx, &th, a->hidden, static_cast<uint64_t>(M), static_cast<uint64_t>(a->H),
-                             static_cast<uint32_t>(pl.N / 2));
+  hola_status s;
+  if (i8) {
+    // 8-bit activations: the same per-row quantiser as for W_lm, into the context's workspace
+    if (!ctx->hid8) return HOLA_ERR_INVALID_ARG;          // (the entry point without a context has no room for it)
+    quantize_rows_int8_kernel<<<static_cast<unsigned>(M), 256, 0, stream>>>(
+        static_cast<const __nv_bfloat16*>(a->hidden), a->H, ctx->hid8, ctx->hid_scale);
+    if (cudaGetLastError() != cudaSuccess) return HOLA_ERR_CUDA;
+    s = encode_map(ctx, &th, ctx->hid8, static_cast<uint64_t>(M), static_cast<uint64_t>(a->H),
+                   static_cast<uint32_t>(pl.N / 2), true, true);
+  } else {
+    s = encode_map(ctx, &th, a->hidden, static_cast<uint64_t>(M), static_cast<uint64_t>(a->H),
+                   static_cast<uint32_t>(pl.N / 2));
+  }
   if (s != HOLA_OK) return s;
-  const bool w8 = a->w_dtype == HOLA_W_INT8;
   s = encode_map(ctx, &tw, a->W_lm, static_cast<uint64_t>(a->V), static_cast<uint64_t>(a->H),
-                 static_cast<uint32_t>(pl.tile_rows), w8);
+                 static_cast<uint32_t>(pl.tile_rows), w8 || i8, i8);
   if (s != HOLA_OK) return s;
   K1Params kp;
   kp.M = M; kp.V = a->V; kp.n_ptiles = pl.n_ptiles; kp.n_kblocks = pl.n_kblocks;
@@ -1320,10 +1369,13 @@ hola_status run_lm_head(hola_ctx* ctx, const hola_verify_args* a, float* logits,
   kp.logits = logits; kp.partials = ctx->partials; kp.part_stride = ctx->max_rows;
   kp.status = a->status_word ? a->status_word : ctx->status;
   kp.w_scale = a->w_scale;
-  cudaError_t e = w8 ? cudaFuncSetAttribute(lm_head_entropy_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  kp.h_scale = ctx->hid_scale;
+  cudaError_t e = i8 ? cudaFuncSetAttribute(lm_head_entropy_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             pl.smem_bytes)
-                     : cudaFuncSetAttribute(lm_head_entropy_kernel<false>,
-                                            cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem_bytes);
+                : w8 ? cudaFuncSetAttribute(lm_head_entropy_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            pl.smem_bytes)
+                     : cudaFuncSetAttribute(lm_head_entropy_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            pl.smem_bytes);
   if (e != cudaSuccess) { set_error(ctx, "cudaFuncSetAttribute", e); return HOLA_ERR_CUDA; }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(static_cast<unsigned>(pl.grid));
@@ -1341,8 +1393,9 @@ hola_status run_lm_head(hola_ctx* ctx, const hola_verify_args* a, float* logits,
     kp.row0 = pass * pl.rows_per_pass;
     kp.rows = M - kp.row0 < pl.rows_per_pass ? M - kp.row0 : pl.rows_per_pass;
     if (kp.rows <= 0) break;
-    e = w8 ? cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<true>, th, tw, kp)
-           : cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<false>, th, tw, kp);
+    e = i8 ? cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<2>, th, tw, kp)
+      : w8 ? cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<1>, th, tw, kp)
+           : cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<0>, th, tw, kp);
     if (e != cudaSuccess) { set_error(ctx, "launch lm_head_entropy_kernel", e); return HOLA_ERR_CUDA; }
   }
   return HOLA_OK;
@@ -1393,8 +1446,8 @@ hola_status check_lm_head_args(const hola_ctx* ctx, const hola_verify_args* a) {
   if (!a->hidden || !a->W_lm) return HOLA_ERR_INVALID_ARG;
   if (!aligned16(a->hidden) || !aligned16(a->W_lm)) return HOLA_ERR_INVALID_ARG;
   if (a->H % 8 != 0) return HOLA_ERR_UNSUPPORTED_SHAPE;
-  if (a->w_dtype != HOLA_W_BF16 && a->w_dtype != HOLA_W_INT8) return HOLA_ERR_INVALID_ARG;
-  if (a->w_dtype == HOLA_W_INT8) {
+  if (a->w_dtype != HOLA_W_BF16 && a->w_dtype != HOLA_W_INT8 && a->w_dtype != HOLA_W8A8) return HOLA_ERR_INVALID_ARG;
+  if (a->w_dtype != HOLA_W_BF16) {
     if (!a->w_scale) return HOLA_ERR_INVALID_ARG;
     if (a->H % 16 != 0) return HOLA_ERR_UNSUPPORTED_SHAPE;     // int8 row pitch must be a multiple of 16 bytes
   }
@@ -1485,6 +1538,8 @@ hola_status hola_create(hola_ctx** out, int device, int maxB, int maxK, int H, i
   ctx->partials = reinterpret_cast<float4*>(ctx->ws + w.partials);
   ctx->status = reinterpret_cast<unsigned*>(ctx->ws + w.status);
   ctx->hq = reinterpret_cast<double*>(ctx->ws + w.hq);
+  ctx->hid8 = reinterpret_cast<signed char*>(ctx->ws + w.hid8);
+  ctx->hid_scale = reinterpret_cast<float*>(ctx->ws + w.hid_scale);
   ctx->st_hidden = ctx->ws + w.st_hidden; ctx->st_tok = reinterpret_cast<int*>(ctx->ws + w.st_tok);
   ctx->st_q = ctx->ws + w.st_q; ctx->st_u = reinterpret_cast<float*>(ctx->ws + w.st_u);
   ctx->st_accept = reinterpret_cast<int*>(ctx->ws + w.st_accept);
@@ -1517,9 +1572,9 @@ hola_status hola_destroy(hola_ctx* ctx) {
 
 hola_status hola_plan_ex(const hola_ctx* ctx, int B, int k, int w_dtype, hola_plan_info* out) {
   if (!ctx || !out || B < 0 || k < 0) return HOLA_ERR_INVALID_ARG;
-  if (w_dtype != HOLA_W_BF16 && w_dtype != HOLA_W_INT8) return HOLA_ERR_INVALID_ARG;
+  if (w_dtype != HOLA_W_BF16 && w_dtype != HOLA_W_INT8 && w_dtype != HOLA_W8A8) return HOLA_ERR_INVALID_ARG;
   if (B > ctx->maxB || k > ctx->maxK) return HOLA_ERR_UNSUPPORTED_SHAPE;
-  const Plan pl = make_plan(ctx, B * (k + 1), w_dtype == HOLA_W_INT8);
+  const Plan pl = make_plan(ctx, B * (k + 1), w_dtype);
   out->tile_v = 2 * pl.tile_rows; out->grid = pl.grid; out->stages = pl.stages; out->rows_per_pass = pl.rows_per_pass;
   out->passes = pl.passes; out->kernels_per_call = pl.passes + 1;
   return HOLA_OK;
@@ -1538,7 +1593,7 @@ hola_status hola_lm_head_entropy(hola_ctx* ctx, const hola_verify_args* a, void*
   DeviceGuard guard(ctx->device);
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   const int M = a->B * (a->k + 1);
-  const Plan pl = make_plan(ctx, M, a->w_dtype == HOLA_W_INT8);
+  const Plan pl = make_plan(ctx, M, a->w_dtype);
   float* logits = a->logits_out ? a->logits_out : ctx->logits;
   const int ldl = a->logits_out ? a->V : ctx->ldl;
   if ((s = run_lm_head(ctx, a, logits, ldl, pl, stream)) != HOLA_OK) return s;
@@ -1566,7 +1621,7 @@ namespace {
 // The whole step on device buffers.  `before_sample`, when given, is an event the accept/sample part waits for
 // (the draft tensor still being copied in by hola_verify_host).
 hola_status verify_device(hola_ctx* ctx, const hola_verify_args* a, cudaStream_t stream, cudaEvent_t before_sample) {
-  const Plan pl = make_plan(ctx, a->B * (a->k + 1), a->w_dtype == HOLA_W_INT8);
+  const Plan pl = make_plan(ctx, a->B * (a->k + 1), a->w_dtype);
   float* logits = a->logits_out ? a->logits_out : ctx->logits;
   const int ldl = a->logits_out ? a->V : ctx->ldl;
   const bool prof = ctx->prof_on && ctx->prof_n < ctx->prof_cap;
@@ -1770,7 +1825,7 @@ extern "C" hola_status hola_lm_head_entropy_static(const hola_verify_args* a, vo
   const int M = static_cast<int>(rows);
   if (a->w_dtype != HOLA_W_BF16 && a->w_dtype != HOLA_W_INT8) return HOLA_ERR_INVALID_ARG;
   if (a->w_dtype == HOLA_W_INT8 && (!a->w_scale || a->H % 16 != 0)) return HOLA_ERR_INVALID_ARG;
-  const Plan pl = make_plan(&local, M, a->w_dtype == HOLA_W_INT8);
+  const Plan pl = make_plan(&local, M, a->w_dtype);
   if (pl.grid > kStaticMaxCtas) return HOLA_ERR_STATIC_LIMIT;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   // The array keeps whatever the last call left.  The statistics slots are fully overwritten for the rows of this

@@ -351,10 +351,15 @@ def test_host_entry_equals_device_entry(binding):
 
 
 # ------------------------------------------------------------------------------------------ 8-bit LM head
-def _w8_oracle(w, q8, scale, **kw):
-    """The oracle on the dequantised head: hidden widened to fp64, W8 = scale * q in fp64."""
+def _w8_oracle(w, q8, scale, a8=False, **kw):
+    """The oracle on the dequantised head: hidden widened to fp64 (or, with a8, quantised row by row with the same
+    rule and dequantised), W8 = scale * q in fp64."""
     from oracle import lobi
     hid = ref.bf16_bits_to_f64(_np(w.hidden))
+    if a8:
+        B, k1, H = hid.shape
+        hq, hs = lobi.quantize_rows_int8(hid.reshape(B * k1, H).astype(np.float32))
+        hid = lobi.dequantize_rows(hq, hs).reshape(B, k1, H)
     W8 = lobi.dequantize_rows(_np(q8), _np(scale))
     return ref.verify(hid, W8, _np(w.draft_tok), _np(w.draft_q), _np(w.uniforms), w.tau, keep_logits=True, **kw)
 
@@ -398,6 +403,64 @@ def test_int8_head_matches_oracle_on_dequantised_weights(binding, B, k, H, V, qd
     # and the quantised head stays close to the bf16 head it came from
     full = compare.run_oracle(w, keep_logits=False)
     assert np.max(np.abs(orc.entropy - full.entropy)) < 0.25
+
+
+@pytest.mark.parametrize("B,k,H,V,qd", [
+    (1, 4, 64, 1000, torch.float32),       # 5 rows: N = 32
+    (37, 6, 256, 5000, torch.bfloat16),    # 259 rows: two MMAs of N = 160 per K step, ragged vocabulary tail
+    (5, 2, 80, 1001, torch.bfloat16),      # K tail (H = 80 < one 128-wide block), odd V
+    (90, 7, 384, 640, torch.float32),      # 720 rows: two passes
+])
+def test_w8a8_head_matches_oracle_on_dequantised_operands(binding, B, k, H, V, qd):
+    w = workloads.gaussian_head("w8a8", B, k, H, V, seed=B + V, device=DEV, w_std=0.3, sigma=1.0, q_dtype=qd,
+                                tau=1.5 + 0.1 * k, sigma_far=0.2)
+    q8, scale = binding.hola_quantize_w8(w.W_lm)
+    with binding.HolaVerify(B, k, H, V) as ctx:
+        out = ctx.hola_verify(w.hidden, q8, w.draft_tok, w.draft_q, w.uniforms, w.tau, want_logits=True, w_scale=scale,
+                              a8=True)
+        torch.cuda.synchronize()
+    assert int(out.status.item()) & binding.FLAG_TIMEOUT == 0
+    orc = _w8_oracle(w, q8, scale, a8=True)
+    rep = compare.compare(orc, _np(w.draft_q), _np(w.uniforms), _np(out.accept_len), _np(out.next_tok),
+                          _np(out.entropy), _np(out.logZ), _np(out.logits))
+    print(rep.summary())
+    assert rep.ok, rep.summary()
+    assert rep.accept_margin_cases <= max(1, B // 20) and rep.token_margin_cases <= max(1, B // 10)
+    check_ranges(w, out)
+
+
+def test_w8a8_integer_operands_are_bit_exact(binding):
+    # integer weights and hidden rows with row maximum 127: both scales are 1, every product and sum is exact
+    g = torch.Generator().manual_seed(10)
+    B, k, H, V = 40, 3, 192, 520
+    hf = torch.randint(-6, 7, (B, k + 1, H), generator=g).float()
+    hf[..., 0] = 127.0
+    Wf = torch.randint(-5, 6, (V, H), generator=g).float()
+    Wf[:, 1] = -127.0
+    hidden, W = hf.bfloat16().to(DEV), Wf.bfloat16().to(DEV)
+    q8, scale = binding.hola_quantize_w8(W)
+    with binding.HolaVerify(B, k, H, V) as ctx:
+        out = ctx.hola_lm_head_entropy(hidden, q8, want_logits=True, w_scale=scale, a8=True)
+        torch.cuda.synchronize()
+    want = ref.logits(_np(hidden).reshape(-1, H), _np(W)).reshape(B, k + 1, V)
+    assert np.array_equal(_np(out.logits).astype(np.float64), want)
+
+
+def test_w8a8_on_the_large_vocabulary_shape(binding):
+    w = workloads.make_config("large_vocab", DEV)
+    q8, scale = binding.hola_quantize_w8(w.W_lm)
+    with binding.HolaVerify(w.B, w.k, w.H, w.V) as ctx:
+        out = ctx.hola_verify(w.hidden, q8, w.draft_tok, w.draft_q, w.uniforms, w.tau, want_logits=True, w_scale=scale,
+                              a8=True)
+        torch.cuda.synchronize()
+    seqs = [1, 22, 63]
+    sub = w.slice(seqs)
+    orc = _w8_oracle(sub, q8, scale, a8=True)
+    idx = np.asarray(seqs)
+    rep = compare.compare(orc, _np(sub.draft_q), _np(sub.uniforms), _np(out.accept_len)[idx], _np(out.next_tok)[idx],
+                          _np(out.entropy)[idx], _np(out.logZ)[idx], _np(out.logits)[idx])
+    assert rep.ok, rep.summary()
+    check_ranges(w, out)
 
 
 def test_int8_head_small_integer_weights_are_bit_exact(binding):
