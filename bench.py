@@ -299,9 +299,11 @@ def main():
     torch.cuda.synchronize()
     e2e_value, _ = hdist.aggregate_throughput(w.M * args.e2e_steps, e0.elapsed_time(e1), dev)
     sampler.stop()
-    h2d = sum(t.numel() * t.element_size() for t in host.values())
-    d2h = sum(getattr(hout, f).numel() * getattr(hout, f).element_size()
-              for f in ("accept_len", "next_tok", "entropy", "logZ", "status"))
+    # bytes the library copied in the last step (every step has the same inputs): counted inside hola_verify_host,
+    # which sends only the rows of the draft tensor that the step reads while the target entropy gates
+    h2d, d2h = ctx.hola_host_traffic()
+    e2e_ms = e0.elapsed_time(e1) / args.e2e_steps
+    host_bytes = sum(t.numel() * t.element_size() for t in host.values())
 
     if rank == 0:
         peaks, peak_kind = load_peaks()
@@ -331,7 +333,8 @@ def main():
                 "config": config_block(w, {"plan": plan, "parallelism": f"replicas x{world}", "gate": args.gate,
                                            "fallback": args.fallback, "weights": args.weights}),
                 "clocks": clocks,
-                "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+                "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                        "ms_per_step": e2e_ms, "host_input_bytes": host_bytes},
                 "gpu_launches": (plan["kernels_per_call"] + (1 if gate_source and w.k > 0 else 0) + (1 if a8 else 0))
                 * args.steps,
                 "accepted_tokens_per_s": accepted_all * args.steps / (ms_max * 1e-3),

@@ -119,9 +119,20 @@ hola_status hola_verify(hola_ctx* ctx, const hola_verify_args* args, void* cuda_
 /* End-to-end form for callers whose per-step data lives in host memory.  Same computation as hola_verify, but
  * hidden, draft_tok, draft_q, uniforms are HOST pointers (pinned memory makes the copies asynchronous) and
  * accept_len, next_tok, entropy, logZ, status_word are HOST outputs; logits_out is ignored.  W_lm stays a
- * DEVICE pointer: weights are resident.  Copies in, runs, copies out and synchronises the stream.  The draft
- * tensor, the largest input, is copied on a stream owned by the context while the LM-head GEMM already runs. */
+ * DEVICE pointer: weights are resident.  Copies in, runs, copies out and synchronises the stream.
+ * While the target entropy gates (gate_source = 0) only the part of draft_q that Algorithm 1's verify step reads
+ * crosses the bus: the k probabilities q_j(x_j) of each sequence, gathered on the host, and the one row q_n that the
+ * residual draw of a sequence needs (none when all k drafts were kept or the fallback is greedy).  The first rows
+ * of every sequence (as many as fit under the LM-head GEMM, at least row 0) are copied ahead on a stream owned by
+ * the context while the GEMM runs; the accept lengths are read back once in the middle of the call and the rows
+ * still missing follow.  Results are identical to hola_verify on the same data.  With the draft-entropy gate every
+ * draft row is read, and for small draft tensors the whole copy hides under the GEMM anyway: then the whole tensor
+ * is copied (on the context's stream, under the GEMM).  The environment variable HOLA_HOST_LAZY_Q (0 / 1, read by
+ * hola_create) forces one or the other.  The host buffers must stay valid until the call returns. */
 hola_status hola_verify_host(hola_ctx* ctx, const hola_verify_args* args, void* cuda_stream);
+
+/* Bytes the last hola_verify_host call on this context copied host-to-device and device-to-host. */
+hola_status hola_host_traffic(const hola_ctx* ctx, unsigned long long* h2d_bytes, unsigned long long* d2h_bytes);
 
 /* Partial entry points, the steps of the path exposed one by one (same argument struct).
  * hola_lm_head_entropy: steps 1-2 only; fills logits (logits_out or scratch), entropy, logZ.

@@ -21,7 +21,7 @@ HOLA_W_BF16, HOLA_W_INT8, HOLA_W8A8 = 0, 1, 2
 FLAG_BAD_TOKEN, FLAG_BAD_UNIFORM, FLAG_TIMEOUT, FLAG_R_ZERO = 1, 2, 4, 8
 
 EXPORTS = ["hola_create", "hola_destroy", "hola_workspace_bytes", "hola_verify", "hola_verify_host",
-           "hola_lm_head_entropy", "hola_accept_sample", "hola_lm_head_entropy_static", "hola_quantize_w8", "hola_plan", "hola_plan_ex", "hola_profile_begin", "hola_profile_end", "hola_strerror", "hola_last_cuda_error",
+           "hola_lm_head_entropy", "hola_accept_sample", "hola_host_traffic", "hola_lm_head_entropy_static", "hola_quantize_w8", "hola_plan", "hola_plan_ex", "hola_profile_begin", "hola_profile_end", "hola_strerror", "hola_last_cuda_error",
            "hola_version"]
 
 
@@ -76,6 +76,9 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
     lib.hola_plan_ex.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.POINTER(hola_plan_info)]
     lib.hola_profile_begin.restype = ctypes.c_int
     lib.hola_profile_begin.argtypes = [ctypes.c_void_p, ctypes.c_int]
+    lib.hola_host_traffic.restype = ctypes.c_int
+    lib.hola_host_traffic.argtypes = [ctypes.c_void_p, ctypes.POINTER(ctypes.c_ulonglong),
+                                      ctypes.POINTER(ctypes.c_ulonglong)]
     lib.hola_profile_end.restype = ctypes.c_int
     lib.hola_profile_end.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(ctypes.c_double),
                                      ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_int)]
@@ -189,6 +192,13 @@ class HolaVerify:
 
     def hola_profile_begin(self, max_calls: int):
         _check(self.lib, self._ctx, self.lib.hola_profile_begin(self._ctx, max_calls), "hola_profile_begin")
+
+    def hola_host_traffic(self) -> tuple[int, int]:
+        """(host-to-device, device-to-host) bytes of the last hola_verify_host call."""
+        up, down = ctypes.c_ulonglong(0), ctypes.c_ulonglong(0)
+        _check(self.lib, self._ctx, self.lib.hola_host_traffic(self._ctx, ctypes.byref(up), ctypes.byref(down)),
+               "hola_host_traffic")
+        return int(up.value), int(down.value)
 
     def hola_profile_end(self, stream=None) -> dict:
         a, b, n = ctypes.c_double(), ctypes.c_double(), ctypes.c_int()

@@ -107,6 +107,8 @@ struct K3Params {
   const int* tok;
   const void* q;
   int q_dtype;
+  const float* q_tok;           // optional fp32 [B][k]: q_j(x_j) already gathered (then q is read at row n only)
+  int phase;                    // 0: the whole step; 1: stop after the accept test (accept_len, statistics written)
   const float* u;
   float tau;
   int gate_source;          // hola_gate_source
@@ -882,8 +884,9 @@ __global__ void __launch_bounds__(kK3Threads) accept_sample_kernel(const K3Param
     if (x >= 0 && x < V) {
       lx = p.logits[static_cast<size_t>(row_first + j) * p.ldl + x];
       const size_t qi = (static_cast<size_t>(b) * k + j) * V + x;
-      qx = (p.q_dtype == HOLA_Q_BF16) ? __bfloat162float(static_cast<const __nv_bfloat16*>(p.q)[qi])
-                                      : static_cast<const float*>(p.q)[qi];
+      if (p.q_tok) qx = p.q_tok[b * k + j];
+      else qx = (p.q_dtype == HOLA_Q_BF16) ? __bfloat162float(static_cast<const __nv_bfloat16*>(p.q)[qi])
+                                           : static_cast<const float*>(p.q)[qi];
     }
     sh_lx[j] = lx; sh_qx[j] = qx;
     float hq = 0.f;
@@ -940,11 +943,13 @@ __global__ void __launch_bounds__(kK3Threads) accept_sample_kernel(const K3Param
       if (p.fallback == HOLA_FALLBACK_GREEDY) {          // greedy: argmax p_n follows the accepted run; no draw
         p.next_tok[b] = min(max(sh_amax[n], 0), V - 1);
         if (flags && p.status) atomicOr(p.status, flags);
+      } else if (p.phase == 1 && flags && p.status) {
+        atomicOr(p.status, flags);
       }
     }
   }
   __syncthreads();
-  if (p.fallback == HOLA_FALLBACK_GREEDY) return;        // same decision in every CTA of the cluster
+  if (p.fallback == HOLA_FALLBACK_GREEDY || p.phase == 1) return;   // same decision in every CTA of the cluster
 
   // ---- this CTA's slice of row n: per-chunk residual mass
   const int n = sh_n;
@@ -1190,6 +1195,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 struct Plan {
   int n_sub, N, rows_per_pass, passes, grid, stages, nbuf, n_ptiles, n_kblocks, smem_bytes, tile_rows;
+  double est_seconds;   // rough duration of all passes (the cost the split was chosen by)
 };
 
 }  // namespace
@@ -1212,6 +1218,12 @@ struct hola_ctx {
   cudaStream_t copy_stream;   // hola_verify_host: the draft tensor travels here while the GEMM runs
   cudaEvent_t copy_done;
   int host_overlap;           // 1: copy the draft tensor on copy_stream while the GEMM runs
+  int host_lazy_q;            // hola_verify_host copies only the draft rows the step reads: 0 never, 1 always,
+                              // -1 when the whole tensor would not fit under the GEMM (the default)
+  float* st_qtok;             // device fp32 [maxB][maxK]: q_j(x_j) gathered on the host
+  float* h_qtok;              // pinned host: the same values before the copy
+  int* h_accept;              // pinned host int32 [maxB]: accept_len read back between the two phases
+  unsigned long long last_h2d, last_d2h;   // bytes the last hola_verify_host call moved
   // optional per-kernel timing (hola_profile_begin / hola_profile_end)
   cudaEvent_t* prof_ev;     // 3 events per recorded call: before the GEMM, after it, after accept/sample
   int prof_cap, prof_n, prof_on;
@@ -1223,7 +1235,7 @@ namespace {
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WsLayout {
-  size_t logits, partials, status, hq, hid8, hid_scale, st_hidden, st_tok, st_q, st_u, st_accept, st_next, st_entropy, st_logZ, total;
+  size_t logits, partials, status, hq, hid8, hid_scale, st_hidden, st_tok, st_q, st_u, st_accept, st_next, st_entropy, st_logZ, st_qtok, total;
 };
 
 WsLayout ws_layout(int maxB, int maxK, int H, int V, int num_sms) {
@@ -1246,6 +1258,7 @@ WsLayout ws_layout(int maxB, int maxK, int H, int V, int num_sms) {
   w.st_next = take(static_cast<size_t>(maxB) * 4);
   w.st_entropy = take(rows * 8);                         // target entropies, then the draft-row entropies
   w.st_logZ = take(rows * 4);
+  w.st_qtok = take(static_cast<size_t>(maxB) * (maxK > 0 ? maxK : 1) * 4);
   w.total = off;
   return w;
 }
@@ -1280,6 +1293,7 @@ Plan make_plan(const hola_ctx* ctx, int M, int w_dtype = HOLA_W_BF16) {
     if (cost < best_cost) {
       best_cost = cost;
       best.n_sub = n_sub; best.N = N; best.rows_per_pass = n_sub * N; best.passes = passes;
+      best.est_seconds = cost;
     }
   }
   // a pass may end up empty when rows_per_pass * (passes - 1) already covers M
@@ -1402,8 +1416,9 @@ hola_status run_lm_head(hola_ctx* ctx, const hola_verify_args* a, float* logits,
 }
 
 hola_status run_accept_sample(hola_ctx* ctx, const hola_verify_args* a, const float* logits, int ldl, int combine,
-                              int nparts, cudaStream_t stream) {
+                              int nparts, cudaStream_t stream, const float* q_tok = nullptr, int phase = 0) {
   K3Params kp;
+  kp.q_tok = q_tok; kp.phase = phase;
   kp.B = a->B; kp.k = a->k; kp.V = a->V; kp.ldl = ldl; kp.logits = logits;
   kp.partials = ctx->partials; kp.nparts = nparts; kp.part_stride = ctx->max_rows; kp.combine = combine;
   kp.tok = a->draft_tok; kp.q = a->draft_q; kp.q_dtype = a->q_dtype; kp.u = a->uniforms; kp.tau = a->tau;
@@ -1423,6 +1438,7 @@ hola_status run_accept_sample(hola_ctx* ctx, const hola_verify_args* a, const fl
   const int nchunks = (a->V + kChunk - 1) / kChunk;
   int S = 8;
   while (S > 1 && (a->B * S > 8 * ctx->num_sms || nchunks / S < 8)) S >>= 1;
+  if (phase == 1) S = 1;                                 // no vocabulary pass: one CTA per sequence
   const int cpc = (nchunks + S - 1) / S;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(static_cast<unsigned>(a->B * S));
@@ -1526,6 +1542,8 @@ hola_status hola_create(hola_ctx** out, int device, int maxB, int maxK, int H, i
   ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
   ctx->host_overlap = 1;
   if (const char* e = getenv("HOLA_HOST_OVERLAP")) ctx->host_overlap = atoi(e) != 0;   // tuning override
+  ctx->host_lazy_q = -1;
+  if (const char* e = getenv("HOLA_HOST_LAZY_Q")) ctx->host_lazy_q = atoi(e) != 0;     // override for tests and sweeps
   if (const char* e = getenv("HOLA_STAGES")) {           // tuning override for sweeps: fewer ring slots
     const int st = atoi(e);
     if (st >= 2 && st <= kMaxStages) ctx->force_stages = st;
@@ -1546,14 +1564,21 @@ hola_status hola_create(hola_ctx** out, int device, int maxB, int maxK, int H, i
   ctx->st_next = reinterpret_cast<int*>(ctx->ws + w.st_next);
   ctx->st_entropy = reinterpret_cast<float*>(ctx->ws + w.st_entropy);
   ctx->st_logZ = reinterpret_cast<float*>(ctx->ws + w.st_logZ);
+  ctx->st_qtok = reinterpret_cast<float*>(ctx->ws + w.st_qtok);
   cudaMemset(ctx->status, 0, 4);
+  const size_t n_qtok = static_cast<size_t>(maxB) * (maxK > 0 ? maxK : 1);
+  void* pinned = nullptr;
   if (cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) != cudaSuccess ||
-      cudaEventCreateWithFlags(&ctx->copy_done, cudaEventDisableTiming) != cudaSuccess) {
+      cudaEventCreateWithFlags(&ctx->copy_done, cudaEventDisableTiming) != cudaSuccess ||
+      cudaHostAlloc(&pinned, (n_qtok + maxB) * 4, cudaHostAllocDefault) != cudaSuccess) {
+    if (ctx->copy_done) cudaEventDestroy(ctx->copy_done);
     if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
     cudaFree(ctx->ws);
     free(ctx);
     return HOLA_ERR_CUDA;
   }
+  ctx->h_qtok = static_cast<float*>(pinned);
+  ctx->h_accept = reinterpret_cast<int*>(ctx->h_qtok + n_qtok);
   *out = ctx;
   return HOLA_OK;
 }
@@ -1565,6 +1590,7 @@ hola_status hola_destroy(hola_ctx* ctx) {
   free(ctx->prof_ev);
   if (ctx->copy_done) cudaEventDestroy(ctx->copy_done);
   if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
+  if (ctx->h_qtok) cudaFreeHost(ctx->h_qtok);
   cudaFree(ctx->ws);
   free(ctx);
   return HOLA_OK;
@@ -1636,6 +1662,113 @@ hola_status verify_device(hola_ctx* ctx, const hola_verify_args* a, cudaStream_t
   return s;
 }
 
+// hola_verify_host while the target entropy gates.  Of the draft tensor the step then reads k single probabilities
+// per sequence (q_j(x_j), gathered here on the host) and at most ONE row per sequence: row accept_len, and none when
+// every draft token was kept or the fallback is greedy.  Rows 0 .. ahead-1 of every sequence (as many as the bus
+// carries while the GEMM runs, at least one) are sent ahead on the context's own stream; after the accept test the
+// accept lengths come back and only the rows still missing follow.  Same kernels, same arithmetic and so the same
+// results as the whole-tensor copy.
+constexpr double kHostBusBytesPerSecond = 50e9;          // what a pinned host-to-device copy reaches here
+
+// Draft rows per sequence that can cross the bus while the GEMM of this call runs.
+int rows_under_gemm(const hola_ctx* ctx, const hola_verify_args* a) {
+  const Plan pl = make_plan(ctx, a->B * (a->k + 1), a->w_dtype);
+  const double group = static_cast<double>(a->B) * a->V * (a->q_dtype == HOLA_Q_BF16 ? 2 : 4);
+  const double n = pl.est_seconds * kHostBusBytesPerSecond / group;
+  return n > 1e6 ? 1000000 : static_cast<int>(n);
+}
+
+hola_status verify_host_lazy(hola_ctx* ctx, const hola_verify_args* a, cudaStream_t stream, int ahead) {
+  const int B = a->B, k = a->k, V = a->V;
+  const size_t rows = static_cast<size_t>(B) * (k + 1);
+  const size_t q_elem = a->q_dtype == HOLA_Q_BF16 ? 2 : 4;
+  const size_t row_bytes = static_cast<size_t>(V) * q_elem;
+  const bool sample = a->fallback != HOLA_FALLBACK_GREEDY;
+  cudaError_t e = cudaSuccess;
+  unsigned long long up = 0, down = 0;
+  auto h2d = [&](void* dst, const void* src, size_t bytes, cudaStream_t st) {
+    if (e == cudaSuccess && bytes) e = cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, st);
+    up += bytes;
+  };
+  auto d2h = [&](void* dst, const void* src, size_t bytes) {
+    if (e == cudaSuccess && bytes) e = cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToHost, stream);
+    down += bytes;
+  };
+  for (int b = 0; b < B; ++b)
+    for (int j = 0; j < k; ++j) {
+      const int x = a->draft_tok[b * k + j];
+      float qx = 0.f;
+      if (x >= 0 && x < V) {
+        const size_t qi = (static_cast<size_t>(b) * k + j) * V + x;
+        if (a->q_dtype == HOLA_Q_BF16) {
+          const uint32_t bits = static_cast<uint32_t>(static_cast<const uint16_t*>(a->draft_q)[qi]) << 16;
+          memcpy(&qx, &bits, 4);
+        } else {
+          qx = static_cast<const float*>(a->draft_q)[qi];
+        }
+      }
+      ctx->h_qtok[b * k + j] = qx;
+    }
+  h2d(ctx->st_hidden, a->hidden, rows * a->H * 2, stream);
+  h2d(ctx->st_tok, a->draft_tok, static_cast<size_t>(B) * k * 4, stream);
+  h2d(ctx->st_u, a->uniforms, rows * 4, stream);
+  h2d(ctx->st_qtok, ctx->h_qtok, static_cast<size_t>(B) * k * 4, stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->status, 0, 4, stream);
+  const size_t seq_pitch = static_cast<size_t>(k) * row_bytes;   // from row (b, 0) to row (b + 1, 0)
+  ahead = ahead < 1 ? 1 : (ahead > k ? k : ahead);
+  const size_t ahead_bytes = static_cast<size_t>(ahead) * row_bytes;     // rows 0 .. ahead-1 of a sequence are adjacent
+  if (sample) {
+    if (seq_pitch < (1ull << 31)) {
+      if (e == cudaSuccess)
+        e = cudaMemcpy2DAsync(ctx->st_q, seq_pitch, a->draft_q, seq_pitch, ahead_bytes, static_cast<size_t>(B),
+                              cudaMemcpyHostToDevice, ctx->copy_stream);
+      up += static_cast<size_t>(B) * ahead_bytes;
+    } else {
+      for (int b = 0; b < B; ++b)
+        h2d(static_cast<char*>(ctx->st_q) + b * seq_pitch, static_cast<const char*>(a->draft_q) + b * seq_pitch,
+            ahead_bytes, ctx->copy_stream);
+    }
+    if (e == cudaSuccess) e = cudaEventRecord(ctx->copy_done, ctx->copy_stream);
+  }
+  if (e != cudaSuccess) { set_error(ctx, "host-to-device copy", e); return HOLA_ERR_CUDA; }
+  hola_verify_args d = *a;
+  d.hidden = ctx->st_hidden; d.draft_tok = ctx->st_tok; d.draft_q = ctx->st_q; d.uniforms = ctx->st_u;
+  d.accept_len = ctx->st_accept; d.next_tok = ctx->st_next; d.entropy = ctx->st_entropy; d.logZ = ctx->st_logZ;
+  d.logits_out = nullptr; d.status_word = ctx->status; d.draft_entropy = nullptr;
+  hola_status s = check_lm_head_args(ctx, &d);
+  if (s != HOLA_OK) return s;
+  const Plan pl = make_plan(ctx, B * (k + 1), a->w_dtype);
+  if ((s = run_lm_head(ctx, &d, ctx->logits, ctx->ldl, pl, stream)) != HOLA_OK) return s;
+  if (!sample) {
+    if ((s = run_accept_sample(ctx, &d, ctx->logits, ctx->ldl, 1, pl.grid, stream, ctx->st_qtok, 0)) != HOLA_OK) return s;
+  } else {
+    if ((s = run_accept_sample(ctx, &d, ctx->logits, ctx->ldl, 1, pl.grid, stream, ctx->st_qtok, 1)) != HOLA_OK) return s;
+    d2h(ctx->h_accept, ctx->st_accept, static_cast<size_t>(B) * 4);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    if (e != cudaSuccess) { set_error(ctx, "accept lengths to host", e); return HOLA_ERR_CUDA; }
+    for (int b = 0; b < B; ++b) {
+      const int n = ctx->h_accept[b];
+      if (n >= ahead && n < k) {
+        const size_t off = (static_cast<size_t>(b) * k + n) * row_bytes;
+        h2d(static_cast<char*>(ctx->st_q) + off, static_cast<const char*>(a->draft_q) + off, row_bytes, stream);
+      }
+    }
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, ctx->copy_done, 0);
+    if (e != cudaSuccess) { set_error(ctx, "host-to-device copy of draft rows", e); return HOLA_ERR_CUDA; }
+    // statistics and accept lengths are in place: this launch repeats the (cheap) accept test and draws the token
+    if ((s = run_accept_sample(ctx, &d, ctx->logits, ctx->ldl, 0, 0, stream, ctx->st_qtok, 0)) != HOLA_OK) return s;
+  }
+  d2h(a->accept_len, ctx->st_accept, static_cast<size_t>(B) * 4);
+  d2h(a->next_tok, ctx->st_next, static_cast<size_t>(B) * 4);
+  d2h(a->entropy, ctx->st_entropy, rows * 4);
+  d2h(a->logZ, ctx->st_logZ, rows * 4);
+  if (a->status_word) d2h(a->status_word, ctx->status, 4);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+  if (e != cudaSuccess) { set_error(ctx, "device-to-host copy", e); return HOLA_ERR_CUDA; }
+  ctx->last_h2d = up; ctx->last_d2h = down;
+  return HOLA_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -1699,12 +1832,21 @@ hola_status hola_verify_host(hola_ctx* ctx, const hola_verify_args* a, void* cud
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   const size_t rows = static_cast<size_t>(a->B) * (a->k + 1);
   const size_t q_elem = a->q_dtype == HOLA_Q_BF16 ? 2 : 4;
+  if (ctx->host_lazy_q && a->k > 0 && a->gate_source == HOLA_GATE_TARGET_ENTROPY) {
+    // when the whole draft tensor crosses the bus under the GEMM anyway, the plain copy below has one launch and
+    // one synchronisation fewer
+    const int ahead = rows_under_gemm(ctx, a);
+    if (ctx->host_lazy_q > 0 || ahead < a->k) return verify_host_lazy(ctx, a, stream, ahead);
+  }
   cudaError_t e = cudaSuccess;
+  unsigned long long up = 0, down = 0;
   auto h2d = [&](void* dst, const void* src, size_t bytes) {
     if (e == cudaSuccess && bytes) e = cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, stream);
+    up += bytes;
   };
   auto d2h = [&](void* dst, const void* src, size_t bytes) {
     if (e == cudaSuccess && bytes) e = cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToHost, stream);
+    down += bytes;
   };
   // The small inputs go first (copies queue on the DMA engine in issue order).  The draft tensor is by far the
   // largest input and only the accept/sample part reads it: it travels on the context's own stream while the
@@ -1717,6 +1859,7 @@ hola_status hola_verify_host(hola_ctx* ctx, const hola_verify_args* a, void* cud
   if (overlap) {
     if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->st_q, a->draft_q, q_bytes, cudaMemcpyHostToDevice, ctx->copy_stream);
     if (e == cudaSuccess) e = cudaEventRecord(ctx->copy_done, ctx->copy_stream);
+    up += q_bytes;
   } else {
     h2d(ctx->st_q, a->draft_q, q_bytes);
   }
@@ -1738,6 +1881,13 @@ hola_status hola_verify_host(hola_ctx* ctx, const hola_verify_args* a, void* cud
     d2h(a->draft_entropy, ctx->st_entropy + rows, static_cast<size_t>(a->B) * a->k * 4);
   if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
   if (e != cudaSuccess) { set_error(ctx, "device-to-host copy", e); return HOLA_ERR_CUDA; }
+  ctx->last_h2d = up; ctx->last_d2h = down;
+  return HOLA_OK;
+}
+
+hola_status hola_host_traffic(const hola_ctx* ctx, unsigned long long* h2d_bytes, unsigned long long* d2h_bytes) {
+  if (!ctx || !h2d_bytes || !d2h_bytes) return HOLA_ERR_INVALID_ARG;
+  *h2d_bytes = ctx->last_h2d; *d2h_bytes = ctx->last_d2h;
   return HOLA_OK;
 }
 

@@ -350,6 +350,46 @@ def test_host_entry_equals_device_entry(binding):
     assert torch.equal(h.entropy, d.entropy.cpu()) and torch.equal(h.logZ, d.logZ.cpu())
 
 
+@pytest.mark.parametrize("q_dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("gate,fallback", [(0, 0), (0, 1), (1, 0)])
+@pytest.mark.parametrize("tau", [0.0, None, 100.0])
+def test_host_entry_sends_only_the_rows_it_reads(binding, monkeypatch, q_dtype, gate, fallback, tau):
+    """hola_verify_host against hola_verify on the same data, over accept lengths from 0 to k (tau = 0: gate off;
+    None: the median entropy; 100: every draft kept), with poisoned staging so that a row that was needed but not copied would show."""
+    w = workloads.gaussian_head("host_rows", 21, 4, 128, 5000, seed=77, device=DEV, w_std=0.3, tau=tau,
+                                q_dtype=q_dtype)
+    pin = lambda t: t.cpu().pin_memory()
+    monkeypatch.setenv("HOLA_HOST_LAZY_Q", "1")          # this small tensor would otherwise be copied whole
+    with binding.HolaVerify(w.B, w.k, w.H, w.V) as ctx:
+        # a first host call with a wrong draft tensor leaves stale rows in the staging area
+        ctx.hola_verify_host(pin(w.hidden), w.W_lm, pin(w.draft_tok), pin(torch.flip(w.draft_q, dims=[2])),
+                             pin(w.uniforms), w.tau, gate_source=gate, fallback=fallback)
+        d = ctx.hola_verify(w.hidden, w.W_lm, w.draft_tok, w.draft_q, w.uniforms, w.tau, gate_source=gate,
+                            fallback=fallback)
+        torch.cuda.synchronize()
+        h = ctx.hola_verify_host(pin(w.hidden), w.W_lm, pin(w.draft_tok), pin(w.draft_q), pin(w.uniforms), w.tau,
+                                 gate_source=gate, fallback=fallback)
+        up, down = ctx.hola_host_traffic()
+    assert torch.equal(h.accept_len, d.accept_len.cpu()) and torch.equal(h.next_tok, d.next_tok.cpu())
+    assert torch.equal(h.entropy, d.entropy.cpu()) and torch.equal(h.logZ, d.logZ.cpu())
+    assert int(h.status.item()) == int(d.status.item())
+    if tau == 0.0 and fallback == 0:
+        assert len(set(h.accept_len.tolist())) >= 3      # the case does spread over several accept lengths
+    q_bytes = w.draft_q.numel() * w.draft_q.element_size()
+    row = w.V * w.draft_q.element_size()
+    small = w.hidden.numel() * 2 + w.draft_tok.numel() * 4 + w.uniforms.numel() * 4
+    if gate == 1:
+        assert up == small + q_bytes                      # the draft entropy reads every row
+    elif fallback == 1:
+        assert up == small + w.B * w.k * 4                # greedy: no row at all
+    else:
+        n = h.accept_len                                  # rows 0 .. ahead-1 go first, then the rows still missing
+        expected = {small + w.B * w.k * 4 + (w.B * ahead + int(((n >= ahead) & (n < w.k)).sum())) * row
+                    for ahead in range(1, w.k + 1)}
+        assert up in expected
+        assert up < small + q_bytes                       # and that is less than the whole tensor
+
+
 # ------------------------------------------------------------------------------------------ 8-bit LM head
 def _w8_oracle(w, q8, scale, a8=False, **kw):
     """The oracle on the dequantised head: hidden widened to fp64 (or, with a8, quantised row by row with the same
