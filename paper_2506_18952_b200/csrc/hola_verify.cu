@@ -47,20 +47,19 @@ constexpr int kPairTile = 2 * kLanes;            // vocabulary rows per CTA pair
 constexpr int kWBlockBytes = kLanes * kBlockK * 2;
 constexpr int kMaxN = 256;                       // verify rows per MMA
 constexpr int kMaxRowsPerPass = 2 * kMaxN;       // two MMAs per K step fill the 512 tensor-memory columns
-constexpr int kDrainWarps = 8;                   // warps 2..9: tensor memory -> logits buffer
-constexpr int kStatsWarps = 8;                   // warps 10..17: softmax statistics from the stored tile
-constexpr int kStatsThreads = kStatsWarps * 32;
-constexpr int kK1Warps = 2 + kDrainWarps + kStatsWarps;   // warp 0 TMA, warp 1 MMA + tensor-memory owner
+constexpr int kEpiWarps = 16;                    // warps 2..17: tensor memory -> logits buffer + softmax statistics
+constexpr int kK1Warps = 2 + kEpiWarps;          // warp 0 TMA, warp 1 MMA + tensor-memory owner
 constexpr int kK1Threads = kK1Warps * 32;
-constexpr int kStatsRowsPerThread = kMaxRowsPerPass * 4 / kStatsThreads;   // four threads share a row
-// 8-bit W_lm: the int8 tile lands in a raw block, converter warps expand it to the bf16 tile the MMA reads.
-// That kernel takes at most 256 rows per pass, so 4 drain warps (2..5) and 4 statistics warps (10..13) are enough;
-// warp 14 loads the hidden blocks and warps 6..9 and 15..17 convert.
+constexpr int kEpiSlots = 4;                     // 32-column chunks of a tile one epilogue warp handles at most
+constexpr int kTransRows = 16;                   // verify rows per transposition step of an epilogue warp
+constexpr int kTransBytes = kTransRows * 32 * 4; // its staging buffer: [16 rows][32 vocabulary entries] fp32
+// 8-bit W_lm, expanded on chip (mode 1): the int8 tile of a K block lands in a raw block of the ring slot and
+// converter warps expand it to the bf16 tile the MMA reads.  Warps 2..9 are epilogue warps, warp 14 loads the
+// hidden blocks, warps 10..13 and 15..17 convert.
 constexpr int kRawBlockBytes = kLanes * kBlockK;  // int8 [128][64]
-constexpr int kW8DrainWarps = 4;
-constexpr int kW8StatsWarps = 4;
-constexpr int kW8HiddenWarp = 2 + kDrainWarps + kW8StatsWarps;     // warp 14
-constexpr int kConvWarps = (kDrainWarps - kW8DrainWarps) + (kK1Warps - kW8HiddenWarp - 1);   // 4 + 3
+constexpr int kW8EpiWarps = 8;
+constexpr int kW8HiddenWarp = 14;
+constexpr int kConvWarps = (kW8HiddenWarp - 2 - kW8EpiWarps) + (kK1Warps - kW8HiddenWarp - 1);   // 4 + 3
 constexpr int kConvThreads = kConvWarps * 32;
 constexpr int kTmemCols = 512;
 constexpr int kMaxStages = 12;
@@ -90,7 +89,6 @@ struct K1Params {
   int n_sub, N;   // MMAs per K step and their N (verify rows each; multiple of 16)
   int tile_rows;  // vocabulary rows per CTA per tile (<= 128, multiple of 4): balances the tiles over the pairs
   int ldl;        // row pitch of the logits buffer, in floats
-  int vec_ok;     // 16-byte loads of the logits buffer allowed (pitch and base aligned)
   const float* w_scale;   // 8-bit W_lm: fp32 scale per vocabulary row, applied to the accumulators
   const float* h_scale;   // 8-bit activations (mode 2): fp32 scale per verify row
   float* logits;
@@ -338,13 +336,12 @@ __device__ __forceinline__ Stats stats_merge(Stats a, Stats b) {
   return r;
 }
 
-// Fold `n` (1..32) logits into the running statistics.  Element i is vocabulary entry
-// vocab0 + 16 * (i / 4) + (i % 4): the statistics threads' interleaved share of a row (ascending in i).
+// Fold the first `n` (1..16) of sixteen logits into the running statistics; element i is vocabulary entry vocab0 + i.
 template <bool kFull>
-__device__ __forceinline__ void stats_fold(const float* v, int n, int vocab0, Stats& st) {
+__device__ __forceinline__ void stats_fold16(const float* v, int n, int vocab0, Stats& st) {
   float cmax = v[0];
 #pragma unroll
-  for (int i = 1; i < 32; ++i)
+  for (int i = 1; i < 16; ++i)
     if (kFull || i < n) cmax = fmaxf(cmax, v[i]);
   if (cmax > st.m) {
     if (st.m != -CUDART_INF_F) {
@@ -356,16 +353,16 @@ __device__ __forceinline__ void stats_fold(const float* v, int n, int vocab0, St
     st.m = cmax;
     int first = 0;
 #pragma unroll
-    for (int i = 31; i > 0; --i)
+    for (int i = 15; i > 0; --i)
       if ((kFull || i < n) && v[i] == cmax) first = i;
     if (v[0] == cmax) first = 0;
-    st.arg = vocab0 + 16 * (first >> 2) + (first & 3);
+    st.arg = vocab0 + first;
   }
   const float m = st.m;
   const float mneg2 = -m * kLog2e;
   float s = st.s, t = st.t;
 #pragma unroll
-  for (int i = 0; i < 32; ++i) {
+  for (int i = 0; i < 16; ++i) {
     if (kFull || i < n) {
       const float e = ex2_approx(fmaf(v[i], kLog2e, mneg2));
       s += e;
@@ -416,12 +413,12 @@ __device__ __forceinline__ float scaled(float acc, float w_scale, const float* h
 //   full[12]   @0    leader CTA's copy is the live one: 2 arrivals (one producer per CTA) + the bytes of both CTAs
 //   empty[12]  @96   per CTA: the MMAs that read this slot have completed (commit, delivered to both CTAs)
 //   tfull[2]   @192  per CTA: the accumulators of a tile are complete (commit, delivered to both CTAs)
-//   tempty[2]  @208  leader's copy: all 16 drain warps of the pair have read their accumulators
-//   lready[2]  @224  per CTA: the 8 drain warps have stored the tile's logits (by tile parity)
-//   sfree[2]   @240  per CTA: the 8 statistics warps are done with that tile (keeps lready from lapping)
+//   tempty[2]  @208  leader's copy: all epilogue warps of the pair have read their accumulators
 //   tensor-memory base @256, abort flag @260
 //   8-bit W_lm only: rawfull[12] @272 per CTA: the int8 tile of the slot has landed; rawempty[12] @368 per CTA: the
 //   converter warps have expanded it.  full[] then collects, besides the hidden bytes, one arrival per converter warp.
+// After the barrier area: one 2 KB transposition buffer per epilogue warp (reused for the final merge of the
+// statistics of the four tensor-memory lane quarters).
 // kMode: 0 bf16 x bf16; 1 int8 W_lm expanded to bf16 on chip (exact); 2 int8 W_lm x int8 hidden on the 8-bit MMA
 // kind (K blocks of 128 elements, so that a block is 128 bytes per row exactly as in mode 0; int32 accumulators).
 template <int kMode>
@@ -451,8 +448,10 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
   const int pair_rows = 2 * p.tile_rows;                 // vocabulary rows of a pair's tile
   const uint32_t bar_base = base + p.stages * stage_bytes;
   const uint32_t full_bar = bar_base, empty_bar = bar_base + 96, tfull_bar = bar_base + 192,
-                 tempty_bar = bar_base + 208, lready_bar = bar_base + 224, sfree_bar = bar_base + 240,
-                 rawfull_bar = bar_base + 272, rawempty_bar = bar_base + 368;
+                 tempty_bar = bar_base + 208, rawfull_bar = bar_base + 272, rawempty_bar = bar_base + 368;
+  constexpr int kNumEpi = kW8 ? kW8EpiWarps : kEpiWarps;      // epilogue warps 2 .. 2 + kNumEpi - 1
+  constexpr int kGroups = kNumEpi / 4;                        // warps per tensor-memory lane quarter
+  float* trans_base = reinterpret_cast<float*>(smem + p.stages * stage_bytes + kBarrierBytes);
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + p.stages * stage_bytes + 256);
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + p.stages * stage_bytes + 260);
 
@@ -467,9 +466,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(tfull_bar + 8 * i, 1);
-      mbar_init(tempty_bar + 8 * i, 2 * (kW8 ? kW8DrainWarps : kDrainWarps));
-      mbar_init(lready_bar + 8 * i, kW8 ? kW8DrainWarps : kDrainWarps);
-      mbar_init(sfree_bar + 8 * i, kW8 ? kW8StatsWarps : kStatsWarps);
+      mbar_init(tempty_bar + 8 * i, 2 * kNumEpi);
     }
     *abort_flag = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -566,122 +563,123 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
         if (ok) umma_commit_pair(tfull_bar + 8 * buf);   // accumulators of this tile are complete in both CTAs
       }
     }
-  } else if (warp < 2 + (kW8 ? kW8DrainWarps : kDrainWarps)) {
-    // ------------------------------------------------------------------ drain warps: tensor memory -> logits
-    const int quarter = warp & 3;                        // tensor-memory lanes 32*quarter .. +31 (fixed by warp id)
-    const int group = (warp - 2) >> 2;                   // the two warps of a quarter alternate over the chunks
-    constexpr int kChunkStep = kW8 ? 1 : 2;              // (one warp per quarter with 8-bit W_lm)
+  } else if (warp < 2 + kNumEpi) {
+    // ------------------------------------------------------------------ epilogue warps
+    // Tensor memory -> registers (thread = vocabulary entry, register = verify row) -> logits buffer, and the same
+    // values, transposed through a small shared-memory buffer 16 rows at a time (thread = verify row and half of the
+    // warp's 32 vocabulary entries), into thread-private softmax statistics that live in registers for the whole
+    // kernel.  A warp owns one lane quarter (fixed by its id) and every kGroups-th 32-column chunk.
+    const int quarter = warp & 3;                        // tensor-memory lanes 32*quarter .. +31
+    const int group = (warp - 2) >> 2;
     const uint32_t leader_tempty = map_to_cta(tempty_bar, 0);
     const int n_chunks = p.n_sub * sub_chunks;
+    const int my_chunks = group < n_chunks ? (n_chunks - 1 - group) / kGroups + 1 : 0;
+    float* tbuf = trans_base + (warp - 2) * (kTransBytes / 4);
+    const int trow = lane & 15, thalf = lane >> 4;       // row of a transposition step; which 16 of the 32 entries
+    Stats st[kEpiSlots][2];
+#pragma unroll
+    for (int i = 0; i < kEpiSlots; ++i) { st[i][0] = stats_empty(); st[i][1] = stats_empty(); }
     bool ok = true;
     for (int t = 0; t < my_tiles && ok; ++t) {
       const int buf = t % p.nbuf;
       const uint32_t acc_phase = static_cast<uint32_t>(t / p.nbuf) & 1u;
-      const int par = t & 1;
       if (!mbar_wait_warp(tfull_bar + 8 * buf, acc_phase, abort_flag, p.status)) { ok = false; break; }
       tc_fence_after();
+      const int vbase = (pair + t * npairs) * pair_rows + static_cast<int>(rank) * p.tile_rows;
       const int tile_lane = quarter * 32 + lane;         // lanes at or beyond tile_rows hold nothing
-      const int vocab = (pair + t * npairs) * pair_rows + static_cast<int>(rank) * p.tile_rows + tile_lane;
+      const int vocab = vbase + tile_lane;
       const bool vocab_ok = tile_lane < p.tile_rows && vocab < p.V;
+      // vocabulary entries of this quarter that exist (a prefix of its 32 lanes), and of this thread's 16
+      const int nv = max(0, min(32, min(p.tile_rows, p.V - vbase) - quarter * 32));
+      const int n16 = max(0, min(16, nv - thalf * 16));
+      const int vocab16 = vbase + quarter * 32 + thalf * 16;
       const float w_scale = ((kW8 || kI8) && vocab_ok) ? p.w_scale[vocab] : 1.f;   // 8-bit W_lm: the row's scale
       const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * 256;
-      for (int ch = group; ch < n_chunks; ch += kChunkStep) {
-        const int s = ch / sub_chunks, j = ch - s * sub_chunks;
-        float v[32];
-        __syncwarp();                                    // tcgen05.ld is warp-collective: reconverge first
-        tmem_ld32(lane_addr + s * 256 + j * 32, v);
-        const int c0 = j * 32;                           // first column of the chunk inside its MMA
-        const int r0 = p.row0 + s * p.N + c0;            // verify row of column c0
-        int n_ok = min(p.N - c0, p.M - r0);              // columns that are real rows
-        n_ok = min(n_ok, 32);
-        if (vocab_ok && n_ok > 0) {
-          float* dst = p.logits + static_cast<size_t>(r0) * p.ldl + vocab;
-          if (n_ok == 32) {
+      if (my_chunks == 0) {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(leader_tempty + 8 * buf);
+      }
 #pragma unroll
-            for (int i = 0; i < 32; ++i) dst[static_cast<size_t>(i) * p.ldl] = scaled<kMode>(v[i], w_scale, p.h_scale, r0 + i);
-          } else {
+      for (int slot = 0; slot < kEpiSlots; ++slot) {
+        if (slot < my_chunks) {
+          const int ch = group + slot * kGroups;
+          const int sub = ch / sub_chunks, j = ch - sub * sub_chunks;
+          float v[32];
+          __syncwarp();                                  // tcgen05.ld is warp-collective: reconverge first
+          tmem_ld32(lane_addr + sub * 256 + j * 32, v);
+          if (slot == my_chunks - 1) {                   // this warp's accumulators may be overwritten
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(leader_tempty + 8 * buf);
+          }
+          const int c0 = j * 32;                         // first column of the chunk inside its MMA
+          const int r0 = p.row0 + sub * p.N + c0;        // verify row of column c0
+          const int n_ok = min(32, min(p.N - c0, p.M - r0));   // columns that are real rows
+          if (n_ok > 0) {
 #pragma unroll
             for (int i = 0; i < 32; ++i)
-              if (i < n_ok) dst[static_cast<size_t>(i) * p.ldl] = scaled<kMode>(v[i], w_scale, p.h_scale, r0 + i);
-          }
-        }
-      }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(leader_tempty + 8 * buf);     // this warp's accumulators may be overwritten
-      // the statistics warps must have finished the tile that used this parity before it is announced again
-      if (t >= 2 && !mbar_wait_warp(sfree_bar + 8 * par, static_cast<uint32_t>((t >> 1) - 1) & 1u, abort_flag, p.status)) {
-        ok = false;
-        break;
-      }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(lready_bar + 8 * par);  // release: this warp's stores are visible to the CTA
-    }
-  } else if (!kW8 || (warp >= 2 + kDrainWarps && warp < kW8HiddenWarp)) {
-    // ------------------------------------------------------------------ statistics warps
-    // Four threads share a verify row: thread `part` takes floats 16*it + 4*part .. +3 (it = 0..7) of the row's 128
-    // logits of this tile, so a warp's load covers 8 rows x 64 contiguous bytes.
-    constexpr int kRowStep = (kW8 ? kW8StatsWarps : kStatsWarps) * 32 / 4;    // rows covered per step of the warps
-    const int ts = threadIdx.x - (2 + kDrainWarps) * 32;
-    const int part = ts & 3, rsub = ts >> 2;
-    Stats st[kStatsRowsPerThread];
+              if (i < n_ok) v[i] = scaled<kMode>(v[i], w_scale, p.h_scale, r0 + i);
+            if (vocab_ok) {
+              float* dst = p.logits + static_cast<size_t>(r0) * p.ldl + vocab;
+              if (n_ok == 32) {
 #pragma unroll
-    for (int i = 0; i < kStatsRowsPerThread; ++i) st[i] = stats_empty();
-    bool ok = true;
-    for (int t = 0; t < my_tiles && ok; ++t) {
-      const int par = t & 1;
-      if (!mbar_wait_warp(lready_bar + 8 * par, static_cast<uint32_t>(t >> 1) & 1u, abort_flag, p.status)) { ok = false; break; }
-      const int vbase = (pair + t * npairs) * pair_rows + static_cast<int>(rank) * p.tile_rows;
-      const int lim = min(p.tile_rows, p.V - vbase);     // logits of this tile that exist
-      if (lim > 0) {
-#pragma unroll
-        for (int i = 0; i < kStatsRowsPerThread; ++i) {
-          const int r = rsub + kRowStep * i;
-          if (r < p.rows) {
-            const float* src = p.logits + static_cast<size_t>(p.row0 + r) * p.ldl + vbase;
-            float v[32];
-            int n = 0;                                   // this thread's columns ascend with the index: a prefix is valid
-#pragma unroll
-            for (int it = 0; it < 8; ++it) {
-              const int col = 16 * it + 4 * part;
-              if (p.vec_ok && col + 4 <= lim) {
-                const float4 x = __ldcg(reinterpret_cast<const float4*>(src + col));
-                v[4 * it] = x.x; v[4 * it + 1] = x.y; v[4 * it + 2] = x.z; v[4 * it + 3] = x.w;
-                n = 4 * it + 4;
+                for (int i = 0; i < 32; ++i) dst[static_cast<size_t>(i) * p.ldl] = v[i];
               } else {
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                  const bool in = col + j < lim;
-                  v[4 * it + j] = in ? __ldcg(src + col + j) : 0.f;
-                  n += in ? 1 : 0;
+                for (int i = 0; i < 32; ++i)
+                  if (i < n_ok) dst[static_cast<size_t>(i) * p.ldl] = v[i];
+              }
+            }
+            if (nv > 0) {
+#pragma unroll
+              for (int half = 0; half < 2; ++half) {
+                if (half * kTransRows < n_ok) {
+                  // entry (row i, vocabulary lane l) at 16-byte group (l / 4) ^ (i % 8) of row i: stores of one
+                  // row and the 16-byte loads of eight neighbouring rows both touch every bank once
+                  __syncwarp();
+#pragma unroll
+                  for (int i = 0; i < kTransRows; ++i)
+                    tbuf[i * 32 + ((((lane >> 2) ^ (i & 7))) << 2) + (lane & 3)] = v[half * kTransRows + i];
+                  __syncwarp();
+                  float e[16];
+#pragma unroll
+                  for (int jj = 0; jj < 4; ++jj) {
+                    const float4 x = *reinterpret_cast<const float4*>(
+                        tbuf + trow * 32 + (((thalf * 4 + jj) ^ (trow & 7)) << 2));
+                    e[4 * jj] = x.x; e[4 * jj + 1] = x.y; e[4 * jj + 2] = x.z; e[4 * jj + 3] = x.w;
+                  }
+                  // (rows at or beyond n_ok fold whatever the unused columns held; they are never written out)
+                  if (n16 == 16) stats_fold16<true>(e, 16, vocab16, st[slot][half]);
+                  else if (n16 > 0) stats_fold16<false>(e, n16, vocab16, st[slot][half]);
                 }
               }
             }
-            if (n == 32) stats_fold<true>(v, 32, vbase + 4 * part, st[i]);
-            else if (n > 0) stats_fold<false>(v, n, vbase + 4 * part, st[i]);
           }
         }
       }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(sfree_bar + 8 * par);
     }
-    if (ok) {
+    // ---- the CTA's statistics of every row: first the two halves of a quarter (lanes L and L ^ 16), then, after
+    // all epilogue warps are done with their buffers, the quarters side by side in shared memory
+    asm volatile("bar.sync 1, %0;" ::"n"(kNumEpi * 32) : "memory");
+    float4* merge = reinterpret_cast<float4*>(trans_base);          // [4 quarters][rows of the pass]
 #pragma unroll
-      for (int i = 0; i < kStatsRowsPerThread; ++i) {
-        Stats a = st[i];
+    for (int slot = 0; slot < kEpiSlots; ++slot) {
 #pragma unroll
-        for (int off = 1; off <= 2; off <<= 1) {
-          Stats o;
-          o.m = __shfl_xor_sync(0xffffffffu, a.m, off);
-          o.s = __shfl_xor_sync(0xffffffffu, a.s, off);
-          o.t = __shfl_xor_sync(0xffffffffu, a.t, off);
-          o.arg = __shfl_xor_sync(0xffffffffu, a.arg, off);
-          a = ((lane & off) == 0) ? stats_merge(a, o) : stats_merge(o, a);
+      for (int half = 0; half < 2; ++half) {
+        Stats a = st[slot][half], o;
+        o.m = __shfl_xor_sync(0xffffffffu, a.m, 16);
+        o.s = __shfl_xor_sync(0xffffffffu, a.s, 16);
+        o.t = __shfl_xor_sync(0xffffffffu, a.t, 16);
+        o.arg = __shfl_xor_sync(0xffffffffu, a.arg, 16);
+        a = stats_merge(a, o);
+        if (slot < my_chunks && thalf == 0) {
+          const int ch = group + slot * kGroups;
+          const int sub = ch / sub_chunks, j = ch - sub * sub_chunks;
+          const int c = j * 32 + half * kTransRows + trow;           // column inside its MMA
+          const int r = sub * p.N + c;                               // row inside the pass
+          if (c < p.N && r < p.rows) merge[quarter * p.rows + r] = make_float4(a.m, a.s, a.t, __int_as_float(a.arg));
         }
-        const int r = rsub + kRowStep * i;
-        if (part == 0 && r < p.rows)
-          p.partials[static_cast<size_t>(blockIdx.x) * p.part_stride + p.row0 + r] =
-              make_float4(a.m, a.s, a.t, __int_as_float(a.arg));
       }
     }
   } else if (warp == kW8HiddenWarp) {
@@ -712,7 +710,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
     // MMA reads: 16-byte chunk c of row r sits at chunk position c ^ (r % 8) of its 128-byte row.  Every int8 value is
     // exact in bf16; the row's scale is applied to the accumulators by the drain warps.
     // All converter warps share every K block (two independent 16-byte pieces per thread), in ring order.
-    const int cw = warp < 2 + kDrainWarps ? warp - (2 + kW8DrainWarps) : warp - (kW8HiddenWarp + 1) + (kDrainWarps - kW8DrainWarps);
+    const int cw = warp < kW8HiddenWarp ? warp - (2 + kW8EpiWarps) : warp - (kW8HiddenWarp + 1) + (kW8HiddenWarp - 2 - kW8EpiWarps);
     const int ct = cw * 32 + lane;
     const uint32_t leader_full = map_to_cta(full_bar, 0);
     const int units = p.tile_rows * 4;                   // 16-byte pieces of the int8 tile
@@ -748,6 +746,20 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
   __syncwarp();                                          // warps 0 and 1 ran one lane apart from the others
   tc_fence_before();
   __syncthreads();
+  if (!*abort_flag) {
+    // one partial per CTA and row: the four quarters merged
+    const float4* merge = reinterpret_cast<const float4*>(trans_base);
+    for (int r = threadIdx.x; r < p.rows; r += kK1Threads) {
+      Stats a = stats_empty();
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const float4 x = merge[q * p.rows + r];
+        a = stats_merge(a, Stats{x.x, x.y, x.z, __float_as_int(x.w)});
+      }
+      p.partials[static_cast<size_t>(blockIdx.x) * p.part_stride + p.row0 + r] =
+          make_float4(a.m, a.s, a.t, __int_as_float(a.arg));
+    }
+  }
   cluster_sync_all();                                    // the peer no longer signals this CTA's barriers or tensor memory
   if (warp == 1) {
     if (*abort_flag) __nanosleep(200000);                // let copies already in flight land before leaving
@@ -1299,7 +1311,8 @@ Plan make_plan(const hola_ctx* ctx, int M, int w_dtype = HOLA_W_BF16) {
   // a pass may end up empty when rows_per_pass * (passes - 1) already covers M
   best.passes = (rows + best.rows_per_pass - 1) / best.rows_per_pass;
   const int stage_bytes = kWBlockBytes + best.n_sub * (best.N / 2) * 128 + (w8 ? kRawBlockBytes : 0);
-  int stages = (kSmemBudget - 1024 - kBarrierBytes) / stage_bytes;
+  const int trans_bytes = (w8 ? kW8EpiWarps : kEpiWarps) * kTransBytes;
+  int stages = (kSmemBudget - 1024 - kBarrierBytes - trans_bytes) / stage_bytes;
   if (stages > kMaxStages) stages = kMaxStages;
   if (ctx->force_stages && ctx->force_stages < stages) stages = ctx->force_stages;
   best.stages = stages;
@@ -1316,7 +1329,7 @@ Plan make_plan(const hola_ctx* ctx, int M, int w_dtype = HOLA_W_BF16) {
   best.n_ptiles = (ctx->V + 2 * tile_rows - 1) / (2 * tile_rows);
   best.grid = 2 * (best.n_ptiles < pairs ? best.n_ptiles : pairs);
   best.n_kblocks = i8 ? (ctx->H + 2 * kBlockK - 1) / (2 * kBlockK) : (ctx->H + kBlockK - 1) / kBlockK;
-  best.smem_bytes = stages * stage_bytes + kBarrierBytes + 1024;
+  best.smem_bytes = stages * stage_bytes + kBarrierBytes + trans_bytes + 1024;
   return best;
 }
 
@@ -1379,7 +1392,6 @@ hola_status run_lm_head(hola_ctx* ctx, const hola_verify_args* a, float* logits,
   K1Params kp;
   kp.M = M; kp.V = a->V; kp.n_ptiles = pl.n_ptiles; kp.n_kblocks = pl.n_kblocks;
   kp.stages = pl.stages; kp.nbuf = pl.nbuf; kp.n_sub = pl.n_sub; kp.N = pl.N; kp.tile_rows = pl.tile_rows; kp.ldl = ldl;
-  kp.vec_ok = (ldl % 4 == 0 && aligned16(logits)) ? 1 : 0;
   kp.logits = logits; kp.partials = ctx->partials; kp.part_stride = ctx->max_rows;
   kp.status = a->status_word ? a->status_word : ctx->status;
   kp.w_scale = a->w_scale;
