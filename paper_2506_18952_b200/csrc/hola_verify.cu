@@ -889,17 +889,27 @@ __global__ void __launch_bounds__(kK3Threads) accept_sample_kernel(const K3Param
 
   // ---- gather the k draft-token logits, draft probabilities and the uniforms (independent of the statistics)
   for (int j = threadIdx.x; j <= k; j += kK3Threads) sh_u[j] = p.u[b * (k + 1) + j];
-  for (int j = threadIdx.x; j < k; j += kK3Threads) {
-    const int x = p.tok[b * k + j];
-    sh_x[j] = x;
-    float lx = 0.f, qx = 0.f;
-    if (x >= 0 && x < V) {
-      lx = p.logits[static_cast<size_t>(row_first + j) * p.ldl + x];
-      const size_t qi = (static_cast<size_t>(b) * k + j) * V + x;
-      if (p.q_tok) qx = p.q_tok[b * k + j];
-      else qx = (p.q_dtype == HOLA_Q_BF16) ? __bfloat162float(static_cast<const __nv_bfloat16*>(p.q)[qi])
-                                           : static_cast<const float*>(p.q)[qi];
+  int x_mine = -1;                                       // (k <= 63 < kK3Threads: one draft position per thread)
+  float qx_mine = 0.f;
+  if (threadIdx.x < k) {
+    const int j = threadIdx.x;
+    x_mine = p.tok[b * k + j];
+    if (x_mine >= 0 && x_mine < V) {
+      const size_t qi = (static_cast<size_t>(b) * k + j) * V + x_mine;
+      if (p.q_tok) qx_mine = p.q_tok[b * k + j];
+      else qx_mine = (p.q_dtype == HOLA_Q_BF16) ? __bfloat162float(static_cast<const __nv_bfloat16*>(p.q)[qi])
+                                                : static_cast<const float*>(p.q)[qi];
     }
+  }
+  // Everything above reads the caller's inputs only.  When this kernel was launched with programmatic stream
+  // serialization it may have started while the GEMM kernel was still running: wait here for its results.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  for (int j = threadIdx.x; j < k; j += kK3Threads) {
+    const int x = x_mine;
+    sh_x[j] = x;
+    float lx = 0.f;
+    const float qx = qx_mine;
+    if (x >= 0 && x < V) lx = p.logits[static_cast<size_t>(row_first + j) * p.ldl + x];
     sh_lx[j] = lx; sh_qx[j] = qx;
     float hq = 0.f;
     if (p.gate_source == HOLA_GATE_DRAFT_ENTROPY) {
@@ -1457,13 +1467,18 @@ hola_status run_accept_sample(hola_ctx* ctx, const hola_verify_args* a, const fl
   cfg.blockDim = dim3(kK3Threads);
   cfg.dynamicSmemBytes = static_cast<size_t>(cpc) * sizeof(double);
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = static_cast<unsigned>(S);
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  // May be scheduled as soon as every CTA of the kernel before it in the stream has exited; it waits for that
+  // kernel's results itself.  (The GEMM kernel does not release its dependents earlier: their CTAs would then pile
+  // up on whichever SMs its first CTAs leave, and the 8-CTA clusters of a large batch run unbalanced.)
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   const cudaError_t e = vec ? cudaLaunchKernelEx(&cfg, accept_sample_kernel<true>, kp)
                             : cudaLaunchKernelEx(&cfg, accept_sample_kernel<false>, kp);
   if (e != cudaSuccess) { set_error(ctx, "launch accept_sample_kernel", e); return HOLA_ERR_CUDA; }
