@@ -87,6 +87,7 @@ struct K1Params {
   int rows;       // rows of this pass (<= n_sub * N)
   int V, n_ptiles, n_kblocks, stages, nbuf;
   int n_sub, N;   // MMAs per K step and their N (verify rows each; multiple of 16)
+  int rot;        // 1: three MMAs of N <= 128 per K step whose accumulators rotate over the four 128-column units
   int tile_rows;  // vocabulary rows per CTA per tile (<= 128, multiple of 4): balances the tiles over the pairs
   int ldl;        // row pitch of the logits buffer, in floats
   const float* w_scale;   // 8-bit W_lm: fp32 scale per vocabulary row, applied to the accumulators
@@ -413,7 +414,8 @@ __device__ __forceinline__ float scaled(float acc, float w_scale, const float* h
 //   full[12]   @0    leader CTA's copy is the live one: 2 arrivals (one producer per CTA) + the bytes of both CTAs
 //   empty[12]  @96   per CTA: the MMAs that read this slot have completed (commit, delivered to both CTAs)
 //   tfull[2]   @192  per CTA: the accumulators of a tile are complete (commit, delivered to both CTAs)
-//   tempty[2]  @208  leader's copy: all epilogue warps of the pair have read their accumulators
+//   tempty[4]  @208  leader's copy: all epilogue warps of the pair have read their accumulators (per buffer; per
+//                    128-column unit when the accumulators rotate)
 //   tensor-memory base @256, abort flag @260
 //   8-bit W_lm only: rawfull[12] @272 per CTA: the int8 tile of the slot has landed; rawempty[12] @368 per CTA: the
 //   converter warps have expanded it.  full[] then collects, besides the hidden bytes, one arrival per converter warp.
@@ -464,10 +466,8 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
         mbar_init(rawempty_bar + 8 * i, kConvWarps);
       }
     }
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(tfull_bar + 8 * i, 1);
-      mbar_init(tempty_bar + 8 * i, 2 * kNumEpi);
-    }
+    for (int i = 0; i < 2; ++i) mbar_init(tfull_bar + 8 * i, 1);
+    for (int i = 0; i < 4; ++i) mbar_init(tempty_bar + 8 * i, 2 * kNumEpi);
     *abort_flag = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_hidden) : "memory");
@@ -483,7 +483,11 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
 
   const int my_tiles = (p.n_ptiles - pair + npairs - 1) / npairs;
   const int sub_chunks = (p.N + 31) >> 5;                // 32-column chunks per MMA's accumulator
-  // accumulator of MMA s of buffer b starts at column b * 256 + s * 256 (two buffers only when n_sub == 1)
+  // Accumulators.  rot == 0: MMA s of buffer b starts at column b * 256 + s * 256 (two buffers only when
+  // n_sub == 1; with two MMAs the next tile waits until the whole tile has been read out).  rot == 1 (257..384 rows):
+  // three MMAs of N <= 128; MMA s of tile t owns the 128-column unit (3 t + s) % 4, so a tile's first unit is always
+  // free and its second and third are the first two the epilogue of the tile before it reads out: the tensor pipe
+  // restarts after one epilogue round instead of after the whole read-out.
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (one per CTA)
@@ -529,6 +533,36 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
+      if (p.rot) {
+        uint32_t used = 0;                               // bit u: parity of the number of tiles that used unit u
+        for (int t = 0; t < my_tiles && ok; ++t) {
+          for (int kb = 0; kb < p.n_kblocks && ok; ++kb) {
+            if (!mbar_wait(full_bar + 8 * stage, phase, abort_flag, p.status)) { ok = false; break; }
+            tc_fence_after();
+            const uint64_t adesc = desc0 + ((stage * stage_bytes) >> 4);
+            const uint64_t bdesc0 = adesc + (kWBlockBytes >> 4);
+#pragma unroll
+            for (int u = 0; u < 3; ++u) {
+              const uint32_t unit = static_cast<uint32_t>(3 * t + u) & 3u;
+              if (kb == 0) {                             // the epilogue must have read this unit's previous tile
+                const uint32_t par = (used >> unit) & 1u;
+                if (!mbar_wait(tempty_bar + 8 * unit, par ^ 1u, abort_flag, p.status)) { ok = false; break; }
+                used ^= 1u << unit;
+                tc_fence_after();
+              }
+              const uint32_t d = tmem_base + unit * 128u;
+              const uint64_t bdesc = bdesc0 + u * (hid_block_bytes >> 4);
+              umma<kI8>(d, adesc, bdesc, idesc, kb != 0 ? 1u : 0u);
+#pragma unroll
+              for (int kk = 1; kk < kBlockK / 16; ++kk) umma<kI8>(d, adesc + 2 * kk, bdesc + 2 * kk, idesc, 1u);
+            }
+            if (!ok) break;
+            umma_commit_pair(empty_bar + 8 * stage);
+            if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+          }
+          if (ok) umma_commit_pair(tfull_bar);           // all three units of this tile are complete in both CTAs
+        }
+      } else
       for (int t = 0; t < my_tiles && ok; ++t) {
         const int buf = t % p.nbuf;
         const uint32_t acc_phase = static_cast<uint32_t>(t / p.nbuf) & 1u;
@@ -568,12 +602,15 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
     // Tensor memory -> registers (thread = vocabulary entry, register = verify row) -> logits buffer, and the same
     // values, transposed through a small shared-memory buffer 16 rows at a time (thread = verify row and half of the
     // warp's 32 vocabulary entries), into thread-private softmax statistics that live in registers for the whole
-    // kernel.  A warp owns one lane quarter (fixed by its id) and every kGroups-th 32-column chunk.
+    // kernel.  A warp owns one lane quarter (fixed by its id) and every kGroups-th 32-column chunk (with rotating
+    // accumulators: chunk `group` of every unit, so that all warps read unit after unit and free each at once).
     const int quarter = warp & 3;                        // tensor-memory lanes 32*quarter .. +31
     const int group = (warp - 2) >> 2;
     const uint32_t leader_tempty = map_to_cta(tempty_bar, 0);
     const int n_chunks = p.n_sub * sub_chunks;
-    const int my_chunks = group < n_chunks ? (n_chunks - 1 - group) / kGroups + 1 : 0;
+    const bool rot = p.rot != 0;
+    const int my_chunks = rot ? (group < sub_chunks ? p.n_sub : 0)
+                              : (group < n_chunks ? (n_chunks - 1 - group) / kGroups + 1 : 0);
     float* tbuf = trans_base + (warp - 2) * (kTransBytes / 4);
     const int trow = lane & 15, thalf = lane >> 4;       // row of a transposition step; which 16 of the 32 entries
     Stats st[kEpiSlots][2];
@@ -594,24 +631,31 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
       const int n16 = max(0, min(16, nv - thalf * 16));
       const int vocab16 = vbase + quarter * 32 + thalf * 16;
       const float w_scale = ((kW8 || kI8) && vocab_ok) ? p.w_scale[vocab] : 1.f;   // 8-bit W_lm: the row's scale
-      const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + buf * 256;
-      if (my_chunks == 0) {
-        tc_fence_before();
+      const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+      if (my_chunks == 0) {                              // nothing to read: the accumulators are free as far as this
+        tc_fence_before();                               // warp is concerned
         __syncwarp();
-        if (lane == 0) mbar_arrive_cluster(leader_tempty + 8 * buf);
+        if (lane == 0) {
+          if (rot) {
+            for (int u = 0; u < p.n_sub; ++u) mbar_arrive_cluster(leader_tempty + 8 * ((3 * t + u) & 3));
+          } else {
+            mbar_arrive_cluster(leader_tempty + 8 * buf);
+          }
+        }
       }
 #pragma unroll
       for (int slot = 0; slot < kEpiSlots; ++slot) {
         if (slot < my_chunks) {
-          const int ch = group + slot * kGroups;
+          const int ch = rot ? slot * sub_chunks + group : group + slot * kGroups;
           const int sub = ch / sub_chunks, j = ch - sub * sub_chunks;
+          const int unit = (3 * t + slot) & 3;           // (rotating accumulators only)
           float v[32];
           __syncwarp();                                  // tcgen05.ld is warp-collective: reconverge first
-          tmem_ld32(lane_addr + sub * 256 + j * 32, v);
-          if (slot == my_chunks - 1) {                   // this warp's accumulators may be overwritten
+          tmem_ld32(lane_addr + (rot ? unit * 128 : buf * 256 + sub * 256) + j * 32, v);
+          if (rot || slot == my_chunks - 1) {            // this warp's accumulators (of this unit) may be overwritten
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(leader_tempty + 8 * buf);
+            if (lane == 0) mbar_arrive_cluster(leader_tempty + 8 * (rot ? unit : buf));
           }
           const int c0 = j * 32;                         // first column of the chunk inside its MMA
           const int r0 = p.row0 + sub * p.N + c0;        // verify row of column c0
@@ -674,7 +718,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
         o.arg = __shfl_xor_sync(0xffffffffu, a.arg, 16);
         a = stats_merge(a, o);
         if (slot < my_chunks && thalf == 0) {
-          const int ch = group + slot * kGroups;
+          const int ch = rot ? slot * sub_chunks + group : group + slot * kGroups;
           const int sub = ch / sub_chunks, j = ch - sub * sub_chunks;
           const int c = j * 32 + half * kTransRows + trow;           // column inside its MMA
           const int r = sub * p.N + c;                               // row inside the pass
@@ -1216,7 +1260,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 struct Plan {
-  int n_sub, N, rows_per_pass, passes, grid, stages, nbuf, n_ptiles, n_kblocks, smem_bytes, tile_rows;
+  int n_sub, N, rows_per_pass, passes, grid, stages, nbuf, rot, n_ptiles, n_kblocks, smem_bytes, tile_rows;
   double est_seconds;   // rough duration of all passes (the cost the split was chosen by)
 };
 
@@ -1237,6 +1281,7 @@ struct hola_ctx {
   void* st_hidden; int* st_tok; void* st_q; float* st_u;
   int* st_accept; int* st_next; float* st_entropy; float* st_logZ;
   int force_stages;
+  int no_rot;                 // tuning override: never use the rotating accumulator units
   cudaStream_t copy_stream;   // hola_verify_host: the draft tensor travels here while the GEMM runs
   cudaEvent_t copy_done;
   int host_overlap;           // 1: copy the draft tensor on copy_stream while the GEMM runs
@@ -1308,7 +1353,9 @@ Plan make_plan(const hola_ctx* ctx, int M, int w_dtype = HOLA_W_BF16) {
   const double t_hbm = (w8 || i8 ? 1.0 : 2.0) * ctx->V * static_cast<double>(ctx->H) / 6.4e12;
   for (int passes = p_min; passes <= p_min + 3; ++passes) {
     const int r = (rows + passes - 1) / passes;
-    const int n_sub = r > kMaxN ? 2 : 1;
+    // up to 256 rows: one MMA, two accumulator buffers; up to 384: three MMAs of N <= 128 on rotating 128-column
+    // units; beyond: two MMAs of N <= 256 that fill the tensor memory
+    const int n_sub = (r > 3 * 128 || (ctx->no_rot && r > kMaxN)) ? 2 : (r > kMaxN ? 3 : 1);
     const int N = round_up((r + n_sub - 1) / n_sub, i8 ? 32 : 16);
     const double t_mma = 2.0 * n_sub * N * static_cast<double>(ctx->V) * ctx->H / (i8 ? 2.8e15 : 1.4e15);
     const double cost = passes * ((t_mma > t_hbm ? t_mma : t_hbm) + 6e-6);
@@ -1327,6 +1374,7 @@ Plan make_plan(const hola_ctx* ctx, int M, int w_dtype = HOLA_W_BF16) {
   if (ctx->force_stages && ctx->force_stages < stages) stages = ctx->force_stages;
   best.stages = stages;
   best.nbuf = best.n_sub == 1 ? 2 : 1;
+  best.rot = best.n_sub == 3 ? 1 : 0;
   // Vocabulary rows per CTA per tile: the smallest multiple of 4 that covers V in the fewest whole rounds over
   // all pairs, so that every pair streams the same number of bytes (V = 32000 on 74 pairs: 2 rounds of 112 + 112
   // rows instead of 1.69 rounds of 128 + 128).
@@ -1401,7 +1449,7 @@ hola_status run_lm_head(hola_ctx* ctx, const hola_verify_args* a, float* logits,
   if (s != HOLA_OK) return s;
   K1Params kp;
   kp.M = M; kp.V = a->V; kp.n_ptiles = pl.n_ptiles; kp.n_kblocks = pl.n_kblocks;
-  kp.stages = pl.stages; kp.nbuf = pl.nbuf; kp.n_sub = pl.n_sub; kp.N = pl.N; kp.tile_rows = pl.tile_rows; kp.ldl = ldl;
+  kp.stages = pl.stages; kp.nbuf = pl.nbuf; kp.rot = pl.rot; kp.n_sub = pl.n_sub; kp.N = pl.N; kp.tile_rows = pl.tile_rows; kp.ldl = ldl;
   kp.logits = logits; kp.partials = ctx->partials; kp.part_stride = ctx->max_rows;
   kp.status = a->status_word ? a->status_word : ctx->status;
   kp.w_scale = a->w_scale;
@@ -1571,6 +1619,7 @@ hola_status hola_create(hola_ctx** out, int device, int maxB, int maxK, int H, i
   if (const char* e = getenv("HOLA_HOST_OVERLAP")) ctx->host_overlap = atoi(e) != 0;   // tuning override
   ctx->host_lazy_q = -1;
   if (const char* e = getenv("HOLA_HOST_LAZY_Q")) ctx->host_lazy_q = atoi(e) != 0;     // override for tests and sweeps
+  if (const char* e = getenv("HOLA_ROT")) ctx->no_rot = atoi(e) == 0;                  // tuning override for sweeps
   if (const char* e = getenv("HOLA_STAGES")) {           // tuning override for sweeps: fewer ring slots
     const int st = atoi(e);
     if (st >= 2 && st <= kMaxStages) ctx->force_stages = st;

@@ -144,6 +144,9 @@ def test_tiny_config(binding, tau):
     (5, 2, 64, 1001, torch.bfloat16),      # odd V: scalar load/store paths
     (130, 0, 64, 777, torch.bfloat16),     # k = 0: plain draw from p
     (90, 7, 128, 640, torch.float32),      # 720 rows: more row blocks than one pass holds
+    (50, 5, 128, 80000, torch.bfloat16),   # 300 rows on rotating accumulator units (N = 112: the last 32-column
+                                           # chunk half empty); five tiles per CTA pair = a full rotation period
+    (46, 5, 64, 60000, torch.bfloat16),    # 276 rows: N = 96, one epilogue warp group without a chunk; four tiles
 ])
 def test_ragged_shapes(binding, B, k, H, V, qd):
     w = workloads.gaussian_head("ragged", B, k, H, V, seed=B + V, device=DEV, w_std=0.3, sigma=1.0, q_dtype=qd,
@@ -447,9 +450,11 @@ def test_int8_head_matches_oracle_on_dequantised_weights(binding, B, k, H, V, qd
 
 @pytest.mark.parametrize("B,k,H,V,qd", [
     (1, 4, 64, 1000, torch.float32),       # 5 rows: N = 32
-    (37, 6, 256, 5000, torch.bfloat16),    # 259 rows: two MMAs of N = 160 per K step, ragged vocabulary tail
+    (37, 6, 256, 5000, torch.bfloat16),    # 259 rows: three MMAs of N = 96 per K step, ragged vocabulary tail
     (5, 2, 80, 1001, torch.bfloat16),      # K tail (H = 80 < one 128-wide block), odd V
     (90, 7, 384, 640, torch.float32),      # 720 rows: two passes
+    (50, 5, 128, 80000, torch.bfloat16),   # 300 rows, N = 128 on rotating units, five tiles per CTA pair
+    (75, 5, 128, 3000, torch.bfloat16),    # 450 rows: two MMAs of N = 256 fill the tensor memory
 ])
 def test_w8a8_head_matches_oracle_on_dequantised_operands(binding, B, k, H, V, qd):
     w = workloads.gaussian_head("w8a8", B, k, H, V, seed=B + V, device=DEV, w_std=0.3, sigma=1.0, q_dtype=qd,
