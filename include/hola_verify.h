@@ -131,6 +131,40 @@ hola_status hola_verify(hola_ctx* ctx, const hola_verify_args* args, void* cuda_
  * hola_create) forces one or the other.  The host buffers must stay valid until the call returns. */
 hola_status hola_verify_host(hola_ctx* ctx, const hola_verify_args* args, void* cuda_stream);
 
+/* Vocabulary-parallel form of the verify step: `world` ranks (normally one GPU each) hold contiguous ranges of the
+ * vocabulary rows of W_lm, and of the vocabulary axis of draft_q; hidden, draft_tok, uniforms and q_j(x_j) are the
+ * same on every rank.  The paper describes the step on one device; this is its natural split over several, with the
+ * same results (the statistics of disjoint vocabulary ranges merge exactly, Eq. 1's entropy included; the draw of
+ * Algorithm 1's fallback is an inverse-CDF search over ranges taken in rank order).  One step is three calls with two
+ * small all-gathers between them, which the caller makes (NCCL, or anything else):
+ *   1. hola_shard_lm_head: logits of this rank's range (scratch or logits_out), and record_out: per verify row the
+ *      statistics of those logits, per draft position the logit of x_j where this rank owns x_j.
+ *      -> all-gather of the records (hola_shard_record_bytes each), in rank order, into `records`.
+ *   2. hola_shard_accept: merged entropy / logZ of all rows, the accept test, accept_len (identical on every rank;
+ *      with the greedy fallback next_tok too, and the step ends here), and mass_out[b] = { mass of max(0, p_n - q_n),
+ *      mass of p_n } of row n = accept_len inside this rank's range.
+ *      -> all-gather of the masses ([B][2] doubles each) into `masses`.
+ *   3. hola_shard_sample: every rank finds the range that holds the point u_k * R; that rank alone searches its
+ *      range and writes the GLOBAL token index to next_tok[b], the others write -1 (a max over ranks gives the step's
+ *      result).
+ * In `args`, V is this rank's share (the context is created for it), W_lm / w_scale / draft_q / logits_out are the
+ * rank's own parts, draft_tok holds global indices.  gate_source must be the target entropy. */
+typedef struct hola_shard_args {
+  int32_t world;          /* ranks the vocabulary is split over, >= 1                                        */
+  int32_t rank;           /* this rank, 0 .. world-1                                                         */
+  int32_t v_offset;       /* global index of this rank's first vocabulary row                                */
+  int32_t V_global;       /* size of the whole vocabulary                                                    */
+  const float* q_tok;     /* dev in  fp32 [B][k]: q_j(x_j), the same on every rank                           */
+  void* record_out;       /* dev out, hola_shard_record_bytes(B, k) bytes, 16-byte aligned (call 1)          */
+  const void* records;    /* dev in, world records in rank order, 16-byte aligned (calls 2 and 3)            */
+  double* mass_out;       /* dev out fp64 [B][2] (call 2)                                                    */
+  const double* masses;   /* dev in  fp64 [world][B][2] (call 3)                                             */
+} hola_shard_args;
+size_t hola_shard_record_bytes(int B, int k);
+hola_status hola_shard_lm_head(hola_ctx* ctx, const hola_verify_args* args, const hola_shard_args* shard, void* cuda_stream);
+hola_status hola_shard_accept(hola_ctx* ctx, const hola_verify_args* args, const hola_shard_args* shard, void* cuda_stream);
+hola_status hola_shard_sample(hola_ctx* ctx, const hola_verify_args* args, const hola_shard_args* shard, void* cuda_stream);
+
 /* Bytes the last hola_verify_host call on this context copied host-to-device and device-to-host. */
 hola_status hola_host_traffic(const hola_ctx* ctx, unsigned long long* h2d_bytes, unsigned long long* d2h_bytes);
 

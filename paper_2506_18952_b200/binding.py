@@ -21,7 +21,8 @@ HOLA_W_BF16, HOLA_W_INT8, HOLA_W8A8 = 0, 1, 2
 FLAG_BAD_TOKEN, FLAG_BAD_UNIFORM, FLAG_TIMEOUT, FLAG_R_ZERO = 1, 2, 4, 8
 
 EXPORTS = ["hola_create", "hola_destroy", "hola_workspace_bytes", "hola_verify", "hola_verify_host",
-           "hola_lm_head_entropy", "hola_accept_sample", "hola_host_traffic", "hola_lm_head_entropy_static", "hola_quantize_w8", "hola_plan", "hola_plan_ex", "hola_profile_begin", "hola_profile_end", "hola_strerror", "hola_last_cuda_error",
+           "hola_lm_head_entropy", "hola_accept_sample", "hola_host_traffic", "hola_shard_record_bytes", "hola_shard_lm_head",
+           "hola_shard_accept", "hola_shard_sample", "hola_lm_head_entropy_static", "hola_quantize_w8", "hola_plan", "hola_plan_ex", "hola_profile_begin", "hola_profile_end", "hola_strerror", "hola_last_cuda_error",
            "hola_version"]
 
 
@@ -38,6 +39,12 @@ class hola_verify_args(ctypes.Structure):
                 ("status_word", ctypes.c_void_p), ("gate_source", ctypes.c_int32), ("fallback", ctypes.c_int32),
                 ("draft_entropy", ctypes.c_void_p), ("w_dtype", ctypes.c_int32), ("reserved_", ctypes.c_int32),
                 ("w_scale", ctypes.c_void_p)]
+
+
+class hola_shard_args(ctypes.Structure):
+    _fields_ = [("world", ctypes.c_int32), ("rank", ctypes.c_int32), ("v_offset", ctypes.c_int32),
+                ("V_global", ctypes.c_int32), ("q_tok", ctypes.c_void_p), ("record_out", ctypes.c_void_p),
+                ("records", ctypes.c_void_p), ("mass_out", ctypes.c_void_p), ("masses", ctypes.c_void_p)]
 
 
 class hola_plan_info(ctypes.Structure):
@@ -76,6 +83,13 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
     lib.hola_plan_ex.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.POINTER(hola_plan_info)]
     lib.hola_profile_begin.restype = ctypes.c_int
     lib.hola_profile_begin.argtypes = [ctypes.c_void_p, ctypes.c_int]
+    lib.hola_shard_record_bytes.restype = ctypes.c_size_t
+    lib.hola_shard_record_bytes.argtypes = [ctypes.c_int, ctypes.c_int]
+    for name in ("hola_shard_lm_head", "hola_shard_accept", "hola_shard_sample"):
+        fn = getattr(lib, name)
+        fn.restype = ctypes.c_int
+        fn.argtypes = [ctypes.c_void_p, ctypes.POINTER(hola_verify_args), ctypes.POINTER(hola_shard_args),
+                       ctypes.c_void_p]
     lib.hola_host_traffic.restype = ctypes.c_int
     lib.hola_host_traffic.argtypes = [ctypes.c_void_p, ctypes.POINTER(ctypes.c_ulonglong),
                                       ctypes.POINTER(ctypes.c_ulonglong)]
@@ -192,6 +206,13 @@ class HolaVerify:
 
     def hola_profile_begin(self, max_calls: int):
         _check(self.lib, self._ctx, self.lib.hola_profile_begin(self._ctx, max_calls), "hola_profile_begin")
+
+    def hola_shard_call(self, which: str, args, shard, stream=None):
+        """hola_shard_lm_head / hola_shard_accept / hola_shard_sample on prepared argument structs."""
+        if which not in ("hola_shard_lm_head", "hola_shard_accept", "hola_shard_sample"):
+            raise HolaError(f"unknown entry point {which}")
+        st = getattr(self.lib, which)(self._ctx, ctypes.byref(args), ctypes.byref(shard), _stream_ptr(stream))
+        _check(self.lib, self._ctx, st, which)
 
     def hola_host_traffic(self) -> tuple[int, int]:
         """(host-to-device, device-to-host) bytes of the last hola_verify_host call."""

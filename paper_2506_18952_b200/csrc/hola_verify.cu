@@ -107,7 +107,16 @@ struct K3Params {
   const void* q;
   int q_dtype;
   const float* q_tok;           // optional fp32 [B][k]: q_j(x_j) already gathered (then q is read at row n only)
-  int phase;                    // 0: the whole step; 1: stop after the accept test (accept_len, statistics written)
+  int phase;                    // 0: the whole step; 1: stop after the accept test (accept_len, statistics written);
+                                // vocabulary-parallel form: 3: stop after the masses of row n inside this shard,
+                                // 4: the draw, by the shard that holds the point u * R
+  // Vocabulary-parallel form (shard_world > 0): V, logits and q cover this rank's V entries starting at v_offset;
+  // draft tokens and next_tok are global indices below V_global.
+  int shard_world, shard_rank, v_offset, V_global;
+  const float* lx_all;          // [world] records, rec_stride floats apart: logit of x_j where its owner found it, else -inf
+  int rec_stride;               // floats from one rank's record to the next
+  double* mass_out;             // phase 3: [B][2] mass of max(0, p_n - q_n) and of p_n inside this shard
+  const double* mass_all;       // phase 4: [world][B][2], the same from every rank
   const float* u;
   float tau;
   int gate_source;          // hola_gate_source
@@ -847,6 +856,32 @@ __global__ void __launch_bounds__(256) finalize_kernel(const float4* partials, i
   if (lane == 0) stats_to_outputs(st, &logZ[row], &entropy[row]);
 }
 
+// Vocabulary-parallel form, first exchange record of a rank: per verify row the statistics of this shard's logits
+// (m, s, t, arg-max as a GLOBAL vocabulary index), then per draft position the logit of the draft token if this shard
+// owns it (-inf otherwise).  Blocks 0 .. ceil(M/8)-1 merge the per-CTA partials, the others gather the logits.
+__global__ void __launch_bounds__(256) shard_record_kernel(const float4* partials, int nparts, int part_stride, int M,
+                                                           int v_offset, int V, const float* logits, int ldl,
+                                                           const int* tok, int B, int k, float4* stats_out,
+                                                           float* lx_out) {
+  const int row_blocks = (M + 7) / 8;
+  if (static_cast<int>(blockIdx.x) < row_blocks) {
+    const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (row >= M) return;
+    Stats st = warp_merge_partials(partials, nparts, part_stride, row, lane);
+    if (lane == 0) {
+      const int arg = st.arg == 0x7fffffff ? st.arg : st.arg + v_offset;
+      stats_out[row] = make_float4(st.m, st.s, st.t, __int_as_float(arg));
+    }
+  } else {
+    const int i = (blockIdx.x - row_blocks) * 256 + threadIdx.x;
+    if (i >= B * k) return;
+    const int b = i / k, j = i - b * k;
+    const int x = tok[i] - v_offset;
+    lx_out[i] = (x >= 0 && x < V) ? logits[static_cast<size_t>(b * (k + 1) + j) * ldl + x] : -CUDART_INF_F;
+  }
+}
+
 // ------------------------------------------------------------------------------------------------ K3
 __device__ __forceinline__ double warp_sum_f64(double x) {
 #pragma unroll
@@ -935,10 +970,12 @@ __global__ void __launch_bounds__(kK3Threads) accept_sample_kernel(const K3Param
   for (int j = threadIdx.x; j <= k; j += kK3Threads) sh_u[j] = p.u[b * (k + 1) + j];
   int x_mine = -1;                                       // (k <= 63 < kK3Threads: one draft position per thread)
   float qx_mine = 0.f;
+  const bool shard = p.shard_world > 0;
+  const int Vtok = shard ? p.V_global : V;               // range of valid token ids
   if (threadIdx.x < k) {
     const int j = threadIdx.x;
     x_mine = p.tok[b * k + j];
-    if (x_mine >= 0 && x_mine < V) {
+    if (x_mine >= 0 && x_mine < Vtok) {
       const size_t qi = (static_cast<size_t>(b) * k + j) * V + x_mine;
       if (p.q_tok) qx_mine = p.q_tok[b * k + j];
       else qx_mine = (p.q_dtype == HOLA_Q_BF16) ? __bfloat162float(static_cast<const __nv_bfloat16*>(p.q)[qi])
@@ -953,7 +990,14 @@ __global__ void __launch_bounds__(kK3Threads) accept_sample_kernel(const K3Param
     sh_x[j] = x;
     float lx = 0.f;
     const float qx = qx_mine;
-    if (x >= 0 && x < V) lx = p.logits[static_cast<size_t>(row_first + j) * p.ldl + x];
+    if (x >= 0 && x < Vtok) {
+      if (shard) {                                       // exactly one shard owns x and left its logit there
+        lx = -CUDART_INF_F;
+        for (int r = 0; r < p.shard_world; ++r) lx = fmaxf(lx, p.lx_all[static_cast<size_t>(r) * p.rec_stride + b * k + j]);
+      } else {
+        lx = p.logits[static_cast<size_t>(row_first + j) * p.ldl + x];
+      }
+    }
     sh_lx[j] = lx; sh_qx[j] = qx;
     float hq = 0.f;
     if (p.gate_source == HOLA_GATE_DRAFT_ENTROPY) {
@@ -989,7 +1033,7 @@ __global__ void __launch_bounds__(kK3Threads) accept_sample_kernel(const K3Param
     int n = k;
     for (int j = 0; j < k; ++j) {
       const int x = sh_x[j];
-      if (x < 0 || x >= V) { flags |= HOLA_FLAG_BAD_TOKEN; n = j; break; }
+      if (x < 0 || x >= Vtok) { flags |= HOLA_FLAG_BAD_TOKEN; n = j; break; }
       const float gate_value = p.gate_source == HOLA_GATE_DRAFT_ENTROPY ? sh_Hq[j] : sh_H[j];
       if (gate_value < p.tau) continue;                  // entropy gate: fast path keeps the draft token
       if (p.fallback == HOLA_FALLBACK_GREEDY) {          // the verifier's own token, or the run ends here
@@ -1007,7 +1051,7 @@ __global__ void __launch_bounds__(kK3Threads) accept_sample_kernel(const K3Param
     if (rank == 0) {
       p.accept_len[b] = n;
       if (p.fallback == HOLA_FALLBACK_GREEDY) {          // greedy: argmax p_n follows the accepted run; no draw
-        p.next_tok[b] = min(max(sh_amax[n], 0), V - 1);
+        p.next_tok[b] = min(max(sh_amax[n], 0), Vtok - 1);
         if (flags && p.status) atomicOr(p.status, flags);
       } else if (p.phase == 1 && flags && p.status) {
         atomicOr(p.status, flags);
@@ -1031,6 +1075,41 @@ __global__ void __launch_bounds__(kK3Threads) accept_sample_kernel(const K3Param
   const int mine = max(0, min(nchunks, c_first + cpc) - c_first);
   const int per_lane = (mine + 31) / 32;
   bool residual = n < k;
+
+  // Vocabulary-parallel draw: every rank holds every rank's two masses of row n, so all of them agree on which mass
+  // counts (the residual's unless it vanishes everywhere), on the total R and on the shard that holds the point u * R.
+  double shard_target = 0.0;
+  if (shard && p.phase == 4) {
+    const double* mass = p.mass_all + static_cast<size_t>(b) * 2;
+    const size_t rs = static_cast<size_t>(p.B) * 2;
+    double tot_res = 0.0;
+    for (int r = 0; r < p.shard_world; ++r) tot_res += mass[r * rs];
+    const bool use_p = !residual || !(tot_res > 0.0);
+    if (use_p && residual) {
+      residual = false;
+      if (threadIdx.x == 0) sh_flags |= HOLA_FLAG_R_ZERO;
+    }
+    const int idx = use_p ? 1 : 0;
+    double total = 0.0;
+    for (int r = 0; r < p.shard_world; ++r) total += mass[r * rs + idx];
+    unsigned uflags = 0;
+    const double target = static_cast<double>(clamp_uniform(sh_u[k], uflags)) * total;
+    int owner = -1, last_mass = 0;
+    double before = 0.0, cum = 0.0;
+    for (int r = 0; r < p.shard_world; ++r) {
+      const double m = mass[r * rs + idx];
+      if (m > 0.0) last_mass = r;
+      if (owner < 0 && cum + m > target) { owner = r; before = cum; }
+      cum += m;
+    }
+    shard_target = target - before;
+    if (owner < 0) { owner = last_mass; shard_target = CUDART_INF; }     // rounding: the last entry with mass
+    if (owner != p.shard_rank) {
+      if (rank == 0 && threadIdx.x == 0) p.next_tok[b] = -1;
+      return;                                            // same decision in every CTA of the cluster
+    }
+    __syncthreads();
+  }
 
   for (int attempt = 0; attempt < 2; ++attempt) {
     for (int c0 = warp; c0 < mine; c0 += kK3Unroll * kK3Warps) {
@@ -1070,7 +1149,22 @@ __global__ void __launch_bounds__(kK3Threads) accept_sample_kernel(const K3Param
     // every CTA: total mass and the slice that holds u * R (identical arithmetic everywhere)
     double R = 0.0;
     for (int r2 = 0; r2 < S; ++r2) R += sh_tot[attempt][r2];
-    if (!(R > 0.0) && residual) {                        // p <= q everywhere: draw from p instead
+    if (shard && p.phase == 3) {
+      // the shard's masses of row n: of the residual, then (second pass, q taken as 0) of p itself
+      if (rank == 0 && threadIdx.x == 0) {
+        p.mass_out[b * 2 + attempt] = R;
+        if (!residual && attempt == 0) p.mass_out[b * 2 + 1] = R;          // bonus position: both are the mass of p
+        const unsigned fl = sh_flags;
+        if (fl && p.status && (attempt == 1 || !residual)) atomicOr(p.status, fl);
+      }
+      if (residual) {
+        residual = false;
+        __syncthreads();
+        continue;
+      }
+      return;
+    }
+    if (!(R > 0.0) && residual && !shard) {              // p <= q everywhere: draw from p instead
       residual = false;
       if (threadIdx.x == 0) sh_flags |= HOLA_FLAG_R_ZERO;
       __syncthreads();
@@ -1078,7 +1172,7 @@ __global__ void __launch_bounds__(kK3Threads) accept_sample_kernel(const K3Param
     }
     unsigned uflags = 0;
     const float uk = clamp_uniform(sh_u[k], uflags);
-    const double target = static_cast<double>(uk) * R;
+    const double target = shard ? shard_target : static_cast<double>(uk) * R;
     int rstar = -1, last_mass = 0;
     double before_slice = 0.0;
     {
@@ -1143,7 +1237,7 @@ __global__ void __launch_bounds__(kK3Threads) accept_sample_kernel(const K3Param
       if (lane == 0) {
         int tokn = (c_first + cstar) * kChunk + src * 4 + idx;
         if (tokn >= V) tokn = V - 1;
-        p.next_tok[b] = tokn;
+        p.next_tok[b] = tokn + (shard ? p.v_offset : 0);
         const unsigned fl = sh_flags | uflags;
         if (fl && p.status) atomicOr(p.status, fl);
       }
@@ -1485,9 +1579,19 @@ hola_status run_lm_head(hola_ctx* ctx, const hola_verify_args* a, float* logits,
   return HOLA_OK;
 }
 
+// What the accept/sample kernel needs to know in the vocabulary-parallel form.
+struct ShardLaunch {
+  int world, rank, v_offset, V_global;
+  const float4* stats_all;   // world records (statistics, then draft-token logits)
+  int rec_floats;            // floats per record
+  double* mass_out;
+  const double* mass_all;
+};
+
 hola_status run_accept_sample(hola_ctx* ctx, const hola_verify_args* a, const float* logits, int ldl, int combine,
-                              int nparts, cudaStream_t stream, const float* q_tok = nullptr, int phase = 0) {
-  K3Params kp;
+                              int nparts, cudaStream_t stream, const float* q_tok = nullptr, int phase = 0,
+                              const ShardLaunch* sh = nullptr) {
+  K3Params kp{};
   kp.q_tok = q_tok; kp.phase = phase;
   kp.B = a->B; kp.k = a->k; kp.V = a->V; kp.ldl = ldl; kp.logits = logits;
   kp.partials = ctx->partials; kp.nparts = nparts; kp.part_stride = ctx->max_rows; kp.combine = combine;
@@ -1503,6 +1607,13 @@ hola_status run_accept_sample(hola_ctx* ctx, const hola_verify_args* a, const fl
   }
   kp.accept_len = a->accept_len; kp.next_tok = a->next_tok; kp.entropy = a->entropy; kp.logZ = a->logZ;
   kp.status = a->status_word ? a->status_word : ctx->status;
+  if (sh) {
+    kp.shard_world = sh->world; kp.shard_rank = sh->rank; kp.v_offset = sh->v_offset; kp.V_global = sh->V_global;
+    kp.lx_all = reinterpret_cast<const float*>(sh->stats_all) + 4 * static_cast<size_t>(a->B) * (a->k + 1);
+    kp.rec_stride = sh->rec_floats;
+    kp.mass_out = sh->mass_out; kp.mass_all = sh->mass_all;
+    if (combine) { kp.partials = sh->stats_all; kp.nparts = sh->world; kp.part_stride = sh->rec_floats / 4; }
+  }
   const bool vec = (a->V % 4 == 0) && (ldl % 4 == 0) && aligned16(logits) && (a->k == 0 || aligned16(a->draft_q));
   // cluster size: as many CTAs per sequence as keeps the grid within a few waves of the SMs
   const int nchunks = (a->V + kChunk - 1) / kChunk;
@@ -1959,6 +2070,80 @@ hola_status hola_verify_host(hola_ctx* ctx, const hola_verify_args* a, void* cud
   if (e != cudaSuccess) { set_error(ctx, "device-to-host copy", e); return HOLA_ERR_CUDA; }
   ctx->last_h2d = up; ctx->last_d2h = down;
   return HOLA_OK;
+}
+
+// ---- vocabulary-parallel form: three calls per step with two small all-gathers between them (made by the caller)
+size_t hola_shard_record_bytes(int B, int k) {
+  if (B <= 0 || k < 0) return 0;
+  const size_t rows = static_cast<size_t>(B) * (k + 1);
+  return rows * 16 + align_up(static_cast<size_t>(B) * k * 4, 16);
+}
+
+static hola_status check_shard(const hola_ctx* ctx, const hola_verify_args* a, const hola_shard_args* sh) {
+  if (!sh || sh->world < 1 || sh->rank < 0 || sh->rank >= sh->world) return HOLA_ERR_INVALID_ARG;
+  if (sh->v_offset < 0 || sh->V_global < sh->v_offset + a->V) return HOLA_ERR_INVALID_ARG;
+  if (a->gate_source != HOLA_GATE_TARGET_ENTROPY) return HOLA_ERR_INVALID_ARG;   // H(q_j) would need q of all shards
+  (void)ctx;
+  return HOLA_OK;
+}
+
+static ShardLaunch shard_launch(const hola_verify_args* a, const hola_shard_args* sh) {
+  ShardLaunch l;
+  l.world = sh->world; l.rank = sh->rank; l.v_offset = sh->v_offset; l.V_global = sh->V_global;
+  l.stats_all = static_cast<const float4*>(sh->records);
+  l.rec_floats = static_cast<int>(hola_shard_record_bytes(a->B, a->k) / 4);
+  l.mass_out = sh->mass_out; l.mass_all = sh->masses;
+  return l;
+}
+
+hola_status hola_shard_lm_head(hola_ctx* ctx, const hola_verify_args* a, const hola_shard_args* sh, void* cuda_stream) {
+  hola_status s = check_common(ctx, a);
+  if (s != HOLA_OK) return s;
+  if (a->B == 0) return HOLA_OK;
+  if ((s = check_lm_head_args(ctx, a)) != HOLA_OK) return s;
+  if ((s = check_shard(ctx, a, sh)) != HOLA_OK) return s;
+  if (!sh->record_out || !aligned16(sh->record_out) || (a->k > 0 && !a->draft_tok)) return HOLA_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const int M = a->B * (a->k + 1);
+  const Plan pl = make_plan(ctx, M, a->w_dtype);
+  float* logits = a->logits_out ? a->logits_out : ctx->logits;
+  const int ldl = a->logits_out ? a->V : ctx->ldl;
+  if ((s = run_lm_head(ctx, a, logits, ldl, pl, stream)) != HOLA_OK) return s;
+  float4* stats_out = static_cast<float4*>(sh->record_out);
+  float* lx_out = reinterpret_cast<float*>(stats_out + M);
+  const int blocks = (M + 7) / 8 + (a->B * a->k + 255) / 256;
+  shard_record_kernel<<<blocks, 256, 0, stream>>>(ctx->partials, pl.grid, ctx->max_rows, M, sh->v_offset, a->V, logits,
+                                                  ldl, a->draft_tok, a->B, a->k, stats_out, lx_out);
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) { set_error(ctx, "launch shard_record_kernel", e); return HOLA_ERR_CUDA; }
+  return HOLA_OK;
+}
+
+static hola_status shard_phase(hola_ctx* ctx, const hola_verify_args* a, const hola_shard_args* sh, void* cuda_stream,
+                               int phase) {
+  hola_status s = check_common(ctx, a);
+  if (s != HOLA_OK) return s;
+  if (a->B == 0) return HOLA_OK;
+  if ((s = check_sample_args(a)) != HOLA_OK) return s;
+  if ((s = check_shard(ctx, a, sh)) != HOLA_OK) return s;
+  if (!sh->records || !aligned16(sh->records) || (a->k > 0 && !sh->q_tok)) return HOLA_ERR_INVALID_ARG;
+  if (phase == 3 && !sh->mass_out) return HOLA_ERR_INVALID_ARG;
+  if (phase == 4 && (!sh->masses || a->fallback == HOLA_FALLBACK_GREEDY)) return HOLA_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  const float* logits = a->logits_out ? a->logits_out : ctx->logits;
+  const int ldl = a->logits_out ? a->V : ctx->ldl;
+  const ShardLaunch l = shard_launch(a, sh);
+  return run_accept_sample(ctx, a, logits, ldl, phase == 3 ? 1 : 0, 0, static_cast<cudaStream_t>(cuda_stream),
+                           sh->q_tok, phase, &l);
+}
+
+hola_status hola_shard_accept(hola_ctx* ctx, const hola_verify_args* a, const hola_shard_args* sh, void* cuda_stream) {
+  return shard_phase(ctx, a, sh, cuda_stream, 3);
+}
+
+hola_status hola_shard_sample(hola_ctx* ctx, const hola_verify_args* a, const hola_shard_args* sh, void* cuda_stream) {
+  return shard_phase(ctx, a, sh, cuda_stream, 4);
 }
 
 hola_status hola_host_traffic(const hola_ctx* ctx, unsigned long long* h2d_bytes, unsigned long long* d2h_bytes) {
