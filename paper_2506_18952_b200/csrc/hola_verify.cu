@@ -7,10 +7,13 @@
 //       dimension of the MMA:  D[v, r] = sum_h W_lm[v, h] * hidden[r, h].  A pair owns up to 256 vocabulary rows
 //       per tile; each CTA streams its (up to 128) rows of W_lm and HALF of the hidden rows per K block with TMA, and one
 //       thread of the leader CTA issues tcgen05.mma.cta_group::2 (bf16 x bf16 -> fp32 in tensor memory) that reads
-//       both halves.  Drain warps copy finished accumulators to the fp32 logits buffer; statistics warps re-read
-//       that tile row-wise (it is still in L2) and keep, per verify position, the running softmax statistics
-//       (m, s, t) = (max, sum e^(l-m), sum e^(l-m)(l-m)) in registers, in the shadow of the next tile's MMAs.
-//       W_lm is read from HBM once per pass.
+//       both halves.  Sixteen epilogue warps copy finished accumulators to the fp32 logits buffer and, from the
+//       same registers transposed through a small shared-memory buffer, keep per verify position the running
+//       softmax statistics (m, s, t) = (max, sum e^(l-m), sum e^(l-m)(l-m)) and the arg-max in registers, in the
+//       shadow of the next tile's MMAs.  W_lm is read from HBM once per pass; the logits are never read back.
+//   quantize_rows_int8_kernel   8-bit case of the Lo-Bi quantiser, per row (W_lm ahead of time, hidden rows per call).
+//   draft_entropy_kernel        H(q_j) of the draft rows, for the gate on the draft distribution.
+//   shard_record_kernel         vocabulary-parallel form: a rank's statistics record for the first all-gather.
 //   finalize_kernel             merges the per-CTA statistics:  logZ = m + ln s,  H = ln s - t/s  (entropy
 //       definition of the HSD section, rearranged around the running maximum).
 //   accept_sample_kernel        one cluster of CTAs per sequence: merges the statistics for its k+1 positions (warp
@@ -761,7 +764,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
     // ------------------------------------------------------------------ 8-bit W_lm: converter warps
     // int8 [tile_rows][64] (row pitch 64 bytes) -> bf16 [tile_rows][64] in the 128-byte-swizzled K-major layout the
     // MMA reads: 16-byte chunk c of row r sits at chunk position c ^ (r % 8) of its 128-byte row.  Every int8 value is
-    // exact in bf16; the row's scale is applied to the accumulators by the drain warps.
+    // exact in bf16; the row's scale is applied to the accumulators by the epilogue warps.
     // All converter warps share every K block (two independent 16-byte pieces per thread), in ring order.
     const int cw = warp < kW8HiddenWarp ? warp - (2 + kW8EpiWarps) : warp - (kW8HiddenWarp + 1) + (kW8HiddenWarp - 2 - kW8EpiWarps);
     const int ct = cw * 32 + lane;
