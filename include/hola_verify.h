@@ -103,7 +103,10 @@ typedef struct {
 } hola_verify_args;
 
 /* Creates a context on `device` able to serve calls with B <= maxB, k <= maxK and exactly this H and V.
- * Allocates the workspace (hola_workspace_bytes) once.  One context serves one stream at a time. */
+ * Allocates the workspace (hola_workspace_bytes) once.  One context serves one stream at a time.
+ * Tuning overrides read from the environment here (for sweeps and tests; the defaults are what was measured best):
+ * HOLA_STAGES=n (fewer shared-memory ring slots), HOLA_ROT=0 (257-384 rows per pass: two MMAs and one accumulator
+ * buffer instead of the rotating 128-column units), HOLA_HOST_OVERLAP=0 and HOLA_HOST_LAZY_Q=0|1 (hola_verify_host). */
 hola_status hola_create(hola_ctx** out, int device, int maxB, int maxK, int H, int V);
 hola_status hola_destroy(hola_ctx* ctx);
 

@@ -827,9 +827,17 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
 __device__ __forceinline__ Stats warp_merge_partials(const float4* partials, int nparts, int part_stride, int row,
                                                      int lane) {
   Stats st = stats_empty();
-  for (int i = lane; i < nparts; i += 32) {
-    const float4 x = partials[static_cast<size_t>(i) * part_stride + row];
-    st = stats_merge(st, Stats{x.x, x.y, x.z, __float_as_int(x.w)});
+  // six loads per lane in flight (192 partials per round: one round on a 148-SM part), then the merges in index order
+  for (int base = 0; base < nparts; base += 192) {
+    float4 x[6];
+#pragma unroll
+    for (int u = 0; u < 6; ++u) {
+      const int i = base + lane + 32 * u;
+      x[u] = i < nparts ? partials[static_cast<size_t>(i) * part_stride + row]
+                        : make_float4(-CUDART_INF_F, 0.f, 0.f, __int_as_float(0x7fffffff));
+    }
+#pragma unroll
+    for (int u = 0; u < 6; ++u) st = stats_merge(st, Stats{x[u].x, x[u].y, x[u].z, __float_as_int(x[u].w)});
   }
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) {
