@@ -50,3 +50,60 @@ def test_quantised_head_logits_are_the_plain_definition_on_w8():
     got = ref.logits(hid, W8)
     np.testing.assert_allclose(got, hid @ W8.T, rtol=1e-13, atol=1e-13)
     assert np.max(np.abs(got - hid @ W.T)) < 0.05           # and stays close to the unquantised head
+
+
+# ---- two 8-bit planes per activation row
+def test_two_plane_rows_error_bound_and_first_plane():
+    rng = np.random.default_rng(5)
+    x = ref.bf16_bits_to_f64(ref.f32_to_bf16_bits(rng.normal(size=(30, 128)).astype(np.float32))).astype(np.float32)
+    x[4] = 0.0
+    q1, q2, s1, s2 = lobi.quantize_rows_two_plane(x)
+    qa, sa = lobi.quantize_rows_int8(x)
+    assert np.array_equal(q1, qa) and np.array_equal(s1, sa)            # the first plane is the plain 8-bit quantiser
+    x16 = lobi.dequantize_two_plane(q1, q2, s1, s2)
+    amax = np.max(np.abs(x), axis=1)
+    # half a step of the second plane, plus the two fp32 roundings that produced the residual (each < 2^-24 of the row
+    # maximum): sixteen bits against the row maximum, 250 times finer than one plane
+    bound = 0.5 * s2.astype(np.float64) + 2.0 ** -22 * amax
+    assert np.all(np.abs(x16 - x) <= bound[:, None])
+    nz = amax > 0
+    one_plane = np.max(np.abs(lobi.dequantize_rows(qa, sa) - x), axis=1)
+    assert np.all(np.max(np.abs(x16 - x), axis=1)[nz] < one_plane[nz] / 100)
+    assert np.abs(q2).max() <= 127 and np.all(q2[4] == 0) and np.all(q1[4] == 0)
+    assert np.allclose(s2 * np.float32(254.0), s1, rtol=1e-6)
+
+
+def test_two_plane_exact_cases_and_symmetry():
+    # integers with row maximum 127: scale 1, the first plane is exact and the second one is zero
+    rng = np.random.default_rng(6)
+    x = rng.integers(-127, 128, size=(5, 64)).astype(np.float32)
+    x[:, 0] = 127.0
+    q1, q2, s1, s2 = lobi.quantize_rows_two_plane(x)
+    assert np.all(s1 == 1.0) and np.array_equal(q1.astype(np.float32), x) and np.all(q2 == 0)
+    # multiples of 1/254 between the integers: the second plane holds them exactly
+    y = x.copy()
+    y[:, 1:] += (rng.integers(-127, 128, size=(5, 63)) / 254.0).astype(np.float32) * 0.999
+    y = np.clip(y, -127, 127).astype(np.float32)
+    q1, q2, s1, s2 = lobi.quantize_rows_two_plane(y)
+    assert np.max(np.abs(lobi.dequantize_two_plane(q1, q2, s1, s2) - y)) <= 0.5 / 254 + 1e-5
+    # odd symmetry, and a power-of-two factor moves into both scales
+    x = rng.normal(size=(8, 96)).astype(np.float32)
+    a = lobi.quantize_rows_two_plane(x)
+    b = lobi.quantize_rows_two_plane(-x)
+    assert np.array_equal(b[0], -a[0]) and np.array_equal(b[1], -a[1]) and np.array_equal(b[2], a[2])
+    c = lobi.quantize_rows_two_plane(x * np.float32(8.0))
+    assert np.array_equal(c[0], a[0]) and np.array_equal(c[1], a[1])
+    assert np.array_equal(c[2], a[2] * np.float32(8.0)) and np.array_equal(c[3], a[3] * np.float32(8.0))
+
+
+def test_two_plane_head_logits_stay_close_to_bf16_activations():
+    rng = np.random.default_rng(7)
+    hid = ref.bf16_bits_to_f64(ref.f32_to_bf16_bits(rng.normal(size=(6, 256)).astype(np.float32)))
+    W = ref.bf16_bits_to_f64(ref.f32_to_bf16_bits((rng.normal(size=(50, 256)) * 0.05).astype(np.float32)))
+    q, s = lobi.quantize_rows_int8(W.astype(np.float32))
+    W8 = lobi.dequantize_rows(q, s)
+    h16 = lobi.dequantize_two_plane(*lobi.quantize_rows_two_plane(hid.astype(np.float32)))
+    h8 = lobi.dequantize_rows(*lobi.quantize_rows_int8(hid.astype(np.float32)))
+    exact = hid @ W8.T
+    assert np.max(np.abs(h16 @ W8.T - exact)) < 2e-4                    # 16-bit-class rows: invisible next to ...
+    assert np.max(np.abs(h8 @ W8.T - exact)) > 2e-3                     # ... what one 8-bit plane does to the logits
