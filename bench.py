@@ -191,9 +191,10 @@ def main():
                     help="which entropy feeds the gate: the verifier's softmax (default) or the draft row")
     ap.add_argument("--fallback", default="sample", choices=["sample", "greedy"],
                     help="what the gate-off branch does: speculative-sampling test (default) or greedy verifier")
-    ap.add_argument("--weights", default="bf16", choices=["bf16", "int8", "w8a8"],
+    ap.add_argument("--weights", default="bf16", choices=["bf16", "int8", "w8a8", "w8a16"],
                     help="bf16 (default); int8: 8-bit W_lm from hola_quantize_w8, expanded exactly on chip; "
-                         "w8a8: 8-bit W_lm and hidden rows quantised on the fly, 8-bit tensor-core kind")
+                         "w8a8: 8-bit W_lm and hidden rows quantised on the fly, 8-bit tensor-core kind; "
+                         "w8a16: the same with the hidden rows as two 8-bit planes (16-bit-class activations)")
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--cpu-budget-s", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -216,14 +217,14 @@ def main():
     w = workloads.make_config(args.workload, dev, seed_offset=hdist.rank_seed_offset(rank))
     ctx = binding.HolaVerify(w.B, w.k, w.H, w.V, device=local)
     plan = ctx.hola_plan(w.B, w.k, {"bf16": binding.HOLA_W_BF16, "int8": binding.HOLA_W_INT8,
-                                    "w8a8": binding.HOLA_W8A8}[args.weights])
+                                    "w8a8": binding.HOLA_W8A8, "w8a16": binding.HOLA_W8A16}[args.weights])
     out = ctx.alloc_outputs(w.B, w.k, False)
     flush = None
     if w.V * w.H * 2 <= 200e6:
         flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
 
     W_dev, w_scale = w.W_lm, None
-    a8 = args.weights == "w8a8"
+    a8 = {"w8a8": True, "w8a16": "a16"}.get(args.weights, False)
     if args.weights != "bf16":
         W_dev, w_scale = binding.hola_quantize_w8(w.W_lm)
         torch.cuda.synchronize()
@@ -310,7 +311,8 @@ def main():
         work = algorithmic_work(w, 2 if args.weights == "bf16" else 1)
         t_mem = work["gemm_bytes"] / (peaks["hbm_gbs"] * 1e9)
         # the 8-bit tensor-core kinds have twice the nominal rate of bf16: measured bf16 peak x 2 for --weights w8a8
-        tensor_peak = peaks["bf16_tflops"] * (2.0 if a8 else 1.0)
+        # (w8a16 runs two 8-bit rows per verify row: per algorithmic flop its peak is the bf16 one again)
+        tensor_peak = peaks["bf16_tflops"] * (2.0 if a8 is True else 1.0)
         t_flop = work["flops"] / (tensor_peak * 1e12)
         t_k1 = k1_ms * 1e-3 * plan["passes"]
         if t_flop >= t_mem:

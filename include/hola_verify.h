@@ -65,9 +65,15 @@ typedef enum {
 typedef enum {
   HOLA_W_BF16 = 0,
   HOLA_W_INT8 = 1, /* int8 weights, bf16 activations: the weights are expanded exactly on chip (W8A16)             */
-  HOLA_W8A8 = 2    /* int8 weights AND the hidden rows quantised the same way (one fp32 scale per verify row) by the
+  HOLA_W8A8 = 2,   /* int8 weights AND the hidden rows quantised the same way (one fp32 scale per verify row) by the
                     * library on the fly; products on the 8-bit tensor-core kind with exact int32 accumulation:
                     * l[r][v] = w_scale[v] * h_scale[r] * sum_h q_hid[r][h] * q_w[v][h].  Needs a context. */
+  HOLA_W8A16 = 3   /* int8 weights, hidden rows kept at 16-bit width as TWO 8-bit planes made on the fly: the coarse
+                    * plane of HOLA_W8A8 (scale s1) and a plane of its remainder (scale s2 = s1 / 254), so that
+                    * |x16 - x| <= max|x| / 64516 per row.  Both planes go through the 8-bit tensor-core kind
+                    * (twice the rows, twice the rate, half the weight bytes of bf16) and
+                    * l[r][v] = w_scale[v] * (s1[r] * sum_h q1[r][h] q_w[v][h] + s2[r] * sum_h q2[r][h] q_w[v][h]).
+                    * At most 256 verify rows per pass over W_lm.  Needs a context. */
 } hola_w_dtype;
 
 /* Bits of the device status word (OR-ed by the kernels; the caller clears it). */
@@ -97,9 +103,9 @@ typedef struct {
   int32_t gate_source;     /* hola_gate_source; 0 (zero-initialised struct) = target entropy                   */
   int32_t fallback;        /* hola_fallback; 0 = speculative sampling.  With GREEDY the uniforms are not read  */
   float* draft_entropy;    /* out fp32 [B][k], optional: H(q_j), written when gate_source = DRAFT_ENTROPY       */
-  int32_t w_dtype;         /* hola_w_dtype; 0 = W_lm is bf16.  INT8 / W8A8: W_lm is int8 [V][H], H % 16 == 0      */
+  int32_t w_dtype;         /* hola_w_dtype; 0 = W_lm is bf16, otherwise W_lm is int8 [V][H] and H % 16 == 0     */
   int32_t reserved_;       /* must be 0                                                                        */
-  const float* w_scale;    /* fp32 [V], required with HOLA_W_INT8 / HOLA_W8A8: scale of each vocabulary row    */
+  const float* w_scale;    /* fp32 [V], required with an int8 W_lm (w_dtype != 0): scale of each vocabulary row  */
 } hola_verify_args;
 
 /* Creates a context on `device` able to serve calls with B <= maxB, k <= maxK and exactly this H and V.

@@ -17,7 +17,7 @@ HOLA_OK = 0
 HOLA_Q_BF16, HOLA_Q_F32 = 0, 1
 HOLA_GATE_TARGET_ENTROPY, HOLA_GATE_DRAFT_ENTROPY = 0, 1
 HOLA_FALLBACK_SAMPLE, HOLA_FALLBACK_GREEDY = 0, 1
-HOLA_W_BF16, HOLA_W_INT8, HOLA_W8A8 = 0, 1, 2
+HOLA_W_BF16, HOLA_W_INT8, HOLA_W8A8, HOLA_W8A16 = 0, 1, 2, 3
 FLAG_BAD_TOKEN, FLAG_BAD_UNIFORM, FLAG_TIMEOUT, FLAG_R_ZERO = 1, 2, 4, 8
 
 EXPORTS = ["hola_create", "hola_destroy", "hola_workspace_bytes", "hola_verify", "hola_verify_host",
@@ -253,9 +253,11 @@ class HolaVerify:
         a.status_word = _dptr(out.status)
         a.gate_source, a.fallback = int(gate_source), int(fallback)
         a.draft_entropy = _dptr(out.draft_entropy)
+        # a8: True = one 8-bit plane per hidden row (W8A8); "a16" = two planes (16-bit-class activations, W8A16)
         if a8 and w_scale is None:
-            raise HolaError("8-bit activations (a8) go with an int8 W_lm and its scales")
-        a.w_dtype = (HOLA_W8A8 if a8 else HOLA_W_INT8) if w_scale is not None else HOLA_W_BF16
+            raise HolaError("8-bit activation planes (a8) go with an int8 W_lm and its scales")
+        act = HOLA_W8A16 if a8 == "a16" else (HOLA_W8A8 if a8 else HOLA_W_INT8)
+        a.w_dtype = act if w_scale is not None else HOLA_W_BF16
         a.w_scale = _dptr(w_scale)
         return a
 

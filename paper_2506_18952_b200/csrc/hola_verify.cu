@@ -94,7 +94,8 @@ struct K1Params {
   int tile_rows;  // vocabulary rows per CTA per tile (<= 128, multiple of 4): balances the tiles over the pairs
   int ldl;        // row pitch of the logits buffer, in floats
   const float* w_scale;   // 8-bit W_lm: fp32 scale per vocabulary row, applied to the accumulators
-  const float* h_scale;   // 8-bit activations (mode 2): fp32 scale per verify row
+  const float* h_scale;   // 8-bit activations (modes 2, 3): fp32 scale per verify row (mode 3: of the coarse plane)
+  const float* h_scale2;  // mode 3: scale of the second plane
   float* logits;
   float4* partials;   // [grid][part_stride] (m, s, t, arg-max index)
   int part_stride;
@@ -299,6 +300,19 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// 16 consecutive 32-bit columns of this thread's tensor-memory lane, as raw words (no wait: the caller waits once
+// for all loads it has issued).
+__device__ __forceinline__ void tmem_ld16_nowait(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -433,6 +447,8 @@ __device__ __forceinline__ float scaled(float acc, float w_scale, const float* h
 //   converter warps have expanded it.  full[] then collects, besides the hidden bytes, one arrival per converter warp.
 // After the barrier area: one 2 KB transposition buffer per epilogue warp (reused for the final merge of the
 // statistics of the four tensor-memory lane quarters).
+// kMode 3 is kMode 2 with every verify row present twice in the hidden operand (coarse 8-bit plane and the plane of
+// its remainder, in alternating blocks of 32 rows): the epilogue adds the two int32 sums with their scales.
 // kMode: 0 bf16 x bf16; 1 int8 W_lm expanded to bf16 on chip (exact); 2 int8 W_lm x int8 hidden on the 8-bit MMA
 // kind (K blocks of 128 elements, so that a block is 128 bytes per row exactly as in mode 0; int32 accumulators).
 template <int kMode>
@@ -440,7 +456,8 @@ __global__ void __launch_bounds__(kK1Threads, 1)
 lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __grid_constant__ CUtensorMap tmap_w,
                        const K1Params p) {
   constexpr bool kW8 = kMode == 1;
-  constexpr bool kI8 = kMode == 2;
+  constexpr bool kI8 = kMode >= 2;                       // both operands 8-bit, 8-bit MMA kind
+  constexpr bool kTwoPlane = kMode == 3;                 // hidden rows as two 8-bit planes, 64 operand rows per 32 verify rows
   constexpr int kKStep = kI8 ? 2 * kBlockK : kBlockK;    // elements of K per ring slot
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -529,7 +546,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
             tma_load_2d(sa, &tmap_w, fb, kx, v0, pol_w);
             for (int s = 0; s < p.n_sub; ++s)
               tma_load_2d(sa + kWBlockBytes + s * hid_block_bytes, &tmap_hidden, fb, kx,
-                          p.row0 + s * p.N + static_cast<int>(rank) * half_n, pol_h);
+                          (kTwoPlane ? 2 : 1) * p.row0 + s * p.N + static_cast<int>(rank) * half_n, pol_h);
           }
           if (++stage == p.stages) { stage = 0; phase ^= 1u; }
         }
@@ -644,6 +661,77 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
       const int vocab16 = vbase + quarter * 32 + thalf * 16;
       const float w_scale = ((kW8 || kI8) && vocab_ok) ? p.w_scale[vocab] : 1.f;   // 8-bit W_lm: the row's scale
       const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+      if (kTwoPlane) {
+        // Two planes: 64 consecutive accumulator columns hold the coarse-plane sums (first 32) and the remainder-plane
+        // sums (last 32) of the same 32 verify rows.  Read 16 + 16 columns at a time, add them with their scales, and
+        // go on as in the other modes (16 rows are exactly one transposition step).
+        const int n_pairs = p.n_sub * p.N / 64;
+        const int my_pairs = group < n_pairs ? (n_pairs - 1 - group) / kGroups + 1 : 0;
+        if (my_pairs == 0) {
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(leader_tempty + 8 * buf);
+        }
+#pragma unroll
+        for (int slot = 0; slot < 2; ++slot) {
+          if (slot < my_pairs) {
+            const int pr = group + slot * kGroups;
+            const int sub = (64 * pr) / p.N, col = 64 * pr - sub * p.N;
+            const uint32_t taddr = lane_addr + buf * 256 + sub * 256 + col;
+            const int vr0 = p.row0 + 32 * pr;            // verify row of the pair's first column
+            const int n_ok = min(32, p.M - vr0);
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+              uint32_t a[16], c[16];
+              __syncwarp();
+              tmem_ld16_nowait(taddr + 16 * half, a);
+              tmem_ld16_nowait(taddr + 32 + 16 * half, c);
+              tmem_ld_wait();
+              if (slot == my_pairs - 1 && half == 1) {   // this warp's accumulators may be overwritten
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(leader_tempty + 8 * buf);
+              }
+              const int rows_here = n_ok - 16 * half;    // real rows among these 16
+              if (rows_here > 0) {
+                float f[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                  f[i] = 0.f;
+                  if (i < rows_here) {
+                    const int r = vr0 + 16 * half + i;
+                    f[i] = fmaf(static_cast<float>(static_cast<int>(c[i])), w_scale * p.h_scale2[r],
+                                static_cast<float>(static_cast<int>(a[i])) * (w_scale * p.h_scale[r]));
+                  }
+                }
+                if (vocab_ok) {
+                  float* dst = p.logits + static_cast<size_t>(vr0 + 16 * half) * p.ldl + vocab;
+#pragma unroll
+                  for (int i = 0; i < 16; ++i)
+                    if (i < rows_here) dst[static_cast<size_t>(i) * p.ldl] = f[i];
+                }
+                if (nv > 0) {
+                  __syncwarp();
+#pragma unroll
+                  for (int i = 0; i < kTransRows; ++i)
+                    tbuf[i * 32 + ((((lane >> 2) ^ (i & 7))) << 2) + (lane & 3)] = f[i];
+                  __syncwarp();
+                  float e[16];
+#pragma unroll
+                  for (int jj = 0; jj < 4; ++jj) {
+                    const float4 x = *reinterpret_cast<const float4*>(
+                        tbuf + trow * 32 + (((thalf * 4 + jj) ^ (trow & 7)) << 2));
+                    e[4 * jj] = x.x; e[4 * jj + 1] = x.y; e[4 * jj + 2] = x.z; e[4 * jj + 3] = x.w;
+                  }
+                  if (n16 == 16) stats_fold16<true>(e, 16, vocab16, st[slot][half]);
+                  else if (n16 > 0) stats_fold16<false>(e, n16, vocab16, st[slot][half]);
+                }
+              }
+            }
+          }
+        }
+        continue;
+      }
       if (my_chunks == 0) {                              // nothing to read: the accumulators are free as far as this
         tc_fence_before();                               // warp is concerned
         __syncwarp();
@@ -729,7 +817,11 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
         o.t = __shfl_xor_sync(0xffffffffu, a.t, 16);
         o.arg = __shfl_xor_sync(0xffffffffu, a.arg, 16);
         a = stats_merge(a, o);
-        if (slot < my_chunks && thalf == 0) {
+        if (kTwoPlane) {
+          const int r = 32 * (group + slot * kGroups) + half * kTransRows + trow;   // row inside the pass
+          if (slot < 2 && thalf == 0 && r < p.rows)
+            merge[quarter * p.rows + r] = make_float4(a.m, a.s, a.t, __int_as_float(a.arg));
+        } else if (slot < my_chunks && thalf == 0) {
           const int ch = rot ? slot * sub_chunks + group : group + slot * kGroups;
           const int sub = ch / sub_chunks, j = ch - sub * sub_chunks;
           const int c = j * 32 + half * kTransRows + trow;           // column inside its MMA
@@ -755,7 +847,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
           mbar_expect_tx_cluster(fb, hid_tx_bytes);
           for (int s = 0; s < p.n_sub; ++s)
             tma_load_2d(sa + kWBlockBytes + s * hid_block_bytes, &tmap_hidden, fb, kx,
-                        p.row0 + s * p.N + static_cast<int>(rank) * half_n, pol_h);
+                        (kTwoPlane ? 2 : 1) * p.row0 + s * p.N + static_cast<int>(rank) * half_n, pol_h);
           if (++stage == p.stages) { stage = 0; phase ^= 1u; }
         }
       }
@@ -1289,6 +1381,49 @@ __global__ void __launch_bounds__(256) quantize_rows_int8_kernel(const __nv_bflo
   }
 }
 
+// Hidden rows as two 8-bit planes (16-bit-class activations for the 8-bit MMA kind): per verify row
+//   s1 = max|x| / 127 (1 if zero), q1 = clip(rint(x / s1));  r = x - s1 q1;  s2 = s1 / 254, q2 = clip(rint(r / s2)),
+// every step one fp32 operation.  Operand layout: blocks of 32 verify rows, each block as 32 rows of q1 followed by
+// 32 rows of q2 (so that 64 consecutive accumulator columns hold both sums of the same 32 rows); rows past M are
+// written as zeros.  One CTA per (padded) verify row.
+__global__ void __launch_bounds__(256) quantize_rows_two_plane_kernel(const __nv_bfloat16* X, int M, int H,
+                                                                      signed char* q, float* s1, float* s2) {
+  __shared__ float sh_max[8];
+  __shared__ float sh_scale;
+  const int row = blockIdx.x;
+  signed char* q1 = q + (static_cast<size_t>(64) * (row >> 5) + (row & 31)) * H;
+  signed char* q2 = q1 + static_cast<size_t>(32) * H;
+  if (row >= M) {
+    for (int h = threadIdx.x; h < H; h += 256) { q1[h] = 0; q2[h] = 0; }
+    return;
+  }
+  const __nv_bfloat16* xr = X + static_cast<size_t>(row) * H;
+  float amax = 0.f;
+  for (int h = threadIdx.x; h < H; h += 256) amax = fmaxf(amax, fabsf(__bfloat162float(xr[h])));
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, off));
+  if ((threadIdx.x & 31) == 0) sh_max[threadIdx.x >> 5] = amax;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float m = 0.f;
+    for (int i = 0; i < 8; ++i) m = fmaxf(m, sh_max[i]);
+    const float sc = m > 0.f ? __fdiv_rn(m, 127.f) : 1.f;
+    sh_scale = sc;
+    s1[row] = sc;
+    s2[row] = __fdiv_rn(sc, 254.f);
+  }
+  __syncthreads();
+  const float sc = sh_scale, sc2 = __fdiv_rn(sc, 254.f);
+  for (int h = threadIdx.x; h < H; h += 256) {
+    const float x = __bfloat162float(xr[h]);
+    const float a = fminf(127.f, fmaxf(-127.f, rintf(__fdiv_rn(x, sc))));
+    const float rem = __fsub_rn(x, __fmul_rn(sc, a));                  // no fused multiply-add: two roundings
+    const float b = fminf(127.f, fmaxf(-127.f, rintf(__fdiv_rn(rem, sc2))));
+    q1[h] = static_cast<signed char>(a);
+    q2[h] = static_cast<signed char>(b);
+  }
+}
+
 // ------------------------------------------------------------------------------------------------ draft entropy
 // H(q) = -sum_v q ln q of each draft row (one CTA per row): the gate value when the gate looks at the draft
 // distribution, as the HSD section words it.  q is used as stored; entries with q <= 0 contribute nothing.
@@ -1420,8 +1555,8 @@ WsLayout ws_layout(int maxB, int maxK, int H, int V, int num_sms) {
   w.partials = take(static_cast<size_t>(num_sms) * rows * 16);
   w.status = take(4);
   w.hq = take(rows * kHqSlices * 8);
-  w.hid8 = take(rows * static_cast<size_t>(H));
-  w.hid_scale = take(rows * 4);
+  w.hid8 = take(2 * align_up(rows, 32) * static_cast<size_t>(H));     // one or two 8-bit planes of the hidden rows
+  w.hid_scale = take(2 * rows * 4);                                   // their scales (second plane after the first)
   w.st_hidden = take(rows * H * 2);
   w.st_tok = take(static_cast<size_t>(maxB) * maxK * 4);
   w.st_q = take(static_cast<size_t>(maxB) * maxK * V * 4);
@@ -1448,25 +1583,31 @@ int round_up(int x, int a) { return (x + a - 1) / a * a; }
 // Cost per pass: the slower of streaming W_lm once and the padded rows' tensor time, plus a fixed launch cost.
 Plan make_plan(const hola_ctx* ctx, int M, int w_dtype = HOLA_W_BF16) {
   const bool w8 = w_dtype == HOLA_W_INT8;        // int8 W_lm expanded on chip
-  const bool i8 = w_dtype == HOLA_W8A8;          // 8-bit MMA: N a multiple of 32, K blocks of 128, twice the rate
+  const bool two = w_dtype == HOLA_W8A16;        // as W8A8, with two operand rows per verify row
+  const bool i8 = w_dtype == HOLA_W8A8 || two;   // 8-bit MMA: N a multiple of 32, K blocks of 128, twice the rate
   Plan best{};
   double best_cost = 1e300;
   const int rows = M > 0 ? M : 1;
   // 8-bit W_lm: one MMA per K step (at most 256 rows per pass), and the slot also holds the int8 block
-  const int max_rows_per_pass = w8 ? kMaxN : kMaxRowsPerPass;
+  const int max_rows_per_pass = (w8 || two) ? kMaxN : kMaxRowsPerPass;
   const int p_min = (rows + max_rows_per_pass - 1) / max_rows_per_pass;
   const double t_hbm = (w8 || i8 ? 1.0 : 2.0) * ctx->V * static_cast<double>(ctx->H) / 6.4e12;
   for (int passes = p_min; passes <= p_min + 3; ++passes) {
     const int r = (rows + passes - 1) / passes;
     // up to 256 rows: one MMA, two accumulator buffers; up to 384: three MMAs of N <= 128 on rotating 128-column
     // units; beyond: two MMAs of N <= 256 that fill the tensor memory
-    const int n_sub = (r > 3 * 128 || (ctx->no_rot && r > kMaxN)) ? 2 : (r > kMaxN ? 3 : 1);
-    const int N = round_up((r + n_sub - 1) / n_sub, i8 ? 32 : 16);
+    int n_sub = (r > 3 * 128 || (ctx->no_rot && r > kMaxN)) ? 2 : (r > kMaxN ? 3 : 1);
+    int N = round_up((r + n_sub - 1) / n_sub, i8 ? 32 : 16);
+    if (two) {                                     // operand rows: 64 per 32 verify rows; one or two MMAs, N % 64 == 0
+      const int r8 = 2 * round_up(r, 32);
+      n_sub = r8 > kMaxN ? 2 : 1;
+      N = round_up(r8 / n_sub, 64);
+    }
     const double t_mma = 2.0 * n_sub * N * static_cast<double>(ctx->V) * ctx->H / (i8 ? 2.8e15 : 1.4e15);
     const double cost = passes * ((t_mma > t_hbm ? t_mma : t_hbm) + 6e-6);
     if (cost < best_cost) {
       best_cost = cost;
-      best.n_sub = n_sub; best.N = N; best.rows_per_pass = n_sub * N; best.passes = passes;
+      best.n_sub = n_sub; best.N = N; best.rows_per_pass = two ? n_sub * N / 2 : n_sub * N; best.passes = passes;
       best.est_seconds = cost;
     }
   }
@@ -1533,10 +1674,19 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 hola_status run_lm_head(hola_ctx* ctx, const hola_verify_args* a, float* logits, int ldl, const Plan& pl,
                         cudaStream_t stream) {
   const int M = a->B * (a->k + 1);
-  const bool w8 = a->w_dtype == HOLA_W_INT8, i8 = a->w_dtype == HOLA_W8A8;
+  const bool w8 = a->w_dtype == HOLA_W_INT8, two = a->w_dtype == HOLA_W8A16, i8 = a->w_dtype == HOLA_W8A8 || two;
   CUtensorMap th, tw;
   hola_status s;
-  if (i8) {
+  if (two) {
+    // 16-bit-class activations: two 8-bit planes per hidden row, blocks of 32 rows, into the context's workspace
+    if (!ctx->hid8) return HOLA_ERR_INVALID_ARG;
+    const int padded = round_up(M, 32);
+    quantize_rows_two_plane_kernel<<<static_cast<unsigned>(padded), 256, 0, stream>>>(
+        static_cast<const __nv_bfloat16*>(a->hidden), M, a->H, ctx->hid8, ctx->hid_scale, ctx->hid_scale + ctx->max_rows);
+    if (cudaGetLastError() != cudaSuccess) return HOLA_ERR_CUDA;
+    s = encode_map(ctx, &th, ctx->hid8, static_cast<uint64_t>(2 * padded), static_cast<uint64_t>(a->H),
+                   static_cast<uint32_t>(pl.N / 2), true, true);
+  } else if (i8) {
     // 8-bit activations: the same per-row quantiser as for W_lm, into the context's workspace
     if (!ctx->hid8) return HOLA_ERR_INVALID_ARG;          // (the entry point without a context has no room for it)
     quantize_rows_int8_kernel<<<static_cast<unsigned>(M), 256, 0, stream>>>(
@@ -1559,7 +1709,10 @@ hola_status run_lm_head(hola_ctx* ctx, const hola_verify_args* a, float* logits,
   kp.status = a->status_word ? a->status_word : ctx->status;
   kp.w_scale = a->w_scale;
   kp.h_scale = ctx->hid_scale;
-  cudaError_t e = i8 ? cudaFuncSetAttribute(lm_head_entropy_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  kp.h_scale2 = ctx->hid_scale ? ctx->hid_scale + ctx->max_rows : nullptr;
+  cudaError_t e = two ? cudaFuncSetAttribute(lm_head_entropy_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             pl.smem_bytes)
+                : i8 ? cudaFuncSetAttribute(lm_head_entropy_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             pl.smem_bytes)
                 : w8 ? cudaFuncSetAttribute(lm_head_entropy_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             pl.smem_bytes)
@@ -1582,7 +1735,8 @@ hola_status run_lm_head(hola_ctx* ctx, const hola_verify_args* a, float* logits,
     kp.row0 = pass * pl.rows_per_pass;
     kp.rows = M - kp.row0 < pl.rows_per_pass ? M - kp.row0 : pl.rows_per_pass;
     if (kp.rows <= 0) break;
-    e = i8 ? cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<2>, th, tw, kp)
+    e = two ? cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<3>, th, tw, kp)
+      : i8 ? cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<2>, th, tw, kp)
       : w8 ? cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<1>, th, tw, kp)
            : cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<0>, th, tw, kp);
     if (e != cudaSuccess) { set_error(ctx, "launch lm_head_entropy_kernel", e); return HOLA_ERR_CUDA; }
@@ -1659,7 +1813,7 @@ hola_status check_lm_head_args(const hola_ctx* ctx, const hola_verify_args* a) {
   if (!a->hidden || !a->W_lm) return HOLA_ERR_INVALID_ARG;
   if (!aligned16(a->hidden) || !aligned16(a->W_lm)) return HOLA_ERR_INVALID_ARG;
   if (a->H % 8 != 0) return HOLA_ERR_UNSUPPORTED_SHAPE;
-  if (a->w_dtype != HOLA_W_BF16 && a->w_dtype != HOLA_W_INT8 && a->w_dtype != HOLA_W8A8) return HOLA_ERR_INVALID_ARG;
+  if (a->w_dtype < HOLA_W_BF16 || a->w_dtype > HOLA_W8A16) return HOLA_ERR_INVALID_ARG;
   if (a->w_dtype != HOLA_W_BF16) {
     if (!a->w_scale) return HOLA_ERR_INVALID_ARG;
     if (a->H % 16 != 0) return HOLA_ERR_UNSUPPORTED_SHAPE;     // int8 row pitch must be a multiple of 16 bytes
@@ -1796,7 +1950,7 @@ hola_status hola_destroy(hola_ctx* ctx) {
 
 hola_status hola_plan_ex(const hola_ctx* ctx, int B, int k, int w_dtype, hola_plan_info* out) {
   if (!ctx || !out || B < 0 || k < 0) return HOLA_ERR_INVALID_ARG;
-  if (w_dtype != HOLA_W_BF16 && w_dtype != HOLA_W_INT8 && w_dtype != HOLA_W8A8) return HOLA_ERR_INVALID_ARG;
+  if (w_dtype < HOLA_W_BF16 || w_dtype > HOLA_W8A16) return HOLA_ERR_INVALID_ARG;
   if (B > ctx->maxB || k > ctx->maxK) return HOLA_ERR_UNSUPPORTED_SHAPE;
   const Plan pl = make_plan(ctx, B * (k + 1), w_dtype);
   out->tile_v = 2 * pl.tile_rows; out->grid = pl.grid; out->stages = pl.stages; out->rows_per_pass = pl.rows_per_pass;

@@ -533,6 +533,81 @@ def test_w8a8_on_the_large_vocabulary_shape(binding):
     check_ranges(w, out)
 
 
+# ---- 8-bit weights, 16-bit-class activations (two 8-bit planes)
+def _w8a16_oracle(w, q8, scale, **kw):
+    """The oracle on both operands as the kernel sees them: hidden rows = s1 q1 + s2 q2 (fp64), W8 = scale * q."""
+    from oracle import lobi
+    hid = ref.bf16_bits_to_f64(_np(w.hidden))
+    B, k1, H = hid.shape
+    h16 = lobi.dequantize_two_plane(*lobi.quantize_rows_two_plane(hid.reshape(B * k1, H).astype(np.float32)))
+    W8 = lobi.dequantize_rows(_np(q8), _np(scale))
+    return ref.verify(h16.reshape(B, k1, H), W8, _np(w.draft_tok), _np(w.draft_q), _np(w.uniforms), w.tau,
+                      keep_logits=True, **kw)
+
+
+@pytest.mark.parametrize("B,k,H,V,qd", [
+    (1, 4, 64, 1000, torch.float32),       # 5 rows: one block of 32, N = 64
+    (37, 6, 256, 5000, torch.bfloat16),    # 259 rows: two passes (at most 256 verify rows each)
+    (5, 2, 80, 1001, torch.bfloat16),      # K tail, odd V
+    (33, 3, 128, 40000, torch.bfloat16),   # 132 rows: two MMAs of N = 192 (five blocks of 32, the last one ragged)
+    (21, 5, 128, 3000, torch.float32),     # 126 rows: N = 256, double-buffered accumulators
+])
+def test_w8a16_head_matches_oracle_on_two_plane_rows(binding, B, k, H, V, qd):
+    w = workloads.gaussian_head("w8a16", B, k, H, V, seed=B + V, device=DEV, w_std=0.3, sigma=1.0, q_dtype=qd,
+                                tau=1.5 + 0.1 * k, sigma_far=0.2)
+    q8, scale = binding.hola_quantize_w8(w.W_lm)
+    with binding.HolaVerify(B, k, H, V) as ctx:
+        out = ctx.hola_verify(w.hidden, q8, w.draft_tok, w.draft_q, w.uniforms, w.tau, want_logits=True, w_scale=scale,
+                              a8="a16")
+        torch.cuda.synchronize()
+    assert int(out.status.item()) & binding.FLAG_TIMEOUT == 0
+    orc = _w8a16_oracle(w, q8, scale)
+    rep = compare.compare(orc, _np(w.draft_q), _np(w.uniforms), _np(out.accept_len), _np(out.next_tok),
+                          _np(out.entropy), _np(out.logZ), _np(out.logits))
+    print(rep.summary())
+    assert rep.ok, rep.summary()
+    assert rep.accept_margin_cases <= max(1, B // 20) and rep.token_margin_cases <= max(1, B // 10)
+    check_ranges(w, out)
+    # and the two planes keep the logits within 1e-3 of the 8-bit head on the unquantised bf16 rows
+    exact = _w8_oracle(w, q8, scale)
+    assert np.max(np.abs(_np(out.logits) - exact.logits)) < 2e-3
+
+
+def test_w8a16_integer_operands_are_bit_exact(binding):
+    # integer rows with maximum 127: s1 = 1, the first plane is the row, the second plane is zero
+    g = torch.Generator().manual_seed(11)
+    B, k, H, V = 40, 3, 192, 520
+    hf = torch.randint(-6, 7, (B, k + 1, H), generator=g).float()
+    hf[..., 0] = 127.0
+    Wf = torch.randint(-5, 6, (V, H), generator=g).float()
+    Wf[:, 1] = -127.0
+    hidden, W = hf.bfloat16().to(DEV), Wf.bfloat16().to(DEV)
+    q8, scale = binding.hola_quantize_w8(W)
+    with binding.HolaVerify(B, k, H, V) as ctx:
+        out = ctx.hola_lm_head_entropy(hidden, q8, want_logits=True, w_scale=scale, a8="a16")
+        torch.cuda.synchronize()
+    want = ref.logits(_np(hidden).reshape(-1, H), _np(W)).reshape(B, k + 1, V)
+    assert np.array_equal(_np(out.logits).astype(np.float64), want)
+
+
+@pytest.mark.parametrize("name", ["edge", "large_vocab_b32"])
+def test_w8a16_on_the_bandwidth_bound_shapes(binding, name):
+    w = workloads.make_config(name, DEV)
+    q8, scale = binding.hola_quantize_w8(w.W_lm)
+    with binding.HolaVerify(w.B, w.k, w.H, w.V) as ctx:
+        out = ctx.hola_verify(w.hidden, q8, w.draft_tok, w.draft_q, w.uniforms, w.tau, want_logits=True, w_scale=scale,
+                              a8="a16")
+        torch.cuda.synchronize()
+    seqs = [0] if w.B == 1 else [0, 13, w.B - 1]
+    sub = w.slice(seqs)
+    orc = _w8a16_oracle(sub, q8, scale)
+    idx = np.asarray(seqs)
+    rep = compare.compare(orc, _np(sub.draft_q), _np(sub.uniforms), _np(out.accept_len)[idx], _np(out.next_tok)[idx],
+                          _np(out.entropy)[idx], _np(out.logZ)[idx], _np(out.logits)[idx])
+    assert rep.ok, rep.summary()
+    check_ranges(w, out)
+
+
 def test_int8_head_small_integer_weights_are_bit_exact(binding):
     # integer weights with row maximum 127: scale = 1, q = W, every product and sum exact
     g = torch.Generator().manual_seed(9)
