@@ -240,6 +240,12 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       : "memory");
 }
 
+// Programmatic dependent launch: the grid may have been started while the kernel before it in the stream was still
+// running.  grid_dependency_wait returns once that kernel has completed and its writes are visible; it must precede
+// every global-memory access of the calling thread that could touch what that kernel reads or writes.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -528,6 +534,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
+      grid_dependency_wait();                            // W_lm and the hidden rows may come from the kernel before
       for (int t = 0; t < my_tiles && ok; ++t) {
         const int v0 = (pair + t * npairs) * pair_rows + static_cast<int>(rank) * p.tile_rows;
         int kx = 0;                                      // K coordinate of the block, in elements
@@ -646,6 +653,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
 #pragma unroll
     for (int i = 0; i < kEpiSlots; ++i) { st[i][0] = stats_empty(); st[i][1] = stats_empty(); }
     bool ok = true;
+    grid_dependency_wait();                              // the logits buffer may still be read by the kernel before
     for (int t = 0; t < my_tiles && ok; ++t) {
       const int buf = t % p.nbuf;
       const uint32_t acc_phase = static_cast<uint32_t>(t / p.nbuf) & 1u;
@@ -838,6 +846,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
+      grid_dependency_wait();
       for (int t = 0; t < my_tiles && ok; ++t) {
         int kx = 0;
         for (int kb = 0; kb < p.n_kblocks; ++kb, kx += kKStep) {
@@ -894,6 +903,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
   __syncwarp();                                          // warps 0 and 1 ran one lane apart from the others
   tc_fence_before();
   __syncthreads();
+  grid_dependency_wait();                                // (every thread that writes below; long since satisfied)
   if (!*abort_flag) {
     // one partial per CTA and row: the four quarters merged
     const float4* merge = reinterpret_cast<const float4*>(trans_base);
@@ -1061,6 +1071,9 @@ __global__ void __launch_bounds__(kK3Threads) accept_sample_kernel(const K3Param
   __shared__ int sh_n;
   __shared__ unsigned sh_flags;
 
+  // The next kernel in the stream (normally the next call's GEMM kernel, which waits for this grid before it touches
+  // memory) may be scheduled from now on: its launch and prologue then hide behind this kernel.
+  grid_dependency_release();
   cg::cluster_group cluster = cg::this_cluster();
   const int S = static_cast<int>(cluster.num_blocks());
   const int rank = static_cast<int>(cluster.block_rank());
@@ -1087,7 +1100,7 @@ __global__ void __launch_bounds__(kK3Threads) accept_sample_kernel(const K3Param
   }
   // Everything above reads the caller's inputs only.  When this kernel was launched with programmatic stream
   // serialization it may have started while the GEMM kernel was still running: wait here for its results.
-  asm volatile("griddepcontrol.wait;" ::: "memory");
+  grid_dependency_wait();
   for (int j = threadIdx.x; j < k; j += kK3Threads) {
     const int x = x_mine;
     sh_x[j] = x;
@@ -1724,13 +1737,17 @@ hola_status run_lm_head(hola_ctx* ctx, const hola_verify_args* a, float* logits,
   cfg.blockDim = dim3(kK1Threads);
   cfg.dynamicSmemBytes = static_cast<size_t>(pl.smem_bytes);
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  // may start while the kernel before it in the stream drains (its threads wait for that kernel before they touch
+  // global memory): launch, barrier set-up and tensor-memory allocation hide behind the previous call's last kernel
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   for (int pass = 0; pass < pl.passes; ++pass) {
     kp.row0 = pass * pl.rows_per_pass;
     kp.rows = M - kp.row0 < pl.rows_per_pass ? M - kp.row0 : pl.rows_per_pass;
