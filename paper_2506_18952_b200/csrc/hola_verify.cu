@@ -1532,7 +1532,8 @@ struct hola_ctx {
   float* hid_scale;         // [max_rows]
   // staging for hola_verify_host
   void* st_hidden; int* st_tok; void* st_q; float* st_u;
-  int* st_accept; int* st_next; float* st_entropy; float* st_logZ;
+  unsigned char* st_out;      // device block of one call's outputs (status, accept_len, next_tok, entropy, logZ, ...)
+  unsigned char* h_out;       // pinned host mirror: the outputs come back in ONE copy
   int force_stages;
   int no_rot;                 // tuning override: never use the rotating accumulator units
   cudaStream_t copy_stream;   // hola_verify_host: the draft tensor travels here while the GEMM runs
@@ -1554,8 +1555,26 @@ namespace {
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Where one call's outputs sit inside the output block of hola_verify_host (16-byte aligned pieces, packed for the
+// call's own B and k so that one copy brings them all back).
+struct OutBlock {
+  size_t status, accept, next, entropy, logZ, dent, total;
+};
+OutBlock out_block(int B, int k) {
+  const size_t rows = static_cast<size_t>(B) * (k + 1);
+  OutBlock o;
+  o.status = 0;
+  o.accept = 16;
+  o.next = o.accept + align_up(static_cast<size_t>(B) * 4, 16);
+  o.entropy = o.next + align_up(static_cast<size_t>(B) * 4, 16);
+  o.logZ = o.entropy + align_up(rows * 4, 16);
+  o.dent = o.logZ + align_up(rows * 4, 16);
+  o.total = o.dent + align_up(static_cast<size_t>(B) * (k > 0 ? k : 1) * 4, 16);
+  return o;
+}
+
 struct WsLayout {
-  size_t logits, partials, status, hq, hid8, hid_scale, st_hidden, st_tok, st_q, st_u, st_accept, st_next, st_entropy, st_logZ, st_qtok, total;
+  size_t logits, partials, status, hq, hid8, hid_scale, st_hidden, st_tok, st_q, st_u, st_out, st_qtok, total;
 };
 
 WsLayout ws_layout(int maxB, int maxK, int H, int V, int num_sms) {
@@ -1574,10 +1593,7 @@ WsLayout ws_layout(int maxB, int maxK, int H, int V, int num_sms) {
   w.st_tok = take(static_cast<size_t>(maxB) * maxK * 4);
   w.st_q = take(static_cast<size_t>(maxB) * maxK * V * 4);
   w.st_u = take(rows * 4);
-  w.st_accept = take(static_cast<size_t>(maxB) * 4);
-  w.st_next = take(static_cast<size_t>(maxB) * 4);
-  w.st_entropy = take(rows * 8);                         // target entropies, then the draft-row entropies
-  w.st_logZ = take(rows * 4);
+  w.st_out = take(out_block(maxB, maxK).total);
   w.st_qtok = take(static_cast<size_t>(maxB) * (maxK > 0 ? maxK : 1) * 4);
   w.total = off;
   return w;
@@ -1929,17 +1945,14 @@ hola_status hola_create(hola_ctx** out, int device, int maxB, int maxK, int H, i
   ctx->hid_scale = reinterpret_cast<float*>(ctx->ws + w.hid_scale);
   ctx->st_hidden = ctx->ws + w.st_hidden; ctx->st_tok = reinterpret_cast<int*>(ctx->ws + w.st_tok);
   ctx->st_q = ctx->ws + w.st_q; ctx->st_u = reinterpret_cast<float*>(ctx->ws + w.st_u);
-  ctx->st_accept = reinterpret_cast<int*>(ctx->ws + w.st_accept);
-  ctx->st_next = reinterpret_cast<int*>(ctx->ws + w.st_next);
-  ctx->st_entropy = reinterpret_cast<float*>(ctx->ws + w.st_entropy);
-  ctx->st_logZ = reinterpret_cast<float*>(ctx->ws + w.st_logZ);
+  ctx->st_out = reinterpret_cast<unsigned char*>(ctx->ws + w.st_out);
   ctx->st_qtok = reinterpret_cast<float*>(ctx->ws + w.st_qtok);
   cudaMemset(ctx->status, 0, 4);
   const size_t n_qtok = static_cast<size_t>(maxB) * (maxK > 0 ? maxK : 1);
   void* pinned = nullptr;
   if (cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) != cudaSuccess ||
       cudaEventCreateWithFlags(&ctx->copy_done, cudaEventDisableTiming) != cudaSuccess ||
-      cudaHostAlloc(&pinned, (n_qtok + maxB) * 4, cudaHostAllocDefault) != cudaSuccess) {
+      cudaHostAlloc(&pinned, (n_qtok + maxB) * 4 + 16 + out_block(maxB, maxK).total, cudaHostAllocDefault) != cudaSuccess) {
     if (ctx->copy_done) cudaEventDestroy(ctx->copy_done);
     if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
     cudaFree(ctx->ws);
@@ -1948,6 +1961,7 @@ hola_status hola_create(hola_ctx** out, int device, int maxB, int maxK, int H, i
   }
   ctx->h_qtok = static_cast<float*>(pinned);
   ctx->h_accept = reinterpret_cast<int*>(ctx->h_qtok + n_qtok);
+  ctx->h_out = reinterpret_cast<unsigned char*>(align_up(reinterpret_cast<size_t>(ctx->h_accept + maxB), 16));
   *out = ctx;
   return HOLA_OK;
 }
@@ -2082,7 +2096,8 @@ hola_status verify_host_lazy(hola_ctx* ctx, const hola_verify_args* a, cudaStrea
   h2d(ctx->st_tok, a->draft_tok, static_cast<size_t>(B) * k * 4, stream);
   h2d(ctx->st_u, a->uniforms, rows * 4, stream);
   h2d(ctx->st_qtok, ctx->h_qtok, static_cast<size_t>(B) * k * 4, stream);
-  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->status, 0, 4, stream);
+  const OutBlock ob = out_block(B, k);
+  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->st_out, 0, 4, stream);
   const size_t seq_pitch = static_cast<size_t>(k) * row_bytes;   // from row (b, 0) to row (b + 1, 0)
   ahead = ahead < 1 ? 1 : (ahead > k ? k : ahead);
   const size_t ahead_bytes = static_cast<size_t>(ahead) * row_bytes;     // rows 0 .. ahead-1 of a sequence are adjacent
@@ -2102,8 +2117,11 @@ hola_status verify_host_lazy(hola_ctx* ctx, const hola_verify_args* a, cudaStrea
   if (e != cudaSuccess) { set_error(ctx, "host-to-device copy", e); return HOLA_ERR_CUDA; }
   hola_verify_args d = *a;
   d.hidden = ctx->st_hidden; d.draft_tok = ctx->st_tok; d.draft_q = ctx->st_q; d.uniforms = ctx->st_u;
-  d.accept_len = ctx->st_accept; d.next_tok = ctx->st_next; d.entropy = ctx->st_entropy; d.logZ = ctx->st_logZ;
-  d.logits_out = nullptr; d.status_word = ctx->status; d.draft_entropy = nullptr;
+  d.accept_len = reinterpret_cast<int*>(ctx->st_out + ob.accept);
+  d.next_tok = reinterpret_cast<int*>(ctx->st_out + ob.next);
+  d.entropy = reinterpret_cast<float*>(ctx->st_out + ob.entropy);
+  d.logZ = reinterpret_cast<float*>(ctx->st_out + ob.logZ);
+  d.logits_out = nullptr; d.status_word = reinterpret_cast<uint32_t*>(ctx->st_out); d.draft_entropy = nullptr;
   hola_status s = check_lm_head_args(ctx, &d);
   if (s != HOLA_OK) return s;
   const Plan pl = make_plan(ctx, B * (k + 1), a->w_dtype);
@@ -2112,7 +2130,7 @@ hola_status verify_host_lazy(hola_ctx* ctx, const hola_verify_args* a, cudaStrea
     if ((s = run_accept_sample(ctx, &d, ctx->logits, ctx->ldl, 1, pl.grid, stream, ctx->st_qtok, 0)) != HOLA_OK) return s;
   } else {
     if ((s = run_accept_sample(ctx, &d, ctx->logits, ctx->ldl, 1, pl.grid, stream, ctx->st_qtok, 1)) != HOLA_OK) return s;
-    d2h(ctx->h_accept, ctx->st_accept, static_cast<size_t>(B) * 4);
+    d2h(ctx->h_accept, d.accept_len, static_cast<size_t>(B) * 4);
     if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
     if (e != cudaSuccess) { set_error(ctx, "accept lengths to host", e); return HOLA_ERR_CUDA; }
     for (int b = 0; b < B; ++b) {
@@ -2127,13 +2145,14 @@ hola_status verify_host_lazy(hola_ctx* ctx, const hola_verify_args* a, cudaStrea
     // statistics and accept lengths are in place: this launch repeats the (cheap) accept test and draws the token
     if ((s = run_accept_sample(ctx, &d, ctx->logits, ctx->ldl, 0, 0, stream, ctx->st_qtok, 0)) != HOLA_OK) return s;
   }
-  d2h(a->accept_len, ctx->st_accept, static_cast<size_t>(B) * 4);
-  d2h(a->next_tok, ctx->st_next, static_cast<size_t>(B) * 4);
-  d2h(a->entropy, ctx->st_entropy, rows * 4);
-  d2h(a->logZ, ctx->st_logZ, rows * 4);
-  if (a->status_word) d2h(a->status_word, ctx->status, 4);
+  d2h(ctx->h_out, ctx->st_out, ob.dent);                 // every output in one copy
   if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
   if (e != cudaSuccess) { set_error(ctx, "device-to-host copy", e); return HOLA_ERR_CUDA; }
+  memcpy(a->accept_len, ctx->h_out + ob.accept, static_cast<size_t>(B) * 4);
+  memcpy(a->next_tok, ctx->h_out + ob.next, static_cast<size_t>(B) * 4);
+  memcpy(a->entropy, ctx->h_out + ob.entropy, rows * 4);
+  memcpy(a->logZ, ctx->h_out + ob.logZ, rows * 4);
+  if (a->status_word) memcpy(a->status_word, ctx->h_out + ob.status, 4);
   ctx->last_h2d = up; ctx->last_d2h = down;
   return HOLA_OK;
 }
@@ -2232,24 +2251,29 @@ hola_status hola_verify_host(hola_ctx* ctx, const hola_verify_args* a, void* cud
   } else {
     h2d(ctx->st_q, a->draft_q, q_bytes);
   }
-  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->status, 0, 4, stream);
+  const OutBlock ob = out_block(a->B, a->k);
+  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->st_out, 0, 4, stream);
   if (e != cudaSuccess) { set_error(ctx, "host-to-device copy", e); return HOLA_ERR_CUDA; }
   hola_verify_args d = *a;
   d.hidden = ctx->st_hidden; d.draft_tok = ctx->st_tok; d.draft_q = ctx->st_q; d.uniforms = ctx->st_u;
-  d.accept_len = ctx->st_accept; d.next_tok = ctx->st_next; d.entropy = ctx->st_entropy; d.logZ = ctx->st_logZ;
-  d.logits_out = nullptr; d.status_word = ctx->status;
-  d.draft_entropy = a->draft_entropy ? ctx->st_entropy + rows : nullptr;   // staged after the entropies
+  d.accept_len = reinterpret_cast<int*>(ctx->st_out + ob.accept);
+  d.next_tok = reinterpret_cast<int*>(ctx->st_out + ob.next);
+  d.entropy = reinterpret_cast<float*>(ctx->st_out + ob.entropy);
+  d.logZ = reinterpret_cast<float*>(ctx->st_out + ob.logZ);
+  d.logits_out = nullptr; d.status_word = reinterpret_cast<uint32_t*>(ctx->st_out);
+  const bool want_dent = a->draft_entropy && a->gate_source == HOLA_GATE_DRAFT_ENTROPY;
+  d.draft_entropy = a->draft_entropy ? reinterpret_cast<float*>(ctx->st_out + ob.dent) : nullptr;
   if ((s = check_lm_head_args(ctx, &d)) != HOLA_OK) return s;
   if ((s = verify_device(ctx, &d, stream, overlap ? ctx->copy_done : nullptr)) != HOLA_OK) return s;
-  d2h(a->accept_len, ctx->st_accept, static_cast<size_t>(a->B) * 4);
-  d2h(a->next_tok, ctx->st_next, static_cast<size_t>(a->B) * 4);
-  d2h(a->entropy, ctx->st_entropy, rows * 4);
-  d2h(a->logZ, ctx->st_logZ, rows * 4);
-  if (a->status_word) d2h(a->status_word, ctx->status, 4);
-  if (a->draft_entropy && a->gate_source == HOLA_GATE_DRAFT_ENTROPY)
-    d2h(a->draft_entropy, ctx->st_entropy + rows, static_cast<size_t>(a->B) * a->k * 4);
+  d2h(ctx->h_out, ctx->st_out, want_dent ? ob.total : ob.dent);      // every output in one copy
   if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
   if (e != cudaSuccess) { set_error(ctx, "device-to-host copy", e); return HOLA_ERR_CUDA; }
+  memcpy(a->accept_len, ctx->h_out + ob.accept, static_cast<size_t>(a->B) * 4);
+  memcpy(a->next_tok, ctx->h_out + ob.next, static_cast<size_t>(a->B) * 4);
+  memcpy(a->entropy, ctx->h_out + ob.entropy, rows * 4);
+  memcpy(a->logZ, ctx->h_out + ob.logZ, rows * 4);
+  if (a->status_word) memcpy(a->status_word, ctx->h_out + ob.status, 4);
+  if (want_dent) memcpy(a->draft_entropy, ctx->h_out + ob.dent, static_cast<size_t>(a->B) * a->k * 4);
   ctx->last_h2d = up; ctx->last_d2h = down;
   return HOLA_OK;
 }
