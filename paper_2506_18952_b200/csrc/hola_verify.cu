@@ -1542,7 +1542,9 @@ struct hola_ctx {
   int host_lazy_q;            // hola_verify_host copies only the draft rows the step reads: 0 never, 1 always,
                               // -1 when the whole tensor would not fit under the GEMM (the default)
   float* st_qtok;             // device fp32 [maxB][maxK]: q_j(x_j) gathered on the host
-  float* h_qtok;              // pinned host: the same values before the copy
+  float* h_qtok;              // pinned host: the same values before the copy (inside h_small)
+  unsigned char* h_small;     // pinned host mirror of the workspace span [st_tok, st_qtok + ...): tokens, uniforms, q_tok
+  size_t small_u_off, small_qtok_off, small_span;   // offsets of the uniforms and of q_tok inside that span; its size
   int* h_accept;              // pinned host int32 [maxB]: accept_len read back between the two phases
   unsigned long long last_h2d, last_d2h;   // bytes the last hola_verify_host call moved
   // optional per-kernel timing (hola_profile_begin / hola_profile_end)
@@ -1574,7 +1576,7 @@ OutBlock out_block(int B, int k) {
 }
 
 struct WsLayout {
-  size_t logits, partials, status, hq, hid8, hid_scale, st_hidden, st_tok, st_q, st_u, st_out, st_qtok, total;
+  size_t logits, partials, status, hq, hid8, hid_scale, st_hidden, st_tok, st_q, st_u, st_out, st_qtok, st_small_end, total;
 };
 
 WsLayout ws_layout(int maxB, int maxK, int H, int V, int num_sms) {
@@ -1590,11 +1592,13 @@ WsLayout ws_layout(int maxB, int maxK, int H, int V, int num_sms) {
   w.hid8 = take(2 * align_up(rows, 32) * static_cast<size_t>(H));     // one or two 8-bit planes of the hidden rows
   w.hid_scale = take(2 * rows * 4);                                   // their scales (second plane after the first)
   w.st_hidden = take(rows * H * 2);
+  // the three small per-step inputs side by side: hola_verify_host sends them as one copy
   w.st_tok = take(static_cast<size_t>(maxB) * maxK * 4);
-  w.st_q = take(static_cast<size_t>(maxB) * maxK * V * 4);
   w.st_u = take(rows * 4);
-  w.st_out = take(out_block(maxB, maxK).total);
   w.st_qtok = take(static_cast<size_t>(maxB) * (maxK > 0 ? maxK : 1) * 4);
+  w.st_small_end = off;
+  w.st_q = take(static_cast<size_t>(maxB) * maxK * V * 4);
+  w.st_out = take(out_block(maxB, maxK).total);
   w.total = off;
   return w;
 }
@@ -1952,15 +1956,21 @@ hola_status hola_create(hola_ctx** out, int device, int maxB, int maxK, int H, i
   void* pinned = nullptr;
   if (cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) != cudaSuccess ||
       cudaEventCreateWithFlags(&ctx->copy_done, cudaEventDisableTiming) != cudaSuccess ||
-      cudaHostAlloc(&pinned, (n_qtok + maxB) * 4 + 16 + out_block(maxB, maxK).total, cudaHostAllocDefault) != cudaSuccess) {
+      cudaHostAlloc(&pinned, (w.st_small_end - w.st_tok) + maxB * 4 + 16 + out_block(maxB, maxK).total,
+                    cudaHostAllocDefault) != cudaSuccess) {
     if (ctx->copy_done) cudaEventDestroy(ctx->copy_done);
     if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
     cudaFree(ctx->ws);
     free(ctx);
     return HOLA_ERR_CUDA;
   }
-  ctx->h_qtok = static_cast<float*>(pinned);
-  ctx->h_accept = reinterpret_cast<int*>(ctx->h_qtok + n_qtok);
+  ctx->h_small = static_cast<unsigned char*>(pinned);
+  ctx->small_u_off = w.st_u - w.st_tok;
+  ctx->small_qtok_off = w.st_qtok - w.st_tok;
+  ctx->small_span = w.st_small_end - w.st_tok;
+  ctx->h_qtok = reinterpret_cast<float*>(ctx->h_small + ctx->small_qtok_off);
+  ctx->h_accept = reinterpret_cast<int*>(ctx->h_small + ctx->small_span);
+  (void)n_qtok;
   ctx->h_out = reinterpret_cast<unsigned char*>(align_up(reinterpret_cast<size_t>(ctx->h_accept + maxB), 16));
   *out = ctx;
   return HOLA_OK;
@@ -1973,7 +1983,7 @@ hola_status hola_destroy(hola_ctx* ctx) {
   free(ctx->prof_ev);
   if (ctx->copy_done) cudaEventDestroy(ctx->copy_done);
   if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
-  if (ctx->h_qtok) cudaFreeHost(ctx->h_qtok);
+  if (ctx->h_small) cudaFreeHost(ctx->h_small);
   cudaFree(ctx->ws);
   free(ctx);
   return HOLA_OK;
@@ -2093,9 +2103,10 @@ hola_status verify_host_lazy(hola_ctx* ctx, const hola_verify_args* a, cudaStrea
       ctx->h_qtok[b * k + j] = qx;
     }
   h2d(ctx->st_hidden, a->hidden, rows * a->H * 2, stream);
-  h2d(ctx->st_tok, a->draft_tok, static_cast<size_t>(B) * k * 4, stream);
-  h2d(ctx->st_u, a->uniforms, rows * 4, stream);
-  h2d(ctx->st_qtok, ctx->h_qtok, static_cast<size_t>(B) * k * 4, stream);
+  // tokens, uniforms and the gathered probabilities: into the pinned mirror, then one copy of the span in use
+  memcpy(ctx->h_small, a->draft_tok, static_cast<size_t>(B) * k * 4);
+  memcpy(ctx->h_small + ctx->small_u_off, a->uniforms, rows * 4);
+  h2d(ctx->st_tok, ctx->h_small, ctx->small_qtok_off + static_cast<size_t>(B) * k * 4, stream);
   const OutBlock ob = out_block(B, k);
   if (e == cudaSuccess) e = cudaMemsetAsync(ctx->st_out, 0, 4, stream);
   const size_t seq_pitch = static_cast<size_t>(k) * row_bytes;   // from row (b, 0) to row (b + 1, 0)
@@ -2240,8 +2251,9 @@ hola_status hola_verify_host(hola_ctx* ctx, const hola_verify_args* a, void* cud
   // largest input and only the accept/sample part reads it: it travels on the context's own stream while the
   // GEMM runs on the caller's.  (The previous call synchronised before returning, so the staging is free.)
   h2d(ctx->st_hidden, a->hidden, rows * a->H * 2);
-  h2d(ctx->st_tok, a->draft_tok, static_cast<size_t>(a->B) * a->k * 4);
-  h2d(ctx->st_u, a->uniforms, rows * 4);
+  memcpy(ctx->h_small, a->draft_tok, static_cast<size_t>(a->B) * a->k * 4);
+  memcpy(ctx->h_small + ctx->small_u_off, a->uniforms, rows * 4);
+  h2d(ctx->st_tok, ctx->h_small, ctx->small_u_off + rows * 4);
   const size_t q_bytes = static_cast<size_t>(a->B) * a->k * a->V * q_elem;
   const bool overlap = q_bytes && ctx->host_overlap;
   if (overlap) {

@@ -405,16 +405,18 @@ def test_host_entry_sends_only_the_rows_it_reads(binding, monkeypatch, q_dtype, 
         assert len(set(h.accept_len.tolist())) >= 3      # the case does spread over several accept lengths
     q_bytes = w.draft_q.numel() * w.draft_q.element_size()
     row = w.V * w.draft_q.element_size()
+    # hidden rows, then tokens + uniforms (+ gathered probabilities) as one copy of a workspace span whose pieces
+    # start on 256-byte boundaries: up to 255 bytes of padding after each piece but the last
     small = w.hidden.numel() * 2 + w.draft_tok.numel() * 4 + w.uniforms.numel() * 4
     if gate == 1:
-        assert up == small + q_bytes                      # the draft entropy reads every row
+        assert 0 <= up - (small + q_bytes) < 256          # the draft entropy reads every row
     elif fallback == 1:
-        assert up == small + w.B * w.k * 4                # greedy: no row at all
+        assert 0 <= up - (small + w.B * w.k * 4) < 512    # greedy: no row at all
     else:
         n = h.accept_len                                  # rows 0 .. ahead-1 go first, then the rows still missing
-        expected = {small + w.B * w.k * 4 + (w.B * ahead + int(((n >= ahead) & (n < w.k)).sum())) * row
-                    for ahead in range(1, w.k + 1)}
-        assert up in expected
+        pad = [up - (small + w.B * w.k * 4 + (w.B * ahead + int(((n >= ahead) & (n < w.k)).sum())) * row)
+               for ahead in range(1, w.k + 1)]
+        assert any(0 <= x < 512 for x in pad)
         assert up < small + q_bytes                       # and that is less than the whole tensor
 
 
