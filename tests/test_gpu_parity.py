@@ -551,7 +551,8 @@ def _w8a16_oracle(w, q8, scale, **kw):
     (1, 4, 64, 1000, torch.float32),       # 5 rows: one block of 32, N = 64
     (37, 6, 256, 5000, torch.bfloat16),    # 259 rows: two passes (at most 256 verify rows each)
     (5, 2, 80, 1001, torch.bfloat16),      # K tail, odd V
-    (33, 3, 128, 40000, torch.bfloat16),   # 132 rows: two MMAs of N = 192 (five blocks of 32, the last one ragged)
+    (33, 3, 128, 40000, torch.bfloat16),   # 132 rows: 320 operand rows, two MMAs of N = 192, last block of 32 ragged
+    (75, 2, 128, 3000, torch.bfloat16),    # 225 rows: 512 operand rows, two MMAs of N = 256
     (21, 5, 128, 3000, torch.float32),     # 126 rows: N = 256, double-buffered accumulators
 ])
 def test_w8a16_head_matches_oracle_on_two_plane_rows(binding, B, k, H, V, qd):
