@@ -1538,6 +1538,8 @@ struct hola_ctx {
   int no_rot;                 // tuning override: never use the rotating accumulator units
   cudaStream_t copy_stream;   // hola_verify_host: the draft tensor travels here while the GEMM runs
   cudaEvent_t copy_done;
+  cudaEvent_t fork_point;     // verify_device: where the side stream branches off the caller's stream
+  int hq_ready;               // the draft-row entropies of this call are already being made on the side stream
   int host_overlap;           // 1: copy the draft tensor on copy_stream while the GEMM runs
   int host_lazy_q;            // hola_verify_host copies only the draft rows the step reads: 0 never, 1 always,
                               // -1 when the whole tensor would not fit under the GEMM (the default)
@@ -1800,11 +1802,14 @@ hola_status run_accept_sample(hola_ctx* ctx, const hola_verify_args* a, const fl
   kp.tok = a->draft_tok; kp.q = a->draft_q; kp.q_dtype = a->q_dtype; kp.u = a->uniforms; kp.tau = a->tau;
   kp.gate_source = a->gate_source; kp.fallback = a->fallback; kp.hq_part = nullptr; kp.draft_entropy = a->draft_entropy;
   if (a->gate_source == HOLA_GATE_DRAFT_ENTROPY && a->k > 0) {
-    // one more pass over the draft rows: H(q_j) for every (sequence, draft position)
-    draft_entropy_kernel<<<dim3(static_cast<unsigned>(a->B * a->k), kHqSlices), 256, 0, stream>>>(
-        a->draft_q, a->q_dtype, a->V, ctx->hq);
-    const cudaError_t e0 = cudaGetLastError();
-    if (e0 != cudaSuccess) { set_error(ctx, "launch draft_entropy_kernel", e0); return HOLA_ERR_CUDA; }
+    // one more pass over the draft rows: H(q_j) for every (sequence, draft position) - unless the caller has put it
+    // on the side stream already, next to the GEMM
+    if (!ctx->hq_ready) {
+      draft_entropy_kernel<<<dim3(static_cast<unsigned>(a->B * a->k), kHqSlices), 256, 0, stream>>>(
+          a->draft_q, a->q_dtype, a->V, ctx->hq);
+      const cudaError_t e0 = cudaGetLastError();
+      if (e0 != cudaSuccess) { set_error(ctx, "launch draft_entropy_kernel", e0); return HOLA_ERR_CUDA; }
+    }
     kp.hq_part = ctx->hq;
   }
   kp.accept_len = a->accept_len; kp.next_tok = a->next_tok; kp.entropy = a->entropy; kp.logZ = a->logZ;
@@ -1956,9 +1961,11 @@ hola_status hola_create(hola_ctx** out, int device, int maxB, int maxK, int H, i
   void* pinned = nullptr;
   if (cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) != cudaSuccess ||
       cudaEventCreateWithFlags(&ctx->copy_done, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&ctx->fork_point, cudaEventDisableTiming) != cudaSuccess ||
       cudaHostAlloc(&pinned, (w.st_small_end - w.st_tok) + maxB * 4 + 16 + out_block(maxB, maxK).total,
                     cudaHostAllocDefault) != cudaSuccess) {
     if (ctx->copy_done) cudaEventDestroy(ctx->copy_done);
+    if (ctx->fork_point) cudaEventDestroy(ctx->fork_point);
     if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
     cudaFree(ctx->ws);
     free(ctx);
@@ -1982,6 +1989,7 @@ hola_status hola_destroy(hola_ctx* ctx) {
   for (int i = 0; i < 3 * ctx->prof_cap; ++i) cudaEventDestroy(ctx->prof_ev[i]);
   free(ctx->prof_ev);
   if (ctx->copy_done) cudaEventDestroy(ctx->copy_done);
+  if (ctx->fork_point) cudaEventDestroy(ctx->fork_point);
   if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
   if (ctx->h_small) cudaFreeHost(ctx->h_small);
   cudaFree(ctx->ws);
@@ -2046,11 +2054,35 @@ hola_status verify_device(hola_ctx* ctx, const hola_verify_args* a, cudaStream_t
   const bool prof = ctx->prof_on && ctx->prof_n < ctx->prof_cap;
   cudaEvent_t* ev = prof ? ctx->prof_ev + 3 * ctx->prof_n : nullptr;
   if (prof) cudaEventRecord(ev[0], stream);
+  cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(stream, &capturing) != cudaSuccess) capturing = cudaStreamCaptureStatusActive;
+  // The pass over the draft rows (draft-entropy gate) depends on nothing the GEMM makes, and its small CTAs fit on the
+  // SMs beside the GEMM's: it runs on the context's side stream (behind the copy of the draft tensor, when the host
+  // entry put one there), branching off the caller's stream before the GEMM and joining it again before the
+  // accept/sample kernel.  It is launched AFTER the GEMM so that the GEMM's CTAs get their SMs first.
+  // (While the caller records a graph everything stays on the caller's stream.)
+  const bool side = a->gate_source == HOLA_GATE_DRAFT_ENTROPY && a->k > 0 &&
+                    (before_sample || capturing == cudaStreamCaptureStatusNone);
+  if (side && !before_sample && cudaEventRecord(ctx->fork_point, stream) != cudaSuccess) return HOLA_ERR_CUDA;
   hola_status s = run_lm_head(ctx, a, logits, ldl, pl, stream);
   if (s != HOLA_OK) return s;
   if (prof) cudaEventRecord(ev[1], stream);
+  if (side) {
+    cudaError_t e = cudaSuccess;
+    if (!before_sample) e = cudaStreamWaitEvent(ctx->copy_stream, ctx->fork_point, 0);
+    if (e == cudaSuccess) {
+      draft_entropy_kernel<<<dim3(static_cast<unsigned>(a->B * a->k), kHqSlices), 256, 0, ctx->copy_stream>>>(
+          a->draft_q, a->q_dtype, a->V, ctx->hq);
+      e = cudaGetLastError();
+    }
+    if (e == cudaSuccess) e = cudaEventRecord(ctx->copy_done, ctx->copy_stream);
+    if (e != cudaSuccess) { set_error(ctx, "draft_entropy_kernel on the side stream", e); return HOLA_ERR_CUDA; }
+    before_sample = ctx->copy_done;
+  }
   if (before_sample && cudaStreamWaitEvent(stream, before_sample, 0) != cudaSuccess) return HOLA_ERR_CUDA;
+  ctx->hq_ready = side ? 1 : 0;
   s = run_accept_sample(ctx, a, logits, ldl, 1, pl.grid, stream);
+  ctx->hq_ready = 0;
   if (prof) { cudaEventRecord(ev[2], stream); ctx->prof_n++; }
   return s;
 }

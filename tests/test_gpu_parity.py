@@ -317,7 +317,8 @@ def test_deterministic_and_batch_order_equivariant(binding):
     assert torch.allclose(c.entropy, a.entropy[idx], atol=1e-5)
 
 
-def test_call_can_be_captured_in_a_cuda_graph(binding):
+@pytest.mark.parametrize("gate", [0, 1])
+def test_call_can_be_captured_in_a_cuda_graph(binding, gate):
     """hola_verify neither allocates nor synchronises: a stream capture records it, and a replay on new contents of
     the same buffers gives what a direct call gives."""
     w = workloads.gaussian_head("graph", 12, 4, 128, 6000, seed=5, device=DEV, w_std=0.3, sigma=1.0, tau=4.0)
@@ -325,18 +326,19 @@ def test_call_can_be_captured_in_a_cuda_graph(binding):
     with binding.HolaVerify(w.B, w.k, w.H, w.V) as ctx:
         bufs = [t.clone() for t in (w.hidden, w.W_lm, w.draft_tok, w.draft_q, w.uniforms)]
         out = ctx.alloc_outputs(w.B, w.k, False)
-        ctx.hola_verify(*bufs, w.tau, out=out)                     # warm-up outside the capture
+        ctx.hola_verify(*bufs, w.tau, out=out, gate_source=gate)   # warm-up outside the capture
         torch.cuda.synchronize()
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph):
-            ctx.hola_verify(*bufs, w.tau, out=out)
+            ctx.hola_verify(*bufs, w.tau, out=out, gate_source=gate)
         for src in (w2, w):
             for dst, t in zip(bufs, (src.hidden, src.W_lm, src.draft_tok, src.draft_q, src.uniforms)):
                 dst.copy_(t)
             out.accept_len.fill_(-1); out.next_tok.fill_(-1)
             graph.replay()
             torch.cuda.synchronize()
-            ref_out = ctx.hola_verify(src.hidden, src.W_lm, src.draft_tok, src.draft_q, src.uniforms, src.tau)
+            ref_out = ctx.hola_verify(src.hidden, src.W_lm, src.draft_tok, src.draft_q, src.uniforms, src.tau,
+                                      gate_source=gate)
             torch.cuda.synchronize()
             assert torch.equal(out.accept_len, ref_out.accept_len) and torch.equal(out.next_tok, ref_out.next_tok)
             assert torch.equal(out.entropy, ref_out.entropy) and torch.equal(out.logZ, ref_out.logZ)
