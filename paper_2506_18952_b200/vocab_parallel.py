@@ -10,7 +10,9 @@ them and a max over ranks at the end:
 
 Everything numeric runs in the library's kernels; this module marshals arguments and moves the records.
 `ShardedHolaVerify.step` does it for one rank over torch.distributed (NCCL on device tensors); `run_ranks_in_turn` runs
-all ranks of a group one after the other in ONE process, which is how a single GPU checks the multi-rank path.
+all ranks of a group one after the other in ONE process, which is how a single GPU checks the multi-rank path - and
+how one GPU runs a head whose vocabulary ranges are stored at different widths (each range is a "rank" with its own
+weight mode; the merges are exact, so the result is the verify step on the mixed-width matrix).
 """
 from __future__ import annotations
 
@@ -152,9 +154,10 @@ def split_inputs(W_lm, draft_q, draft_tok, world: int, w_scale=None):
 def run_ranks_in_turn(ranks: list[ShardedHolaVerify], hidden, parts, draft_tok, q_tok, uniforms, tau, **kw):
     """All ranks of a group in one process, one after the other (no kernel waits for another): call 1 on every rank,
     the records side by side, call 2 on every rank, the masses side by side, call 3 on every rank, the max."""
-    a8 = kw.pop("a8", False)
+    a8 = kw.pop("a8", False)                                 # (a part may carry its own "a8": ranges of mixed width)
     records = torch.stack([r.lm_head(hidden, p["W_lm"], draft_tok, p["draft_q"], q_tok, uniforms, tau,
-                                     w_scale=p["w_scale"], a8=a8, **kw) for r, p in zip(ranks, parts)])
+                                     w_scale=p["w_scale"], a8=p.get("a8", a8) if p["w_scale"] is not None else False,
+                                     **kw) for r, p in zip(ranks, parts)])
     masses = [r.accept(records) for r in ranks]
     if masses[0] is None:
         return ranks[0].outputs(), [r.outputs() for r in ranks]

@@ -259,6 +259,37 @@ def test_sharded_step_with_the_8bit_head():
 
 
 @gpu
+def test_ranges_of_mixed_width_on_one_device():
+    """A head whose first vocabulary range stays bf16 and whose second range is 8-bit (weights, and rows as two planes):
+    the ranges run as two "ranks" in turn and merge exactly, so the result is the verify step on the mixed matrix."""
+    from oracle import lobi
+    from paper_2506_18952_b200 import binding
+    w = workloads.gaussian_head("vp_mixed", 14, 4, 128, 6000, seed=17, device=DEV, w_std=0.3, sigma=1.0, tau=None)
+    parts, q_tok = vp.split_inputs(w.W_lm, w.draft_q, w.draft_tok, 2)
+    lo1, n1 = vp.shard_range(w.V, 1, 2)
+    q8, scale = binding.hola_quantize_w8(parts[1]["W_lm"])
+    parts[1].update(W_lm=q8, w_scale=scale, a8="a16")
+    ranks = [vp.ShardedHolaVerify(w.B, w.k, w.H, w.V, r, 2) for r in range(2)]
+    try:
+        merged, _ = vp.run_ranks_in_turn(ranks, w.hidden, parts, w.draft_tok, q_tok, w.uniforms, w.tau)
+        torch.cuda.synchronize()
+        got = [t.clone() for t in (merged.accept_len, merged.next_tok, merged.entropy, merged.logZ)]
+    finally:
+        for r in ranks:
+            r.close()
+    # oracle: logits of range 0 from the bf16 operands, of range 1 from the two-plane rows and the dequantised weights
+    hid = ref.bf16_bits_to_f64(_np(w.hidden))
+    B, k1, H = hid.shape
+    h16 = lobi.dequantize_two_plane(*lobi.quantize_rows_two_plane(hid.reshape(B * k1, H).astype(np.float32)))
+    W0 = ref.bf16_bits_to_f64(_np(w.W_lm))[:lo1]
+    W1 = lobi.dequantize_rows(_np(q8), _np(scale))
+    logits = np.concatenate([hid.reshape(B * k1, H) @ W0.T, h16 @ W1.T], axis=1).reshape(B, k1, w.V)
+    orc = ref.verify_from_logits(logits, _np(w.draft_tok), _np(w.draft_q), _np(w.uniforms), w.tau)
+    rep = compare.compare(orc, _np(w.draft_q), _np(w.uniforms), _np(got[0]), _np(got[1]), _np(got[2]), _np(got[3]), None)
+    assert rep.ok, rep.summary()
+
+
+@gpu
 def test_shard_calls_validate_their_arguments():
     from paper_2506_18952_b200 import binding
     w = workloads.gaussian_head("vp_args", 3, 2, 64, 1000, seed=1, device=DEV, w_std=0.3)
