@@ -152,6 +152,13 @@ __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release;" ::: "memory");
   asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
 }
+// Execution barrier only: orders no memory operations.  For the end of the kernel, where the point is that the peer CTA
+// has stopped using this CTA's barriers and tensor memory; a release here would make every thread wait until its last
+// stores of logits (hundreds of KB per CTA) have drained to L2 before the CTA may leave.
+__device__ __forceinline__ void cluster_sync_execution_only() {
+  asm volatile("barrier.cluster.arrive.relaxed;" ::: "memory");
+  asm volatile("barrier.cluster.wait;" ::: "memory");
+}
 
 // True in exactly one lane of a converged warp.  Unlike a lane-id test, the compiler knows that a single thread
 // runs the guarded region, so TMA / tcgen05 operands can stay in uniform registers.
@@ -918,7 +925,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
           make_float4(a.m, a.s, a.t, __int_as_float(a.arg));
     }
   }
-  cluster_sync_all();                                    // the peer no longer signals this CTA's barriers or tensor memory
+  cluster_sync_execution_only();                         // the peer no longer signals this CTA's barriers or tensor memory
   if (warp == 1) {
     if (*abort_flag) __nanosleep(200000);                // let copies already in flight land before leaving
     tmem_dealloc(tmem_base, kTmemCols);
