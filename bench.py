@@ -37,7 +37,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # in profiles/lm_head_entropy_kernel__batched__ncu_full.md (workload "batched": B=64 k=5 H=4096 V=32000).  The
 # traffic is W_lm + hidden + logits write-back, all proportional to V at fixed B, k, H, so a workload with the same
 # B, k, H gets the captured figure scaled by V; any other workload reports null.
-NCU_TRAFFIC = {"shape": (64, 5, 4096), "V": 32000, "bytes": 265955072 + 7874560}
+NCU_TRAFFIC = {"shape": (64, 5, 4096), "V": 32000, "bytes": 266059520 + 8002048}
 
 
 def ncu_traffic_bytes(w):
