@@ -344,6 +344,37 @@ def test_call_can_be_captured_in_a_cuda_graph(binding, gate):
             assert torch.equal(out.entropy, ref_out.entropy) and torch.equal(out.logZ, ref_out.logZ)
 
 
+@pytest.mark.parametrize("quant", [False, True])
+def test_back_to_back_calls_do_not_disturb_each_other(binding, quant):
+    """Calls queue on one stream without synchronisation, and each call's kernels may be scheduled while the call
+    before still runs (programmatic dependent launch): 60 calls alternating between two problems must each give
+    exactly what the problem gives alone."""
+    ws = [workloads.gaussian_head(f"b2b{i}", 6, 4, 256, 20000, seed=40 + i, device=DEV, w_std=0.3, sigma=1.0, tau=4.0)
+          for i in range(2)]
+    with binding.HolaVerify(6, 4, 256, 20000) as ctx:
+        Ws, scales = [], []
+        for w in ws:
+            if quant:
+                q8, sc = binding.hola_quantize_w8(w.W_lm)
+                Ws.append(q8); scales.append(sc)
+            else:
+                Ws.append(w.W_lm); scales.append(None)
+        kw = [dict(w_scale=sc, a8=True) if quant else {} for sc in scales]
+        alone = []
+        for w, W, k in zip(ws, Ws, kw):
+            alone.append(ctx.hola_verify(w.hidden, W, w.draft_tok, w.draft_q, w.uniforms, w.tau, **k))
+            torch.cuda.synchronize()
+        outs = [ctx.alloc_outputs(6, 4, False) for _ in range(60)]
+        for i, o in enumerate(outs):
+            w, W, k = ws[i & 1], Ws[i & 1], kw[i & 1]
+            ctx.hola_verify(w.hidden, W, w.draft_tok, w.draft_q, w.uniforms, w.tau, out=o, **k)
+        torch.cuda.synchronize()
+    for i, o in enumerate(outs):
+        r = alone[i & 1]
+        assert torch.equal(o.accept_len, r.accept_len) and torch.equal(o.next_tok, r.next_tok), i
+        assert torch.equal(o.entropy, r.entropy) and torch.equal(o.logZ, r.logZ), i
+
+
 def test_outputs_stay_inside_their_buffers(binding):
     # canary words before and after every output
     B, k, H, V = 6, 3, 64, 333
