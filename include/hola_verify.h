@@ -18,7 +18,8 @@
  * y = argmax p, instead of the speculative-sampling test).  A zero-initialised struct gives steps 1-5 as listed.
  *
  * All pointers in hola_verify_args are DEVICE pointers unless a field says otherwise.  Every buffer is owned by
- * the caller.  The library allocates device memory only inside hola_create and frees it in hola_destroy.
+ * the caller.  The library allocates device memory (and a few KB of pinned host memory for hola_verify_host) only
+ * inside hola_create and frees it in hola_destroy.
  * No function throws, aborts or exits; each returns a hola_status.
  */
 #ifndef HOLA_VERIFY_H_
@@ -122,7 +123,14 @@ size_t hola_workspace_bytes(int maxB, int maxK, int H, int V);
 
 /* Enqueues the whole verify step (steps 1-5 above) on `cuda_stream` (a cudaStream_t; NULL = default stream).
  * Asynchronous: no synchronisation, no host read-back.  The return code covers host-detectable errors only;
- * device-detected conditions are reported through status_word and never fault. */
+ * device-detected conditions are reported through status_word and never fault.
+ * Stream semantics are those of ordinary work on `cuda_stream`, with two things to know.  (1) The kernels are
+ * launched with programmatic stream serialization and the last one lets its successor be scheduled early; the
+ * library's own kernels wait for their predecessor before touching memory, and so does any ordinarily launched work.
+ * Only a kernel that the CALLER launches right behind this call with programmatic stream serialization must execute
+ * griddepcontrol.wait (cudaGridDependencySynchronize) before it reads this call's outputs.  (2) With the
+ * draft-entropy gate one kernel runs on a stream owned by the context, forked from and joined back to `cuda_stream`
+ * by events (it stays on `cuda_stream` while that stream is being captured into a graph). */
 hola_status hola_verify(hola_ctx* ctx, const hola_verify_args* args, void* cuda_stream);
 
 /* End-to-end form for callers whose per-step data lives in host memory.  Same computation as hola_verify, but
