@@ -1378,6 +1378,7 @@ __global__ void __launch_bounds__(256) quantize_rows_int8_kernel(const __nv_bflo
                                                                  float* scale) {
   __shared__ float sh_max[8];
   __shared__ float sh_scale;
+  grid_dependency_wait();                                // (no-op unless launched with programmatic serialization)
   const size_t row = blockIdx.x;
   const __nv_bfloat16* wr = W + row * H;
   float amax = 0.f;
@@ -1410,6 +1411,7 @@ __global__ void __launch_bounds__(256) quantize_rows_two_plane_kernel(const __nv
                                                                       signed char* q, float* s1, float* s2) {
   __shared__ float sh_max[8];
   __shared__ float sh_scale;
+  grid_dependency_wait();
   const int row = blockIdx.x;
   signed char* q1 = q + (static_cast<size_t>(64) * (row >> 5) + (row & 31)) * H;
   signed char* q2 = q1 + static_cast<size_t>(32) * H;
@@ -1723,17 +1725,29 @@ hola_status run_lm_head(hola_ctx* ctx, const hola_verify_args* a, float* logits,
     // 16-bit-class activations: two 8-bit planes per hidden row, blocks of 32 rows, into the context's workspace
     if (!ctx->hid8) return HOLA_ERR_INVALID_ARG;
     const int padded = round_up(M, 32);
-    quantize_rows_two_plane_kernel<<<static_cast<unsigned>(padded), 256, 0, stream>>>(
-        static_cast<const __nv_bfloat16*>(a->hidden), M, a->H, ctx->hid8, ctx->hid_scale, ctx->hid_scale + ctx->max_rows);
-    if (cudaGetLastError() != cudaSuccess) return HOLA_ERR_CUDA;
+    cudaLaunchConfig_t qc = {};
+    qc.gridDim = dim3(static_cast<unsigned>(padded)); qc.blockDim = dim3(256); qc.stream = stream;
+    cudaLaunchAttribute qa[1];
+    qa[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // launch latency hides behind the call before
+    qa[0].val.programmaticStreamSerializationAllowed = 1;
+    qc.attrs = qa; qc.numAttrs = 1;
+    if (cudaLaunchKernelEx(&qc, quantize_rows_two_plane_kernel, static_cast<const __nv_bfloat16*>(a->hidden), M, a->H,
+                           ctx->hid8, ctx->hid_scale, ctx->hid_scale + ctx->max_rows) != cudaSuccess)
+      return HOLA_ERR_CUDA;
     s = encode_map(ctx, &th, ctx->hid8, static_cast<uint64_t>(2 * padded), static_cast<uint64_t>(a->H),
                    static_cast<uint32_t>(pl.N / 2), true, true);
   } else if (i8) {
     // 8-bit activations: the same per-row quantiser as for W_lm, into the context's workspace
     if (!ctx->hid8) return HOLA_ERR_INVALID_ARG;          // (the entry point without a context has no room for it)
-    quantize_rows_int8_kernel<<<static_cast<unsigned>(M), 256, 0, stream>>>(
-        static_cast<const __nv_bfloat16*>(a->hidden), a->H, ctx->hid8, ctx->hid_scale);
-    if (cudaGetLastError() != cudaSuccess) return HOLA_ERR_CUDA;
+    cudaLaunchConfig_t qc = {};
+    qc.gridDim = dim3(static_cast<unsigned>(M)); qc.blockDim = dim3(256); qc.stream = stream;
+    cudaLaunchAttribute qa[1];
+    qa[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // launch latency hides behind the call before
+    qa[0].val.programmaticStreamSerializationAllowed = 1;
+    qc.attrs = qa; qc.numAttrs = 1;
+    if (cudaLaunchKernelEx(&qc, quantize_rows_int8_kernel, static_cast<const __nv_bfloat16*>(a->hidden), a->H, ctx->hid8,
+                           ctx->hid_scale) != cudaSuccess)
+      return HOLA_ERR_CUDA;
     s = encode_map(ctx, &th, ctx->hid8, static_cast<uint64_t>(M), static_cast<uint64_t>(a->H),
                    static_cast<uint32_t>(pl.N / 2), true, true);
   } else {
