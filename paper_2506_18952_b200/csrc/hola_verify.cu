@@ -96,6 +96,7 @@ struct K1Params {
   const float* w_scale;   // 8-bit W_lm: fp32 scale per vocabulary row, applied to the accumulators
   const float* h_scale;   // 8-bit activations (modes 2, 3): fp32 scale per verify row (mode 3: of the coarse plane)
   const float* h_scale2;  // mode 3: scale of the second plane
+  int stream_logits;      // 1: store the logits with the streaming hint (they exceed what the L2 keeps until they are read)
   float* logits;
   float4* partials;   // [grid][part_stride] (m, s, t, arg-max index)
   int part_stride;
@@ -437,6 +438,14 @@ __device__ __forceinline__ void expand_int8x16(const uint4 x, uint8_t* tile, int
   *reinterpret_cast<uint4*>(drow + (((2 * c + 1) ^ (row & 7)) << 4)) = make_uint4(o[4], o[5], o[6], o[7]);
 }
 
+// A logit on its way to the buffer.  Only one verify row per sequence is ever read back (row accept_len, by the
+// accept/sample kernel); when the buffer is much larger than the L2 the streaming hint lets the lines leave early
+// instead of displacing what the next kernel reads.
+__device__ __forceinline__ void store_logit(float* dst, float x, int streaming) {
+  if (streaming) __stcs(dst, x);
+  else *dst = x;
+}
+
 // One accumulator on its way to the logits buffer.  Mode 0: as is.  Mode 1: times the scale of the vocabulary row.
 // Mode 2: the accumulator is an int32 (bit pattern in `acc`); times the scales of the vocabulary row and of the
 // verify row.
@@ -723,7 +732,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
                   float* dst = p.logits + static_cast<size_t>(vr0 + 16 * half) * p.ldl + vocab;
 #pragma unroll
                   for (int i = 0; i < 16; ++i)
-                    if (i < rows_here) dst[static_cast<size_t>(i) * p.ldl] = f[i];
+                    if (i < rows_here) store_logit(dst + static_cast<size_t>(i) * p.ldl, f[i], p.stream_logits);
                 }
                 if (nv > 0) {
                   __syncwarp();
@@ -783,11 +792,11 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
               float* dst = p.logits + static_cast<size_t>(r0) * p.ldl + vocab;
               if (n_ok == 32) {
 #pragma unroll
-                for (int i = 0; i < 32; ++i) dst[static_cast<size_t>(i) * p.ldl] = v[i];
+                for (int i = 0; i < 32; ++i) store_logit(dst + static_cast<size_t>(i) * p.ldl, v[i], p.stream_logits);
               } else {
 #pragma unroll
                 for (int i = 0; i < 32; ++i)
-                  if (i < n_ok) dst[static_cast<size_t>(i) * p.ldl] = v[i];
+                  if (i < n_ok) store_logit(dst + static_cast<size_t>(i) * p.ldl, v[i], p.stream_logits);
               }
             }
             if (nv > 0) {
@@ -1766,6 +1775,7 @@ hola_status run_lm_head(hola_ctx* ctx, const hola_verify_args* a, float* logits,
   kp.w_scale = a->w_scale;
   kp.h_scale = ctx->hid_scale;
   kp.h_scale2 = ctx->hid_scale ? ctx->hid_scale + ctx->max_rows : nullptr;
+  kp.stream_logits = static_cast<double>(M) * a->V * 4.0 > 96e6 ? 1 : 0;     // beyond ~3/4 of the L2
   cudaError_t e = two ? cudaFuncSetAttribute(lm_head_entropy_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              pl.smem_bytes)
                 : i8 ? cudaFuncSetAttribute(lm_head_entropy_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
