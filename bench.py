@@ -33,17 +33,15 @@ METRIC = "verify_positions_per_s"
 UNIT = "positions/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of lm_head_entropy_kernel, from the ncu capture summarised
-# in profiles/lm_head_entropy_kernel__batched__ncu_full.md (workload "batched": B=64 k=5 H=4096 V=32000).  The
-# traffic is W_lm + hidden + logits write-back, all proportional to V at fixed B, k, H, so a workload with the same
-# B, k, H gets the captured figure scaled by V; any other workload reports null.
-NCU_TRAFFIC = {"shape": (64, 5, 4096), "V": 32000, "bytes": 266059520 + 8002048}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of lm_head_entropy_kernel<0>, from the ncu captures
+# summarised under profiles/: "batched" (--set full capture) and "large_vocab" (a capture of the three DRAM / time
+# counters on the full-size launch; its logits are stored with the streaming hint, so most of the 197 MB reach DRAM
+# inside the kernel).  Other workloads, and the other weight modes, report null.
+NCU_TRAFFIC = {"batched": 266059520 + 8002048, "large_vocab": 1054992640 + 165308416}
 
 
 def ncu_traffic_bytes(w):
-    if (w.B, w.k, w.H) != NCU_TRAFFIC["shape"]:
-        return None
-    return NCU_TRAFFIC["bytes"] * w.V / NCU_TRAFFIC["V"]
+    return NCU_TRAFFIC.get(w.name)
 
 
 def load_peaks():
