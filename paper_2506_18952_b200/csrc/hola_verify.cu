@@ -790,9 +790,12 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
               if (i < n_ok) v[i] = scaled<kMode>(v[i], w_scale, p.h_scale, r0 + i);
             if (vocab_ok) {
               float* dst = p.logits + static_cast<size_t>(r0) * p.ldl + vocab;
-              if (n_ok == 32) {
+              if (n_ok == 32 && p.stream_logits) {       // (the common cases without a test per store)
 #pragma unroll
-                for (int i = 0; i < 32; ++i) store_logit(dst + static_cast<size_t>(i) * p.ldl, v[i], p.stream_logits);
+                for (int i = 0; i < 32; ++i) __stcs(dst + static_cast<size_t>(i) * p.ldl, v[i]);
+              } else if (n_ok == 32) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) dst[static_cast<size_t>(i) * p.ldl] = v[i];
               } else {
 #pragma unroll
                 for (int i = 0; i < 32; ++i)
