@@ -37,7 +37,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # summarised under profiles/: "batched" (--set full capture) and "large_vocab" (a capture of the three DRAM / time
 # counters on the full-size launch; its logits are stored with the streaming hint, so most of the 197 MB reach DRAM
 # inside the kernel).  Other workloads, and the other weight modes, report null.
-NCU_TRAFFIC = {"batched": 266059520 + 8002048, "large_vocab": 1054992640 + 165308416}
+NCU_TRAFFIC = {"batched": 265883392 + 7073536, "large_vocab": 1055344896 + 165309952}
 
 
 def ncu_traffic_bytes(w):
