@@ -32,7 +32,7 @@
 extern "C" {
 #endif
 
-typedef struct hola_ctx hola_ctx; /* opaque: workspace, cached TMA descriptors, device properties */
+typedef struct hola_ctx hola_ctx; /* opaque: workspace, side stream, pinned staging, device properties */
 
 typedef enum {
   HOLA_OK = 0,
