@@ -6,7 +6,7 @@
  *      (the "higher-fidelity verifier" f_ver of the HSD section, restricted to its output layer);
  *   2. softmax statistics and Shannon entropy per position,  H = -sum_i p_i log p_i  in nats (HSD section);
  *   3. the entropy gate  g(t) = 1[H < tau]  and Eq. (1): a gated position keeps its draft token, any other
- *      position falls back to the verifier (Algorithm 1, lines 4-8);
+ *      position falls back to the verifier (Algorithm 1, the HSD loop);
  *   4. the fallback itself, which the paper leaves open, is the speculative-sampling test: accept draft token x
  *      iff  u * q(x) < p(x)  (u < min(1, p/q)); the first position that is not accepted ends the run;
  *   5. one new token per sequence: from the normalised residual max(0, p - q) at the first rejected position,
@@ -14,7 +14,7 @@
  *      (ascending token id, first token whose cumulative mass exceeds u * total).
  *
  * Two switches select the other readings of the paper's text: gate_source (entropy of the draft row instead of the
- * verifier's softmax, the HSD section's "uncertainty in the draft distribution") and fallback (a greedy verifier,
+ * verifier's softmax: the HSD section's prose ties H to the draft model's uncertainty) and fallback (a greedy verifier,
  * y = argmax p, instead of the speculative-sampling test).  A zero-initialised struct gives steps 1-5 as listed.
  *
  * All pointers in hola_verify_args are DEVICE pointers unless a field says otherwise.  Every buffer is owned by
@@ -46,8 +46,8 @@ typedef enum {
 
 typedef enum { HOLA_Q_BF16 = 0, HOLA_Q_F32 = 1 } hola_q_dtype;
 
-/* Which distribution's entropy feeds the gate g(t) = 1[H < tau].  The HSD section calls H "uncertainty in the draft
- * distribution" but writes it with the verifier's symbol p; both readings are available. */
+/* Which distribution's entropy feeds the gate g(t) = 1[H < tau].  The HSD section's prose ties H to how
+ * unsure the draft model is, yet writes it with the verifier's symbol p; both readings are available. */
 typedef enum {
   HOLA_GATE_TARGET_ENTROPY = 0, /* H of the verifier's softmax at the position (default) */
   HOLA_GATE_DRAFT_ENTROPY = 1   /* H(q_j) = -sum_v q_j(v) ln q_j(v) of the draft row, q used as given */
@@ -110,12 +110,27 @@ typedef struct {
 } hola_verify_args;
 
 /* Creates a context on `device` able to serve calls with B <= maxB, k <= maxK and exactly this H and V.
- * Allocates the workspace (hola_workspace_bytes) once.  One context serves one stream at a time.
- * Tuning overrides read from the environment here (for sweeps and tests; the defaults are what was measured best):
- * HOLA_STAGES=n (fewer shared-memory ring slots), HOLA_ROT=0 (257-384 rows per pass: two MMAs and one accumulator
- * buffer instead of the rotating 128-column units), HOLA_HOST_OVERLAP=0 and HOLA_HOST_LAZY_Q=0|1 (hola_verify_host). */
+ * Allocates the workspace (hola_workspace_bytes) once and tells the runtime once how much shared memory the kernels
+ * use.  One context serves one stream at a time.  The context also remembers, from call to call, the launch geometry
+ * of each (B * (k+1), w_dtype) it has seen and the tensor maps of each (hidden, W_lm) pointer pair: a call that
+ * repeats an earlier call's pointers and sizes does no set-up work on the host.  The library reads no environment
+ * variable. */
 hola_status hola_create(hola_ctx** out, int device, int maxB, int maxK, int H, int V);
 hola_status hola_destroy(hola_ctx* ctx);
+
+/* Debug and tuning switches of a context (for sweeps and tests; the defaults are what was measured best).  Results
+ * do not depend on them, only speed and the copies hola_verify_host makes.  Setting one drops the remembered launch
+ * geometry and tensor maps. */
+typedef enum {
+  HOLA_OPT_RING_SLOTS = 1,          /* shared-memory ring slots of the GEMM kernel: 0 = as many as fit, else 2..12      */
+  HOLA_OPT_ROTATING_UNITS = 2,      /* 257-384 rows per pass: 1 = three MMAs on rotating 128-column accumulator units
+                                     * (default), 0 = two MMAs and one accumulator buffer                              */
+  HOLA_OPT_HOST_OVERLAP = 3,        /* hola_verify_host: 1 = the draft tensor travels on the context's stream while
+                                     * the GEMM runs (default), 0 = every copy on the caller's stream                  */
+  HOLA_OPT_HOST_ROWS_ON_DEMAND = 4  /* hola_verify_host: 1 = always send only the draft rows the step reads,
+                                     * 0 = always the whole tensor, -1 = decide per call (default)                     */
+} hola_option;
+hola_status hola_set_option(hola_ctx* ctx, int option, int value);
 
 /* Device bytes a context of these limits holds: fp32 logits scratch [B(k+1)][V], per-CTA softmax partials,
  * staging for hola_verify_host, a status word. */
@@ -125,8 +140,12 @@ size_t hola_workspace_bytes(int maxB, int maxK, int H, int V);
  * Asynchronous: no synchronisation, no host read-back.  The return code covers host-detectable errors only;
  * device-detected conditions are reported through status_word and never fault.
  * Stream semantics are those of ordinary work on `cuda_stream`, with two things to know.  (1) The kernels are
- * launched with programmatic stream serialization and the last one lets its successor be scheduled early; the
- * library's own kernels wait for their predecessor before touching memory, and so does any ordinarily launched work.
+ * launched with programmatic stream serialization and each lets its successor be scheduled early; the library's own
+ * kernels wait for their predecessor before they touch anything it writes, and so does any ordinarily launched work.
+ * The first kernel of a call waits for the kernel in front of the call before it reads its inputs, and nothing behind
+ * it is scheduled before that wait has returned, so inputs written by the kernel just before the call are seen by all
+ * of the call.  (The step-by-step entry points hola_accept_sample, hola_shard_accept and hola_shard_sample wait
+ * before their first read of any input.)
  * Only a kernel that the CALLER launches right behind this call with programmatic stream serialization must execute
  * griddepcontrol.wait (cudaGridDependencySynchronize) before it reads this call's outputs.  (2) With the
  * draft-entropy gate one kernel runs on a stream owned by the context, forked from and joined back to `cuda_stream`
@@ -144,8 +163,8 @@ hola_status hola_verify(hola_ctx* ctx, const hola_verify_args* args, void* cuda_
  * the context while the GEMM runs; the accept lengths are read back once in the middle of the call and the rows
  * still missing follow.  Results are identical to hola_verify on the same data.  With the draft-entropy gate every
  * draft row is read, and for small draft tensors the whole copy hides under the GEMM anyway: then the whole tensor
- * is copied (on the context's stream, under the GEMM).  The environment variable HOLA_HOST_LAZY_Q (0 / 1, read by
- * hola_create) forces one or the other.  The host buffers must stay valid until the call returns. */
+ * is copied (on the context's stream, under the GEMM).  HOLA_OPT_HOST_ROWS_ON_DEMAND forces one or the
+ * other.  The host buffers must stay valid until the call returns. */
 hola_status hola_verify_host(hola_ctx* ctx, const hola_verify_args* args, void* cuda_stream);
 
 /* Vocabulary-parallel form of the verify step: `world` ranks (normally one GPU each) hold contiguous ranges of the
@@ -202,7 +221,10 @@ hola_status hola_accept_sample(hola_ctx* ctx, const hola_verify_args* args, void
  * part of the library image (every GPU that loads the library holds it until the process exits), and everything
  * else is the caller's: hidden, W_lm (inputs), logits_out (REQUIRED here, fp32 [B][k+1][V]), entropy, logZ
  * (outputs), all device pointers with the layouts given above; draft_*, uniforms, tau, accept_len, next_tok are
- * ignored.  Limit: B*(k+1) <= 512 verify rows, else HOLA_ERR_STATIC_LIMIT and nothing is launched.
+ * ignored.  W_lm must be bf16 (w_dtype = 0): the 8-bit modes need a context's workspace and are refused here.
+ * status_word is honoured and is the only way to learn that an on-chip wait ran out (HOLA_FLAG_TIMEOUT: entropy and
+ * logZ of that call are then invalid); without it such a call cannot be told from a good one.
+ * Limit: B*(k+1) <= 512 verify rows, else HOLA_ERR_STATIC_LIMIT and nothing is launched.
  * Runs on the CURRENT device, asynchronously on cuda_stream.  It calls no cudaMalloc, cudaFree or other allocating
  * routine.  The first call on each device also looks up the array's device address and the driver's tensor-map
  * encoder; make that first call outside any stream capture.
@@ -233,6 +255,17 @@ hola_status hola_plan_ex(const hola_ctx* ctx, int B, int k, int w_dtype, hola_pl
 hola_status hola_profile_begin(hola_ctx* ctx, int max_calls);
 hola_status hola_profile_end(hola_ctx* ctx, void* cuda_stream, double* lm_head_ms, double* accept_sample_ms,
                              int* calls);
+
+/* Self-test of the bounded waits (the paper has no counterpart; it is how the library's failure path is exercised
+ * without breaking anything).  Every on-chip wait of the kernels gives up after a fixed number of SM cycles, raises
+ * HOLA_FLAG_TIMEOUT and makes its CTA leave in good order.  This call launches a two-CTA miniature of the GEMM
+ * kernel's set-up (barriers, tensor memory of the pair) in which one thread and one warp per CTA wait, for at most
+ * `limit_cycles` SM cycles (1e3 .. 2e8), on a barrier that nothing ever signals.  Afterwards *status_word has
+ * HOLA_FLAG_TIMEOUT set (it is OR-ed in: clear it first), counters[0] = 128 (every thread reached the end) and
+ * counters[1] = 4 (each of the four waits returned "give up"); the device stays usable.  status_word and counters
+ * (uint32 [2], zeroed by the call) are device pointers.  Asynchronous on cuda_stream. */
+hola_status hola_selftest_bounded_wait(hola_ctx* ctx, long long limit_cycles, uint32_t* status_word,
+                                       uint32_t* counters, void* cuda_stream);
 
 const char* hola_strerror(hola_status s);
 /* Text of the last CUDA error seen by this context (empty string if none). */

@@ -9,7 +9,7 @@
 //   * HSD section, entropy definition  H = -sum_i p_i log p_i  (natural log), p = softmax of the verifier's
 //     LM-head logits at one verify position.
 //   * HSD section, gate  g(t) = 1[H < tau]  (strict), and Eq. (1): a gated position takes the draft token,
-//     any other position falls back to the verifier (Algorithm 1, lines 4-8).
+//     any other position falls back to the verifier (Algorithm 1, the HSD loop).
 //   * The paper does not say how the verifier decides.  The reading taken here is the speculative-sampling
 //     rule: accept the draft token x with probability min(1, p(x)/q(x)); at the first rejection draw the
 //     replacement from the normalised residual max(0, p - q); when all k drafts pass, draw one more token from
@@ -27,7 +27,7 @@
 //
 // Two variants of steps 4-5, selected by arguments (defaults reproduce the steps above):
 //   gate_source = 1: the gate looks at the entropy of the DRAFT distribution, H^q_j = -sum_v q_j(v) ln q_j(v), which
-//      is what the HSD section literally says ("uncertainty in the draft distribution"); q is used as given, terms
+//      is how the HSD section's prose describes H (a measure of how unsure the draft model is); q is used as given, terms
 //      with q = 0 contribute 0, the result is clamped at >= 0.  The target entropy is still computed and returned.
 //   fallback = 1: the verifier decides greedily (Eq. 1 read as "take the verifier's own token"): at a position
 //      where the gate is off the draft token is kept iff it equals argmax_v p_j(v) (lowest token id on ties);

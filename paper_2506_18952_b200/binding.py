@@ -19,10 +19,11 @@ HOLA_GATE_TARGET_ENTROPY, HOLA_GATE_DRAFT_ENTROPY = 0, 1
 HOLA_FALLBACK_SAMPLE, HOLA_FALLBACK_GREEDY = 0, 1
 HOLA_W_BF16, HOLA_W_INT8, HOLA_W8A8, HOLA_W8A16 = 0, 1, 2, 3
 FLAG_BAD_TOKEN, FLAG_BAD_UNIFORM, FLAG_TIMEOUT, FLAG_R_ZERO = 1, 2, 4, 8
+HOLA_OPT_RING_SLOTS, HOLA_OPT_ROTATING_UNITS, HOLA_OPT_HOST_OVERLAP, HOLA_OPT_HOST_ROWS_ON_DEMAND = 1, 2, 3, 4
 
 EXPORTS = ["hola_create", "hola_destroy", "hola_workspace_bytes", "hola_verify", "hola_verify_host",
            "hola_lm_head_entropy", "hola_accept_sample", "hola_host_traffic", "hola_shard_record_bytes", "hola_shard_lm_head",
-           "hola_shard_accept", "hola_shard_sample", "hola_lm_head_entropy_static", "hola_quantize_w8", "hola_plan", "hola_plan_ex", "hola_profile_begin", "hola_profile_end", "hola_strerror", "hola_last_cuda_error",
+           "hola_shard_accept", "hola_shard_sample", "hola_lm_head_entropy_static", "hola_quantize_w8", "hola_plan", "hola_plan_ex", "hola_set_option", "hola_selftest_bounded_wait", "hola_profile_begin", "hola_profile_end", "hola_strerror", "hola_last_cuda_error",
            "hola_version"]
 
 
@@ -83,6 +84,11 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
     lib.hola_plan_ex.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.POINTER(hola_plan_info)]
     lib.hola_profile_begin.restype = ctypes.c_int
     lib.hola_profile_begin.argtypes = [ctypes.c_void_p, ctypes.c_int]
+    lib.hola_set_option.restype = ctypes.c_int
+    lib.hola_set_option.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int]
+    lib.hola_selftest_bounded_wait.restype = ctypes.c_int
+    lib.hola_selftest_bounded_wait.argtypes = [ctypes.c_void_p, ctypes.c_longlong, ctypes.c_void_p, ctypes.c_void_p,
+                                               ctypes.c_void_p]
     lib.hola_shard_record_bytes.restype = ctypes.c_size_t
     lib.hola_shard_record_bytes.argtypes = [ctypes.c_int, ctypes.c_int]
     for name in ("hola_shard_lm_head", "hola_shard_accept", "hola_shard_sample"):
@@ -137,7 +143,7 @@ def hola_quantize_w8(W_lm: torch.Tensor, stream=None):
     return q, scale
 
 
-def hola_lm_head_entropy_static(hidden, W_lm, logits, entropy, logZ, stream=None) -> None:
+def hola_lm_head_entropy_static(hidden, W_lm, logits, entropy, logZ, stream=None, status=None) -> None:
     """Steps 1-2 through the entry point that allocates no device memory (no context needed).
 
     For callers that cannot call cudaMalloc (all of HBM already handed to their own pool, a fixed memory budget,
@@ -145,7 +151,8 @@ def hola_lm_head_entropy_static(hidden, W_lm, logits, entropy, logZ, stream=None
     built into it.  Every tensor is the caller's and lives on the current device: hidden bf16 [B, k+1, H],
     W_lm bf16 [V, H], and the outputs logits fp32 [B, k+1, V], entropy and logZ fp32 [B, k+1].
     At most 512 verify rows (B * (k+1)); larger calls raise HolaError and launch nothing.  Calls share the
-    built-in array, so do not let two of them overlap on one GPU.
+    built-in array, so do not let two of them overlap on one GPU.  `status` (int32 [1] on the device, optional) gets
+    HOLA_FLAG_TIMEOUT OR-ed in should an on-chip wait run out: it is the only way to learn of that here.
     """
     lib = load_library()
     B, k1, H = hidden.shape
@@ -153,6 +160,7 @@ def hola_lm_head_entropy_static(hidden, W_lm, logits, entropy, logZ, stream=None
     a.B, a.k, a.H, a.V = B, k1 - 1, H, W_lm.shape[0]
     a.hidden, a.W_lm = _dptr(hidden), _dptr(W_lm)
     a.logits_out, a.entropy, a.logZ = _dptr(logits), _dptr(entropy), _dptr(logZ)
+    a.status_word = _dptr(status)
     _check(lib, None, lib.hola_lm_head_entropy_static(ctypes.byref(a), _stream_ptr(stream)),
            "hola_lm_head_entropy_static")
 
@@ -203,6 +211,21 @@ class HolaVerify:
         info = hola_plan_info()
         _check(self.lib, self._ctx, self.lib.hola_plan_ex(self._ctx, B, k, w_dtype, ctypes.byref(info)), "hola_plan_ex")
         return {n: getattr(info, n) for n, _ in info._fields_}
+
+    def hola_set_option(self, option: int, value: int):
+        _check(self.lib, self._ctx, self.lib.hola_set_option(self._ctx, int(option), int(value)), "hola_set_option")
+
+    def hola_selftest_bounded_wait(self, limit_cycles: int = 100000, stream=None) -> tuple[int, int, int]:
+        """Runs the bounded-wait self-test; returns (status word, threads that reached the end, waits that gave up)
+        after synchronising the stream."""
+        dev = torch.device("cuda", self.device)
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+        counters = torch.zeros(2, dtype=torch.int32, device=dev)
+        st = self.lib.hola_selftest_bounded_wait(self._ctx, int(limit_cycles), _dptr(status), _dptr(counters),
+                                                 _stream_ptr(stream))
+        _check(self.lib, self._ctx, st, "hola_selftest_bounded_wait")
+        (torch.cuda.current_stream() if stream is None else stream).synchronize()
+        return int(status.item()), int(counters[0].item()), int(counters[1].item())
 
     def hola_profile_begin(self, max_calls: int):
         _check(self.lib, self._ctx, self.lib.hola_profile_begin(self._ctx, max_calls), "hola_profile_begin")

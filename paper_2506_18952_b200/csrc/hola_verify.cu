@@ -1,5 +1,5 @@
 // hola_verify.cu - sm_100a kernels and C ABI for the entropy-aware verify step of Hierarchical Speculative
-// Decoding (HSD section, Eq. 1, Algorithm 1 lines 4-8).  See include/hola_verify.h for the contract.
+// Decoding (HSD section, Eq. 1, the HSD loop of Algorithm 1).  See include/hola_verify.h for the contract.
 //
 // Kernels
 //   lm_head_entropy_kernel      persistent, warp-specialised weight-streaming GEMM run by pairs of CTAs (clusters of
@@ -72,13 +72,13 @@ constexpr long long kWaitLimitCycles = 4000000000ll;   // about 2 s of SM clock 
 
 constexpr int kK3Threads = 256;
 constexpr int kK3Warps = kK3Threads / 32;
+constexpr int kK3MaxPerSm = 4;                   // CTAs of the accept/sample kernel an SM holds (register budget: 64 per thread)
+constexpr size_t kSmTotalSmem = 228 * 1024;      // shared memory of an SM
+constexpr size_t kK3SmemOverhead = 1024 + 2048 + 256;   // per CTA: the system's reserve, static arrays (rounded up), slack
 constexpr int kChunk = 128;                      // vocabulary entries per warp step (32 lanes x 4)
 constexpr int kMaxChunks = 4096;                 // => V <= 524288
 constexpr int kMaxK1 = 64;                       // k + 1 <= 64
-#ifndef K3_UNROLL
-#define K3_UNROLL 4
-#endif
-constexpr int kK3Unroll = K3_UNROLL;             // vocabulary chunks a warp has in flight per step
+constexpr int kK3Unroll = 4;                     // vocabulary chunks a warp has in flight per step
 
 constexpr int kHqSlices = 8;                     // CTAs that share one draft row in draft_entropy_kernel
 
@@ -86,6 +86,8 @@ constexpr float kLog2e = 1.4426950408889634f;
 
 struct K1Params {
   int M;          // total verify rows B(k+1)
+  int first_pass; // 1: the first launch of a call (its producers wait for the kernel before it in the stream);
+                  // later passes are only scheduled once every CTA of the pass before has passed that wait
   int row0;       // first row of this pass
   int rows;       // rows of this pass (<= n_sub * N)
   int V, n_ptiles, n_kblocks, stages, nbuf;
@@ -112,6 +114,9 @@ struct K3Params {
   const void* q;
   int q_dtype;
   const float* q_tok;           // optional fp32 [B][k]: q_j(x_j) already gathered (then q is read at row n only)
+  int inputs_settled;           // 1: launched right behind this call's own GEMM kernel, whose CTAs have waited for the
+                                // kernel before the call: tokens, uniforms and draft probabilities may be read
+                                // before this grid's dependency wait.  0: wait first.
   int phase;                    // 0: the whole step; 1: stop after the accept test (accept_len, statistics written);
                                 // vocabulary-parallel form: 3: stop after the masses of row n inside this shard,
                                 // 4: the draw, by the shard that holds the point u * R
@@ -198,7 +203,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // Bounded wait.  Returns false when the CTA is aborting (this wait or another one ran out of time).
 // The clock is the SM's cycle counter (cheap to read), looked at only every 256 unsuccessful polls.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                          unsigned* status) {
+                                          unsigned* status, long long limit_cycles = kWaitLimitCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   long long t0 = 0;
   uint32_t spins = 0;
@@ -208,7 +213,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       if (*abort_flag) return false;
       const long long now = clock64();
       if (t0 == 0) t0 = now;
-      if (now - t0 > kWaitLimitCycles) {
+      if (now - t0 > limit_cycles) {
         *abort_flag = 1u;
         if (status) atomicOr(status, HOLA_FLAG_TIMEOUT);
         return false;
@@ -219,9 +224,9 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 
 // Whole-warp form: lane 0 polls, every lane gets the same answer (and, through the shuffle, the same ordering).
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                               unsigned* status) {
+                                               unsigned* status, long long limit_cycles = kWaitLimitCycles) {
   int r = 1;
-  if ((threadIdx.x & 31) == 0) r = mbar_wait(bar, parity, abort_flag, status) ? 1 : 0;
+  if ((threadIdx.x & 31) == 0) r = mbar_wait(bar, parity, abort_flag, status, limit_cycles) ? 1 : 0;
   r = __shfl_sync(0xffffffffu, r, 0);
   return r != 0;
 }
@@ -532,6 +537,14 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
   tc_fence_after();
   const uint32_t tmem_base = *tmem_holder;
 
+  // Programmatic dependent launch.  The kernel behind this one in the stream (the next pass over W_lm, or the
+  // accept/sample kernel) may be scheduled as soon as every CTA here has said so: its CTAs then start on the SMs this
+  // grid's CTAs leave, set themselves up under this grid's tail, and wait for this grid to complete before they touch
+  // what it writes.  One thread per CTA, the TMA producer, says so only after its own dependency wait (first pass):
+  // whatever runs behind this kernel therefore never starts before the kernel in front of the call has completed.
+  const bool producer = warp == 0 && elect_one();
+  if (!producer) grid_dependency_release();
+
   const int my_tiles = (p.n_ptiles - pair + npairs - 1) / npairs;
   const int sub_chunks = (p.N + 31) >> 5;                // 32-column chunks per MMA's accumulator
   // Accumulators.  rot == 0: MMA s of buffer b starts at column b * 256 + s * 256 (two buffers only when
@@ -542,7 +555,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (one per CTA)
-    if (elect_one()) {
+    if (producer) {
       const uint64_t pol_w = l2_policy_evict_first();    // W_lm is streamed once
       const uint64_t pol_h = l2_policy_evict_last();     // hidden is re-read for every tile
       const uint32_t leader_full = map_to_cta(full_bar, 0);
@@ -550,7 +563,8 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      grid_dependency_wait();                            // W_lm and the hidden rows may come from the kernel before
+      if (p.first_pass) grid_dependency_wait();          // W_lm and the hidden rows may come from the kernel before
+      grid_dependency_release();
       for (int t = 0; t < my_tiles && ok; ++t) {
         const int v0 = (pair + t * npairs) * pair_rows + static_cast<int>(rank) * p.tile_rows;
         int kx = 0;                                      // K coordinate of the block, in elements
@@ -944,6 +958,46 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
   }
 }
 
+// ------------------------------------------------------------------------------------------------ self-test
+// The way a GEMM CTA pair gives up, in miniature and on purpose: a pair of CTAs sets up barriers and tensor memory as
+// the GEMM kernel does, then one thread and one whole warp of each CTA wait (with the limit given) on a barrier that
+// nothing ever arrives on.  The wait must run out, raise HOLA_FLAG_TIMEOUT and the CTA's abort flag, the other waiters
+// must see that flag, and every thread must reach the common tail, where the tensor memory is released.
+// out[0] counts the threads that got there, out[1] the waits that returned "give up".
+__global__ void __launch_bounds__(64, 1) bounded_wait_selftest_kernel(long long limit_cycles, unsigned* status,
+                                                                      unsigned* out) {
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ uint32_t tmem_holder;
+  __shared__ uint32_t abort_word;
+  volatile uint32_t* abort_flag = &abort_word;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_word = 0u;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncwarp();
+  if (warp == 1) tmem_alloc(smem_u32(&tmem_holder), 32);
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_holder;
+  unsigned gave_up = 0;
+  if (warp == 0) {
+    if (lane == 0) gave_up = mbar_wait(smem_u32(&bar), 0u, abort_flag, status, limit_cycles) ? 0u : 1u;
+  } else {
+    gave_up = mbar_wait_warp(smem_u32(&bar), 0u, abort_flag, status, limit_cycles) ? 0u : (lane == 0 ? 1u : 0u);
+  }
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (gave_up) atomicAdd(out + 1, 1u);
+  atomicAdd(out, 1u);
+  cluster_sync_execution_only();
+  if (warp == 1) tmem_dealloc(tmem_base, 32);
+}
+
 // ------------------------------------------------------------------------------------------------ K2
 __device__ __forceinline__ Stats warp_merge_partials(const float4* partials, int nparts, int part_stride, int row,
                                                      int lane) {
@@ -1021,6 +1075,20 @@ __device__ __forceinline__ double warp_sum_f64(double x) {
   return x;
 }
 
+// Four sums over the warp at once, in the addition order of warp_sum_f64 (pairs 16 apart, then 8, 4, 2, 1) and so with
+// the same bits, for a third of the shuffles: the first two rounds halve the number of values a lane carries instead of
+// adding all of them everywhere.  Lanes 8 i .. 8 i + 7 return the sum of v[i].
+__device__ __forceinline__ double warp_sum4_f64(const double v[4], int lane) {
+  const bool hi16 = (lane & 16) != 0;
+  const double a = (hi16 ? v[2] : v[0]) + __shfl_xor_sync(0xffffffffu, hi16 ? v[0] : v[2], 16);
+  const double b = (hi16 ? v[3] : v[1]) + __shfl_xor_sync(0xffffffffu, hi16 ? v[1] : v[3], 16);
+  const bool hi8 = (lane & 8) != 0;
+  double c = (hi8 ? b : a) + __shfl_xor_sync(0xffffffffu, hi8 ? a : b, 8);
+#pragma unroll
+  for (int off = 4; off > 0; off >>= 1) c += __shfl_xor_sync(0xffffffffu, c, off);
+  return c;
+}
+
 // Logits and draft probabilities of vocabulary entries base..base+3 of one row (q = 0 when the row is drawn
 // from p itself; entries at or beyond V get l = -inf, q = 0 and so no mass).  Loads only: a caller can issue
 // several of these before using any, which keeps more requests in flight.
@@ -1082,11 +1150,13 @@ __device__ __forceinline__ float clamp_uniform(float u, unsigned& flags) {
 // total to all CTAs of the cluster through distributed shared memory.  After one cluster barrier each CTA knows
 // the total mass R and which slice holds the point u*R; that CTA alone finishes the inverse-CDF search.
 template <bool kVec>
-__global__ void __launch_bounds__(kK3Threads) accept_sample_kernel(const K3Params p) {
+__global__ void __launch_bounds__(kK3Threads, kK3MaxPerSm) accept_sample_kernel(const K3Params p) {
   extern __shared__ double csum[];                       // per-chunk residual mass of this CTA's slice
   __shared__ double sh_tot[2][8];                        // slice totals of the whole cluster, per attempt
-  __shared__ float sh_logZ[kMaxK1], sh_H[kMaxK1], sh_lx[kMaxK1], sh_qx[kMaxK1], sh_u[kMaxK1], sh_Hq[kMaxK1];
-  __shared__ int sh_x[kMaxK1], sh_amax[kMaxK1];
+  __shared__ float sh_logZ[kMaxK1], sh_H[kMaxK1], sh_u[kMaxK1 + 1];
+  __shared__ int sh_amax[kMaxK1];
+  __shared__ int sh_stop[2];                             // first draft position not accepted, per gathering warp
+  __shared__ unsigned sh_wflags[2];
   __shared__ int sh_n;
   __shared__ unsigned sh_flags;
 
@@ -1100,16 +1170,23 @@ __global__ void __launch_bounds__(kK3Threads) accept_sample_kernel(const K3Param
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int k = p.k, V = p.V;
   const int row_first = b * (k + 1);
-
-  // ---- gather the k draft-token logits, draft probabilities and the uniforms (independent of the statistics)
-  for (int j = threadIdx.x; j <= k; j += kK3Threads) sh_u[j] = p.u[b * (k + 1) + j];
-  int x_mine = -1;                                       // (k <= 63 < kK3Threads: one draft position per thread)
-  float qx_mine = 0.f;
   const bool shard = p.shard_world > 0;
   const int Vtok = shard ? p.V_global : V;               // range of valid token ids
-  if (threadIdx.x < k) {
-    const int j = threadIdx.x;
+
+  // Inputs that come from the caller and not from the GEMM kernel.  Behind this call's own GEMM kernel they are known
+  // to be in place (its CTAs waited for whatever ran before the call) and are fetched under that kernel's tail;
+  // in every other launch the dependency wait comes first.
+  if (!p.inputs_settled) grid_dependency_wait();
+  // The last two warps own the draft positions (k <= 63: one position per thread, j = gthread); the other warps
+  // start on the softmax statistics at once, so the two chains of dependent loads run side by side.
+  const int gthread = static_cast<int>(threadIdx.x) - (kK3Threads - 64);
+  const bool gatherer = gthread >= 0 && gthread < k;
+  int x_mine = -1;
+  float qx_mine = 0.f, u_mine = 0.f, lx_mine = 0.f;
+  if (gatherer) {
+    const int j = gthread;
     x_mine = p.tok[b * k + j];
+    u_mine = p.u[b * (k + 1) + j];
     if (x_mine >= 0 && x_mine < Vtok) {
       const size_t qi = (static_cast<size_t>(b) * k + j) * V + x_mine;
       if (p.q_tok) qx_mine = p.q_tok[b * k + j];
@@ -1117,31 +1194,27 @@ __global__ void __launch_bounds__(kK3Threads) accept_sample_kernel(const K3Param
                                                 : static_cast<const float*>(p.q)[qi];
     }
   }
-  // Everything above reads the caller's inputs only.  When this kernel was launched with programmatic stream
-  // serialization it may have started while the GEMM kernel was still running: wait here for its results.
-  grid_dependency_wait();
-  for (int j = threadIdx.x; j < k; j += kK3Threads) {
-    const int x = x_mine;
-    sh_x[j] = x;
-    float lx = 0.f;
-    const float qx = qx_mine;
+  if (threadIdx.x == 0) sh_u[k] = p.u[b * (k + 1) + k];
+  // From here on the GEMM kernel's results are read.
+  if (p.inputs_settled) grid_dependency_wait();
+  float hq_mine = 0.f;
+  if (gatherer) {
+    const int j = gthread, x = x_mine;
     if (x >= 0 && x < Vtok) {
       if (shard) {                                       // exactly one shard owns x and left its logit there
-        lx = -CUDART_INF_F;
-        for (int r = 0; r < p.shard_world; ++r) lx = fmaxf(lx, p.lx_all[static_cast<size_t>(r) * p.rec_stride + b * k + j]);
+        lx_mine = -CUDART_INF_F;
+        for (int r = 0; r < p.shard_world; ++r)
+          lx_mine = fmaxf(lx_mine, p.lx_all[static_cast<size_t>(r) * p.rec_stride + b * k + j]);
       } else {
-        lx = p.logits[static_cast<size_t>(row_first + j) * p.ldl + x];
+        lx_mine = p.logits[static_cast<size_t>(row_first + j) * p.ldl + x];
       }
     }
-    sh_lx[j] = lx; sh_qx[j] = qx;
-    float hq = 0.f;
     if (p.gate_source == HOLA_GATE_DRAFT_ENTROPY) {
       double tot = 0.0;
       for (int sl = 0; sl < kHqSlices; ++sl) tot += p.hq_part[(static_cast<size_t>(b) * k + j) * kHqSlices + sl];
-      hq = fmaxf(0.f, static_cast<float>(-tot));
-      if (rank == 0 && p.draft_entropy) p.draft_entropy[b * k + j] = hq;
+      hq_mine = fmaxf(0.f, static_cast<float>(-tot));
+      if (rank == 0 && p.draft_entropy) p.draft_entropy[b * k + j] = hq_mine;
     }
-    sh_Hq[j] = hq;
   }
   // ---- softmax statistics of this sequence's k+1 positions
   if (p.combine) {
@@ -1162,25 +1235,53 @@ __global__ void __launch_bounds__(kK3Threads) accept_sample_kernel(const K3Param
   }
   __syncthreads();
 
-  // ---- gate and ratio test in draft order; stop at the first position that is not accepted
-  if (threadIdx.x == 0) {
+  // ---- gate and ratio test, every draft position on its own thread; the run of kept drafts ends at the first
+  // position that is not accepted (a token outside the vocabulary counts as one)
+  {
     unsigned flags = 0;
-    int n = k;
-    for (int j = 0; j < k; ++j) {
-      const int x = sh_x[j];
-      if (x < 0 || x >= Vtok) { flags |= HOLA_FLAG_BAD_TOKEN; n = j; break; }
-      const float gate_value = p.gate_source == HOLA_GATE_DRAFT_ENTROPY ? sh_Hq[j] : sh_H[j];
-      if (gate_value < p.tau) continue;                  // entropy gate: fast path keeps the draft token
-      if (p.fallback == HOLA_FALLBACK_GREEDY) {          // the verifier's own token, or the run ends here
-        if (x != sh_amax[j]) { n = j; break; }
-        continue;
+    bool stop = false, bad = false;
+    if (gatherer) {
+      const int j = gthread, x = x_mine;
+      if (x < 0 || x >= Vtok) {
+        stop = true; bad = true;
+      } else {
+        const float gate_value = p.gate_source == HOLA_GATE_DRAFT_ENTROPY ? hq_mine : sh_H[j];
+        if (!(gate_value < p.tau)) {                     // entropy gate off: the verifier decides
+          if (p.fallback == HOLA_FALLBACK_GREEDY) {
+            stop = x != sh_amax[j];
+          } else {
+            const float u = clamp_uniform(u_mine, flags);
+            const float px = expf(lx_mine - sh_logZ[j]);
+            const float qx = qx_mine;
+            stop = !((qx > 0.f) ? (u * qx < px) : (px > 0.f));
+          }
+        }
       }
-      const float u = clamp_uniform(sh_u[j], flags);
-      const float px = expf(sh_lx[j] - sh_logZ[j]);
-      const float qx = sh_qx[j];
-      const bool accept = (qx > 0.f) ? (u * qx < px) : (px > 0.f);
-      if (!accept) { n = j; break; }
     }
+    // positions j = gthread live in the last two warps: first stop per warp, then the earlier of the two
+    const unsigned stops = __ballot_sync(0xffffffffu, stop);
+    const int first = stops ? __ffs(stops) - 1 : 32;     // lane of the first stop in this warp
+    // flags count only for positions that were evaluated: those up to and including the first stop
+    unsigned fl = (lane <= first) ? flags : 0u;
+    if (bad && lane == first) fl |= HOLA_FLAG_BAD_TOKEN;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) fl |= __shfl_xor_sync(0xffffffffu, fl, off);
+    if (warp >= kK3Warps - 2 && lane == 0) {
+      sh_stop[warp - (kK3Warps - 2)] = first;
+      sh_wflags[warp - (kK3Warps - 2)] = fl;
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int n = k;
+    unsigned flags = 0;
+    if (sh_stop[0] < 32) { n = sh_stop[0]; flags = sh_wflags[0]; }
+    else {
+      flags = sh_wflags[0];
+      if (sh_stop[1] < 32) n = 32 + sh_stop[1];
+      flags |= sh_wflags[1];
+    }
+    if (n > k) n = k;
     sh_n = n;
     sh_flags = flags;
     if (rank == 0) {
@@ -1254,16 +1355,21 @@ __global__ void __launch_bounds__(kK3Threads) accept_sample_kernel(const K3Param
         const int c = c0 + i * kK3Warps;
         if (c < mine) fetch4<kVec>(lrow, qrow, p.q_dtype, residual, (c_first + c) * kChunk + lane * 4, V, l[i], q[i]);
       }
+      double part[kK3Unroll];
 #pragma unroll
       for (int i = 0; i < kK3Unroll; ++i) {
         const int c = c0 + i * kK3Warps;
+        part[i] = 0.0;
         if (c < mine) {
           float r[4];
           resid4(l[i], q[i], logZ, r);
-          const double sum = warp_sum_f64(((static_cast<double>(r[0]) + r[1]) + r[2]) + r[3]);
-          if (lane == 0) csum[c] = sum;
+          part[i] = ((static_cast<double>(r[0]) + r[1]) + r[2]) + r[3];
         }
       }
+      // the four chunk sums of this step: lanes 0, 8, 16, 24 end up with chunks 0, 1, 2, 3
+      const double sum = warp_sum4_f64(part, lane);
+      const int c = c0 + (lane >> 3) * kK3Warps;
+      if ((lane & 7) == 0 && c < mine) csum[c] = sum;
     }
     __syncthreads();
     // warp 0: scan of the slice; lane L owns chunks [lo, hi)
@@ -1472,59 +1578,74 @@ __device__ __forceinline__ float qlnq8(const uint4 raw) {     // sum over eight 
   return part;
 }
 __device__ __forceinline__ float qlnq4(const float4 x) { return (qlnq(x.x) + qlnq(x.y)) + (qlnq(x.z) + qlnq(x.w)); }
+__device__ __forceinline__ float qlnq_vec(const uint4 raw) { return qlnq8(raw); }
+__device__ __forceinline__ float qlnq_vec(const float4 x) { return qlnq4(x); }
 
-// Grid (rows, kHqSlices): CTA (r, s) sums slice s of row r and leaves the partial sum in part[r][s]; the
-// accept/sample kernel adds the slices in index order.
-__global__ void __launch_bounds__(256) draft_entropy_kernel(const void* q, int q_dtype, int V, double* part) {
-  __shared__ double sh_part[8];
-  const size_t row = blockIdx.x;
-  const int slice = blockIdx.y;
+// Work items are (row, slice) pairs, kHqSlices slices per draft row; a CTA takes items blockIdx.x, blockIdx.x + grid, ...
+// and leaves each item's partial sum in part[row][slice]; the accept/sample kernel adds the slices in index order.
+// The grid is sized to the machine (a few CTAs per SM) and every thread keeps eight 16-byte loads in flight, so the
+// pass runs at the rate the memory system delivers the rows instead of at the rate CTAs can be launched.
+template <typename Vec, int kPerVec>
+__device__ __forceinline__ double draft_entropy_slice(const void* rowp, int V, int slice, bool scalar_tail) {
+  constexpr int kInFlight = 8;                           // independent 16-byte loads per thread and step
+  const bool vec = (reinterpret_cast<uintptr_t>(rowp) & 15u) == 0;
+  const int nvec = vec ? V / kPerVec : 0;
+  const Vec* q16 = static_cast<const Vec*>(rowp);
+  const int per = (nvec + kHqSlices - 1) / kHqSlices, end = min(nvec, (slice + 1) * per);
   double acc = 0.0;
-  constexpr int kInFlight = 4;                           // independent 16-byte loads per thread and step
-  if (q_dtype == HOLA_Q_BF16) {
-    const __nv_bfloat16* qr = static_cast<const __nv_bfloat16*>(q) + row * V;
-    const bool vec = (reinterpret_cast<uintptr_t>(qr) & 15u) == 0;
-    const int nvec = vec ? V / 8 : 0;
-    const uint4* q16 = reinterpret_cast<const uint4*>(qr);
-    const int per = (nvec + kHqSlices - 1) / kHqSlices, end = min(nvec, (slice + 1) * per);
-    int i = slice * per + threadIdx.x;
-    for (; i + (kInFlight - 1) * 256 < end; i += kInFlight * 256) {
-      uint4 raw[kInFlight];
+  int i = slice * per + threadIdx.x;
+  for (; i + (kInFlight - 1) * 256 < end; i += kInFlight * 256) {
+    Vec raw[kInFlight];
 #pragma unroll
-      for (int u = 0; u < kInFlight; ++u) raw[u] = q16[i + u * 256];
+    for (int u = 0; u < kInFlight; ++u) raw[u] = __ldcs(q16 + i + u * 256);
+    float part = 0.f;
 #pragma unroll
-      for (int u = 0; u < kInFlight; ++u) acc += qlnq8(raw[u]);
-    }
-    for (; i < end; i += 256) acc += qlnq8(q16[i]);
-    for (int v = nvec * 8 + threadIdx.x; slice == 0 && v < V; v += 256) {    // scalar tail (or whole row): slice 0
-      acc += qlnq(__bfloat162float(qr[v]));
-    }
-  } else {
-    const float* qr = static_cast<const float*>(q) + row * V;
-    const bool vec = (reinterpret_cast<uintptr_t>(qr) & 15u) == 0;
-    const int nvec = vec ? V / 4 : 0;
-    const float4* q16 = reinterpret_cast<const float4*>(qr);
-    const int per = (nvec + kHqSlices - 1) / kHqSlices, end = min(nvec, (slice + 1) * per);
-    int i = slice * per + threadIdx.x;
-    for (; i + (kInFlight - 1) * 256 < end; i += kInFlight * 256) {
-      float4 raw[kInFlight];
+    for (int u = 0; u < kInFlight; ++u) part += qlnq_vec(raw[u]);
+    acc += part;
+  }
+  {
+    Vec raw[kInFlight];
 #pragma unroll
-      for (int u = 0; u < kInFlight; ++u) raw[u] = q16[i + u * 256];
+    for (int u = 0; u < kInFlight; ++u)
+      if (i + u * 256 < end) raw[u] = __ldcs(q16 + i + u * 256);
+    float part = 0.f;
 #pragma unroll
-      for (int u = 0; u < kInFlight; ++u) acc += qlnq4(raw[u]);
-    }
-    for (; i < end; i += 256) acc += qlnq4(q16[i]);
-    for (int v = nvec * 4 + threadIdx.x; slice == 0 && v < V; v += 256) {
-      acc += qlnq(qr[v]);
+    for (int u = 0; u < kInFlight; ++u)
+      if (i + u * 256 < end) part += qlnq_vec(raw[u]);
+    acc += part;
+  }
+  if (scalar_tail) {                                     // what the 16-byte loads do not cover (or the whole row)
+    if (kPerVec == 8) {
+      const __nv_bfloat16* qr = static_cast<const __nv_bfloat16*>(rowp);
+      for (int v = nvec * kPerVec + threadIdx.x; v < V; v += 256) acc += qlnq(__bfloat162float(qr[v]));
+    } else {
+      const float* qr = static_cast<const float*>(rowp);
+      for (int v = nvec * kPerVec + threadIdx.x; v < V; v += 256) acc += qlnq(qr[v]);
     }
   }
-  acc = warp_sum_f64(acc);
-  if ((threadIdx.x & 31) == 0) sh_part[threadIdx.x >> 5] = acc;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    double tot = 0.0;
-    for (int i = 0; i < 8; ++i) tot += sh_part[i];
-    part[row * kHqSlices + slice] = tot;
+  return acc;
+}
+
+__global__ void __launch_bounds__(256) draft_entropy_kernel(const void* q, int q_dtype, int V, int rows, double* part) {
+  __shared__ double sh_part[8];
+  const int items = rows * kHqSlices;
+  for (int it = blockIdx.x; it < items; it += gridDim.x) {
+    const size_t row = static_cast<size_t>(it / kHqSlices);
+    const int slice = it % kHqSlices;
+    double acc;
+    if (q_dtype == HOLA_Q_BF16)
+      acc = draft_entropy_slice<uint4, 8>(static_cast<const __nv_bfloat16*>(q) + row * V, V, slice, slice == 0);
+    else
+      acc = draft_entropy_slice<float4, 4>(static_cast<const float*>(q) + row * V, V, slice, slice == 0);
+    acc = warp_sum_f64(acc);
+    if ((threadIdx.x & 31) == 0) sh_part[threadIdx.x >> 5] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      double tot = 0.0;
+      for (int i = 0; i < 8; ++i) tot += sh_part[i];
+      part[row * kHqSlices + slice] = tot;
+    }
+    __syncthreads();
   }
 }
 
@@ -1540,9 +1661,18 @@ struct Plan {
 
 }  // namespace
 
+// What a call needs besides its arguments, kept from one call to the next: the launch geometry of a (rows, weight
+// mode) pair and the two tensor maps of a (hidden pointer, W_lm pointer, rows, weight mode) quadruple.
+struct PlanEntry { int valid, M, w_dtype; Plan pl; };
+struct MapEntry { int valid, M, w_dtype; const void* hidden; const void* W; CUtensorMap th, tw; };
+constexpr int kPlanCache = 8, kMapCache = 8;
+
 struct hola_ctx {
   int device, num_sms, maxB, maxK, H, V, ldl, max_rows;
   EncodeTiledFn encode;
+  PlanEntry plans[kPlanCache];
+  MapEntry maps[kMapCache];
+  int plan_next, map_next;
   char* ws;                 // one device allocation, carved below
   size_t ws_bytes;
   float* logits;            // [max_rows][ldl]
@@ -1693,6 +1823,18 @@ Plan make_plan(const hola_ctx* ctx, int M, int w_dtype = HOLA_W_BF16) {
   return best;
 }
 
+// make_plan through the context's cache (the geometry depends on the context's shape and tuning options, on the number
+// of verify rows and on the weight mode only).
+const Plan& plan_for(hola_ctx* ctx, int M, int w_dtype) {
+  for (int i = 0; i < kPlanCache; ++i)
+    if (ctx->plans[i].valid && ctx->plans[i].M == M && ctx->plans[i].w_dtype == w_dtype) return ctx->plans[i].pl;
+  PlanEntry& e = ctx->plans[ctx->plan_next];
+  ctx->plan_next = (ctx->plan_next + 1) % kPlanCache;
+  e.pl = make_plan(ctx, M, w_dtype);
+  e.M = M; e.w_dtype = w_dtype; e.valid = 1;
+  return e.pl;
+}
+
 // K-major 2-D tensor map with a box of 64 elements x box_rows.  bf16: 128-byte swizzle (the layout the MMA reads);
 // int8: plain rows of 64 bytes (the converter warps read them).
 // int8 with swizzle (8-bit MMA): box of 128 elements = 128 bytes, 128-byte swizzle, the same bytes as a bf16 block.
@@ -1731,45 +1873,52 @@ hola_status run_lm_head(hola_ctx* ctx, const hola_verify_args* a, float* logits,
                         cudaStream_t stream) {
   const int M = a->B * (a->k + 1);
   const bool w8 = a->w_dtype == HOLA_W_INT8, two = a->w_dtype == HOLA_W8A16, i8 = a->w_dtype == HOLA_W8A8 || two;
-  CUtensorMap th, tw;
   hola_status s;
-  if (two) {
-    // 16-bit-class activations: two 8-bit planes per hidden row, blocks of 32 rows, into the context's workspace
-    if (!ctx->hid8) return HOLA_ERR_INVALID_ARG;
+  // 8-bit activations: the hidden operand is the context's own buffer of 8-bit planes, filled per call below
+  const void* hid_src = (two || i8) ? static_cast<const void*>(ctx->hid8) : a->hidden;
+  if ((two || i8) && !ctx->hid8) return HOLA_ERR_INVALID_ARG;   // (the entry point without a context has no room for it)
+  if (two || i8) {
+    // the same per-row quantiser as for W_lm (one plane), or the two-plane form in blocks of 32 rows
     const int padded = round_up(M, 32);
     cudaLaunchConfig_t qc = {};
-    qc.gridDim = dim3(static_cast<unsigned>(padded)); qc.blockDim = dim3(256); qc.stream = stream;
+    qc.gridDim = dim3(static_cast<unsigned>(two ? padded : M)); qc.blockDim = dim3(256); qc.stream = stream;
     cudaLaunchAttribute qa[1];
     qa[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // launch latency hides behind the call before
     qa[0].val.programmaticStreamSerializationAllowed = 1;
     qc.attrs = qa; qc.numAttrs = 1;
-    if (cudaLaunchKernelEx(&qc, quantize_rows_two_plane_kernel, static_cast<const __nv_bfloat16*>(a->hidden), M, a->H,
-                           ctx->hid8, ctx->hid_scale, ctx->hid_scale + ctx->max_rows) != cudaSuccess)
-      return HOLA_ERR_CUDA;
-    s = encode_map(ctx, &th, ctx->hid8, static_cast<uint64_t>(2 * padded), static_cast<uint64_t>(a->H),
-                   static_cast<uint32_t>(pl.N / 2), true, true);
-  } else if (i8) {
-    // 8-bit activations: the same per-row quantiser as for W_lm, into the context's workspace
-    if (!ctx->hid8) return HOLA_ERR_INVALID_ARG;          // (the entry point without a context has no room for it)
-    cudaLaunchConfig_t qc = {};
-    qc.gridDim = dim3(static_cast<unsigned>(M)); qc.blockDim = dim3(256); qc.stream = stream;
-    cudaLaunchAttribute qa[1];
-    qa[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // launch latency hides behind the call before
-    qa[0].val.programmaticStreamSerializationAllowed = 1;
-    qc.attrs = qa; qc.numAttrs = 1;
-    if (cudaLaunchKernelEx(&qc, quantize_rows_int8_kernel, static_cast<const __nv_bfloat16*>(a->hidden), a->H, ctx->hid8,
-                           ctx->hid_scale) != cudaSuccess)
-      return HOLA_ERR_CUDA;
-    s = encode_map(ctx, &th, ctx->hid8, static_cast<uint64_t>(M), static_cast<uint64_t>(a->H),
-                   static_cast<uint32_t>(pl.N / 2), true, true);
-  } else {
-    s = encode_map(ctx, &th, a->hidden, static_cast<uint64_t>(M), static_cast<uint64_t>(a->H),
-                   static_cast<uint32_t>(pl.N / 2));
+    const cudaError_t qe =
+        two ? cudaLaunchKernelEx(&qc, quantize_rows_two_plane_kernel, static_cast<const __nv_bfloat16*>(a->hidden), M,
+                                 a->H, ctx->hid8, ctx->hid_scale, ctx->hid_scale + ctx->max_rows)
+            : cudaLaunchKernelEx(&qc, quantize_rows_int8_kernel, static_cast<const __nv_bfloat16*>(a->hidden), a->H,
+                                 ctx->hid8, ctx->hid_scale);
+    if (qe != cudaSuccess) { set_error(ctx, "launch of the hidden-row quantiser", qe); return HOLA_ERR_CUDA; }
   }
-  if (s != HOLA_OK) return s;
-  s = encode_map(ctx, &tw, a->W_lm, static_cast<uint64_t>(a->V), static_cast<uint64_t>(a->H),
-                 static_cast<uint32_t>(pl.tile_rows), w8 || i8, i8);
-  if (s != HOLA_OK) return s;
+  MapEntry* me = nullptr;
+  for (int i = 0; i < kMapCache; ++i) {
+    MapEntry& c = ctx->maps[i];
+    if (c.valid && c.hidden == hid_src && c.W == a->W_lm && c.M == M && c.w_dtype == a->w_dtype) { me = &c; break; }
+  }
+  if (!me) {
+    me = &ctx->maps[ctx->map_next];
+    ctx->map_next = (ctx->map_next + 1) % kMapCache;
+    me->valid = 0;
+    if (two)
+      s = encode_map(ctx, &me->th, hid_src, static_cast<uint64_t>(2 * round_up(M, 32)), static_cast<uint64_t>(a->H),
+                     static_cast<uint32_t>(pl.N / 2), true, true);
+    else if (i8)
+      s = encode_map(ctx, &me->th, hid_src, static_cast<uint64_t>(M), static_cast<uint64_t>(a->H),
+                     static_cast<uint32_t>(pl.N / 2), true, true);
+    else
+      s = encode_map(ctx, &me->th, hid_src, static_cast<uint64_t>(M), static_cast<uint64_t>(a->H),
+                     static_cast<uint32_t>(pl.N / 2));
+    if (s != HOLA_OK) return s;
+    s = encode_map(ctx, &me->tw, a->W_lm, static_cast<uint64_t>(a->V), static_cast<uint64_t>(a->H),
+                   static_cast<uint32_t>(pl.tile_rows), w8 || i8, i8);
+    if (s != HOLA_OK) return s;
+    me->hidden = hid_src; me->W = a->W_lm; me->M = M; me->w_dtype = a->w_dtype; me->valid = 1;
+  }
+  const CUtensorMap& th = me->th;
+  const CUtensorMap& tw = me->tw;
   K1Params kp;
   kp.M = M; kp.V = a->V; kp.n_ptiles = pl.n_ptiles; kp.n_kblocks = pl.n_kblocks;
   kp.stages = pl.stages; kp.nbuf = pl.nbuf; kp.rot = pl.rot; kp.n_sub = pl.n_sub; kp.N = pl.N; kp.tile_rows = pl.tile_rows; kp.ldl = ldl;
@@ -1779,15 +1928,7 @@ hola_status run_lm_head(hola_ctx* ctx, const hola_verify_args* a, float* logits,
   kp.h_scale = ctx->hid_scale;
   kp.h_scale2 = ctx->hid_scale ? ctx->hid_scale + ctx->max_rows : nullptr;
   kp.stream_logits = static_cast<double>(M) * a->V * 4.0 > 96e6 ? 1 : 0;     // beyond ~3/4 of the L2
-  cudaError_t e = two ? cudaFuncSetAttribute(lm_head_entropy_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             pl.smem_bytes)
-                : i8 ? cudaFuncSetAttribute(lm_head_entropy_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            pl.smem_bytes)
-                : w8 ? cudaFuncSetAttribute(lm_head_entropy_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            pl.smem_bytes)
-                     : cudaFuncSetAttribute(lm_head_entropy_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            pl.smem_bytes);
-  if (e != cudaSuccess) { set_error(ctx, "cudaFuncSetAttribute", e); return HOLA_ERR_CUDA; }
+  cudaError_t e = cudaSuccess;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(static_cast<unsigned>(pl.grid));
   cfg.blockDim = dim3(kK1Threads);
@@ -1806,6 +1947,7 @@ hola_status run_lm_head(hola_ctx* ctx, const hola_verify_args* a, float* logits,
   cfg.numAttrs = 2;
   for (int pass = 0; pass < pl.passes; ++pass) {
     kp.row0 = pass * pl.rows_per_pass;
+    kp.first_pass = pass == 0 ? 1 : 0;
     kp.rows = M - kp.row0 < pl.rows_per_pass ? M - kp.row0 : pl.rows_per_pass;
     if (kp.rows <= 0) break;
     e = two ? cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<3>, th, tw, kp)
@@ -1817,6 +1959,12 @@ hola_status run_lm_head(hola_ctx* ctx, const hola_verify_args* a, float* logits,
   return HOLA_OK;
 }
 
+// CTAs of the pass over the draft rows: one per (row, slice) item up to four per SM.
+unsigned draft_entropy_grid(const hola_ctx* ctx, int rows) {
+  const int items = rows * kHqSlices, cap = 4 * ctx->num_sms;
+  return static_cast<unsigned>(items < cap ? items : cap);
+}
+
 // What the accept/sample kernel needs to know in the vocabulary-parallel form.
 struct ShardLaunch {
   int world, rank, v_offset, V_global;
@@ -1826,11 +1974,12 @@ struct ShardLaunch {
   const double* mass_all;
 };
 
+// `settled`: the launch sits right behind this call's own GEMM kernel (see K3Params::inputs_settled).
 hola_status run_accept_sample(hola_ctx* ctx, const hola_verify_args* a, const float* logits, int ldl, int combine,
                               int nparts, cudaStream_t stream, const float* q_tok = nullptr, int phase = 0,
-                              const ShardLaunch* sh = nullptr) {
+                              const ShardLaunch* sh = nullptr, bool settled = false) {
   K3Params kp{};
-  kp.q_tok = q_tok; kp.phase = phase;
+  kp.q_tok = q_tok; kp.phase = phase; kp.inputs_settled = settled ? 1 : 0;
   kp.B = a->B; kp.k = a->k; kp.V = a->V; kp.ldl = ldl; kp.logits = logits;
   kp.partials = ctx->partials; kp.nparts = nparts; kp.part_stride = ctx->max_rows; kp.combine = combine;
   kp.tok = a->draft_tok; kp.q = a->draft_q; kp.q_dtype = a->q_dtype; kp.u = a->uniforms; kp.tau = a->tau;
@@ -1839,8 +1988,8 @@ hola_status run_accept_sample(hola_ctx* ctx, const hola_verify_args* a, const fl
     // one more pass over the draft rows: H(q_j) for every (sequence, draft position) - unless the caller has put it
     // on the side stream already, next to the GEMM
     if (!ctx->hq_ready) {
-      draft_entropy_kernel<<<dim3(static_cast<unsigned>(a->B * a->k), kHqSlices), 256, 0, stream>>>(
-          a->draft_q, a->q_dtype, a->V, ctx->hq);
+      draft_entropy_kernel<<<draft_entropy_grid(ctx, a->B * a->k), 256, 0, stream>>>(
+          a->draft_q, a->q_dtype, a->V, a->B * a->k, ctx->hq);
       const cudaError_t e0 = cudaGetLastError();
       if (e0 != cudaSuccess) { set_error(ctx, "launch draft_entropy_kernel", e0); return HOLA_ERR_CUDA; }
     }
@@ -1859,13 +2008,24 @@ hola_status run_accept_sample(hola_ctx* ctx, const hola_verify_args* a, const fl
   // cluster size: as many CTAs per sequence as keeps the grid within a few waves of the SMs
   const int nchunks = (a->V + kChunk - 1) / kChunk;
   int S = 8;
-  while (S > 1 && (a->B * S > 8 * ctx->num_sms || nchunks / S < 8)) S >>= 1;
+  while (S > 1 && (a->B * S > kK3MaxPerSm * ctx->num_sms || nchunks / S < 8)) S >>= 1;   // one wave of CTAs
   if (phase == 1) S = 1;                                 // no vocabulary pass: one CTA per sequence
   const int cpc = (nchunks + S - 1) / S;
+  // The grid may be scheduled while the GEMM kernel's CTAs are still leaving their SMs one by one.  Left alone, its
+  // small CTAs would pile up eight deep on the first SMs to come free; asking for as much shared memory as keeps
+  // ceil(grid / SMs) CTAs on an SM, and no more, spreads them over the machine whatever the order of arrival.
+  const int grid = a->B * S;
+  int per_sm = (grid + ctx->num_sms - 1) / ctx->num_sms;
+  per_sm = per_sm < 1 ? 1 : (per_sm > kK3MaxPerSm ? kK3MaxPerSm : per_sm);
+  size_t smem = static_cast<size_t>(cpc) * sizeof(double);
+  if (per_sm < kK3MaxPerSm) {
+    const size_t spread = kSmTotalSmem / per_sm - kK3SmemOverhead;
+    if (spread > smem) smem = spread;
+  }
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(static_cast<unsigned>(a->B * S));
+  cfg.gridDim = dim3(static_cast<unsigned>(grid));
   cfg.blockDim = dim3(kK3Threads);
-  cfg.dynamicSmemBytes = static_cast<size_t>(cpc) * sizeof(double);
+  cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -1902,6 +2062,24 @@ hola_status check_sample_args(const hola_verify_args* a) {
   if (!a->uniforms || !a->accept_len || !a->next_tok || !a->entropy || !a->logZ) return HOLA_ERR_INVALID_ARG;
   if (a->k > 0 && (!a->draft_tok || !a->draft_q)) return HOLA_ERR_INVALID_ARG;
   return HOLA_OK;
+}
+
+// Once per context (and once per device for the entry point without one), with the device current: the kernels that
+// ask for more dynamic shared memory than the default limit are told so here, not on every call.
+cudaError_t configure_kernels() {
+  cudaError_t e = cudaFuncSetAttribute(lm_head_entropy_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(lm_head_entropy_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(lm_head_entropy_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(lm_head_entropy_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+  const int k3_max = static_cast<int>(kSmTotalSmem - kK3SmemOverhead);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(accept_sample_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, k3_max);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(accept_sample_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, k3_max);
+  return e;
 }
 
 struct DeviceGuard {
@@ -1968,14 +2146,8 @@ hola_status hola_create(hola_ctx** out, int device, int maxB, int maxK, int H, i
   ctx->max_rows = maxB * (maxK + 1);
   ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
   ctx->host_overlap = 1;
-  if (const char* e = getenv("HOLA_HOST_OVERLAP")) ctx->host_overlap = atoi(e) != 0;   // tuning override
   ctx->host_lazy_q = -1;
-  if (const char* e = getenv("HOLA_HOST_LAZY_Q")) ctx->host_lazy_q = atoi(e) != 0;     // override for tests and sweeps
-  if (const char* e = getenv("HOLA_ROT")) ctx->no_rot = atoi(e) == 0;                  // tuning override for sweeps
-  if (const char* e = getenv("HOLA_STAGES")) {           // tuning override for sweeps: fewer ring slots
-    const int st = atoi(e);
-    if (st >= 2 && st <= kMaxStages) ctx->force_stages = st;
-  }
+  if (configure_kernels() != cudaSuccess) { free(ctx); return HOLA_ERR_CUDA; }
   const WsLayout w = ws_layout(maxB, maxK, H, V, ctx->num_sms);
   const cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&ctx->ws), w.total);
   if (e != cudaSuccess) { free(ctx); return HOLA_ERR_WORKSPACE; }
@@ -2045,6 +2217,45 @@ hola_status hola_plan(const hola_ctx* ctx, int B, int k, hola_plan_info* out) {
   return hola_plan_ex(ctx, B, k, HOLA_W_BF16, out);
 }
 
+hola_status hola_set_option(hola_ctx* ctx, int option, int value) {
+  if (!ctx) return HOLA_ERR_INVALID_ARG;
+  switch (option) {
+    case HOLA_OPT_RING_SLOTS:
+      if (value != 0 && (value < 2 || value > kMaxStages)) return HOLA_ERR_INVALID_ARG;
+      ctx->force_stages = value;
+      break;
+    case HOLA_OPT_ROTATING_UNITS: ctx->no_rot = value == 0; break;
+    case HOLA_OPT_HOST_OVERLAP: ctx->host_overlap = value != 0; break;
+    case HOLA_OPT_HOST_ROWS_ON_DEMAND:
+      if (value < -1 || value > 1) return HOLA_ERR_INVALID_ARG;
+      ctx->host_lazy_q = value;
+      break;
+    default: return HOLA_ERR_INVALID_ARG;
+  }
+  for (int i = 0; i < kPlanCache; ++i) ctx->plans[i].valid = 0;     // the launch geometry may have changed
+  for (int i = 0; i < kMapCache; ++i) ctx->maps[i].valid = 0;
+  return HOLA_OK;
+}
+
+hola_status hola_selftest_bounded_wait(hola_ctx* ctx, long long limit_cycles, uint32_t* status_word,
+                                       uint32_t* counters, void* cuda_stream) {
+  if (!ctx || !status_word || !counters) return HOLA_ERR_INVALID_ARG;
+  if (limit_cycles < 1000 || limit_cycles > 200000000ll) return HOLA_ERR_INVALID_ARG;   // at most ~0.1 s of SM clock
+  DeviceGuard guard(ctx->device);
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemsetAsync(counters, 0, 2 * sizeof(uint32_t), stream) != cudaSuccess) return HOLA_ERR_CUDA;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2); cfg.blockDim = dim3(64); cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, bounded_wait_selftest_kernel, limit_cycles,
+                                           static_cast<unsigned*>(status_word), static_cast<unsigned*>(counters));
+  if (e != cudaSuccess) { set_error(ctx, "launch bounded_wait_selftest_kernel", e); return HOLA_ERR_CUDA; }
+  return HOLA_OK;
+}
+
 hola_status hola_lm_head_entropy(hola_ctx* ctx, const hola_verify_args* a, void* cuda_stream) {
   hola_status s = check_common(ctx, a);
   if (s != HOLA_OK) return s;
@@ -2054,7 +2265,7 @@ hola_status hola_lm_head_entropy(hola_ctx* ctx, const hola_verify_args* a, void*
   DeviceGuard guard(ctx->device);
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   const int M = a->B * (a->k + 1);
-  const Plan pl = make_plan(ctx, M, a->w_dtype);
+  const Plan& pl = plan_for(ctx, M, a->w_dtype);
   float* logits = a->logits_out ? a->logits_out : ctx->logits;
   const int ldl = a->logits_out ? a->V : ctx->ldl;
   if ((s = run_lm_head(ctx, a, logits, ldl, pl, stream)) != HOLA_OK) return s;
@@ -2082,7 +2293,7 @@ namespace {
 // The whole step on device buffers.  `before_sample`, when given, is an event the accept/sample part waits for
 // (the draft tensor still being copied in by hola_verify_host).
 hola_status verify_device(hola_ctx* ctx, const hola_verify_args* a, cudaStream_t stream, cudaEvent_t before_sample) {
-  const Plan pl = make_plan(ctx, a->B * (a->k + 1), a->w_dtype);
+  const Plan& pl = plan_for(ctx, a->B * (a->k + 1), a->w_dtype);
   float* logits = a->logits_out ? a->logits_out : ctx->logits;
   const int ldl = a->logits_out ? a->V : ctx->ldl;
   const bool prof = ctx->prof_on && ctx->prof_n < ctx->prof_cap;
@@ -2105,8 +2316,8 @@ hola_status verify_device(hola_ctx* ctx, const hola_verify_args* a, cudaStream_t
     cudaError_t e = cudaSuccess;
     if (!before_sample) e = cudaStreamWaitEvent(ctx->copy_stream, ctx->fork_point, 0);
     if (e == cudaSuccess) {
-      draft_entropy_kernel<<<dim3(static_cast<unsigned>(a->B * a->k), kHqSlices), 256, 0, ctx->copy_stream>>>(
-          a->draft_q, a->q_dtype, a->V, ctx->hq);
+      draft_entropy_kernel<<<draft_entropy_grid(ctx, a->B * a->k), 256, 0, ctx->copy_stream>>>(
+          a->draft_q, a->q_dtype, a->V, a->B * a->k, ctx->hq);
       e = cudaGetLastError();
     }
     if (e == cudaSuccess) e = cudaEventRecord(ctx->copy_done, ctx->copy_stream);
@@ -2115,7 +2326,8 @@ hola_status verify_device(hola_ctx* ctx, const hola_verify_args* a, cudaStream_t
   }
   if (before_sample && cudaStreamWaitEvent(stream, before_sample, 0) != cudaSuccess) return HOLA_ERR_CUDA;
   ctx->hq_ready = side ? 1 : 0;
-  s = run_accept_sample(ctx, a, logits, ldl, 1, pl.grid, stream);
+  // (an event wait between the two kernels makes the second an ordinary launch; its inputs are settled either way)
+  s = run_accept_sample(ctx, a, logits, ldl, 1, pl.grid, stream, nullptr, 0, nullptr, true);
   ctx->hq_ready = 0;
   if (prof) { cudaEventRecord(ev[2], stream); ctx->prof_n++; }
   return s;
@@ -2130,8 +2342,8 @@ hola_status verify_device(hola_ctx* ctx, const hola_verify_args* a, cudaStream_t
 constexpr double kHostBusBytesPerSecond = 50e9;          // what a pinned host-to-device copy reaches here
 
 // Draft rows per sequence that can cross the bus while the GEMM of this call runs.
-int rows_under_gemm(const hola_ctx* ctx, const hola_verify_args* a) {
-  const Plan pl = make_plan(ctx, a->B * (a->k + 1), a->w_dtype);
+int rows_under_gemm(hola_ctx* ctx, const hola_verify_args* a) {
+  const Plan& pl = plan_for(ctx, a->B * (a->k + 1), a->w_dtype);
   const double group = static_cast<double>(a->B) * a->V * (a->q_dtype == HOLA_Q_BF16 ? 2 : 4);
   const double n = pl.est_seconds * kHostBusBytesPerSecond / group;
   return n > 1e6 ? 1000000 : static_cast<int>(n);
@@ -2201,7 +2413,7 @@ hola_status verify_host_lazy(hola_ctx* ctx, const hola_verify_args* a, cudaStrea
   d.logits_out = nullptr; d.status_word = reinterpret_cast<uint32_t*>(ctx->st_out); d.draft_entropy = nullptr;
   hola_status s = check_lm_head_args(ctx, &d);
   if (s != HOLA_OK) return s;
-  const Plan pl = make_plan(ctx, B * (k + 1), a->w_dtype);
+  const Plan& pl = plan_for(ctx, B * (k + 1), a->w_dtype);
   if ((s = run_lm_head(ctx, &d, ctx->logits, ctx->ldl, pl, stream)) != HOLA_OK) return s;
   if (!sample) {
     if ((s = run_accept_sample(ctx, &d, ctx->logits, ctx->ldl, 1, pl.grid, stream, ctx->st_qtok, 0)) != HOLA_OK) return s;
@@ -2390,7 +2602,7 @@ hola_status hola_shard_lm_head(hola_ctx* ctx, const hola_verify_args* a, const h
   DeviceGuard guard(ctx->device);
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   const int M = a->B * (a->k + 1);
-  const Plan pl = make_plan(ctx, M, a->w_dtype);
+  const Plan& pl = plan_for(ctx, M, a->w_dtype);
   float* logits = a->logits_out ? a->logits_out : ctx->logits;
   const int ldl = a->logits_out ? a->V : ctx->ldl;
   if ((s = run_lm_head(ctx, a, logits, ldl, pl, stream)) != HOLA_OK) return s;
@@ -2487,6 +2699,7 @@ hola_status static_setup(int dev, hola_ctx* out) {
     void* base = nullptr;
     const cudaError_t e = cudaGetSymbolAddress(&base, g_static_scratch);
     if (e != cudaSuccess || !base) return HOLA_ERR_CUDA;
+    if (configure_kernels() != cudaSuccess) return HOLA_ERR_CUDA;
     memset(c, 0, sizeof *c);
     c->device = dev;
     c->num_sms = prop.multiProcessorCount;
@@ -2518,10 +2731,11 @@ extern "C" hola_status hola_lm_head_entropy_static(const hola_verify_args* a, vo
   if (s != HOLA_OK) return s;
   local.H = a->H; local.V = a->V; local.maxB = a->B; local.maxK = a->k;
   const int M = static_cast<int>(rows);
-  if (a->w_dtype != HOLA_W_BF16 && a->w_dtype != HOLA_W_INT8) return HOLA_ERR_INVALID_ARG;
-  if (a->w_dtype == HOLA_W_INT8 && (!a->w_scale || a->H % 16 != 0)) return HOLA_ERR_INVALID_ARG;
+  if (a->w_dtype != HOLA_W_BF16) return HOLA_ERR_INVALID_ARG;   // the 8-bit weight modes need a context's workspace
   const Plan pl = make_plan(&local, M, a->w_dtype);
   if (pl.grid > kStaticMaxCtas) return HOLA_ERR_STATIC_LIMIT;
+  // a timed-out wait must be visible to the caller: the kernels report to the caller's status word when there is one
+  // (run_lm_head picks it), else to the word inside the array, which nobody outside can read
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   // The array keeps whatever the last call left.  The statistics slots are fully overwritten for the rows of this
   // call before they are read; the internal status word is the one thing that must start at zero.

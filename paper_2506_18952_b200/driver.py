@@ -1,4 +1,4 @@
-"""Multi-round HSD decode loop around hola_verify (Algorithm 1, lines 1-10, run as a loop).
+"""Multi-round HSD decode loop around hola_verify (the HSD part of Algorithm 1, run as a loop).
 
 Each round: the draft model proposes k tokens with their distributions q, the verifier's hidden states for the
 k+1 positions are formed, ONE hola_verify call decides how many drafts survive (entropy gate, Eq. 1, then the

@@ -57,6 +57,18 @@ class TorchDistExchange:
         return t
 
 
+class LocalExchange:
+    """The exchange of a group of one: every collective is the identity."""
+
+    world, rank = 1, 0
+
+    def all_gather(self, t: torch.Tensor) -> torch.Tensor:
+        return t.contiguous().unsqueeze(0)
+
+    def all_reduce_max_(self, t: torch.Tensor) -> torch.Tensor:
+        return t
+
+
 class ShardedHolaVerify:
     """One rank of the vocabulary-parallel verify step."""
 

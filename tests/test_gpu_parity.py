@@ -49,9 +49,10 @@ def check_against_oracle(binding, w, seqs=None, want_logits=True, tau=None, out=
     orc = compare.run_oracle(sub, keep_logits=True, gate_source=gate_source, fallback=fallback)
     if gate_source == 1 and w.k > 0:
         assert np.max(np.abs(_np(out.draft_entropy)[idx] - orc.draft_entropy)) <= compare.ENTROPY_ATOL
-    rep = compare.compare(orc, _np(sub.draft_q), _np(sub.uniforms), _np(out.accept_len)[idx], _np(out.next_tok)[idx],
-                          _np(out.entropy)[idx], _np(out.logZ)[idx],
-                          _np(out.logits)[idx] if out.logits is not None else None)
+    pick = torch.as_tensor(idx, device=out.accept_len.device)
+    rep = compare.compare(orc, _np(sub.draft_q), _np(sub.uniforms), _np(out.accept_len[pick]), _np(out.next_tok[pick]),
+                          _np(out.entropy[pick]), _np(out.logZ[pick]),
+                          _np(out.logits[pick]) if out.logits is not None else None)
     print(w.name, "tau", tau, rep.summary())
     assert rep.ok, rep.summary() + f" accept_fail={rep.accept_failures[:5]} token_fail={rep.token_failures[:5]}"
     # margin cases are reported, and must stay rare
@@ -414,14 +415,14 @@ def test_host_entry_equals_device_entry(binding):
 @pytest.mark.parametrize("q_dtype", [torch.bfloat16, torch.float32])
 @pytest.mark.parametrize("gate,fallback", [(0, 0), (0, 1), (1, 0)])
 @pytest.mark.parametrize("tau", [0.0, None, 100.0])
-def test_host_entry_sends_only_the_rows_it_reads(binding, monkeypatch, q_dtype, gate, fallback, tau):
+def test_host_entry_sends_only_the_rows_it_reads(binding, q_dtype, gate, fallback, tau):
     """hola_verify_host against hola_verify on the same data, over accept lengths from 0 to k (tau = 0: gate off;
     None: the median entropy; 100: every draft kept), with poisoned staging so that a row that was needed but not copied would show."""
     w = workloads.gaussian_head("host_rows", 21, 4, 128, 5000, seed=77, device=DEV, w_std=0.3, tau=tau,
                                 q_dtype=q_dtype)
     pin = lambda t: t.cpu().pin_memory()
-    monkeypatch.setenv("HOLA_HOST_LAZY_Q", "1")          # this small tensor would otherwise be copied whole
     with binding.HolaVerify(w.B, w.k, w.H, w.V) as ctx:
+        ctx.hola_set_option(binding.HOLA_OPT_HOST_ROWS_ON_DEMAND, 1)     # this small tensor would otherwise be copied whole
         # a first host call with a wrong draft tensor leaves stale rows in the staging area
         ctx.hola_verify_host(pin(w.hidden), w.W_lm, pin(w.draft_tok), pin(torch.flip(w.draft_q, dims=[2])),
                              pin(w.uniforms), w.tau, gate_source=gate, fallback=fallback)
@@ -704,6 +705,91 @@ def test_multi_round_decode_loop(binding, gate_source, fallback):
     assert res.verify_ms > 0 and res.total_ms >= res.verify_ms
 
 
+# ------------------------------------------------------------------------------------------ failure path, options
+def test_a_wait_that_runs_out_is_reported_and_leaves_the_device_usable(binding):
+    """The bounded waits, exercised for real but in miniature: a barrier that nothing signals, a limit of 1e5 cycles.
+    The wait must give up, raise the time-out flag, make the whole CTA pair leave through the common tail (tensor
+    memory released), and an ordinary verify call right behind it must be unaffected."""
+    w = workloads.gaussian_head("after-timeout", 6, 3, 128, 3000, seed=5, device=DEV, w_std=0.3)
+    with binding.HolaVerify(w.B, w.k, w.H, w.V) as ctx:
+        want = ctx.hola_verify(w.hidden, w.W_lm, w.draft_tok, w.draft_q, w.uniforms, w.tau)
+        torch.cuda.synchronize()
+        for limit in (20000, 100000):
+            status, reached, gave_up = ctx.hola_selftest_bounded_wait(limit)
+            assert status & binding.FLAG_TIMEOUT and status & ~binding.FLAG_TIMEOUT == 0
+            assert reached == 128 and gave_up == 4
+        got = ctx.hola_verify(w.hidden, w.W_lm, w.draft_tok, w.draft_q, w.uniforms, w.tau)
+        torch.cuda.synchronize()
+        assert int(got.status.item()) == 0
+        for f in ("accept_len", "next_tok", "entropy", "logZ"):
+            assert torch.equal(getattr(got, f), getattr(want, f))
+        with pytest.raises(binding.HolaError):
+            ctx.hola_selftest_bounded_wait(10)                       # below the accepted range: nothing launched
+        with pytest.raises(binding.HolaError):
+            ctx.hola_selftest_bounded_wait(10 ** 12)
+    check_against_oracle(binding, w, out=got, want_logits=False)
+
+
+def test_inputs_written_by_the_kernel_just_before_the_call_are_seen(binding):
+    """Tokens, uniforms and draft probabilities produced on the same stream right before the call (no synchronisation in
+    between) must be the ones the step uses: the accept/sample kernel may be scheduled early, but reads its inputs only
+    once the work in front of it is known to be complete."""
+    w = workloads.gaussian_head("fresh-inputs", 40, 5, 128, 6000, seed=31, device=DEV, w_std=0.3, sigma=1.0)
+    orc = compare.run_oracle(w, keep_logits=True)
+    lg = torch.from_numpy(orc.logits).float().to(DEV)
+    ent = torch.from_numpy(orc.entropy).float().to(DEV)
+    lz = torch.from_numpy(orc.logZ).float().to(DEV)
+    with binding.HolaVerify(w.B, w.k, w.H, w.V) as ctx:
+        for _ in range(5):
+            tok = torch.full_like(w.draft_tok, -1)                   # stale values a too-early read would pick up
+            u = torch.full_like(w.uniforms, 2.0)
+            q = torch.zeros_like(w.draft_q)
+            big = torch.empty(64 << 20, dtype=torch.uint8, device=DEV)
+            torch.cuda.synchronize()
+            big.zero_()                                              # keeps the stream busy while the copies queue up
+            tok.copy_(w.draft_tok); u.copy_(w.uniforms); q.copy_(w.draft_q)
+            a = ctx.hola_accept_sample(lg, ent, lz, tok, q, u, w.tau)
+            b = ctx.hola_verify(w.hidden, w.W_lm, tok, q, u, w.tau)
+            torch.cuda.synchronize()
+            for out in (a, b):
+                assert int(out.status.item()) == 0
+                rep = compare.compare(orc, _np(w.draft_q), _np(w.uniforms), _np(out.accept_len), _np(out.next_tok),
+                                      _np(out.entropy), _np(out.logZ))
+                assert rep.ok and rep.accept_margin_cases + rep.token_margin_cases <= 2, rep.summary()
+
+
+def test_options_change_speed_knobs_not_results(binding):
+    w = workloads.gaussian_head("options", 50, 5, 256, 9000, seed=17, device=DEV, w_std=0.3)     # 300 rows: rotating units
+    with binding.HolaVerify(w.B, w.k, w.H, w.V) as ctx:
+        base = ctx.hola_verify(w.hidden, w.W_lm, w.draft_tok, w.draft_q, w.uniforms, w.tau)
+        plan0 = ctx.hola_plan(w.B, w.k)
+        torch.cuda.synchronize()
+        for opt, val in ((binding.HOLA_OPT_RING_SLOTS, 3), (binding.HOLA_OPT_ROTATING_UNITS, 0)):
+            ctx.hola_set_option(opt, val)
+            out = ctx.hola_verify(w.hidden, w.W_lm, w.draft_tok, w.draft_q, w.uniforms, w.tau)
+            torch.cuda.synchronize()
+            assert torch.equal(out.accept_len, base.accept_len) and torch.equal(out.next_tok, base.next_tok)
+            assert torch.allclose(out.entropy, base.entropy, atol=1e-5) and torch.allclose(out.logZ, base.logZ, atol=1e-5)
+        assert ctx.hola_plan(w.B, w.k)["stages"] == 3 and plan0["stages"] > 3
+        with pytest.raises(binding.HolaError):
+            ctx.hola_set_option(99, 1)
+        with pytest.raises(binding.HolaError):
+            ctx.hola_set_option(binding.HOLA_OPT_RING_SLOTS, 1)
+
+
+def test_repeated_calls_reuse_the_set_up_and_new_pointers_do_not(binding):
+    """Same pointers and sizes: the second call takes its tensor maps from the context.  Other tensors of the same shape,
+    or another batch size, must not be served from what the first call left."""
+    w1 = workloads.gaussian_head("cache-1", 12, 3, 128, 4000, seed=1, device=DEV, w_std=0.3)
+    w2 = workloads.gaussian_head("cache-2", 12, 3, 128, 4000, seed=2, device=DEV, w_std=0.3)
+    w3 = workloads.gaussian_head("cache-3", 7, 3, 128, 4000, seed=3, device=DEV, w_std=0.3)
+    with binding.HolaVerify(12, 3, 128, 4000) as ctx:
+        for w in (w1, w1, w2, w3, w1, w2):
+            out = ctx.hola_verify(w.hidden, w.W_lm, w.draft_tok, w.draft_q, w.uniforms, w.tau, want_logits=True)
+            torch.cuda.synchronize()
+            check_against_oracle(binding, w, out=out)
+
+
 # ------------------------------------------------------------------------------------------ the named workloads
 def test_edge_decode_config_full(binding):
     w = workloads.make_config("edge", DEV)
@@ -714,25 +800,53 @@ def test_edge_decode_config_full(binding):
 
 def test_batched_serving_config(binding):
     w = workloads.make_config("batched", DEV)
-    seqs = [0, 13, 31, 32, 47, 63]
-    out, orc, _ = check_against_oracle(binding, w, seqs=seqs)
+    out, orc, rep = check_against_oracle(binding, w)       # all 64 sequences, logits included
+    assert rep.n_seq == w.B
     check_ranges(w, out)
     acc = _np(out.accept_len)
     assert acc[:32].mean() > acc[32:].mean() + 1.0      # near-p half keeps more drafts than the far half
 
 
-@pytest.mark.parametrize("tau", [1.0, 2.0, 4.0])
-def test_large_vocab_config(binding, tau):
+def test_large_vocab_config(binding):
+    """All 64 sequences, all three thresholds of the sweep.  The fp64 logits do not depend on tau, so the oracle makes
+    them once and repeats only its steps 2-6 for each threshold."""
     w = workloads.make_config("large_vocab", DEV)
-    out, _, _ = check_against_oracle(binding, w, seqs=[1, 22, 40, 63], tau=tau)
-    check_ranges(w, out)
+    lg = ref.logits(_np(w.hidden).reshape(w.M, w.H), _np(w.W_lm)).reshape(w.B, w.k + 1, w.V)
+    with binding.HolaVerify(w.B, w.k, w.H, w.V) as ctx:
+        for tau in (1.0, 2.0, 4.0):
+            out = run_gpu(binding, w, want_logits=True, tau=tau, ctx=ctx)
+            assert int(out.status.item()) & binding.FLAG_TIMEOUT == 0
+            orc = ref.verify_from_logits(lg, _np(w.draft_tok), _np(w.draft_q), _np(w.uniforms), tau)
+            rep = compare.compare(orc, _np(w.draft_q), _np(w.uniforms), _np(out.accept_len), _np(out.next_tok),
+                                  _np(out.entropy), _np(out.logZ), _np(out.logits))
+            print("large_vocab tau", tau, rep.summary())
+            assert rep.ok and rep.n_seq == w.B, rep.summary() + f" {rep.accept_failures[:5]} {rep.token_failures[:5]}"
+            assert rep.accept_margin_cases <= 3 and rep.token_margin_cases <= 6
+            check_ranges(w, out)
+            gated = (_np(out.entropy)[:, :w.k] < tau).sum()
+            assert 0 < gated < w.B * w.k                    # the sweep exercises both branches of the gate
     H = _np(out.entropy)
     assert H.min() < 1.0 and H.max() > 6.0              # the entropy spread the workload asks for
 
 
+def wide_sample(B=256, k1=9, rows_per_pass=384, n=32):
+    """Sequences of the `wide` workload, evenly spread, such that every pass over W_lm and every 128-row accumulator
+    unit inside a pass holds rows of at least one of them, peaked and flat rows alike."""
+    seqs = sorted({round(i * (B - 1) / (n - 1)) for i in range(n)})
+    hit = {((b * k1 + j) // rows_per_pass, ((b * k1 + j) % rows_per_pass) // 128) for b in seqs for j in range(k1)}
+    passes = (B * k1 + rows_per_pass - 1) // rows_per_pass
+    assert hit == {(p, u) for p in range(passes) for u in range(3)}
+    return seqs
+
+
 def test_wide_head_config(binding):
     w = workloads.make_config("wide", DEV)
-    out, _, _ = check_against_oracle(binding, w, seqs=[0, 101, 255], want_logits=False)
+    with binding.HolaVerify(w.B, w.k, w.H, w.V) as ctx:
+        plan = ctx.hola_plan(w.B, w.k)
+    seqs = wide_sample(w.B, w.k + 1, plan["rows_per_pass"])
+    assert len(seqs) >= 32
+    out, _, rep = check_against_oracle(binding, w, seqs=seqs, want_logits=True)
+    assert rep.n_seq == len(seqs)
     check_ranges(w, out)
     H = _np(out.entropy).reshape(-1)
     assert (H[0::2] < 1.5).mean() > 0.9 and (H[1::2] > 10).mean() > 0.9     # peaked and flat rows

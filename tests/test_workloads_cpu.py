@@ -6,6 +6,7 @@ import sys
 import textwrap
 
 import numpy as np
+import pytest
 import torch
 
 from oracle import compare
@@ -81,3 +82,31 @@ def test_replica_plumbing_two_ranks_gloo(tmp_path):
 def test_single_process_defaults():
     assert hdist.env_world()[1] >= 1
     assert hdist.max_over_ranks(3.5) == 3.5 and hdist.sum_over_ranks(2.0) == 2.0
+
+
+def _bench(*argv, timeout=300):
+    """Runs bench.py as a user would, with no launcher variables in the environment; returns its JSON lines."""
+    import json
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")}
+    p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), *argv], env=env, capture_output=True, text=True,
+                       timeout=timeout)
+    assert p.returncode == 0, p.stderr[-2000:]
+    return [json.loads(l) for l in p.stdout.splitlines() if l.startswith("{")]
+
+
+@pytest.mark.parametrize("mode,scaling", [("replicas", "weak"), ("vocab", "strong")])
+def test_bench_starts_its_own_ranks(mode, scaling):
+    """`python bench.py --gpus 2` without a launcher starts two ranks itself; they meet on the loopback address, make the
+    collectives of the chosen parallelism (gloo, no GPU work) and rank 0 alone prints the one line, with n_gpus = 2."""
+    lines = _bench("--gpus", "2", "--dry-run", "--steps", "2", "--parallelism", mode)
+    assert len(lines) == 1
+    assert lines[0]["n_gpus"] == 2 and lines[0]["scaling"] == scaling and lines[0]["parallelism"] == mode
+
+
+def test_bench_reference_arm_runs_on_rank_zero_only():
+    lines = _bench("--gpus", "2", "--impl", "reference", "--workload", "tiny", "--steps", "2", "--warmup", "1")
+    assert len(lines) == 1
+    line = lines[0]
+    assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["value"] > 0
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["value"] == line["value"]
+    assert line["e2e"]["h2d_bytes_per_step"] == 0 and "1 of 1 sequences" in line["config"]["sample"]
