@@ -73,8 +73,6 @@ constexpr long long kWaitLimitCycles = 4000000000ll;   // about 2 s of SM clock 
 constexpr int kK3Threads = 256;
 constexpr int kK3Warps = kK3Threads / 32;
 constexpr int kK3MaxPerSm = 4;                   // CTAs of the accept/sample kernel an SM holds (register budget: 64 per thread)
-constexpr size_t kSmTotalSmem = 228 * 1024;      // shared memory of an SM
-constexpr size_t kK3SmemOverhead = 1024 + 2048 + 256;   // per CTA: the system's reserve, static arrays (rounded up), slack
 constexpr int kChunk = 128;                      // vocabulary entries per warp step (32 lanes x 4)
 constexpr int kMaxChunks = 4096;                 // => V <= 524288
 constexpr int kMaxK1 = 64;                       // k + 1 <= 64
@@ -86,8 +84,6 @@ constexpr float kLog2e = 1.4426950408889634f;
 
 struct K1Params {
   int M;          // total verify rows B(k+1)
-  int first_pass; // 1: the first launch of a call (its producers wait for the kernel before it in the stream);
-                  // later passes are only scheduled once every CTA of the pass before has passed that wait
   int row0;       // first row of this pass
   int rows;       // rows of this pass (<= n_sub * N)
   int V, n_ptiles, n_kblocks, stages, nbuf;
@@ -419,6 +415,75 @@ __device__ __forceinline__ void stats_fold16(const float* v, int n, int vocab0, 
   st.t = t;
 }
 
+// Two fp32 values in one 64-bit register, for the packed fp32 instructions of sm_100 (two results per issue slot).
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t r, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(r));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
+// stats_fold16<true> with half the issue slots: the maximum by three-input comparisons, the exponents' arguments, the
+// sum of the exponentials and the sum of e * l two at a time.  The centred sum of the sixteen entries,
+// sum e (l - m), is taken as  sum e l - m sum e : both terms are of size |m| * (sum e), so the rounding of the
+// difference is about 1e-7 |m| relative to s, far inside the tolerance on H = ln s - t / s.
+__device__ __forceinline__ void stats_fold16_packed(const float* v, int vocab0, Stats& st) {
+  const float c0 = max3(v[0], v[1], v[2]), c1 = max3(v[3], v[4], v[5]), c2 = max3(v[6], v[7], v[8]),
+              c3 = max3(v[9], v[10], v[11]), c4 = max3(v[12], v[13], v[14]);
+  const float cmax = fmaxf(max3(c0, c1, c2), max3(c3, c4, v[15]));
+  if (cmax > st.m) {
+    if (st.m != -CUDART_INF_F) {
+      const float d = st.m - cmax;
+      const float sc = ex2_approx(d * kLog2e);
+      st.t = sc * (st.t + d * st.s);
+      st.s *= sc;
+    }
+    st.m = cmax;
+    int first = 0;
+#pragma unroll
+    for (int i = 15; i > 0; --i)
+      if (v[i] == cmax) first = i;
+    if (v[0] == cmax) first = 0;
+    st.arg = vocab0 + first;
+  }
+  const float m = st.m;
+  const float mneg2 = -m * kLog2e;
+  const uint64_t l2e = pack2(kLog2e, kLog2e), mn = pack2(mneg2, mneg2);
+  uint64_t s2 = pack2(0.f, 0.f), a2 = pack2(0.f, 0.f);
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const uint64_t vp = pack2(v[2 * j], v[2 * j + 1]);
+    float x0, x1;
+    unpack2(fma2(vp, l2e, mn), x0, x1);
+    const uint64_t ep = pack2(ex2_approx(x0), ex2_approx(x1));
+    s2 = add2(s2, ep);
+    a2 = fma2(ep, vp, a2);
+  }
+  float sa, sb, aa, ab;
+  unpack2(s2, sa, sb);
+  unpack2(a2, aa, ab);
+  const float sc = sa + sb;
+  st.s += sc;
+  st.t += fmaf(-m, sc, aa + ab);
+}
+
 // Sixteen int8 values (one 16-byte piece c of row `row` of the raw block) -> sixteen bf16 values at their place in
 // the 128-byte-swizzled K-major tile that starts at `tile`: chunk 2c and 2c+1 of the row, each XOR-ed with row % 8.
 __device__ __forceinline__ void expand_int8x16(const uint4 x, uint8_t* tile, int row, int c) {
@@ -478,7 +543,9 @@ __device__ __forceinline__ float scaled(float acc, float w_scale, const float* h
 // its remainder, in alternating blocks of 32 rows): the epilogue adds the two int32 sums with their scales.
 // kMode: 0 bf16 x bf16; 1 int8 W_lm expanded to bf16 on chip (exact); 2 int8 W_lm x int8 hidden on the 8-bit MMA
 // kind (K blocks of 128 elements, so that a block is 128 bytes per row exactly as in mode 0; int32 accumulators).
-template <int kMode>
+// kRot: 257..384 rows per pass, three MMAs of N <= 128 per K step on rotating 128-column accumulator units (a
+// specialisation of its own because its epilogue holds a different set of values in registers).
+template <int kMode, bool kRot>
 __global__ void __launch_bounds__(kK1Threads, 1)
 lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __grid_constant__ CUtensorMap tmap_w,
                        const K1Params p) {
@@ -509,6 +576,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
                  tempty_bar = bar_base + 208, rawfull_bar = bar_base + 272, rawempty_bar = bar_base + 368;
   constexpr int kNumEpi = kW8 ? kW8EpiWarps : kEpiWarps;      // epilogue warps 2 .. 2 + kNumEpi - 1
   constexpr int kGroups = kNumEpi / 4;                        // warps per tensor-memory lane quarter
+  constexpr int kWarpTransBytes = kRot ? 2 * kTransBytes : kTransBytes;   // rotating units: a whole 32-row chunk at once
   float* trans_base = reinterpret_cast<float*>(smem + p.stages * stage_bytes + kBarrierBytes);
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + p.stages * stage_bytes + 256);
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + p.stages * stage_bytes + 260);
@@ -537,14 +605,6 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
   tc_fence_after();
   const uint32_t tmem_base = *tmem_holder;
 
-  // Programmatic dependent launch.  The kernel behind this one in the stream (the next pass over W_lm, or the
-  // accept/sample kernel) may be scheduled as soon as every CTA here has said so: its CTAs then start on the SMs this
-  // grid's CTAs leave, set themselves up under this grid's tail, and wait for this grid to complete before they touch
-  // what it writes.  One thread per CTA, the TMA producer, says so only after its own dependency wait (first pass):
-  // whatever runs behind this kernel therefore never starts before the kernel in front of the call has completed.
-  const bool producer = warp == 0 && elect_one();
-  if (!producer) grid_dependency_release();
-
   const int my_tiles = (p.n_ptiles - pair + npairs - 1) / npairs;
   const int sub_chunks = (p.N + 31) >> 5;                // 32-column chunks per MMA's accumulator
   // Accumulators.  rot == 0: MMA s of buffer b starts at column b * 256 + s * 256 (two buffers only when
@@ -555,7 +615,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (one per CTA)
-    if (producer) {
+    if (elect_one()) {
       const uint64_t pol_w = l2_policy_evict_first();    // W_lm is streamed once
       const uint64_t pol_h = l2_policy_evict_last();     // hidden is re-read for every tile
       const uint32_t leader_full = map_to_cta(full_bar, 0);
@@ -563,8 +623,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      if (p.first_pass) grid_dependency_wait();          // W_lm and the hidden rows may come from the kernel before
-      grid_dependency_release();
+      grid_dependency_wait();                            // W_lm and the hidden rows may come from the kernel before
       for (int t = 0; t < my_tiles && ok; ++t) {
         const int v0 = (pair + t * npairs) * pair_rows + static_cast<int>(rank) * p.tile_rows;
         int kx = 0;                                      // K coordinate of the block, in elements
@@ -599,7 +658,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      if (p.rot) {
+      if (kRot) {
         uint32_t used = 0;                               // bit u: parity of the number of tiles that used unit u
         for (int t = 0; t < my_tiles && ok; ++t) {
           for (int kb = 0; kb < p.n_kblocks && ok; ++kb) {
@@ -674,14 +733,15 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
     const int group = (warp - 2) >> 2;
     const uint32_t leader_tempty = map_to_cta(tempty_bar, 0);
     const int n_chunks = p.n_sub * sub_chunks;
-    const bool rot = p.rot != 0;
+    constexpr bool rot = kRot;
     const int my_chunks = rot ? (group < sub_chunks ? p.n_sub : 0)
                               : (group < n_chunks ? (n_chunks - 1 - group) / kGroups + 1 : 0);
-    float* tbuf = trans_base + (warp - 2) * (kTransBytes / 4);
+    float* tbuf = trans_base + (warp - 2) * (kWarpTransBytes / 4);
     const int trow = lane & 15, thalf = lane >> 4;       // row of a transposition step; which 16 of the 32 entries
-    Stats st[kEpiSlots][2];
+    constexpr int kSlots = kRot ? 3 : kEpiSlots;         // chunks per tile this warp keeps statistics for
+    Stats st[kSlots][2];
 #pragma unroll
-    for (int i = 0; i < kEpiSlots; ++i) { st[i][0] = stats_empty(); st[i][1] = stats_empty(); }
+    for (int i = 0; i < kSlots; ++i) { st[i][0] = stats_empty(); st[i][1] = stats_empty(); }
     bool ok = true;
     grid_dependency_wait();                              // the logits buffer may still be read by the kernel before
     for (int t = 0; t < my_tiles && ok; ++t) {
@@ -761,7 +821,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
                         tbuf + trow * 32 + (((thalf * 4 + jj) ^ (trow & 7)) << 2));
                     e[4 * jj] = x.x; e[4 * jj + 1] = x.y; e[4 * jj + 2] = x.z; e[4 * jj + 3] = x.w;
                   }
-                  if (n16 == 16) stats_fold16<true>(e, 16, vocab16, st[slot][half]);
+                  if (n16 == 16) stats_fold16_packed(e, vocab16, st[slot][half]);
                   else if (n16 > 0) stats_fold16<false>(e, n16, vocab16, st[slot][half]);
                 }
               }
@@ -781,8 +841,81 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
           }
         }
       }
+      if (kRot) {
+        // Rotating units.  The next tile's MMAs wait for this tile's first two units, so a unit is read and handed back
+        // as early as possible: a chunk goes from the registers to the logits buffer and, whole, into the warp's
+        // 4 KB staging buffer; the registers then take the next unit's chunk at once, and the statistics of the chunk
+        // before are folded from the staging buffer while that unit is already free.
+        if (my_chunks > 0) {
+          float v[32];
+          __syncwarp();
+          tmem_ld32(lane_addr + ((3 * t) & 3) * 128 + group * 32, v);
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(leader_tempty + 8 * ((3 * t) & 3));
 #pragma unroll
-      for (int slot = 0; slot < kEpiSlots; ++slot) {
+          for (int slot = 0; slot < 3; ++slot) {
+            const int c0 = group * 32;                   // first column of the chunk inside its MMA
+            const int r0 = p.row0 + slot * p.N + c0;     // verify row of column c0
+            const int n_ok = min(32, min(p.N - c0, p.M - r0));   // columns that are real rows
+            if (n_ok > 0) {
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                if (i < n_ok) v[i] = scaled<kMode>(v[i], w_scale, p.h_scale, r0 + i);
+              if (vocab_ok) {
+                float* dst = p.logits + static_cast<size_t>(r0) * p.ldl + vocab;
+                if (n_ok == 32 && p.stream_logits) {
+#pragma unroll
+                  for (int i = 0; i < 32; ++i) __stcs(dst + static_cast<size_t>(i) * p.ldl, v[i]);
+                } else if (n_ok == 32) {
+#pragma unroll
+                  for (int i = 0; i < 32; ++i) dst[static_cast<size_t>(i) * p.ldl] = v[i];
+                } else {
+#pragma unroll
+                  for (int i = 0; i < 32; ++i)
+                    if (i < n_ok) store_logit(dst + static_cast<size_t>(i) * p.ldl, v[i], p.stream_logits);
+                }
+              }
+            }
+            const bool fold = n_ok > 0 && nv > 0;
+            __syncwarp();                                // every lane has folded the chunk before out of the buffer
+            if (fold) {
+              // two blocks of 16 rows, each laid out as in the 16-row scheme: entry (row i, vocabulary lane l) at
+              // 16-byte group (l / 4) ^ (i % 8) of row i
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                tbuf[i * 32 + ((((lane >> 2) ^ (i & 7))) << 2) + (lane & 3)] = v[i];
+            }
+            __syncwarp();
+            if (slot < 2) {                              // the registers are free: take the next unit's chunk, free the unit
+              const int unit = (3 * t + slot + 1) & 3;
+              tmem_ld32(lane_addr + unit * 128 + group * 32, v);
+              tc_fence_before();
+              __syncwarp();
+              if (lane == 0) mbar_arrive_cluster(leader_tempty + 8 * unit);
+            }
+            if (fold) {
+#pragma unroll
+              for (int half = 0; half < 2; ++half) {
+                if (half * kTransRows < n_ok) {
+                  float e[16];
+#pragma unroll
+                  for (int jj = 0; jj < 4; ++jj) {
+                    const float4 x = *reinterpret_cast<const float4*>(
+                        tbuf + (half * kTransRows + trow) * 32 + (((thalf * 4 + jj) ^ (trow & 7)) << 2));
+                    e[4 * jj] = x.x; e[4 * jj + 1] = x.y; e[4 * jj + 2] = x.z; e[4 * jj + 3] = x.w;
+                  }
+                  if (n16 == 16) stats_fold16_packed(e, vocab16, st[slot][half]);
+                  else if (n16 > 0) stats_fold16<false>(e, n16, vocab16, st[slot][half]);
+                }
+              }
+            }
+          }
+        }
+        continue;
+      }
+#pragma unroll
+      for (int slot = 0; slot < kSlots; ++slot) {
         if (slot < my_chunks) {
           const int ch = rot ? slot * sub_chunks + group : group + slot * kGroups;
           const int sub = ch / sub_chunks, j = ch - sub * sub_chunks;
@@ -835,7 +968,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
                     e[4 * jj] = x.x; e[4 * jj + 1] = x.y; e[4 * jj + 2] = x.z; e[4 * jj + 3] = x.w;
                   }
                   // (rows at or beyond n_ok fold whatever the unused columns held; they are never written out)
-                  if (n16 == 16) stats_fold16<true>(e, 16, vocab16, st[slot][half]);
+                  if (n16 == 16) stats_fold16_packed(e, vocab16, st[slot][half]);
                   else if (n16 > 0) stats_fold16<false>(e, n16, vocab16, st[slot][half]);
                 }
               }
@@ -849,7 +982,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
     asm volatile("bar.sync 1, %0;" ::"n"(kNumEpi * 32) : "memory");
     float4* merge = reinterpret_cast<float4*>(trans_base);          // [4 quarters][rows of the pass]
 #pragma unroll
-    for (int slot = 0; slot < kEpiSlots; ++slot) {
+    for (int slot = 0; slot < kSlots; ++slot) {
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
         Stats a = st[slot][half], o;
@@ -1153,10 +1286,8 @@ template <bool kVec>
 __global__ void __launch_bounds__(kK3Threads, kK3MaxPerSm) accept_sample_kernel(const K3Params p) {
   extern __shared__ double csum[];                       // per-chunk residual mass of this CTA's slice
   __shared__ double sh_tot[2][8];                        // slice totals of the whole cluster, per attempt
-  __shared__ float sh_logZ[kMaxK1], sh_H[kMaxK1], sh_u[kMaxK1 + 1];
-  __shared__ int sh_amax[kMaxK1];
-  __shared__ int sh_stop[2];                             // first draft position not accepted, per gathering warp
-  __shared__ unsigned sh_wflags[2];
+  __shared__ float sh_logZ[kMaxK1], sh_H[kMaxK1], sh_lx[kMaxK1], sh_qx[kMaxK1], sh_u[kMaxK1], sh_Hq[kMaxK1];
+  __shared__ int sh_x[kMaxK1], sh_amax[kMaxK1];
   __shared__ int sh_n;
   __shared__ unsigned sh_flags;
 
@@ -1170,23 +1301,20 @@ __global__ void __launch_bounds__(kK3Threads, kK3MaxPerSm) accept_sample_kernel(
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int k = p.k, V = p.V;
   const int row_first = b * (k + 1);
+
+  // ---- gather the k draft-token logits, draft probabilities and the uniforms (independent of the statistics).
+  // These come from the caller, not from the GEMM kernel.  Behind this call's own GEMM kernel they are known to be in
+  // place (its CTAs waited for whatever ran before the call) and are fetched before this grid's dependency wait; in
+  // every other launch the wait comes first.
+  if (!p.inputs_settled) grid_dependency_wait();
+  for (int j = threadIdx.x; j <= k; j += kK3Threads) sh_u[j] = p.u[b * (k + 1) + j];
+  int x_mine = -1;                                       // (k <= 63 < kK3Threads: one draft position per thread)
+  float qx_mine = 0.f;
   const bool shard = p.shard_world > 0;
   const int Vtok = shard ? p.V_global : V;               // range of valid token ids
-
-  // Inputs that come from the caller and not from the GEMM kernel.  Behind this call's own GEMM kernel they are known
-  // to be in place (its CTAs waited for whatever ran before the call) and are fetched under that kernel's tail;
-  // in every other launch the dependency wait comes first.
-  if (!p.inputs_settled) grid_dependency_wait();
-  // The last two warps own the draft positions (k <= 63: one position per thread, j = gthread); the other warps
-  // start on the softmax statistics at once, so the two chains of dependent loads run side by side.
-  const int gthread = static_cast<int>(threadIdx.x) - (kK3Threads - 64);
-  const bool gatherer = gthread >= 0 && gthread < k;
-  int x_mine = -1;
-  float qx_mine = 0.f, u_mine = 0.f, lx_mine = 0.f;
-  if (gatherer) {
-    const int j = gthread;
+  if (threadIdx.x < k) {
+    const int j = threadIdx.x;
     x_mine = p.tok[b * k + j];
-    u_mine = p.u[b * (k + 1) + j];
     if (x_mine >= 0 && x_mine < Vtok) {
       const size_t qi = (static_cast<size_t>(b) * k + j) * V + x_mine;
       if (p.q_tok) qx_mine = p.q_tok[b * k + j];
@@ -1194,27 +1322,30 @@ __global__ void __launch_bounds__(kK3Threads, kK3MaxPerSm) accept_sample_kernel(
                                                 : static_cast<const float*>(p.q)[qi];
     }
   }
-  if (threadIdx.x == 0) sh_u[k] = p.u[b * (k + 1) + k];
   // From here on the GEMM kernel's results are read.
   if (p.inputs_settled) grid_dependency_wait();
-  float hq_mine = 0.f;
-  if (gatherer) {
-    const int j = gthread, x = x_mine;
+  for (int j = threadIdx.x; j < k; j += kK3Threads) {
+    const int x = x_mine;
+    sh_x[j] = x;
+    float lx = 0.f;
+    const float qx = qx_mine;
     if (x >= 0 && x < Vtok) {
       if (shard) {                                       // exactly one shard owns x and left its logit there
-        lx_mine = -CUDART_INF_F;
-        for (int r = 0; r < p.shard_world; ++r)
-          lx_mine = fmaxf(lx_mine, p.lx_all[static_cast<size_t>(r) * p.rec_stride + b * k + j]);
+        lx = -CUDART_INF_F;
+        for (int r = 0; r < p.shard_world; ++r) lx = fmaxf(lx, p.lx_all[static_cast<size_t>(r) * p.rec_stride + b * k + j]);
       } else {
-        lx_mine = p.logits[static_cast<size_t>(row_first + j) * p.ldl + x];
+        lx = p.logits[static_cast<size_t>(row_first + j) * p.ldl + x];
       }
     }
+    sh_lx[j] = lx; sh_qx[j] = qx;
+    float hq = 0.f;
     if (p.gate_source == HOLA_GATE_DRAFT_ENTROPY) {
       double tot = 0.0;
       for (int sl = 0; sl < kHqSlices; ++sl) tot += p.hq_part[(static_cast<size_t>(b) * k + j) * kHqSlices + sl];
-      hq_mine = fmaxf(0.f, static_cast<float>(-tot));
-      if (rank == 0 && p.draft_entropy) p.draft_entropy[b * k + j] = hq_mine;
+      hq = fmaxf(0.f, static_cast<float>(-tot));
+      if (rank == 0 && p.draft_entropy) p.draft_entropy[b * k + j] = hq;
     }
+    sh_Hq[j] = hq;
   }
   // ---- softmax statistics of this sequence's k+1 positions
   if (p.combine) {
@@ -1235,53 +1366,25 @@ __global__ void __launch_bounds__(kK3Threads, kK3MaxPerSm) accept_sample_kernel(
   }
   __syncthreads();
 
-  // ---- gate and ratio test, every draft position on its own thread; the run of kept drafts ends at the first
-  // position that is not accepted (a token outside the vocabulary counts as one)
-  {
-    unsigned flags = 0;
-    bool stop = false, bad = false;
-    if (gatherer) {
-      const int j = gthread, x = x_mine;
-      if (x < 0 || x >= Vtok) {
-        stop = true; bad = true;
-      } else {
-        const float gate_value = p.gate_source == HOLA_GATE_DRAFT_ENTROPY ? hq_mine : sh_H[j];
-        if (!(gate_value < p.tau)) {                     // entropy gate off: the verifier decides
-          if (p.fallback == HOLA_FALLBACK_GREEDY) {
-            stop = x != sh_amax[j];
-          } else {
-            const float u = clamp_uniform(u_mine, flags);
-            const float px = expf(lx_mine - sh_logZ[j]);
-            const float qx = qx_mine;
-            stop = !((qx > 0.f) ? (u * qx < px) : (px > 0.f));
-          }
-        }
-      }
-    }
-    // positions j = gthread live in the last two warps: first stop per warp, then the earlier of the two
-    const unsigned stops = __ballot_sync(0xffffffffu, stop);
-    const int first = stops ? __ffs(stops) - 1 : 32;     // lane of the first stop in this warp
-    // flags count only for positions that were evaluated: those up to and including the first stop
-    unsigned fl = (lane <= first) ? flags : 0u;
-    if (bad && lane == first) fl |= HOLA_FLAG_BAD_TOKEN;
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) fl |= __shfl_xor_sync(0xffffffffu, fl, off);
-    if (warp >= kK3Warps - 2 && lane == 0) {
-      sh_stop[warp - (kK3Warps - 2)] = first;
-      sh_wflags[warp - (kK3Warps - 2)] = fl;
-    }
-  }
-  __syncthreads();
+  // ---- gate and ratio test in draft order; stop at the first position that is not accepted
   if (threadIdx.x == 0) {
-    int n = k;
     unsigned flags = 0;
-    if (sh_stop[0] < 32) { n = sh_stop[0]; flags = sh_wflags[0]; }
-    else {
-      flags = sh_wflags[0];
-      if (sh_stop[1] < 32) n = 32 + sh_stop[1];
-      flags |= sh_wflags[1];
+    int n = k;
+    for (int j = 0; j < k; ++j) {
+      const int x = sh_x[j];
+      if (x < 0 || x >= Vtok) { flags |= HOLA_FLAG_BAD_TOKEN; n = j; break; }
+      const float gate_value = p.gate_source == HOLA_GATE_DRAFT_ENTROPY ? sh_Hq[j] : sh_H[j];
+      if (gate_value < p.tau) continue;                  // entropy gate: fast path keeps the draft token
+      if (p.fallback == HOLA_FALLBACK_GREEDY) {          // the verifier's own token, or the run ends here
+        if (x != sh_amax[j]) { n = j; break; }
+        continue;
+      }
+      const float u = clamp_uniform(sh_u[j], flags);
+      const float px = expf(sh_lx[j] - sh_logZ[j]);
+      const float qx = sh_qx[j];
+      const bool accept = (qx > 0.f) ? (u * qx < px) : (px > 0.f);
+      if (!accept) { n = j; break; }
     }
-    if (n > k) n = k;
     sh_n = n;
     sh_flags = flags;
     if (rank == 0) {
@@ -1355,21 +1458,16 @@ __global__ void __launch_bounds__(kK3Threads, kK3MaxPerSm) accept_sample_kernel(
         const int c = c0 + i * kK3Warps;
         if (c < mine) fetch4<kVec>(lrow, qrow, p.q_dtype, residual, (c_first + c) * kChunk + lane * 4, V, l[i], q[i]);
       }
-      double part[kK3Unroll];
 #pragma unroll
       for (int i = 0; i < kK3Unroll; ++i) {
         const int c = c0 + i * kK3Warps;
-        part[i] = 0.0;
         if (c < mine) {
           float r[4];
           resid4(l[i], q[i], logZ, r);
-          part[i] = ((static_cast<double>(r[0]) + r[1]) + r[2]) + r[3];
+          const double sum = warp_sum_f64(((static_cast<double>(r[0]) + r[1]) + r[2]) + r[3]);
+          if (lane == 0) csum[c] = sum;
         }
       }
-      // the four chunk sums of this step: lanes 0, 8, 16, 24 end up with chunks 0, 1, 2, 3
-      const double sum = warp_sum4_f64(part, lane);
-      const int c = c0 + (lane >> 3) * kK3Warps;
-      if ((lane & 7) == 0 && c < mine) csum[c] = sum;
     }
     __syncthreads();
     // warp 0: scan of the slice; lane L owns chunks [lo, hi)
@@ -1800,7 +1898,8 @@ Plan make_plan(const hola_ctx* ctx, int M, int w_dtype = HOLA_W_BF16) {
   // a pass may end up empty when rows_per_pass * (passes - 1) already covers M
   best.passes = (rows + best.rows_per_pass - 1) / best.rows_per_pass;
   const int stage_bytes = kWBlockBytes + best.n_sub * (best.N / 2) * 128 + (w8 ? kRawBlockBytes : 0);
-  const int trans_bytes = (w8 ? kW8EpiWarps : kEpiWarps) * kTransBytes;
+  // (rotating units: every epilogue warp stages a whole 32-row chunk, twice the bytes)
+  const int trans_bytes = (w8 ? kW8EpiWarps : kEpiWarps) * kTransBytes * (best.n_sub == 3 ? 2 : 1);
   int stages = (kSmemBudget - 1024 - kBarrierBytes - trans_bytes) / stage_bytes;
   if (stages > kMaxStages) stages = kMaxStages;
   if (ctx->force_stages && ctx->force_stages < stages) stages = ctx->force_stages;
@@ -1947,13 +2046,14 @@ hola_status run_lm_head(hola_ctx* ctx, const hola_verify_args* a, float* logits,
   cfg.numAttrs = 2;
   for (int pass = 0; pass < pl.passes; ++pass) {
     kp.row0 = pass * pl.rows_per_pass;
-    kp.first_pass = pass == 0 ? 1 : 0;
     kp.rows = M - kp.row0 < pl.rows_per_pass ? M - kp.row0 : pl.rows_per_pass;
     if (kp.rows <= 0) break;
-    e = two ? cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<3>, th, tw, kp)
-      : i8 ? cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<2>, th, tw, kp)
-      : w8 ? cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<1>, th, tw, kp)
-           : cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<0>, th, tw, kp);
+    e = two ? cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<3, false>, th, tw, kp)
+      : i8 ? (pl.rot ? cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<2, true>, th, tw, kp)
+                     : cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<2, false>, th, tw, kp))
+      : w8 ? cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<1, false>, th, tw, kp)
+           : (pl.rot ? cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<0, true>, th, tw, kp)
+                     : cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<0, false>, th, tw, kp));
     if (e != cudaSuccess) { set_error(ctx, "launch lm_head_entropy_kernel", e); return HOLA_ERR_CUDA; }
   }
   return HOLA_OK;
@@ -2011,21 +2111,10 @@ hola_status run_accept_sample(hola_ctx* ctx, const hola_verify_args* a, const fl
   while (S > 1 && (a->B * S > kK3MaxPerSm * ctx->num_sms || nchunks / S < 8)) S >>= 1;   // one wave of CTAs
   if (phase == 1) S = 1;                                 // no vocabulary pass: one CTA per sequence
   const int cpc = (nchunks + S - 1) / S;
-  // The grid may be scheduled while the GEMM kernel's CTAs are still leaving their SMs one by one.  Left alone, its
-  // small CTAs would pile up eight deep on the first SMs to come free; asking for as much shared memory as keeps
-  // ceil(grid / SMs) CTAs on an SM, and no more, spreads them over the machine whatever the order of arrival.
-  const int grid = a->B * S;
-  int per_sm = (grid + ctx->num_sms - 1) / ctx->num_sms;
-  per_sm = per_sm < 1 ? 1 : (per_sm > kK3MaxPerSm ? kK3MaxPerSm : per_sm);
-  size_t smem = static_cast<size_t>(cpc) * sizeof(double);
-  if (per_sm < kK3MaxPerSm) {
-    const size_t spread = kSmTotalSmem / per_sm - kK3SmemOverhead;
-    if (spread > smem) smem = spread;
-  }
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(static_cast<unsigned>(grid));
+  cfg.gridDim = dim3(static_cast<unsigned>(a->B * S));
   cfg.blockDim = dim3(kK3Threads);
-  cfg.dynamicSmemBytes = smem;
+  cfg.dynamicSmemBytes = static_cast<size_t>(cpc) * sizeof(double);
   cfg.stream = stream;
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -2067,18 +2156,15 @@ hola_status check_sample_args(const hola_verify_args* a) {
 // Once per context (and once per device for the entry point without one), with the device current: the kernels that
 // ask for more dynamic shared memory than the default limit are told so here, not on every call.
 cudaError_t configure_kernels() {
-  cudaError_t e = cudaFuncSetAttribute(lm_head_entropy_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(lm_head_entropy_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(lm_head_entropy_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(lm_head_entropy_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
-  const int k3_max = static_cast<int>(kSmTotalSmem - kK3SmemOverhead);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(accept_sample_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, k3_max);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(accept_sample_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, k3_max);
+  cudaError_t e = cudaSuccess;
+  const void* kernels[] = {reinterpret_cast<const void*>(lm_head_entropy_kernel<0, false>),
+                           reinterpret_cast<const void*>(lm_head_entropy_kernel<0, true>),
+                           reinterpret_cast<const void*>(lm_head_entropy_kernel<1, false>),
+                           reinterpret_cast<const void*>(lm_head_entropy_kernel<2, false>),
+                           reinterpret_cast<const void*>(lm_head_entropy_kernel<2, true>),
+                           reinterpret_cast<const void*>(lm_head_entropy_kernel<3, false>)};
+  for (const void* k : kernels)
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
   return e;
 }
 
@@ -2326,7 +2412,7 @@ hola_status verify_device(hola_ctx* ctx, const hola_verify_args* a, cudaStream_t
   }
   if (before_sample && cudaStreamWaitEvent(stream, before_sample, 0) != cudaSuccess) return HOLA_ERR_CUDA;
   ctx->hq_ready = side ? 1 : 0;
-  // (an event wait between the two kernels makes the second an ordinary launch; its inputs are settled either way)
+  // (behind the GEMM kernel: the caller's inputs are settled; an event wait in between makes it an ordinary launch)
   s = run_accept_sample(ctx, a, logits, ldl, 1, pl.grid, stream, nullptr, 0, nullptr, true);
   ctx->hq_ready = 0;
   if (prof) { cudaEventRecord(ev[2], stream); ctx->prof_n++; }
