@@ -1208,15 +1208,14 @@ __device__ __forceinline__ double warp_sum_f64(double x) {
   return x;
 }
 
-// Four sums over the warp at once, in the addition order of warp_sum_f64 (pairs 16 apart, then 8, 4, 2, 1) and so with
-// the same bits, for a third of the shuffles: the first two rounds halve the number of values a lane carries instead of
-// adding all of them everywhere.  Lanes 8 i .. 8 i + 7 return the sum of v[i].
-__device__ __forceinline__ double warp_sum4_f64(const double v[4], int lane) {
+// Four sums over the warp at once (lanes 8 i .. 8 i + 7 return the sum of v[i]): the first two rounds halve the
+// number of values a lane carries instead of adding all of them everywhere, six shuffles in all.
+__device__ __forceinline__ float warp_sum4_f32(const float v[4], int lane) {
   const bool hi16 = (lane & 16) != 0;
-  const double a = (hi16 ? v[2] : v[0]) + __shfl_xor_sync(0xffffffffu, hi16 ? v[0] : v[2], 16);
-  const double b = (hi16 ? v[3] : v[1]) + __shfl_xor_sync(0xffffffffu, hi16 ? v[1] : v[3], 16);
+  const float a = (hi16 ? v[2] : v[0]) + __shfl_xor_sync(0xffffffffu, hi16 ? v[0] : v[2], 16);
+  const float b = (hi16 ? v[3] : v[1]) + __shfl_xor_sync(0xffffffffu, hi16 ? v[1] : v[3], 16);
   const bool hi8 = (lane & 8) != 0;
-  double c = (hi8 ? b : a) + __shfl_xor_sync(0xffffffffu, hi8 ? a : b, 8);
+  float c = (hi8 ? b : a) + __shfl_xor_sync(0xffffffffu, hi8 ? a : b, 8);
 #pragma unroll
   for (int off = 4; off > 0; off >>= 1) c += __shfl_xor_sync(0xffffffffu, c, off);
   return c;
@@ -1258,10 +1257,12 @@ __device__ __forceinline__ void fetch4(const float* lrow, const void* qrow, int 
   }
 }
 
-// The four residual masses  r = max(0, p - q)  with  p = e^(l - logZ)  (q = 0: r = p).
+// The four residual masses  r = max(0, p - q)  with  p = e^(l - logZ)  (q = 0: r = p).  The exponential is the
+// hardware's 2^x on (l - logZ) log2 e: relative error about 1e-6 at l - logZ = -30, against a decision margin of 1e-4
+// on the cumulative mass; the pass over the row and the final search inside a chunk both come through here.
 __device__ __forceinline__ void resid4(const float l[4], const float q[4], float logZ, float r[4]) {
 #pragma unroll
-  for (int i = 0; i < 4; ++i) r[i] = fmaxf(0.f, expf(l[i] - logZ) - q[i]);
+  for (int i = 0; i < 4; ++i) r[i] = fmaxf(0.f, ex2_approx((l[i] - logZ) * kLog2e) - q[i]);
 }
 
 template <bool kVec>
@@ -1349,7 +1350,9 @@ __global__ void __launch_bounds__(kK3Threads, kK3MaxPerSm) accept_sample_kernel(
   }
   // ---- softmax statistics of this sequence's k+1 positions
   if (p.combine) {
-    for (int j = warp; j <= k; j += kK3Warps) {
+    // (rows are dealt to the warps from the last warp down: warp 0, whose threads are still waiting for the gathers
+    // above, gets a row only when there are more than seven)
+    for (int j = kK3Warps - 1 - warp; j <= k; j += kK3Warps) {
       Stats st = warp_merge_partials(p.partials, p.nparts, p.part_stride, row_first + j, lane);
       if (lane == 0) {
         float lz, h;
@@ -1458,16 +1461,22 @@ __global__ void __launch_bounds__(kK3Threads, kK3MaxPerSm) accept_sample_kernel(
         const int c = c0 + i * kK3Warps;
         if (c < mine) fetch4<kVec>(lrow, qrow, p.q_dtype, residual, (c_first + c) * kChunk + lane * 4, V, l[i], q[i]);
       }
+      // the mass of each chunk in fp32 (128 non-negative terms added pairwise: relative error a few 1e-7), kept as
+      // fp64 for the scans that follow; lanes 0, 8, 16, 24 end up with chunks 0, 1, 2, 3 of this step
+      float part[kK3Unroll];
 #pragma unroll
       for (int i = 0; i < kK3Unroll; ++i) {
         const int c = c0 + i * kK3Warps;
+        part[i] = 0.f;
         if (c < mine) {
           float r[4];
           resid4(l[i], q[i], logZ, r);
-          const double sum = warp_sum_f64(((static_cast<double>(r[0]) + r[1]) + r[2]) + r[3]);
-          if (lane == 0) csum[c] = sum;
+          part[i] = (r[0] + r[1]) + (r[2] + r[3]);
         }
       }
+      const float sum = warp_sum4_f32(part, lane);
+      const int c = c0 + (lane >> 3) * kK3Warps;
+      if ((lane & 7) == 0 && c < mine) csum[c] = static_cast<double>(sum);
     }
     __syncthreads();
     // warp 0: scan of the slice; lane L owns chunks [lo, hi)
