@@ -107,3 +107,87 @@ def test_two_plane_head_logits_stay_close_to_bf16_activations():
     exact = hid @ W8.T
     assert np.max(np.abs(h16 @ W8.T - exact)) < 2e-4                    # 16-bit-class rows: invisible next to ...
     assert np.max(np.abs(h8 @ W8.T - exact)) > 2e-3                     # ... what one 8-bit plane does to the logits
+
+
+# ---- 4-bit sub-blocks with a shared power-of-two exponent per sub-block --------------------------------------------
+def _w4_rows(seed, V=12, nb=3):
+    """Rows that ARE of the 4-bit form with row scale 1: entry = c << e with c in [-7, 7], e per sub-block, and one
+    entry equal to 112 so that the row maximum gives scale exactly 1."""
+    rng = np.random.default_rng(seed)
+    c = rng.integers(-7, 8, size=(V, nb, 128))
+    e = rng.integers(0, 5, size=(V, nb))
+    c[:, :, 0] = 7                                          # every sub-block reaches its top code: e is forced
+    e[:, 0] = 4                                             # sub-block 0 holds 7 << 4 = 112, the row maximum
+    W = (c << e[:, :, None]).reshape(V, nb * 128).astype(np.float32)
+    return W, c.reshape(V, -1).astype(np.int8), e.astype(np.uint8)
+
+
+def test_w4_rows_of_the_format_are_reproduced_exactly():
+    W, c, e = _w4_rows(3)
+    codes, shifts, scale = lobi.quantize_rows_w4(W)
+    assert np.all(scale == 1.0)
+    assert np.array_equal(shifts, e) and np.array_equal(codes, c)
+    assert np.array_equal(lobi.dequantize_rows_w4(codes, shifts, scale), W.astype(np.float64))
+    # a power-of-two factor moves into the row scale and changes neither codes nor exponents
+    codes2, shifts2, scale2 = lobi.quantize_rows_w4(W * np.float32(0.125))
+    assert np.array_equal(codes2, codes) and np.array_equal(shifts2, shifts) and np.all(scale2 == 0.125)
+
+
+def test_w4_exponent_is_the_smallest_that_covers_the_sub_block():
+    W = np.zeros((1, 4 * 128), np.float32)
+    W[0, 0] = 112.0                                         # row scale 1; sub-block 0 needs e = 4
+    W[0, 128] = 7.0                                         # sub-block 1: 7 * 2^0 covers it
+    W[0, 256] = 7.5                                         # sub-block 2: just beyond 7, so e = 1
+    W[0, 384] = 56.0                                        # sub-block 3: 7 * 2^3
+    codes, shifts, scale = lobi.quantize_rows_w4(W)
+    assert scale[0] == 1.0 and shifts[0].tolist() == [4, 0, 1, 3]
+    assert codes[0, 0] == 7 and codes[0, 128] == 7 and codes[0, 384] == 7
+    assert codes[0, 256] == 4                               # 7.5 / 2 = 3.75 -> 4
+
+
+def test_w4_error_bound_symmetry_zero_rows_and_ties():
+    rng = np.random.default_rng(4)
+    W = (rng.normal(size=(30, 512)) * 0.02).astype(np.float32)
+    W[:, 128:256] *= 0.1                                    # a quiet sub-block in every row: it gets a smaller exponent
+    W[5] = 0.0
+    codes, shifts, scale = lobi.quantize_rows_w4(W)
+    deq = lobi.dequantize_rows_w4(codes, shifts, scale)
+    step = scale[:, None].astype(np.float64) * np.exp2(shifts.astype(np.float64))          # [V, nb]
+    err = np.abs(deq - W).reshape(30, 4, 128)
+    assert np.all(err <= 0.5 * step[:, :, None] * (1 + 1e-6))          # nothing clips: at most half a step per sub-block
+    assert np.all(shifts[np.arange(30) != 5, 1] < 4)                   # the quiet sub-block uses a finer step
+    assert codes.min() >= -7 and codes.max() <= 7                      # -8 is never used
+    assert np.all(codes[5] == 0) and scale[5] == 1.0
+    c2, e2, s2 = lobi.quantize_rows_w4(-W)
+    assert np.array_equal(c2, -codes) and np.array_equal(e2, shifts) and np.array_equal(s2, scale)
+    # ties go to the even code: row scale 1 (maximum 112), second sub-block at e = 0 holds x.5 values
+    T = np.zeros((1, 256), np.float32)
+    T[0, 0] = 112.0
+    T[0, 128:134] = [0.5, 1.5, 2.5, -0.5, -1.5, 6.5]
+    T[0, 134] = 7.0
+    c, e, s = lobi.quantize_rows_w4(T)
+    assert s[0] == 1.0 and e[0].tolist() == [4, 0] and c[0, 128:135].tolist() == [0, 2, 2, 0, -2, 6, 7]
+
+
+def test_nibble_packing_round_trip_and_layout():
+    rng = np.random.default_rng(5)
+    c = rng.integers(-8, 8, size=(7, 64)).astype(np.int8)
+    p = lobi.pack_nibbles(c)
+    assert p.shape == (7, 32) and p.dtype == np.uint8
+    assert np.array_equal(lobi.unpack_nibbles(p), c)
+    one = np.array([[3, -2]], np.int8)                      # low nibble 0x3, high nibble 0xE (-2 in 4-bit two's complement)
+    assert lobi.pack_nibbles(one)[0, 0] == 0xE3
+
+
+def test_mixed_width_head_takes_each_group_from_its_own_quantiser():
+    rng = np.random.default_rng(6)
+    V, H = 2 * 256 + 100, 256                               # three groups, the last one ragged
+    W = ref.bf16_bits_to_f64(ref.f32_to_bf16_bits((rng.normal(size=(V, H)) * 0.02).astype(np.float32))).astype(np.float32)
+    D = lobi.dequantize_mixed(W, [16, 4, 8])
+    assert np.array_equal(D[:256], W[:256].astype(np.float64))                              # 16 bits: untouched
+    assert np.array_equal(D[256:512], lobi.dequantize_rows_w4(*lobi.quantize_rows_w4(W[256:512])))
+    assert np.array_equal(D[512:], lobi.dequantize_rows(*lobi.quantize_rows_int8(W[512:])))
+    # wider is closer: the 8-bit group's error is well below the 4-bit group's
+    e4 = np.abs(D[256:512] - W[256:512]).max() / np.abs(W[256:512]).max()
+    e8 = np.abs(D[512:] - W[512:]).max() / np.abs(W[512:]).max()
+    assert e8 < 0.005 and 0.02 < e4 < 0.08
