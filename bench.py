@@ -315,10 +315,12 @@ def main():
                     help="which entropy feeds the gate: the verifier's softmax (default) or the draft row")
     ap.add_argument("--fallback", default="sample", choices=["sample", "greedy"],
                     help="what the gate-off branch does: speculative-sampling test (default) or greedy verifier")
-    ap.add_argument("--weights", default="bf16", choices=["bf16", "int8", "w8a8", "w8a16"],
+    ap.add_argument("--weights", default="bf16", choices=["bf16", "int8", "w8a8", "w8a16", "mixed", "w4"],
                     help="bf16 (default); int8: 8-bit W_lm from hola_quantize_w8, expanded exactly on chip; "
                          "w8a8: 8-bit W_lm and hidden rows quantised on the fly, 8-bit tensor-core kind; "
-                         "w8a16: the same with the hidden rows as two 8-bit planes (16-bit-class activations)")
+                         "w8a16: the same with the hidden rows as two 8-bit planes (16-bit-class activations); "
+                         "mixed: groups of 256 vocabulary rows at 4 / 8 / 16 bits in the proportions 20 / 70 / 10 %% "
+                         "(seeded), expanded on chip; w4: every group at 4 bits")
     ap.add_argument("--flush-l2", default="auto", choices=["auto", "on", "off"],
                     help="rewrite a 256 MB buffer between timed steps (auto: when the weights streamed per step do not "
                          "clearly exceed the L2)")
@@ -353,7 +355,8 @@ def main():
     w = workloads.make_config(args.workload, dev, seed_offset=hdist.rank_seed_offset(rank))
     ctx = binding.HolaVerify(w.B, w.k, w.H, w.V, device=local)
     plan = ctx.hola_plan(w.B, w.k, {"bf16": binding.HOLA_W_BF16, "int8": binding.HOLA_W_INT8,
-                                    "w8a8": binding.HOLA_W8A8, "w8a16": binding.HOLA_W8A16}[args.weights])
+                                    "w8a8": binding.HOLA_W8A8, "w8a16": binding.HOLA_W8A16,
+                                    "mixed": binding.HOLA_W_MIXED, "w4": binding.HOLA_W_MIXED}[args.weights])
     out = ctx.alloc_outputs(w.B, w.k, False)
     global L2_BYTES
     L2_BYTES = int(getattr(torch.cuda.get_device_properties(dev), "L2_cache_size", L2_BYTES)) or L2_BYTES
@@ -363,7 +366,16 @@ def main():
 
     W_dev, w_scale = w.W_lm, None
     a8 = {"w8a8": True, "w8a16": "a16"}.get(args.weights, False)
-    if args.weights != "bf16":
+    head_bytes = None
+    if args.weights in ("mixed", "w4"):
+        import numpy as np
+        ng = -(-w.V // binding.GROUP_ROWS)
+        widths = ([4] * ng if args.weights == "w4" else
+                  np.random.default_rng(250618952).choice([4, 8, 16], size=ng, p=[0.2, 0.7, 0.1]).tolist())
+        W_dev = binding.hola_quantize_mixed(w.W_lm, widths)
+        head_bytes = W_dev.weight_bytes()
+        torch.cuda.synchronize()
+    elif args.weights != "bf16":
         W_dev, w_scale = binding.hola_quantize_w8(w.W_lm)
         torch.cuda.synchronize()
     gate_source = 1 if args.gate == "draft" else 0
@@ -437,6 +449,10 @@ def main():
     if rank == 0:
         peaks, peak_kind = load_peaks()
         work = algorithmic_work(w, 2 if args.weights == "bf16" else 1)
+        if head_bytes is not None:                          # mixed widths: the bytes of the stored head, as they are
+            delta = head_bytes - (work["gemm_bytes"] - w.M * w.H * 2)
+            work["gemm_bytes"] += delta
+            work["step_bytes"] += delta
         # the 8-bit tensor-core kinds have twice the nominal rate of bf16: measured bf16 peak x 2 for --weights w8a8
         # (w8a16 runs two 8-bit rows per verify row: per algorithmic flop its peak is the bf16 one again)
         roof = fractions(work, peaks, k1_ms * 1e-3 * plan["passes"], ms_max / args.steps * 1e-3,
@@ -452,6 +468,7 @@ def main():
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms_max / args.steps, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "int8" if a8 else "bf16", "data": "synthetic",
+                "weight_bytes": head_bytes if head_bytes is not None else w.V * w.H * w_elem,
                 "repeats": {"regions": len(per_region), "ms_per_step_min": min(per_region) / args.steps,
                             "ms_per_step_median": ms_total / args.steps, "ms_per_step_max": max(per_region) / args.steps},
                 "config": config_block(w, {"plan": plan, "parallelism": f"replicas x{world}", "gate": args.gate,

@@ -69,13 +69,38 @@ typedef enum {
   HOLA_W8A8 = 2,   /* int8 weights AND the hidden rows quantised the same way (one fp32 scale per verify row) by the
                     * library on the fly; products on the 8-bit tensor-core kind with exact int32 accumulation:
                     * l[r][v] = w_scale[v] * h_scale[r] * sum_h q_hid[r][h] * q_w[v][h].  Needs a context. */
-  HOLA_W8A16 = 3   /* int8 weights, hidden rows kept at 16-bit width as TWO 8-bit planes made on the fly: the coarse
+  HOLA_W8A16 = 3,  /* int8 weights, hidden rows kept at 16-bit width as TWO 8-bit planes made on the fly: the coarse
                     * plane of HOLA_W8A8 (scale s1) and a plane of its remainder (scale s2 = s1 / 254), so that
                     * |x16 - x| <= max|x| / 64516 per row.  Both planes go through the 8-bit tensor-core kind
                     * (twice the rows, twice the rate, half the weight bytes of bf16) and
                     * l[r][v] = w_scale[v] * (s1[r] * sum_h q1[r][h] q_w[v][h] + s2[r] * sum_h q2[r][h] q_w[v][h]).
                     * At most 256 verify rows per pass over W_lm.  Needs a context. */
+  HOLA_W_MIXED = 4 /* the Lo-Bi section's mixed precision on the LM head: groups of 256 vocabulary rows stored at 4, 8 or 16
+                    * bits (hola_wmix below), all expanded exactly to bf16 on chip, bf16 activations as given.  W_lm of
+                    * the arguments is not read.  At most 256 verify rows per pass; H a multiple of 128. */
 } hola_w_dtype;
+
+/* The weights of HOLA_W_MIXED (args->wmix points to one of these, in HOST memory; its pointers are DEVICE pointers).
+ * The paper's quantiser maps sub-blocks of a weight matrix to 4, 8 or 16 bits and leaves format and sub-block open;
+ * the reading built here: a sub-block is 128 consecutive hidden channels of one vocabulary row, and widths are
+ * assigned per GROUP of 256 consecutive vocabulary rows (group g = rows 256 g .. 256 g + 255, the last one ragged).
+ *   16 bits: the bf16 row as it is (w_scale[v] must be 1).
+ *    8 bits: int8 codes, one scale per row (hola_quantize_w8): W[v][h] = w_scale[v] * q[v][h].
+ *    4 bits: codes c in [-7, 7], two per byte (even h in the low nibble, two's complement), and per sub-block b an
+ *            exponent e in 0..4 (hola_quantize_w4): W[v][h] = w_scale[v] * (c[v][h] << e[v][b]), so a sub-block's scale
+ *            is w_scale[v] * 2^e.
+ * Rows of one width are stored compactly, in vocabulary order, in that width's buffer; group_row[g] is the index of
+ * group g's first row inside the buffer of its width.  w_scale (args) is indexed by vocabulary row as usual. */
+typedef struct hola_wmix {
+  const void* W16;             /* bf16 [rows16][H]                                                       */
+  const void* W8;              /* int8 [rows8][H]                                                        */
+  const void* W4;              /* bytes [rows4][H/2], two 4-bit codes each                               */
+  const uint8_t* shift4;       /* uint8 [H/128][rows4]: exponent of each 4-bit sub-block, sub-block-major */
+  const uint8_t* group_width;  /* uint8 [ceil(V/256)]: 4, 8 or 16                                        */
+  const int32_t* group_row;    /* int32 [ceil(V/256)]                                                    */
+  int32_t rows16, rows8, rows4;/* rows in each buffer (0: that width does not occur, its pointers may be null) */
+  int32_t reserved_;
+} hola_wmix;
 
 /* Bits of the device status word (OR-ed by the kernels; the caller clears it). */
 #define HOLA_FLAG_BAD_TOKEN 1u   /* a draft token outside [0,V): treated as a rejection at that position    */
@@ -107,6 +132,7 @@ typedef struct {
   int32_t w_dtype;         /* hola_w_dtype; 0 = W_lm is bf16, otherwise W_lm is int8 [V][H] and H % 16 == 0     */
   int32_t reserved_;       /* must be 0                                                                        */
   const float* w_scale;    /* fp32 [V], required with an int8 W_lm (w_dtype != 0): scale of each vocabulary row  */
+  const hola_wmix* wmix;   /* HOST pointer, required with w_dtype = HOLA_W_MIXED, else ignored                   */
 } hola_verify_args;
 
 /* Creates a context on `device` able to serve calls with B <= maxB, k <= maxK and exactly this H and V.
@@ -239,6 +265,16 @@ hola_status hola_lm_head_entropy_static(const hola_verify_args* args, void* cuda
  * fp32 with ties to even.  q_out is int8 [V][H], scale_out fp32 [V], both device buffers of the caller.  Allocates
  * nothing and needs no context. */
 hola_status hola_quantize_w8(const void* W_bf16, int V, int H, void* q_out, float* scale_out, void* cuda_stream);
+
+/* The 4-bit case of the same quantiser (Lo-Bi Optimization section; format as described at hola_wmix): `rows` bf16 rows
+ * of H channels (H a multiple of 128) -> packed_out bytes [rows][H/2], scale_out fp32 [rows] = max|w| / 112 (1 for an
+ * all-zero row), and per sub-block b the smallest exponent e in 0..4 with 7 * 2^e * scale >= max |w| over the sub-block
+ * (4 if none), written to shift_out[b * shift_stride + row]; codes = clip(rint(w / (scale * 2^e)), -7, 7), every step
+ * one fp32 operation, ties to even.  shift_stride is the row count of the whole exponent array (>= rows), so that a
+ * range of rows can be written into a larger buffer by offsetting the three output pointers.  Current device,
+ * asynchronous on the stream, allocates nothing. */
+hola_status hola_quantize_w4(const void* W_bf16, int rows, int H, void* packed_out, uint8_t* shift_out, int shift_stride,
+                             float* scale_out, void* cuda_stream);
 
 /* Launch geometry chosen for a shape (for reports): vocabulary rows per tile of a CTA pair, grid size (CTAs),
  * shared-memory ring slots, verify rows per pass, passes over W_lm, kernel launches per hola_verify call. */

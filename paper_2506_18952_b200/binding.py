@@ -17,13 +17,14 @@ HOLA_OK = 0
 HOLA_Q_BF16, HOLA_Q_F32 = 0, 1
 HOLA_GATE_TARGET_ENTROPY, HOLA_GATE_DRAFT_ENTROPY = 0, 1
 HOLA_FALLBACK_SAMPLE, HOLA_FALLBACK_GREEDY = 0, 1
-HOLA_W_BF16, HOLA_W_INT8, HOLA_W8A8, HOLA_W8A16 = 0, 1, 2, 3
+HOLA_W_BF16, HOLA_W_INT8, HOLA_W8A8, HOLA_W8A16, HOLA_W_MIXED = 0, 1, 2, 3, 4
+GROUP_ROWS, SUB_BLOCK = 256, 128
 FLAG_BAD_TOKEN, FLAG_BAD_UNIFORM, FLAG_TIMEOUT, FLAG_R_ZERO = 1, 2, 4, 8
 HOLA_OPT_RING_SLOTS, HOLA_OPT_ROTATING_UNITS, HOLA_OPT_HOST_OVERLAP, HOLA_OPT_HOST_ROWS_ON_DEMAND = 1, 2, 3, 4
 
 EXPORTS = ["hola_create", "hola_destroy", "hola_workspace_bytes", "hola_verify", "hola_verify_host",
            "hola_lm_head_entropy", "hola_accept_sample", "hola_host_traffic", "hola_shard_record_bytes", "hola_shard_lm_head",
-           "hola_shard_accept", "hola_shard_sample", "hola_lm_head_entropy_static", "hola_quantize_w8", "hola_plan", "hola_plan_ex", "hola_set_option", "hola_selftest_bounded_wait", "hola_profile_begin", "hola_profile_end", "hola_strerror", "hola_last_cuda_error",
+           "hola_shard_accept", "hola_shard_sample", "hola_lm_head_entropy_static", "hola_quantize_w8", "hola_quantize_w4", "hola_plan", "hola_plan_ex", "hola_set_option", "hola_selftest_bounded_wait", "hola_profile_begin", "hola_profile_end", "hola_strerror", "hola_last_cuda_error",
            "hola_version"]
 
 
@@ -39,7 +40,13 @@ class hola_verify_args(ctypes.Structure):
                 ("entropy", ctypes.c_void_p), ("logZ", ctypes.c_void_p), ("logits_out", ctypes.c_void_p),
                 ("status_word", ctypes.c_void_p), ("gate_source", ctypes.c_int32), ("fallback", ctypes.c_int32),
                 ("draft_entropy", ctypes.c_void_p), ("w_dtype", ctypes.c_int32), ("reserved_", ctypes.c_int32),
-                ("w_scale", ctypes.c_void_p)]
+                ("w_scale", ctypes.c_void_p), ("wmix", ctypes.c_void_p)]
+
+
+class hola_wmix(ctypes.Structure):
+    _fields_ = [("W16", ctypes.c_void_p), ("W8", ctypes.c_void_p), ("W4", ctypes.c_void_p), ("shift4", ctypes.c_void_p),
+                ("group_width", ctypes.c_void_p), ("group_row", ctypes.c_void_p), ("rows16", ctypes.c_int32),
+                ("rows8", ctypes.c_int32), ("rows4", ctypes.c_int32), ("reserved_", ctypes.c_int32)]
 
 
 class hola_shard_args(ctypes.Structure):
@@ -78,6 +85,9 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
     lib.hola_quantize_w8.restype = ctypes.c_int
     lib.hola_quantize_w8.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p,
                                      ctypes.c_void_p]
+    lib.hola_quantize_w4.restype = ctypes.c_int
+    lib.hola_quantize_w4.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p,
+                                     ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p]
     lib.hola_plan.restype = ctypes.c_int
     lib.hola_plan.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.POINTER(hola_plan_info)]
     lib.hola_plan_ex.restype = ctypes.c_int
@@ -141,6 +151,85 @@ def hola_quantize_w8(W_lm: torch.Tensor, stream=None):
         _check(lib, None, lib.hola_quantize_w8(_dptr(W_lm), V, H, _dptr(q), _dptr(scale), _stream_ptr(stream)),
                "hola_quantize_w8")
     return q, scale
+
+
+@dataclass
+class MixedHead:
+    """An LM head stored as groups of 256 vocabulary rows at 4, 8 or 16 bits (HOLA_W_MIXED): the device buffers and the
+    hola_wmix struct that points at them.  Keep the object alive while calls that use it are in flight."""
+    V: int
+    H: int
+    widths: list
+    W16: torch.Tensor | None
+    W8: torch.Tensor | None
+    W4: torch.Tensor | None
+    shift4: torch.Tensor | None
+    w_scale: torch.Tensor
+    group_width: torch.Tensor
+    group_row: torch.Tensor
+    struct: "hola_wmix" = None
+
+    def weight_bytes(self) -> int:
+        """Bytes of weights, scales and exponents one pass over the head streams."""
+        n = self.w_scale.numel() * 4
+        for t in (self.W16, self.W8, self.W4, self.shift4):
+            n += 0 if t is None else t.numel() * t.element_size()
+        return n
+
+
+def hola_quantize_mixed(W_lm: torch.Tensor, widths, stream=None) -> MixedHead:
+    """bf16 W_lm [V, H] -> the mixed-width form: widths[g] in {4, 8, 16} for group g of 256 vocabulary rows.  The codes,
+    scales and exponents are made by the library's quantiser kernels, each run of groups of one width in one launch that
+    writes straight into that width's compact buffer; 16-bit rows are copied as they are.  torch provides the buffers."""
+    if W_lm.dtype != torch.bfloat16 or not W_lm.is_cuda or not W_lm.is_contiguous():
+        raise HolaError("hola_quantize_mixed takes a contiguous bfloat16 device tensor")
+    lib = load_library()
+    V, H = W_lm.shape
+    ng = -(-V // GROUP_ROWS)
+    widths = [int(x) for x in widths]
+    if len(widths) != ng or any(x not in (4, 8, 16) for x in widths) or H % SUB_BLOCK:
+        raise HolaError(f"need {ng} widths out of 4, 8, 16 and H a multiple of {SUB_BLOCK}")
+    dev = W_lm.device
+    rows = {4: 0, 8: 0, 16: 0}
+    group_row = []
+    for g, wd in enumerate(widths):
+        group_row.append(rows[wd])
+        rows[wd] += min(V, (g + 1) * GROUP_ROWS) - g * GROUP_ROWS
+    W16 = torch.empty((rows[16], H), dtype=torch.bfloat16, device=dev) if rows[16] else None
+    W8 = torch.empty((rows[8], H), dtype=torch.int8, device=dev) if rows[8] else None
+    W4 = torch.empty((rows[4], H // 2), dtype=torch.uint8, device=dev) if rows[4] else None
+    shift4 = torch.zeros((H // SUB_BLOCK, rows[4]), dtype=torch.uint8, device=dev) if rows[4] else None
+    w_scale = torch.ones((V,), dtype=torch.float32, device=dev)
+    sp = _stream_ptr(stream)
+    with torch.cuda.device(dev):
+        g = 0
+        while g < ng:                                            # runs of consecutive groups of one width
+            g1 = g
+            while g1 < ng and widths[g1] == widths[g]:
+                g1 += 1
+            v0, v1 = g * GROUP_ROWS, min(V, g1 * GROUP_ROWS)
+            n, r0, wd = v1 - v0, group_row[g], widths[g]
+            src = ctypes.c_void_p(W_lm.data_ptr() + v0 * H * 2)
+            scale = ctypes.c_void_p(w_scale.data_ptr() + v0 * 4)
+            if wd == 16:
+                W16[r0:r0 + n].copy_(W_lm[v0:v1])
+            elif wd == 8:
+                _check(lib, None, lib.hola_quantize_w8(src, n, H, ctypes.c_void_p(W8.data_ptr() + r0 * H), scale, sp),
+                       "hola_quantize_w8")
+            else:
+                _check(lib, None, lib.hola_quantize_w4(src, n, H, ctypes.c_void_p(W4.data_ptr() + r0 * (H // 2)),
+                                                       ctypes.c_void_p(shift4.data_ptr() + r0), rows[4], scale, sp),
+                       "hola_quantize_w4")
+            g = g1
+    head = MixedHead(V, H, widths, W16, W8, W4, shift4, w_scale,
+                     torch.tensor(widths, dtype=torch.uint8, device=dev),
+                     torch.tensor(group_row, dtype=torch.int32, device=dev))
+    st = hola_wmix()
+    st.W16, st.W8, st.W4, st.shift4 = (t.data_ptr() if t is not None else None for t in (W16, W8, W4, shift4))
+    st.group_width, st.group_row = head.group_width.data_ptr(), head.group_row.data_ptr()
+    st.rows16, st.rows8, st.rows4 = rows[16], rows[8], rows[4]
+    head.struct = st
+    return head
 
 
 def hola_lm_head_entropy_static(hidden, W_lm, logits, entropy, logZ, stream=None, status=None) -> None:
@@ -253,9 +342,14 @@ class HolaVerify:
     def _args(self, hidden, W_lm, draft_tok, draft_q, uniforms, tau, out: VerifyOutputs, B, k,
               gate_source: int = HOLA_GATE_TARGET_ENTROPY, fallback: int = HOLA_FALLBACK_SAMPLE, w_scale=None,
               a8: bool = False):
-        if hidden.dtype != torch.bfloat16 or W_lm.dtype not in (torch.bfloat16, torch.int8):
+        mixed = W_lm if isinstance(W_lm, MixedHead) else None
+        if mixed is not None:
+            if mixed.V != self.V or mixed.H != self.H or w_scale is not None or a8:
+                raise HolaError("a MixedHead carries its own scales and takes bf16 activations; its shape must be the context's")
+            W_lm, w_scale = (mixed.W8 if mixed.W8 is not None else (mixed.W4 if mixed.W4 is not None else mixed.W16)), mixed.w_scale
+        if hidden.dtype != torch.bfloat16 or (mixed is None and W_lm.dtype not in (torch.bfloat16, torch.int8)):
             raise HolaError("hidden must be bfloat16, W_lm bfloat16 or int8")
-        if (W_lm.dtype == torch.int8) != (w_scale is not None):
+        if mixed is None and (W_lm.dtype == torch.int8) != (w_scale is not None):
             raise HolaError("an int8 W_lm goes with w_scale (fp32 per vocabulary row), a bfloat16 one without")
         if draft_q is not None and draft_q.dtype not in (torch.bfloat16, torch.float32):
             raise HolaError("draft_q must be bfloat16 or float32")
@@ -282,6 +376,9 @@ class HolaVerify:
         act = HOLA_W8A16 if a8 == "a16" else (HOLA_W8A8 if a8 else HOLA_W_INT8)
         a.w_dtype = act if w_scale is not None else HOLA_W_BF16
         a.w_scale = _dptr(w_scale)
+        if mixed is not None:
+            a.w_dtype, a.W_lm = HOLA_W_MIXED, None
+            a.wmix = ctypes.addressof(mixed.struct)
         return a
 
     def alloc_outputs(self, B: int, k: int, want_logits: bool = False, device=None) -> VerifyOutputs:
@@ -341,7 +438,7 @@ class HolaVerify:
         """End-to-end form: per-step inputs and all outputs are HOST tensors (pinned for async copies);
         W_lm is the resident device weight.  Returns after the stream has been synchronised."""
         B, k = hidden.shape[0], hidden.shape[1] - 1
-        if W_lm.device.type != "cuda":
+        if not isinstance(W_lm, MixedHead) and W_lm.device.type != "cuda":
             raise HolaError("W_lm must be resident on the device")
         for t in (hidden, draft_tok, draft_q, uniforms):
             if t is not None and t.device.type != "cpu":

@@ -60,6 +60,8 @@ constexpr int kTransBytes = kTransRows * 32 * 4; // its staging buffer: [16 rows
 // converter warps expand it to the bf16 tile the MMA reads.  Warps 2..9 are epilogue warps, warp 14 loads the
 // hidden blocks, warps 10..13 and 15..17 convert.
 constexpr int kRawBlockBytes = kLanes * kBlockK;  // int8 [128][64]
+constexpr int kSubBlock = 128;                    // hidden channels per 4-bit sub-block (one shared exponent each)
+constexpr int kGroupRows = 256;                   // vocabulary rows per group of one width
 constexpr int kW8EpiWarps = 8;
 constexpr int kW8HiddenWarp = 14;
 constexpr int kConvWarps = (kW8HiddenWarp - 2 - kW8EpiWarps) + (kK1Warps - kW8HiddenWarp - 1);   // 4 + 3
@@ -94,6 +96,13 @@ struct K1Params {
   const float* w_scale;   // 8-bit W_lm: fp32 scale per vocabulary row, applied to the accumulators
   const float* h_scale;   // 8-bit activations (modes 2, 3): fp32 scale per verify row (mode 3: of the coarse plane)
   const float* h_scale2;  // mode 3: scale of the second plane
+  // Mode 1 with vocabulary groups of mixed width (null: every row is 8-bit and lives at its own index in W_lm): width
+  // (4, 8 or 16) of each group of 256 vocabulary rows, first row of the group inside the buffer of its width, and the
+  // exponents of the 4-bit sub-blocks, [sub-block][row of the 4-bit buffer].
+  const uint8_t* group_width;
+  const int* group_row;
+  const uint8_t* shift4;
+  int rows4;
   int stream_logits;      // 1: store the logits with the streaming hint (they exceed what the L2 keeps until they are read)
   float* logits;
   float4* partials;   // [grid][part_stride] (m, s, t, arg-max index)
@@ -508,6 +517,31 @@ __device__ __forceinline__ void expand_int8x16(const uint4 x, uint8_t* tile, int
   *reinterpret_cast<uint4*>(drow + (((2 * c + 1) ^ (row & 7)) << 4)) = make_uint4(o[4], o[5], o[6], o[7]);
 }
 
+// Thirty-two 4-bit codes (one 16-byte piece c, 0 or 1, of row `row` of the raw block; two's complement nibbles, even
+// entry in the low nibble) -> thirty-two bf16 values  code << shift  at their place in the 128-byte-swizzled K-major
+// tile: chunks 4c .. 4c+3 of the row, each XOR-ed with row % 8.  Every value (magnitude <= 7 * 2^4) is exact in bf16.
+__device__ __forceinline__ void expand_int4x32(const uint4 x, uint8_t* tile, int row, int c, int shift) {
+  const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+  // nibble n (as unsigned, after flipping its sign bit: n ^ 8 = code + 8) in the low mantissa bits of 2^23 is the float
+  // 2^23 + code + 8; times 2^shift minus (2^23 + 8) 2^shift leaves code * 2^shift, all exact.
+  const float mul = __int_as_float((127 + shift) << 23);
+  const float sub = -(8388608.f + 8.f) * mul;
+  uint8_t* drow = tile + (row >> 3) * 1024 + (row & 7) * 128;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const uint32_t u = w[j] ^ 0x88888888u;
+    uint32_t o[4];
+#pragma unroll
+    for (int h = 0; h < 4; ++h) {
+      const float f0 = fmaf(__uint_as_float(0x4B000000u | ((u >> (8 * h)) & 0xFu)), mul, sub);
+      const float f1 = fmaf(__uint_as_float(0x4B000000u | ((u >> (8 * h + 4)) & 0xFu)), mul, sub);
+      const __nv_bfloat162 b = __floats2bfloat162_rn(f0, f1);
+      o[h] = *reinterpret_cast<const uint32_t*>(&b);
+    }
+    *reinterpret_cast<uint4*>(drow + (((4 * c + j) ^ (row & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+}
+
 // A logit on its way to the buffer.  Only one verify row per sequence is ever read back (row accept_len, by the
 // accept/sample kernel); when the buffer is much larger than the L2 the streaming hint lets the lines leave early
 // instead of displacing what the next kernel reads.
@@ -548,6 +582,7 @@ __device__ __forceinline__ float scaled(float acc, float w_scale, const float* h
 template <int kMode, bool kRot>
 __global__ void __launch_bounds__(kK1Threads, 1)
 lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __grid_constant__ CUtensorMap tmap_w,
+                       const __grid_constant__ CUtensorMap tmap_w4, const __grid_constant__ CUtensorMap tmap_w16,
                        const K1Params p) {
   constexpr bool kW8 = kMode == 1;
   constexpr bool kI8 = kMode >= 2;                       // both operands 8-bit, 8-bit MMA kind
@@ -626,15 +661,30 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
       grid_dependency_wait();                            // W_lm and the hidden rows may come from the kernel before
       for (int t = 0; t < my_tiles && ok; ++t) {
         const int v0 = (pair + t * npairs) * pair_rows + static_cast<int>(rank) * p.tile_rows;
+        int tile_width = 8, w_row = v0;                  // (mode 1) width of this tile's rows and where they are stored
+        if (kW8 && p.group_width) {
+          const int g = pair + t * npairs;
+          tile_width = p.group_width[g];
+          w_row = p.group_row[g] + static_cast<int>(rank) * p.tile_rows;
+        }
         int kx = 0;                                      // K coordinate of the block, in elements
         for (int kb = 0; kb < p.n_kblocks; ++kb, kx += kKStep) {
           const uint32_t sa = base + stage * stage_bytes;
           if (kW8) {
-            // only the int8 tile: its slot is free again as soon as the converters have read it
+            // only the raw tile: its slot is free again as soon as the converters have read it
             if (!mbar_wait(rawempty_bar + 8 * stage, phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
             const uint32_t rb = own_rawfull + 8 * stage;
-            mbar_expect_tx_cluster(rb, raw_tx_bytes);
-            tma_load_2d(sa + raw_off, &tmap_w, rb, kx, v0, pol_w);
+            if (tile_width == 8) {
+              mbar_expect_tx_cluster(rb, raw_tx_bytes);
+              tma_load_2d(sa + raw_off, &tmap_w, rb, kx, w_row, pol_w);
+            } else if (tile_width == 4) {                  // two codes per byte: 32 bytes per row and K block
+              mbar_expect_tx_cluster(rb, raw_tx_bytes >> 1);
+              tma_load_2d(sa + raw_off, &tmap_w4, rb, kx >> 1, w_row, pol_w);
+            } else {                                       // bf16 rows go straight into the tile the MMA reads,
+              if (!mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
+              mbar_expect_tx_cluster(rb, raw_tx_bytes << 1);   // once the MMAs of its previous use are done
+              tma_load_2d(sa, &tmap_w16, rb, kx, w_row, pol_w);
+            }
           } else {
             if (!mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
             const uint32_t fb = leader_full + 8 * stage;
@@ -1040,25 +1090,45 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
     int stage = 0;
     uint32_t phase = 0;
     bool ok = true;
+    grid_dependency_wait();                              // the width table and the exponents may come from the kernel before
     for (int t = 0; t < my_tiles && ok; ++t) {
+      int tile_width = 8, w_row = 0;                     // width of this tile's rows; first row in the 4-bit buffer
+      if (p.group_width) {
+        const int g = pair + t * npairs;
+        tile_width = p.group_width[g];
+        w_row = p.group_row[g] + static_cast<int>(rank) * p.tile_rows;
+      }
       for (int kb = 0; kb < p.n_kblocks; ++kb) {
         if (!mbar_wait_warp(rawfull_bar + 8 * stage, phase, abort_flag, p.status) ||
             !mbar_wait_warp(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
         uint8_t* slot = smem + stage * stage_bytes;
-        for (int u0 = ct; u0 < units; u0 += 2 * kConvThreads) {
-          const int u1 = u0 + kConvThreads;
-          const bool has1 = u1 < units;
-          const uint4 x0 = *reinterpret_cast<const uint4*>(slot + raw_off + (u0 >> 2) * 64 + (u0 & 3) * 16);
-          uint4 x1 = make_uint4(0u, 0u, 0u, 0u);
-          if (has1) x1 = *reinterpret_cast<const uint4*>(slot + raw_off + (u1 >> 2) * 64 + (u1 & 3) * 16);
-          expand_int8x16(x0, slot, u0 >> 2, u0 & 3);
-          if (has1) expand_int8x16(x1, slot, u1 >> 2, u1 & 3);
+        if (tile_width == 8) {
+          for (int u0 = ct; u0 < units; u0 += 2 * kConvThreads) {
+            const int u1 = u0 + kConvThreads;
+            const bool has1 = u1 < units;
+            const uint4 x0 = *reinterpret_cast<const uint4*>(slot + raw_off + (u0 >> 2) * 64 + (u0 & 3) * 16);
+            uint4 x1 = make_uint4(0u, 0u, 0u, 0u);
+            if (has1) x1 = *reinterpret_cast<const uint4*>(slot + raw_off + (u1 >> 2) * 64 + (u1 & 3) * 16);
+            expand_int8x16(x0, slot, u0 >> 2, u0 & 3);
+            if (has1) expand_int8x16(x1, slot, u1 >> 2, u1 & 3);
+          }
+        } else if (tile_width == 4) {
+          // 32-byte rows: two 16-byte pieces per row; a sub-block of 128 hidden channels spans two K blocks
+          const uint8_t* sh = p.shift4 + static_cast<size_t>(kb >> 1) * p.rows4;
+          for (int u0 = ct; u0 < (units >> 1); u0 += kConvThreads) {
+            const int row = u0 >> 1, c = u0 & 1;
+            const uint4 x0 = *reinterpret_cast<const uint4*>(slot + raw_off + row * 32 + c * 16);
+            const int r4 = w_row + row;
+            const int shift = (r4 >= 0 && r4 < p.rows4) ? min(static_cast<int>(sh[r4]), 4) : 0;
+            expand_int4x32(x0, slot, row, c, shift);
+          }
         }
+        // (16-bit rows were loaded into the tile as they are)
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // generic-proxy writes, read by the MMA
         __syncwarp();
         if (lane == 0) {
           mbar_arrive_cluster(leader_full + 8 * stage);  // this warp's share of the bf16 tile is in place
-          mbar_arrive(rawempty_bar + 8 * stage);         // and the int8 block may be refilled
+          mbar_arrive(rawempty_bar + 8 * stage);         // and the raw block may be refilled
         }
         if (++stage == p.stages) { stage = 0; phase ^= 1u; }
       }
@@ -1627,6 +1697,57 @@ __global__ void __launch_bounds__(256) quantize_rows_int8_kernel(const __nv_bflo
   }
 }
 
+// The 4-bit case of the Lo-Bi quantiser on the LM head (reading: a sub-block is 128 hidden channels of one vocabulary
+// row; symmetric codes in [-7, 7]; the sub-block's scale is the row's fp32 scale times a power of two):
+//   s = max|w| / 112 (1 for an all-zero row);  e_b = the smallest e in 0..4 with  7 * 2^e * s >= max_{h in b} |w|  (else 4);
+//   c = clip(rint(w / (s * 2^e_b)), -7, 7),  every step one fp32 operation, ties to even.
+// Two codes per byte (even channel in the low nibble, 4-bit two's complement).  Exponents go to
+// shift[b * shift_stride + row].  One CTA per row; warp w takes sub-blocks w, w + 8, ...; a lane holds four channels.
+__global__ void __launch_bounds__(256) quantize_rows_w4_kernel(const __nv_bfloat16* W, int H, uint8_t* packed,
+                                                               uint8_t* shift, int shift_stride, float* scale) {
+  __shared__ float sh_max[8];
+  __shared__ float sh_scale;
+  const size_t row = blockIdx.x;
+  const __nv_bfloat16* wr = W + row * H;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  float amax = 0.f;
+  for (int h = threadIdx.x; h < H; h += 256) amax = fmaxf(amax, fabsf(__bfloat162float(wr[h])));
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, off));
+  if (lane == 0) sh_max[warp] = amax;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float m = 0.f;
+    for (int i = 0; i < 8; ++i) m = fmaxf(m, sh_max[i]);
+    const float sc = m > 0.f ? __fdiv_rn(m, 112.f) : 1.f;
+    sh_scale = sc;
+    scale[row] = sc;
+  }
+  __syncthreads();
+  const float sc = sh_scale;
+  for (int b = warp; b < H / kSubBlock; b += 8) {
+    float w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) w[i] = __bfloat162float(wr[b * kSubBlock + lane * 4 + i]);
+    float bmax = fmaxf(fmaxf(fabsf(w[0]), fabsf(w[1])), fmaxf(fabsf(w[2]), fabsf(w[3])));
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, off));
+    int e = 4;
+#pragma unroll
+    for (int c = 3; c >= 0; --c)
+      if (__fmul_rn(sc, static_cast<float>(7 << c)) >= bmax) e = c;
+    const float step = sc * static_cast<float>(1 << e);              // exact
+    uint32_t bits = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float r = fminf(7.f, fmaxf(-7.f, rintf(__fdiv_rn(w[i], step))));
+      bits |= (static_cast<uint32_t>(static_cast<int>(r)) & 0xFu) << (4 * i);
+    }
+    *reinterpret_cast<uint16_t*>(packed + row * (H / 2) + b * (kSubBlock / 2) + lane * 2) = static_cast<uint16_t>(bits);
+    if (lane == 0) shift[static_cast<size_t>(b) * shift_stride + row] = static_cast<uint8_t>(e);
+  }
+}
+
 // Hidden rows as two 8-bit planes (16-bit-class activations for the 8-bit MMA kind): per verify row
 //   s1 = max|x| / 127 (1 if zero), q1 = clip(rint(x / s1));  r = x - s1 q1;  s2 = s1 / 254, q2 = clip(rint(r / s2)),
 // every step one fp32 operation.  Operand layout: blocks of 32 verify rows, each block as 32 rows of q1 followed by
@@ -1771,7 +1892,8 @@ struct Plan {
 // What a call needs besides its arguments, kept from one call to the next: the launch geometry of a (rows, weight
 // mode) pair and the two tensor maps of a (hidden pointer, W_lm pointer, rows, weight mode) quadruple.
 struct PlanEntry { int valid, M, w_dtype; Plan pl; };
-struct MapEntry { int valid, M, w_dtype; const void* hidden; const void* W; CUtensorMap th, tw; };
+struct MapEntry { int valid, M, w_dtype; const void* hidden; const void* W; const void* W4; const void* W16;
+                  CUtensorMap th, tw, tw4, tw16; };
 constexpr int kPlanCache = 8, kMapCache = 8;
 
 struct hola_ctx {
@@ -1875,7 +1997,8 @@ int round_up(int x, int a) { return (x + a - 1) / a * a; }
 // A pass holds at most 512 rows (two MMAs of N <= 256 fill the tensor memory); N is a multiple of 16.
 // Cost per pass: the slower of streaming W_lm once and the padded rows' tensor time, plus a fixed launch cost.
 Plan make_plan(const hola_ctx* ctx, int M, int w_dtype = HOLA_W_BF16) {
-  const bool w8 = w_dtype == HOLA_W_INT8;        // int8 W_lm expanded on chip
+  const bool mixed = w_dtype == HOLA_W_MIXED;    // vocabulary groups of 4-, 8- and 16-bit rows, expanded on chip
+  const bool w8 = w_dtype == HOLA_W_INT8 || mixed;   // int8 W_lm expanded on chip
   const bool two = w_dtype == HOLA_W8A16;        // as W8A8, with two operand rows per verify row
   const bool i8 = w_dtype == HOLA_W8A8 || two;   // 8-bit MMA: N a multiple of 32, K blocks of 128, twice the rate
   Plan best{};
@@ -1923,6 +2046,7 @@ Plan make_plan(const hola_ctx* ctx, int M, int w_dtype = HOLA_W_BF16) {
   int tile_rows = round_up((ctx->V + 2 * pairs * rounds - 1) / (2 * pairs * rounds), 4);
   if (tile_rows < 8) tile_rows = 8;
   if (tile_rows > kLanes) tile_rows = kLanes;
+  if (mixed) tile_rows = kLanes;                 // a pair's tile is one group of 256 rows of one width
   best.tile_rows = tile_rows;
   best.n_ptiles = (ctx->V + 2 * tile_rows - 1) / (2 * tile_rows);
   best.grid = 2 * (best.n_ptiles < pairs ? best.n_ptiles : pairs);
@@ -1946,11 +2070,14 @@ const Plan& plan_for(hola_ctx* ctx, int M, int w_dtype) {
 // K-major 2-D tensor map with a box of 64 elements x box_rows.  bf16: 128-byte swizzle (the layout the MMA reads);
 // int8: plain rows of 64 bytes (the converter warps read them).
 // int8 with swizzle (8-bit MMA): box of 128 elements = 128 bytes, 128-byte swizzle, the same bytes as a bf16 block.
+// `packed4`: rows of cols / 2 bytes holding two 4-bit codes each; box of 32 bytes (64 codes) x box_rows, plain rows.
 hola_status encode_map(hola_ctx* ctx, CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols,
-                       uint32_t box_rows, bool int8 = false, bool int8_swizzled = false) {
+                       uint32_t box_rows, bool int8 = false, bool int8_swizzled = false, bool packed4 = false) {
+  if (packed4) { cols /= 2; int8 = true; int8_swizzled = false; }
   const cuuint64_t dims[2] = {cols, rows};
   const cuuint64_t strides[1] = {cols * (int8 ? 1u : 2u)};
-  const cuuint32_t box[2] = {static_cast<cuuint32_t>(int8_swizzled ? 2 * kBlockK : kBlockK), box_rows};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(packed4 ? kBlockK / 2 : (int8_swizzled ? 2 * kBlockK : kBlockK)),
+                             box_rows};
   const cuuint32_t estr[2] = {1, 1};
   const CUresult r = ctx->encode(map, int8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
                                  const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
@@ -1980,7 +2107,12 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 hola_status run_lm_head(hola_ctx* ctx, const hola_verify_args* a, float* logits, int ldl, const Plan& pl,
                         cudaStream_t stream) {
   const int M = a->B * (a->k + 1);
-  const bool w8 = a->w_dtype == HOLA_W_INT8, two = a->w_dtype == HOLA_W8A16, i8 = a->w_dtype == HOLA_W8A8 || two;
+  const bool mixed = a->w_dtype == HOLA_W_MIXED;
+  const bool w8 = a->w_dtype == HOLA_W_INT8 || mixed, two = a->w_dtype == HOLA_W8A16,
+             i8 = a->w_dtype == HOLA_W8A8 || two;
+  const hola_wmix* mx = mixed ? a->wmix : nullptr;
+  // (mixed widths: W_lm of the arguments is not read; the 8-bit buffer takes its place in the cache key and the map)
+  const void* w_main = mixed ? (mx->rows8 > 0 ? mx->W8 : (mx->rows4 > 0 ? mx->W4 : mx->W16)) : a->W_lm;
   hola_status s;
   // 8-bit activations: the hidden operand is the context's own buffer of 8-bit planes, filled per call below
   const void* hid_src = (two || i8) ? static_cast<const void*>(ctx->hid8) : a->hidden;
@@ -2004,7 +2136,8 @@ hola_status run_lm_head(hola_ctx* ctx, const hola_verify_args* a, float* logits,
   MapEntry* me = nullptr;
   for (int i = 0; i < kMapCache; ++i) {
     MapEntry& c = ctx->maps[i];
-    if (c.valid && c.hidden == hid_src && c.W == a->W_lm && c.M == M && c.w_dtype == a->w_dtype) { me = &c; break; }
+    if (c.valid && c.hidden == hid_src && c.W == w_main && c.M == M && c.w_dtype == a->w_dtype &&
+        (!mixed || (c.W4 == mx->W4 && c.W16 == mx->W16))) { me = &c; break; }
   }
   if (!me) {
     me = &ctx->maps[ctx->map_next];
@@ -2020,13 +2153,43 @@ hola_status run_lm_head(hola_ctx* ctx, const hola_verify_args* a, float* logits,
       s = encode_map(ctx, &me->th, hid_src, static_cast<uint64_t>(M), static_cast<uint64_t>(a->H),
                      static_cast<uint32_t>(pl.N / 2));
     if (s != HOLA_OK) return s;
-    s = encode_map(ctx, &me->tw, a->W_lm, static_cast<uint64_t>(a->V), static_cast<uint64_t>(a->H),
-                   static_cast<uint32_t>(pl.tile_rows), w8 || i8, i8);
-    if (s != HOLA_OK) return s;
-    me->hidden = hid_src; me->W = a->W_lm; me->M = M; me->w_dtype = a->w_dtype; me->valid = 1;
+    const uint32_t trows = static_cast<uint32_t>(pl.tile_rows);
+    if (!mixed) {
+      s = encode_map(ctx, &me->tw, a->W_lm, static_cast<uint64_t>(a->V), static_cast<uint64_t>(a->H), trows, w8 || i8, i8);
+      if (s != HOLA_OK) return s;
+      me->tw4 = me->tw; me->tw16 = me->tw;               // (never read outside the mixed-width form)
+      me->W4 = nullptr; me->W16 = nullptr;
+    } else {
+      // one map per width that occurs; a width that does not occur gets a copy of one that does (never used)
+      bool have = false;
+      if (mx->rows8 > 0) {
+        s = encode_map(ctx, &me->tw, mx->W8, static_cast<uint64_t>(mx->rows8), static_cast<uint64_t>(a->H), trows, true);
+        if (s != HOLA_OK) return s;
+        have = true;
+      }
+      if (mx->rows4 > 0) {
+        s = encode_map(ctx, &me->tw4, mx->W4, static_cast<uint64_t>(mx->rows4), static_cast<uint64_t>(a->H), trows, true,
+                       false, true);
+        if (s != HOLA_OK) return s;
+        if (!have) me->tw = me->tw4;
+        have = true;
+      }
+      if (mx->rows16 > 0) {
+        s = encode_map(ctx, &me->tw16, mx->W16, static_cast<uint64_t>(mx->rows16), static_cast<uint64_t>(a->H), trows);
+        if (s != HOLA_OK) return s;
+        if (!have) me->tw = me->tw16;
+        have = true;
+      }
+      if (mx->rows4 <= 0) me->tw4 = me->tw;
+      if (mx->rows16 <= 0) me->tw16 = me->tw;
+      me->W4 = mx->W4; me->W16 = mx->W16;
+    }
+    me->hidden = hid_src; me->W = w_main; me->M = M; me->w_dtype = a->w_dtype; me->valid = 1;
   }
   const CUtensorMap& th = me->th;
   const CUtensorMap& tw = me->tw;
+  const CUtensorMap& tw4 = me->tw4;
+  const CUtensorMap& tw16 = me->tw16;
   K1Params kp;
   kp.M = M; kp.V = a->V; kp.n_ptiles = pl.n_ptiles; kp.n_kblocks = pl.n_kblocks;
   kp.stages = pl.stages; kp.nbuf = pl.nbuf; kp.rot = pl.rot; kp.n_sub = pl.n_sub; kp.N = pl.N; kp.tile_rows = pl.tile_rows; kp.ldl = ldl;
@@ -2036,6 +2199,10 @@ hola_status run_lm_head(hola_ctx* ctx, const hola_verify_args* a, float* logits,
   kp.h_scale = ctx->hid_scale;
   kp.h_scale2 = ctx->hid_scale ? ctx->hid_scale + ctx->max_rows : nullptr;
   kp.stream_logits = static_cast<double>(M) * a->V * 4.0 > 96e6 ? 1 : 0;     // beyond ~3/4 of the L2
+  kp.group_width = mixed ? mx->group_width : nullptr;
+  kp.group_row = mixed ? mx->group_row : nullptr;
+  kp.shift4 = mixed ? mx->shift4 : nullptr;
+  kp.rows4 = mixed ? mx->rows4 : 0;
   cudaError_t e = cudaSuccess;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(static_cast<unsigned>(pl.grid));
@@ -2057,12 +2224,12 @@ hola_status run_lm_head(hola_ctx* ctx, const hola_verify_args* a, float* logits,
     kp.row0 = pass * pl.rows_per_pass;
     kp.rows = M - kp.row0 < pl.rows_per_pass ? M - kp.row0 : pl.rows_per_pass;
     if (kp.rows <= 0) break;
-    e = two ? cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<3, false>, th, tw, kp)
-      : i8 ? (pl.rot ? cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<2, true>, th, tw, kp)
-                     : cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<2, false>, th, tw, kp))
-      : w8 ? cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<1, false>, th, tw, kp)
-           : (pl.rot ? cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<0, true>, th, tw, kp)
-                     : cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<0, false>, th, tw, kp));
+    e = two ? cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<3, false>, th, tw, tw4, tw16, kp)
+      : i8 ? (pl.rot ? cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<2, true>, th, tw, tw4, tw16, kp)
+                     : cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<2, false>, th, tw, tw4, tw16, kp))
+      : w8 ? cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<1, false>, th, tw, tw4, tw16, kp)
+           : (pl.rot ? cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<0, true>, th, tw, tw4, tw16, kp)
+                     : cudaLaunchKernelEx(&cfg, lm_head_entropy_kernel<0, false>, th, tw, tw4, tw16, kp));
     if (e != cudaSuccess) { set_error(ctx, "launch lm_head_entropy_kernel", e); return HOLA_ERR_CUDA; }
   }
   return HOLA_OK;
@@ -2144,10 +2311,22 @@ hola_status run_accept_sample(hola_ctx* ctx, const hola_verify_args* a, const fl
 }
 
 hola_status check_lm_head_args(const hola_ctx* ctx, const hola_verify_args* a) {
+  if (a->w_dtype < HOLA_W_BF16 || a->w_dtype > HOLA_W_MIXED) return HOLA_ERR_INVALID_ARG;
+  if (a->w_dtype == HOLA_W_MIXED) {
+    // vocabulary groups of mixed width: the weights come through args->wmix, W_lm is not read
+    const hola_wmix* mx = a->wmix;
+    if (!a->hidden || !aligned16(a->hidden) || !mx || !a->w_scale) return HOLA_ERR_INVALID_ARG;
+    if (a->H % kSubBlock != 0) return HOLA_ERR_UNSUPPORTED_SHAPE;          // whole sub-blocks of 128 hidden channels
+    if (mx->rows4 < 0 || mx->rows8 < 0 || mx->rows16 < 0 || !mx->group_width || !mx->group_row) return HOLA_ERR_INVALID_ARG;
+    if (static_cast<long long>(mx->rows4) + mx->rows8 + mx->rows16 < a->V) return HOLA_ERR_INVALID_ARG;
+    if ((mx->rows4 > 0 && (!mx->W4 || !mx->shift4 || !aligned16(mx->W4))) || (mx->rows8 > 0 && (!mx->W8 || !aligned16(mx->W8))) ||
+        (mx->rows16 > 0 && (!mx->W16 || !aligned16(mx->W16))))
+      return HOLA_ERR_INVALID_ARG;
+    return HOLA_OK;
+  }
   if (!a->hidden || !a->W_lm) return HOLA_ERR_INVALID_ARG;
   if (!aligned16(a->hidden) || !aligned16(a->W_lm)) return HOLA_ERR_INVALID_ARG;
   if (a->H % 8 != 0) return HOLA_ERR_UNSUPPORTED_SHAPE;
-  if (a->w_dtype < HOLA_W_BF16 || a->w_dtype > HOLA_W8A16) return HOLA_ERR_INVALID_ARG;
   if (a->w_dtype != HOLA_W_BF16) {
     if (!a->w_scale) return HOLA_ERR_INVALID_ARG;
     if (a->H % 16 != 0) return HOLA_ERR_UNSUPPORTED_SHAPE;     // int8 row pitch must be a multiple of 16 bytes
@@ -2300,7 +2479,7 @@ hola_status hola_destroy(hola_ctx* ctx) {
 
 hola_status hola_plan_ex(const hola_ctx* ctx, int B, int k, int w_dtype, hola_plan_info* out) {
   if (!ctx || !out || B < 0 || k < 0) return HOLA_ERR_INVALID_ARG;
-  if (w_dtype < HOLA_W_BF16 || w_dtype > HOLA_W8A16) return HOLA_ERR_INVALID_ARG;
+  if (w_dtype < HOLA_W_BF16 || w_dtype > HOLA_W_MIXED) return HOLA_ERR_INVALID_ARG;
   if (B > ctx->maxB || k > ctx->maxK) return HOLA_ERR_UNSUPPORTED_SHAPE;
   const Plan pl = make_plan(ctx, B * (k + 1), w_dtype);
   out->tile_v = 2 * pl.tile_rows; out->grid = pl.grid; out->stages = pl.stages; out->rows_per_pass = pl.rows_per_pass;
@@ -2741,6 +2920,16 @@ hola_status hola_host_traffic(const hola_ctx* ctx, unsigned long long* h2d_bytes
   if (!ctx || !h2d_bytes || !d2h_bytes) return HOLA_ERR_INVALID_ARG;
   *h2d_bytes = ctx->last_h2d; *d2h_bytes = ctx->last_d2h;
   return HOLA_OK;
+}
+
+hola_status hola_quantize_w4(const void* W_bf16, int rows, int H, void* packed_out, uint8_t* shift_out, int shift_stride,
+                             float* scale_out, void* cuda_stream) {
+  if (!W_bf16 || !packed_out || !shift_out || !scale_out || rows <= 0 || H <= 0 || shift_stride < rows)
+    return HOLA_ERR_INVALID_ARG;
+  if (H % kSubBlock != 0) return HOLA_ERR_UNSUPPORTED_SHAPE;
+  quantize_rows_w4_kernel<<<static_cast<unsigned>(rows), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+      static_cast<const __nv_bfloat16*>(W_bf16), H, static_cast<uint8_t*>(packed_out), shift_out, shift_stride, scale_out);
+  return cudaGetLastError() == cudaSuccess ? HOLA_OK : HOLA_ERR_CUDA;
 }
 
 hola_status hola_quantize_w8(const void* W_bf16, int V, int H, void* q_out, float* scale_out, void* cuda_stream) {

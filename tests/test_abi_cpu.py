@@ -43,8 +43,9 @@ def test_strerror_version_and_workspace(lib):
 def test_struct_layout_matches_header():
     from paper_2506_18952_b200 import binding
     a = binding.hola_verify_args
-    # 4 int32, 4 pointers, int32 (+pad), pointer, float (+pad), 6 pointers, 2 int32, pointer, 2 int32, pointer
-    assert ctypes.sizeof(a) == 16 + 4 * 8 + 8 + 8 + 8 + 6 * 8 + 8 + 8 + 8 + 8
+    # 4 int32, 4 pointers, int32 (+pad), pointer, float (+pad), 6 pointers, 2 int32, pointer, 2 int32, 2 pointers
+    assert ctypes.sizeof(a) == 16 + 4 * 8 + 8 + 8 + 8 + 6 * 8 + 8 + 8 + 8 + 8 + 8
+    assert a.wmix.offset == 152 and ctypes.sizeof(binding.hola_wmix) == 6 * 8 + 4 * 4
     assert a.w_dtype.offset == 136 and a.w_scale.offset == 144
     assert a.gate_source.offset == 120 and a.fallback.offset == 124 and a.draft_entropy.offset == 128
     assert a.uniforms.offset == 56 and a.tau.offset == 64 and a.accept_len.offset == 72
