@@ -493,24 +493,33 @@ __device__ __forceinline__ void stats_fold16_packed(const float* v, int vocab0, 
   st.t += fmaf(-m, sc, aa + ab);
 }
 
+// Integer codes to bf16 without conversion instructions: 0x4300 | n is the bf16 number 128 + n for 0 <= n < 128 (seven
+// mantissa bits, unit steps), two such numbers sit in one register, and one packed bf16 subtraction or multiply-add
+// (exact: every intermediate is an integer of at most eight bits) leaves the codes themselves.
+__device__ __forceinline__ uint32_t bf16x2_sub(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("sub.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+__device__ __forceinline__ uint32_t bf16x2_fma(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t d;
+  asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
+
 // Sixteen int8 values (one 16-byte piece c of row `row` of the raw block) -> sixteen bf16 values at their place in
 // the 128-byte-swizzled K-major tile that starts at `tile`: chunk 2c and 2c+1 of the row, each XOR-ed with row % 8.
 __device__ __forceinline__ void expand_int8x16(const uint4 x, uint8_t* tile, int row, int c) {
   const uint32_t w[4] = {x.x, x.y, x.z, x.w};
   uint32_t o[8];
-  // int8 -> float without conversion instructions: byte b + 128 placed in the low mantissa bits of 2^23 gives the
-  // float 2^23 + 128 + b exactly; one subtraction leaves b.  Two such floats pack into a bf16 pair (exact: |b| <= 128).
-  constexpr float kMagic = 8388608.f + 128.f;
+  // byte b as n = b + 128 in 0..255 = 128 hi + lo:  b = (128 + lo) - (hi ? 128 : 256); the subtrahend's bits are
+  // 0x4380 (256) with bit 7 cleared when hi is set (0x4300 = 128)
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
     const uint32_t u = w[j] ^ 0x80808080u;
-    const float f0 = __uint_as_float(__byte_perm(u, 0x4B000000u, 0x7650)) - kMagic;
-    const float f1 = __uint_as_float(__byte_perm(u, 0x4B000000u, 0x7651)) - kMagic;
-    const float f2 = __uint_as_float(__byte_perm(u, 0x4B000000u, 0x7652)) - kMagic;
-    const float f3 = __uint_as_float(__byte_perm(u, 0x4B000000u, 0x7653)) - kMagic;
-    const __nv_bfloat162 a = __floats2bfloat162_rn(f0, f1), b = __floats2bfloat162_rn(f2, f3);
-    o[2 * j] = *reinterpret_cast<const uint32_t*>(&a);
-    o[2 * j + 1] = *reinterpret_cast<const uint32_t*>(&b);
+    const uint32_t t0 = __byte_perm(u, 0u, 0x4140), t1 = __byte_perm(u, 0u, 0x4342);   // bytes 0,1 and 2,3 in 16-bit lanes
+    o[2 * j] = bf16x2_sub((t0 & 0x007F007Fu) | 0x43004300u, (t0 & 0x00800080u) ^ 0x43804380u);
+    o[2 * j + 1] = bf16x2_sub((t1 & 0x007F007Fu) | 0x43004300u, (t1 & 0x00800080u) ^ 0x43804380u);
   }
   uint8_t* drow = tile + (row >> 3) * 1024 + (row & 7) * 128;
   *reinterpret_cast<uint4*>(drow + (((2 * c) ^ (row & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
@@ -522,23 +531,24 @@ __device__ __forceinline__ void expand_int8x16(const uint4 x, uint8_t* tile, int
 // tile: chunks 4c .. 4c+3 of the row, each XOR-ed with row % 8.  Every value (magnitude <= 7 * 2^4) is exact in bf16.
 __device__ __forceinline__ void expand_int4x32(const uint4 x, uint8_t* tile, int row, int c, int shift) {
   const uint32_t w[4] = {x.x, x.y, x.z, x.w};
-  // nibble n (as unsigned, after flipping its sign bit: n ^ 8 = code + 8) in the low mantissa bits of 2^23 is the float
-  // 2^23 + code + 8; times 2^shift minus (2^23 + 8) 2^shift leaves code * 2^shift, all exact.
-  const float mul = __int_as_float((127 + shift) << 23);
-  const float sub = -(8388608.f + 8.f) * mul;
+  // nibble n with its sign bit flipped is code + 8; (128 + code + 8) * 2^shift - 136 * 2^shift = code * 2^shift
+  const uint32_t mul1 = static_cast<uint32_t>(127 + shift) << 7;           // bf16 bits of 2^shift
+  const uint32_t mul = mul1 | (mul1 << 16);
+  const uint32_t sub1 = 0xC308u + (static_cast<uint32_t>(shift) << 7);     // bf16 bits of -136 * 2^shift
+  const uint32_t sub = sub1 | (sub1 << 16);
   uint8_t* drow = tile + (row >> 3) * 1024 + (row & 7) * 128;
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
     const uint32_t u = w[j] ^ 0x88888888u;
-    uint32_t o[4];
-#pragma unroll
-    for (int h = 0; h < 4; ++h) {
-      const float f0 = fmaf(__uint_as_float(0x4B000000u | ((u >> (8 * h)) & 0xFu)), mul, sub);
-      const float f1 = fmaf(__uint_as_float(0x4B000000u | ((u >> (8 * h + 4)) & 0xFu)), mul, sub);
-      const __nv_bfloat162 b = __floats2bfloat162_rn(f0, f1);
-      o[h] = *reinterpret_cast<const uint32_t*>(&b);
-    }
-    *reinterpret_cast<uint4*>(drow + (((4 * c + j) ^ (row & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+    // entries (0,4), (1,5), (2,6), (3,7) of this word side by side in 16-bit lanes
+    const uint32_t r0 = bf16x2_fma((u & 0x000F000Fu) | 0x43004300u, mul, sub);
+    const uint32_t r1 = bf16x2_fma(((u >> 4) & 0x000F000Fu) | 0x43004300u, mul, sub);
+    const uint32_t r2 = bf16x2_fma(((u >> 8) & 0x000F000Fu) | 0x43004300u, mul, sub);
+    const uint32_t r3 = bf16x2_fma(((u >> 12) & 0x000F000Fu) | 0x43004300u, mul, sub);
+    // back into channel order: (0,1) (2,3) (4,5) (6,7)
+    *reinterpret_cast<uint4*>(drow + (((4 * c + j) ^ (row & 7)) << 4)) =
+        make_uint4(__byte_perm(r0, r1, 0x5410), __byte_perm(r2, r3, 0x5410), __byte_perm(r0, r1, 0x7632),
+                   __byte_perm(r2, r3, 0x7632));
   }
 }
 
@@ -2777,7 +2787,7 @@ hola_status hola_verify_host(hola_ctx* ctx, const hola_verify_args* a, void* cud
   hola_status s = check_common(ctx, a);
   if (s != HOLA_OK) return s;
   if (a->B == 0) return HOLA_OK;
-  if (!a->hidden || !a->W_lm) return HOLA_ERR_INVALID_ARG;
+  if (!a->hidden || (!a->W_lm && a->w_dtype != HOLA_W_MIXED)) return HOLA_ERR_INVALID_ARG;
   if ((s = check_sample_args(a)) != HOLA_OK) return s;
   DeviceGuard guard(ctx->device);
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
