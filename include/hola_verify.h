@@ -153,8 +153,10 @@ typedef enum {
                                      * (default), 0 = two MMAs and one accumulator buffer                              */
   HOLA_OPT_HOST_OVERLAP = 3,        /* hola_verify_host: 1 = the draft tensor travels on the context's stream while
                                      * the GEMM runs (default), 0 = every copy on the caller's stream                  */
-  HOLA_OPT_HOST_ROWS_ON_DEMAND = 4  /* hola_verify_host: 1 = always send only the draft rows the step reads,
+  HOLA_OPT_HOST_ROWS_ON_DEMAND = 4, /* hola_verify_host: 1 = always send only the draft rows the step reads,
                                      * 0 = always the whole tensor, -1 = decide per call (default)                     */
+  HOLA_OPT_PASSES = 5               /* passes over W_lm the verify rows are split into: 0 = chosen by estimated cost
+                                     * (default), else that many when the rows fit (at most 512 per pass)             */
 } hola_option;
 hola_status hola_set_option(hola_ctx* ctx, int option, int value);
 

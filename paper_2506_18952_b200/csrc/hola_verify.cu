@@ -1816,74 +1816,62 @@ __device__ __forceinline__ float qlnq8(const uint4 raw) {     // sum over eight 
   return part;
 }
 __device__ __forceinline__ float qlnq4(const float4 x) { return (qlnq(x.x) + qlnq(x.y)) + (qlnq(x.z) + qlnq(x.w)); }
-__device__ __forceinline__ float qlnq_vec(const uint4 raw) { return qlnq8(raw); }
-__device__ __forceinline__ float qlnq_vec(const float4 x) { return qlnq4(x); }
 
-// Work items are (row, slice) pairs, kHqSlices slices per draft row; a CTA takes items blockIdx.x, blockIdx.x + grid, ...
-// and leaves each item's partial sum in part[row][slice]; the accept/sample kernel adds the slices in index order.
-// The grid is sized to the machine (a few CTAs per SM) and every thread keeps eight 16-byte loads in flight, so the
-// pass runs at the rate the memory system delivers the rows instead of at the rate CTAs can be launched.
-template <typename Vec, int kPerVec>
-__device__ __forceinline__ double draft_entropy_slice(const void* rowp, int V, int slice, bool scalar_tail) {
-  constexpr int kInFlight = 8;                           // independent 16-byte loads per thread and step
-  const bool vec = (reinterpret_cast<uintptr_t>(rowp) & 15u) == 0;
-  const int nvec = vec ? V / kPerVec : 0;
-  const Vec* q16 = static_cast<const Vec*>(rowp);
-  const int per = (nvec + kHqSlices - 1) / kHqSlices, end = min(nvec, (slice + 1) * per);
-  double acc = 0.0;
-  int i = slice * per + threadIdx.x;
-  for (; i + (kInFlight - 1) * 256 < end; i += kInFlight * 256) {
-    Vec raw[kInFlight];
-#pragma unroll
-    for (int u = 0; u < kInFlight; ++u) raw[u] = __ldcs(q16 + i + u * 256);
-    float part = 0.f;
-#pragma unroll
-    for (int u = 0; u < kInFlight; ++u) part += qlnq_vec(raw[u]);
-    acc += part;
-  }
-  {
-    Vec raw[kInFlight];
-#pragma unroll
-    for (int u = 0; u < kInFlight; ++u)
-      if (i + u * 256 < end) raw[u] = __ldcs(q16 + i + u * 256);
-    float part = 0.f;
-#pragma unroll
-    for (int u = 0; u < kInFlight; ++u)
-      if (i + u * 256 < end) part += qlnq_vec(raw[u]);
-    acc += part;
-  }
-  if (scalar_tail) {                                     // what the 16-byte loads do not cover (or the whole row)
-    if (kPerVec == 8) {
-      const __nv_bfloat16* qr = static_cast<const __nv_bfloat16*>(rowp);
-      for (int v = nvec * kPerVec + threadIdx.x; v < V; v += 256) acc += qlnq(__bfloat162float(qr[v]));
-    } else {
-      const float* qr = static_cast<const float*>(rowp);
-      for (int v = nvec * kPerVec + threadIdx.x; v < V; v += 256) acc += qlnq(qr[v]);
-    }
-  }
-  return acc;
-}
-
-__global__ void __launch_bounds__(256) draft_entropy_kernel(const void* q, int q_dtype, int V, int rows, double* part) {
+// Grid (rows, kHqSlices): CTA (r, s) sums slice s of row r and leaves the partial sum in part[r][s]; the
+// accept/sample kernel adds the slices in index order.  Small CTAs of 32 registers per thread on purpose: the pass
+// runs on a side stream while the GEMM kernel holds every SM, and only a CTA of this size fits into the registers
+// that kernel leaves free (a persistent form with eight loads in flight per thread, 100 registers, could not start
+// before the GEMM kernel had finished and made the step 45 us longer).
+__global__ void __launch_bounds__(256) draft_entropy_kernel(const void* q, int q_dtype, int V, double* part) {
   __shared__ double sh_part[8];
-  const int items = rows * kHqSlices;
-  for (int it = blockIdx.x; it < items; it += gridDim.x) {
-    const size_t row = static_cast<size_t>(it / kHqSlices);
-    const int slice = it % kHqSlices;
-    double acc;
-    if (q_dtype == HOLA_Q_BF16)
-      acc = draft_entropy_slice<uint4, 8>(static_cast<const __nv_bfloat16*>(q) + row * V, V, slice, slice == 0);
-    else
-      acc = draft_entropy_slice<float4, 4>(static_cast<const float*>(q) + row * V, V, slice, slice == 0);
-    acc = warp_sum_f64(acc);
-    if ((threadIdx.x & 31) == 0) sh_part[threadIdx.x >> 5] = acc;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      double tot = 0.0;
-      for (int i = 0; i < 8; ++i) tot += sh_part[i];
-      part[row * kHqSlices + slice] = tot;
+  const size_t row = blockIdx.x;
+  const int slice = blockIdx.y;
+  double acc = 0.0;
+  constexpr int kInFlight = 4;                           // independent 16-byte loads per thread and step
+  if (q_dtype == HOLA_Q_BF16) {
+    const __nv_bfloat16* qr = static_cast<const __nv_bfloat16*>(q) + row * V;
+    const bool vec = (reinterpret_cast<uintptr_t>(qr) & 15u) == 0;
+    const int nvec = vec ? V / 8 : 0;
+    const uint4* q16 = reinterpret_cast<const uint4*>(qr);
+    const int per = (nvec + kHqSlices - 1) / kHqSlices, end = min(nvec, (slice + 1) * per);
+    int i = slice * per + threadIdx.x;
+    for (; i + (kInFlight - 1) * 256 < end; i += kInFlight * 256) {
+      uint4 raw[kInFlight];
+#pragma unroll
+      for (int u = 0; u < kInFlight; ++u) raw[u] = q16[i + u * 256];
+#pragma unroll
+      for (int u = 0; u < kInFlight; ++u) acc += qlnq8(raw[u]);
     }
-    __syncthreads();
+    for (; i < end; i += 256) acc += qlnq8(q16[i]);
+    for (int v = nvec * 8 + threadIdx.x; slice == 0 && v < V; v += 256) {    // scalar tail (or whole row): slice 0
+      acc += qlnq(__bfloat162float(qr[v]));
+    }
+  } else {
+    const float* qr = static_cast<const float*>(q) + row * V;
+    const bool vec = (reinterpret_cast<uintptr_t>(qr) & 15u) == 0;
+    const int nvec = vec ? V / 4 : 0;
+    const float4* q16 = reinterpret_cast<const float4*>(qr);
+    const int per = (nvec + kHqSlices - 1) / kHqSlices, end = min(nvec, (slice + 1) * per);
+    int i = slice * per + threadIdx.x;
+    for (; i + (kInFlight - 1) * 256 < end; i += kInFlight * 256) {
+      float4 raw[kInFlight];
+#pragma unroll
+      for (int u = 0; u < kInFlight; ++u) raw[u] = q16[i + u * 256];
+#pragma unroll
+      for (int u = 0; u < kInFlight; ++u) acc += qlnq4(raw[u]);
+    }
+    for (; i < end; i += 256) acc += qlnq4(q16[i]);
+    for (int v = nvec * 4 + threadIdx.x; slice == 0 && v < V; v += 256) {
+      acc += qlnq(qr[v]);
+    }
+  }
+  acc = warp_sum_f64(acc);
+  if ((threadIdx.x & 31) == 0) sh_part[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double tot = 0.0;
+    for (int i = 0; i < 8; ++i) tot += sh_part[i];
+    part[row * kHqSlices + slice] = tot;
   }
 }
 
@@ -1926,6 +1914,7 @@ struct hola_ctx {
   unsigned char* h_out;       // pinned host mirror: the outputs come back in ONE copy
   int force_stages;
   int no_rot;                 // tuning override: never use the rotating accumulator units
+  int force_passes;           // tuning override: passes over W_lm (0: chosen by cost)
   cudaStream_t copy_stream;   // hola_verify_host: the draft tensor travels here while the GEMM runs
   cudaEvent_t copy_done;
   cudaEvent_t fork_point;     // verify_device: where the side stream branches off the caller's stream
@@ -2019,6 +2008,7 @@ Plan make_plan(const hola_ctx* ctx, int M, int w_dtype = HOLA_W_BF16) {
   const int p_min = (rows + max_rows_per_pass - 1) / max_rows_per_pass;
   const double t_hbm = (w8 || i8 ? 1.0 : 2.0) * ctx->V * static_cast<double>(ctx->H) / 6.4e12;
   for (int passes = p_min; passes <= p_min + 3; ++passes) {
+    if (ctx->force_passes && passes != ctx->force_passes && ctx->force_passes >= p_min) continue;
     const int r = (rows + passes - 1) / passes;
     // up to 256 rows: one MMA, two accumulator buffers; up to 384: three MMAs of N <= 128 on rotating 128-column
     // units; beyond: two MMAs of N <= 256 that fill the tensor memory
@@ -2245,12 +2235,6 @@ hola_status run_lm_head(hola_ctx* ctx, const hola_verify_args* a, float* logits,
   return HOLA_OK;
 }
 
-// CTAs of the pass over the draft rows: one per (row, slice) item up to four per SM.
-unsigned draft_entropy_grid(const hola_ctx* ctx, int rows) {
-  const int items = rows * kHqSlices, cap = 4 * ctx->num_sms;
-  return static_cast<unsigned>(items < cap ? items : cap);
-}
-
 // What the accept/sample kernel needs to know in the vocabulary-parallel form.
 struct ShardLaunch {
   int world, rank, v_offset, V_global;
@@ -2274,8 +2258,8 @@ hola_status run_accept_sample(hola_ctx* ctx, const hola_verify_args* a, const fl
     // one more pass over the draft rows: H(q_j) for every (sequence, draft position) - unless the caller has put it
     // on the side stream already, next to the GEMM
     if (!ctx->hq_ready) {
-      draft_entropy_kernel<<<draft_entropy_grid(ctx, a->B * a->k), 256, 0, stream>>>(
-          a->draft_q, a->q_dtype, a->V, a->B * a->k, ctx->hq);
+      draft_entropy_kernel<<<dim3(static_cast<unsigned>(a->B * a->k), kHqSlices), 256, 0, stream>>>(
+          a->draft_q, a->q_dtype, a->V, ctx->hq);
       const cudaError_t e0 = cudaGetLastError();
       if (e0 != cudaSuccess) { set_error(ctx, "launch draft_entropy_kernel", e0); return HOLA_ERR_CUDA; }
     }
@@ -2509,6 +2493,10 @@ hola_status hola_set_option(hola_ctx* ctx, int option, int value) {
       ctx->force_stages = value;
       break;
     case HOLA_OPT_ROTATING_UNITS: ctx->no_rot = value == 0; break;
+    case HOLA_OPT_PASSES:
+      if (value < 0 || value > 64) return HOLA_ERR_INVALID_ARG;
+      ctx->force_passes = value;
+      break;
     case HOLA_OPT_HOST_OVERLAP: ctx->host_overlap = value != 0; break;
     case HOLA_OPT_HOST_ROWS_ON_DEMAND:
       if (value < -1 || value > 1) return HOLA_ERR_INVALID_ARG;
@@ -2600,8 +2588,8 @@ hola_status verify_device(hola_ctx* ctx, const hola_verify_args* a, cudaStream_t
     cudaError_t e = cudaSuccess;
     if (!before_sample) e = cudaStreamWaitEvent(ctx->copy_stream, ctx->fork_point, 0);
     if (e == cudaSuccess) {
-      draft_entropy_kernel<<<draft_entropy_grid(ctx, a->B * a->k), 256, 0, ctx->copy_stream>>>(
-          a->draft_q, a->q_dtype, a->V, a->B * a->k, ctx->hq);
+      draft_entropy_kernel<<<dim3(static_cast<unsigned>(a->B * a->k), kHqSlices), 256, 0, ctx->copy_stream>>>(
+          a->draft_q, a->q_dtype, a->V, ctx->hq);
       e = cudaGetLastError();
     }
     if (e == cudaSuccess) e = cudaEventRecord(ctx->copy_done, ctx->copy_stream);
