@@ -47,7 +47,7 @@ NOMINAL_PEAKS = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
 # summarised under profiles/: "batched" (--set full capture) and "large_vocab" (a capture of the three DRAM / time
 # counters on the full-size launch; its logits are stored with the streaming hint, so most of the 197 MB reach DRAM
 # inside the kernel).  Other workloads, and the other weight modes, report null.
-NCU_TRAFFIC = {"batched": 265883392 + 7073536, "large_vocab": 1055344896 + 165309952}
+NCU_TRAFFIC = {"batched": 265922304 + 8190720, "large_vocab": 1055559936 + 172039680}
 
 
 def ncu_traffic_bytes(w):
