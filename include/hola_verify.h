@@ -155,6 +155,8 @@ typedef enum {
                                      * the GEMM runs (default), 0 = every copy on the caller's stream                  */
   HOLA_OPT_HOST_ROWS_ON_DEMAND = 4, /* hola_verify_host: 1 = always send only the draft rows the step reads,
                                      * 0 = always the whole tensor, -1 = decide per call (default)                     */
+  HOLA_OPT_PAIR_MMA = 6,            /* 384-row passes on rotating units: 1 = one MMA of N = 256 over two adjacent units
+                                     * plus one of N = 128 per K step (default), 0 = three MMAs of N = 128             */
   HOLA_OPT_PASSES = 5               /* passes over W_lm the verify rows are split into: 0 = chosen by estimated cost
                                      * (default), else that many when the rows fit (at most 512 per pass)             */
 } hola_option;

@@ -91,6 +91,7 @@ struct K1Params {
   int V, n_ptiles, n_kblocks, stages, nbuf;
   int n_sub, N;   // MMAs per K step and their N (verify rows each; multiple of 16)
   int rot;        // 1: three MMAs of N <= 128 per K step whose accumulators rotate over the four 128-column units
+  int pair256;    // rot with N = 128 exactly: two of the three units of a tile are adjacent and take ONE MMA of N = 256
   int tile_rows;  // vocabulary rows per CTA per tile (<= 128, multiple of 4): balances the tiles over the pairs
   int ldl;        // row pitch of the logits buffer, in floats
   const float* w_scale;   // 8-bit W_lm: fp32 scale per vocabulary row, applied to the accumulators
@@ -700,9 +701,21 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
             const uint32_t fb = leader_full + 8 * stage;
             mbar_expect_tx_cluster(fb, tx_bytes);
             tma_load_2d(sa, &tmap_w, fb, kx, v0, pol_w);
-            for (int s = 0; s < p.n_sub; ++s)
-              tma_load_2d(sa + kWBlockBytes + s * hid_block_bytes, &tmap_hidden, fb, kx,
-                          (kTwoPlane ? 2 : 1) * p.row0 + s * p.N + static_cast<int>(rank) * half_n, pol_h);
+            if (kRot && p.pair256) {
+              // Row blocks 0, 1, 2 (128 rows each) sit on units (3t, 3t+1, 3t+2) mod 4.  Two of them that are adjacent
+              // without wrapping (blocks 0, 1, or blocks 1, 2 when the tile starts on unit 3) share one MMA of N = 256:
+              // this CTA then supplies ONE of the two blocks whole, and its half of the third block as before.
+              const bool late_pair = ((3 * t) & 3) == 3;
+              const int pair_row = (late_pair ? 128 : 0) + static_cast<int>(rank) * 128;
+              const int single_row = (late_pair ? 0 : 256) + static_cast<int>(rank) * 64;
+              tma_load_2d(sa + kWBlockBytes, &tmap_hidden, fb, kx, p.row0 + pair_row, pol_h);
+              tma_load_2d(sa + kWBlockBytes + hid_block_bytes, &tmap_hidden, fb, kx, p.row0 + pair_row + 64, pol_h);
+              tma_load_2d(sa + kWBlockBytes + 2 * hid_block_bytes, &tmap_hidden, fb, kx, p.row0 + single_row, pol_h);
+            } else {
+              for (int s = 0; s < p.n_sub; ++s)
+                tma_load_2d(sa + kWBlockBytes + s * hid_block_bytes, &tmap_hidden, fb, kx,
+                            (kTwoPlane ? 2 : 1) * p.row0 + s * p.N + static_cast<int>(rank) * half_n, pol_h);
+            }
           }
           if (++stage == p.stages) { stage = 0; phase ^= 1u; }
         }
@@ -713,6 +726,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
     if (rank == 0 && elect_one()) {
       const uint32_t idesc = kI8 ? make_idesc_s8_m256(static_cast<uint32_t>(p.N))
                                  : make_idesc_bf16_m256(static_cast<uint32_t>(p.N));
+      const uint32_t idesc_pair = kI8 ? make_idesc_s8_m256(256u) : make_idesc_bf16_m256(256u);
       const uint64_t desc0 = make_kmajor_sw128_desc(base);
       const bool two_mmas = p.n_sub == 2;
       int stage = 0;
@@ -726,6 +740,32 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
             tc_fence_after();
             const uint64_t adesc = desc0 + ((stage * stage_bytes) >> 4);
             const uint64_t bdesc0 = adesc + (kWBlockBytes >> 4);
+            if (p.pair256) {
+              // one MMA of N = 256 over the two adjacent units, one of N = 128 over the third: the W_lm block is read
+              // from shared memory twice per K step instead of three times
+              const uint32_t a0 = static_cast<uint32_t>(3 * t) & 3u;
+              const bool late_pair = a0 == 3u;
+              const uint32_t unit_pair = late_pair ? 0u : a0, unit_single = late_pair ? 3u : ((a0 + 2u) & 3u);
+              if (kb == 0) {                             // the epilogue must have read these units' previous tiles
+#pragma unroll
+                for (int u = 0; u < 3; ++u) {
+                  const uint32_t unit = (a0 + u) & 3u;
+                  const uint32_t par = (used >> unit) & 1u;
+                  if (!mbar_wait(tempty_bar + 8 * unit, par ^ 1u, abort_flag, p.status)) { ok = false; break; }
+                  used ^= 1u << unit;
+                }
+                if (!ok) break;
+                tc_fence_after();
+              }
+              const uint32_t acc = kb != 0 ? 1u : 0u;
+              const uint32_t dp = tmem_base + unit_pair * 128u, ds = tmem_base + unit_single * 128u;
+              const uint64_t bdesc_s = bdesc0 + 2 * (hid_block_bytes >> 4);
+#pragma unroll
+              for (int kk = 0; kk < kBlockK / 16; ++kk) {
+                umma<kI8>(dp, adesc + 2 * kk, bdesc0 + 2 * kk, idesc_pair, kk == 0 ? acc : 1u);
+                umma<kI8>(ds, adesc + 2 * kk, bdesc_s + 2 * kk, idesc, kk == 0 ? acc : 1u);
+              }
+            } else
 #pragma unroll
             for (int u = 0; u < 3; ++u) {
               const uint32_t unit = static_cast<uint32_t>(3 * t + u) & 3u;
@@ -1915,6 +1955,7 @@ struct hola_ctx {
   int force_stages;
   int no_rot;                 // tuning override: never use the rotating accumulator units
   int force_passes;           // tuning override: passes over W_lm (0: chosen by cost)
+  int no_pair256;             // tuning override: rotating units always as three MMAs of N = 128
   cudaStream_t copy_stream;   // hola_verify_host: the draft tensor travels here while the GEMM runs
   cudaEvent_t copy_done;
   cudaEvent_t fork_point;     // verify_device: where the side stream branches off the caller's stream
@@ -2192,6 +2233,7 @@ hola_status run_lm_head(hola_ctx* ctx, const hola_verify_args* a, float* logits,
   const CUtensorMap& tw16 = me->tw16;
   K1Params kp;
   kp.M = M; kp.V = a->V; kp.n_ptiles = pl.n_ptiles; kp.n_kblocks = pl.n_kblocks;
+  kp.pair256 = (pl.rot && pl.N == 128 && !ctx->no_pair256) ? 1 : 0;
   kp.stages = pl.stages; kp.nbuf = pl.nbuf; kp.rot = pl.rot; kp.n_sub = pl.n_sub; kp.N = pl.N; kp.tile_rows = pl.tile_rows; kp.ldl = ldl;
   kp.logits = logits; kp.partials = ctx->partials; kp.part_stride = ctx->max_rows;
   kp.status = a->status_word ? a->status_word : ctx->status;
@@ -2493,6 +2535,7 @@ hola_status hola_set_option(hola_ctx* ctx, int option, int value) {
       ctx->force_stages = value;
       break;
     case HOLA_OPT_ROTATING_UNITS: ctx->no_rot = value == 0; break;
+    case HOLA_OPT_PAIR_MMA: ctx->no_pair256 = value == 0; break;
     case HOLA_OPT_PASSES:
       if (value < 0 || value > 64) return HOLA_ERR_INVALID_ARG;
       ctx->force_passes = value;

@@ -777,6 +777,30 @@ def test_options_change_speed_knobs_not_results(binding):
             ctx.hola_set_option(binding.HOLA_OPT_RING_SLOTS, 1)
 
 
+@pytest.mark.parametrize("a8", [False, True])
+def test_pair_mma_on_rotating_units_matches_oracle_and_the_three_mma_form(binding, a8):
+    """378 rows: three row blocks of 128 (the last one ragged) on rotating units, two of them under one MMA of N = 256;
+    20 000 vocabulary rows give every CTA pair a tile, the first pairs two, so both placements of the pair occur."""
+    w = workloads.gaussian_head("pair-mma", 63, 5, 256, 20000, seed=23, device=DEV, w_std=0.3, sigma=1.0, sigma_far=0.2)
+    W, sc = (binding.hola_quantize_w8(w.W_lm) if a8 else (w.W_lm, None))
+    with binding.HolaVerify(w.B, w.k, w.H, w.V) as ctx:
+        out = ctx.hola_verify(w.hidden, W, w.draft_tok, w.draft_q, w.uniforms, w.tau, want_logits=True, w_scale=sc, a8=a8)
+        torch.cuda.synchronize()
+        ctx.hola_set_option(binding.HOLA_OPT_PAIR_MMA, 0)
+        three = ctx.hola_verify(w.hidden, W, w.draft_tok, w.draft_q, w.uniforms, w.tau, want_logits=True, w_scale=sc, a8=a8)
+        torch.cuda.synchronize()
+    assert int(out.status.item()) == 0
+    assert torch.equal(out.accept_len, three.accept_len) and torch.equal(out.next_tok, three.next_tok)
+    assert torch.allclose(out.logits, three.logits, rtol=1e-5, atol=1e-5)
+    if a8:
+        orc = _w8_oracle(w, W, sc, a8=True)
+        rep = compare.compare(orc, _np(w.draft_q), _np(w.uniforms), _np(out.accept_len), _np(out.next_tok),
+                              _np(out.entropy), _np(out.logZ), _np(out.logits))
+        assert rep.ok, rep.summary()
+    else:
+        check_against_oracle(binding, w, out=out)
+
+
 def test_repeated_calls_reuse_the_set_up_and_new_pointers_do_not(binding):
     """Same pointers and sizes: the second call takes its tensor maps from the context.  Other tensors of the same shape,
     or another batch size, must not be served from what the first call left."""
