@@ -146,6 +146,8 @@ def oracle_sample_size(w, steps: int, warmup: int) -> tuple[int, float]:
     n = int(max(1, min(w.B, per_step_budget / max(per_seq, 1e-4))))
     if n > 0.8 * w.B:                                               # the whole batch when it nearly fits anyway
         n = w.B
+    elif n >= 8:                                                    # (a multiple of 8: the probe's jitter must not move it)
+        n -= n % 8
     return n, per_seq
 
 
