@@ -157,6 +157,9 @@ typedef enum {
                                      * 0 = always the whole tensor, -1 = decide per call (default)                     */
   HOLA_OPT_PAIR_MMA = 6,            /* 384-row passes on rotating units: 1 = one MMA of N = 256 over two adjacent units
                                      * plus one of N = 128 per K step (default), 0 = three MMAs of N = 128             */
+  HOLA_OPT_HOST_IN_PLACE = 7,       /* hola_verify_host with rows on demand: 1 = where draft_q is pinned host memory the
+                                     * device can address, the accept/sample kernel reads the rows not sent ahead in
+                                     * place over the bus (default), 0 = they are copied after a read-back of accept_len */
   HOLA_OPT_PASSES = 5               /* passes over W_lm the verify rows are split into: 0 = chosen by estimated cost
                                      * (default), else that many when the rows fit (at most 512 per pass)             */
 } hola_option;

@@ -120,6 +120,8 @@ struct K3Params {
   const void* q;
   int q_dtype;
   const float* q_tok;           // optional fp32 [B][k]: q_j(x_j) already gathered (then q is read at row n only)
+  const void* q_far;            // optional: the same draft tensor in pinned HOST memory, as the device sees it; rows
+  int q_far_from;               //   n >= q_far_from of a sequence are read from there (rows before it were copied to q)
   int inputs_settled;           // 1: launched right behind this call's own GEMM kernel, whose CTAs have waited for the
                                 // kernel before the call: tokens, uniforms and draft probabilities may be read
                                 // before this grid's dependency wait.  0: wait first.
@@ -1528,9 +1530,8 @@ __global__ void __launch_bounds__(kK3Threads, kK3MaxPerSm) accept_sample_kernel(
   const float logZ = sh_logZ[n];
   const float* lrow = p.logits + static_cast<size_t>(row_first + n) * p.ldl;
   const size_t q_elem = (p.q_dtype == HOLA_Q_BF16) ? 2 : 4;
-  const void* qrow = (n < k) ? static_cast<const void*>(static_cast<const char*>(p.q) +
-                                                        (static_cast<size_t>(b) * k + n) * V * q_elem)
-                             : nullptr;
+  const char* qbase = static_cast<const char*>((p.q_far && n >= p.q_far_from) ? p.q_far : p.q);
+  const void* qrow = (n < k) ? static_cast<const void*>(qbase + (static_cast<size_t>(b) * k + n) * V * q_elem) : nullptr;
   const int nchunks = (V + kChunk - 1) / kChunk;
   const int cpc = (nchunks + S - 1) / S;                 // chunks per CTA
   const int c_first = rank * cpc;
@@ -1956,6 +1957,7 @@ struct hola_ctx {
   int no_rot;                 // tuning override: never use the rotating accumulator units
   int force_passes;           // tuning override: passes over W_lm (0: chosen by cost)
   int no_pair256;             // tuning override: rotating units always as three MMAs of N = 128
+  int host_in_place;          // hola_verify_host: read draft rows not sent ahead in place from pinned host memory
   cudaStream_t copy_stream;   // hola_verify_host: the draft tensor travels here while the GEMM runs
   cudaEvent_t copy_done;
   cudaEvent_t fork_point;     // verify_device: where the side stream branches off the caller's stream
@@ -2289,8 +2291,10 @@ struct ShardLaunch {
 // `settled`: the launch sits right behind this call's own GEMM kernel (see K3Params::inputs_settled).
 hola_status run_accept_sample(hola_ctx* ctx, const hola_verify_args* a, const float* logits, int ldl, int combine,
                               int nparts, cudaStream_t stream, const float* q_tok = nullptr, int phase = 0,
-                              const ShardLaunch* sh = nullptr, bool settled = false) {
+                              const ShardLaunch* sh = nullptr, bool settled = false, const void* q_far = nullptr,
+                              int q_far_from = 0) {
   K3Params kp{};
+  kp.q_far = q_far; kp.q_far_from = q_far_from;
   kp.q_tok = q_tok; kp.phase = phase; kp.inputs_settled = settled ? 1 : 0;
   kp.B = a->B; kp.k = a->k; kp.V = a->V; kp.ldl = ldl; kp.logits = logits;
   kp.partials = ctx->partials; kp.nparts = nparts; kp.part_stride = ctx->max_rows; kp.combine = combine;
@@ -2457,6 +2461,7 @@ hola_status hola_create(hola_ctx** out, int device, int maxB, int maxK, int H, i
   ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
   ctx->host_overlap = 1;
   ctx->host_lazy_q = -1;
+  ctx->host_in_place = 1;
   if (configure_kernels() != cudaSuccess) { free(ctx); return HOLA_ERR_CUDA; }
   const WsLayout w = ws_layout(maxB, maxK, H, V, ctx->num_sms);
   const cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&ctx->ws), w.total);
@@ -2536,6 +2541,7 @@ hola_status hola_set_option(hola_ctx* ctx, int option, int value) {
       break;
     case HOLA_OPT_ROTATING_UNITS: ctx->no_rot = value == 0; break;
     case HOLA_OPT_PAIR_MMA: ctx->no_pair256 = value == 0; break;
+    case HOLA_OPT_HOST_IN_PLACE: ctx->host_in_place = value != 0; break;
     case HOLA_OPT_PASSES:
       if (value < 0 || value > 64) return HOLA_ERR_INVALID_ARG;
       ctx->force_passes = value;
@@ -2730,8 +2736,25 @@ hola_status verify_host_lazy(hola_ctx* ctx, const hola_verify_args* a, cudaStrea
   if (s != HOLA_OK) return s;
   const Plan& pl = plan_for(ctx, B * (k + 1), a->w_dtype);
   if ((s = run_lm_head(ctx, &d, ctx->logits, ctx->ldl, pl, stream)) != HOLA_OK) return s;
+  // Where the caller's draft tensor is pinned host memory that the device can address, the rows still missing after the
+  // accept test are not copied at all: the accept/sample kernel reads row accept_len of a sequence in place, over the
+  // bus, when that row is not among the ones sent ahead.  One launch, no read-back in the middle of the call.
+  const void* q_far = nullptr;
+  if (sample && ctx->host_in_place) {
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, a->draft_q) == cudaSuccess && at.type == cudaMemoryTypeHost && at.devicePointer)
+      q_far = at.devicePointer;
+    else
+      cudaGetLastError();                                // (an unregistered pointer is not an error of this call)
+  }
   if (!sample) {
     if ((s = run_accept_sample(ctx, &d, ctx->logits, ctx->ldl, 1, pl.grid, stream, ctx->st_qtok, 0)) != HOLA_OK) return s;
+  } else if (q_far) {
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, ctx->copy_done, 0);
+    if (e != cudaSuccess) { set_error(ctx, "wait for the draft rows sent ahead", e); return HOLA_ERR_CUDA; }
+    if ((s = run_accept_sample(ctx, &d, ctx->logits, ctx->ldl, 1, pl.grid, stream, ctx->st_qtok, 0, nullptr, false, q_far,
+                               ahead)) != HOLA_OK)
+      return s;
   } else {
     if ((s = run_accept_sample(ctx, &d, ctx->logits, ctx->ldl, 1, pl.grid, stream, ctx->st_qtok, 1)) != HOLA_OK) return s;
     d2h(ctx->h_accept, d.accept_len, static_cast<size_t>(B) * 4);
@@ -2757,6 +2780,12 @@ hola_status verify_host_lazy(hola_ctx* ctx, const hola_verify_args* a, cudaStrea
   memcpy(a->entropy, ctx->h_out + ob.entropy, rows * 4);
   memcpy(a->logZ, ctx->h_out + ob.logZ, rows * 4);
   if (a->status_word) memcpy(a->status_word, ctx->h_out + ob.status, 4);
+  if (q_far) {                                           // rows the kernel read over the bus count as bytes sent
+    for (int b = 0; b < B; ++b) {
+      const int n = a->accept_len[b];
+      if (n >= ahead && n < k) up += row_bytes;
+    }
+  }
   ctx->last_h2d = up; ctx->last_d2h = down;
   return HOLA_OK;
 }

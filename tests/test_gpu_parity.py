@@ -412,6 +412,30 @@ def test_host_entry_equals_device_entry(binding):
     assert torch.equal(h.entropy, d.entropy.cpu()) and torch.equal(h.logZ, d.logZ.cpu())
 
 
+@pytest.mark.parametrize("pinned", [True, False])
+def test_host_entry_reads_missing_rows_in_place_or_copies_them(binding, pinned):
+    """With the draft tensor in pinned host memory the rows not sent ahead are read in place by the accept/sample kernel;
+    with pageable memory, or with the option off, they are copied after a read-back of accept_len.  Same results, same
+    byte count, either way."""
+    w = workloads.gaussian_head("in-place", 21, 4, 128, 5000, seed=78, device=DEV, w_std=0.3, tau=0.0)
+    mem = (lambda t: t.cpu().pin_memory()) if pinned else (lambda t: t.cpu().clone())
+    host = [mem(t) for t in (w.hidden, w.draft_tok, w.draft_q, w.uniforms)]
+    outs, traffic = [], []
+    with binding.HolaVerify(w.B, w.k, w.H, w.V) as ctx:
+        ctx.hola_set_option(binding.HOLA_OPT_HOST_ROWS_ON_DEMAND, 1)
+        d = ctx.hola_verify(w.hidden, w.W_lm, w.draft_tok, w.draft_q, w.uniforms, w.tau)
+        torch.cuda.synchronize()
+        for in_place in (1, 0):
+            ctx.hola_set_option(binding.HOLA_OPT_HOST_IN_PLACE, in_place)
+            outs.append(ctx.hola_verify_host(host[0], w.W_lm, host[1], host[2], host[3], w.tau))
+            traffic.append(ctx.hola_host_traffic()[0])
+    for h in outs:
+        assert torch.equal(h.accept_len, d.accept_len.cpu()) and torch.equal(h.next_tok, d.next_tok.cpu())
+        assert torch.equal(h.entropy, d.entropy.cpu()) and torch.equal(h.logZ, d.logZ.cpu())
+    assert traffic[0] == traffic[1]
+    assert len(set(d.accept_len.tolist())) >= 3              # rows beyond the ones sent ahead are needed
+
+
 @pytest.mark.parametrize("q_dtype", [torch.bfloat16, torch.float32])
 @pytest.mark.parametrize("gate,fallback", [(0, 0), (0, 1), (1, 0)])
 @pytest.mark.parametrize("tau", [0.0, None, 100.0])
