@@ -11,7 +11,13 @@
 //       same registers transposed through a small shared-memory buffer, keep per verify position the running
 //       softmax statistics (m, s, t) = (max, sum e^(l-m), sum e^(l-m)(l-m)) and the arg-max in registers, in the
 //       shadow of the next tile's MMAs.  W_lm is read from HBM once per pass; the logits are never read back.
+//       With 257..384 verify rows the accumulators rotate over the four 128-column units of the tensor memory and a
+//       unit is handed back as soon as its chunk has gone to the logits buffer and a staging buffer.  In its
+//       on-chip-expansion mode the kernel streams groups of 256 vocabulary rows stored at 4, 8 or 16 bits and
+//       converter warps expand the codes exactly to bf16 (mixed-precision quantiser of the Lo-Bi Optimization section).
 //   quantize_rows_int8_kernel   8-bit case of the Lo-Bi quantiser, per row (W_lm ahead of time, hidden rows per call).
+//   quantize_rows_w4_kernel     4-bit case: codes in [-7, 7] with one shared exponent per sub-block of 128 channels.
+//   bounded_wait_selftest_kernel  a wait that is made to run out, to exercise the give-up path without breaking anything.
 //   draft_entropy_kernel        H(q_j) of the draft rows, for the gate on the draft distribution.
 //   shard_record_kernel         vocabulary-parallel form: a rank's statistics record for the first all-gather.
 //   finalize_kernel             merges the per-CTA statistics:  logZ = m + ln s,  H = ln s - t/s  (entropy
