@@ -160,6 +160,9 @@ typedef enum {
   HOLA_OPT_HOST_IN_PLACE = 7,       /* hola_verify_host with rows on demand: 1 = where draft_q is pinned host memory the
                                      * device can address, the accept/sample kernel reads the rows not sent ahead in
                                      * place over the bus (default), 0 = they are copied after a read-back of accept_len */
+  HOLA_OPT_CONVERTER_GROUP = 8,     /* on-chip expansion (HOLA_W_INT8, HOLA_W_MIXED): converter warps that share one K
+                                     * block, 1..8; groups of that many of the eight converter warps take whole blocks
+                                     * in turn.  0 = the default (2)                                                  */
   HOLA_OPT_PASSES = 5               /* passes over W_lm the verify rows are split into: 0 = chosen by estimated cost
                                      * (default), else that many when the rows fit (at most 512 per pass)             */
 } hola_option;

@@ -63,15 +63,13 @@ constexpr int kEpiSlots = 4;                     // 32-column chunks of a tile o
 constexpr int kTransRows = 16;                   // verify rows per transposition step of an epilogue warp
 constexpr int kTransBytes = kTransRows * 32 * 4; // its staging buffer: [16 rows][32 vocabulary entries] fp32
 // 8-bit W_lm, expanded on chip (mode 1): the int8 tile of a K block lands in a raw block of the ring slot and
-// converter warps expand it to the bf16 tile the MMA reads.  Warps 2..9 are epilogue warps, warp 14 loads the
-// hidden blocks, warps 10..13 and 15..17 convert.
+// converter warps expand it to the bf16 tile the MMA reads.  Warps 2..9 are epilogue warps, warps 10..17 convert (and
+// the first lane of a group also fetches the hidden blocks of the K blocks the group owns).
 constexpr int kRawBlockBytes = kLanes * kBlockK;  // int8 [128][64]
 constexpr int kSubBlock = 128;                    // hidden channels per 4-bit sub-block (one shared exponent each)
 constexpr int kGroupRows = 256;                   // vocabulary rows per group of one width
 constexpr int kW8EpiWarps = 8;
-constexpr int kW8HiddenWarp = 14;
-constexpr int kConvWarps = (kW8HiddenWarp - 2 - kW8EpiWarps) + (kK1Warps - kW8HiddenWarp - 1);   // 4 + 3
-constexpr int kConvThreads = kConvWarps * 32;
+constexpr int kConvWarps = kK1Warps - 2 - kW8EpiWarps;   // 8
 constexpr int kTmemCols = 512;
 constexpr int kMaxStages = 12;
 constexpr int kSmemBudget = 227 * 1024;          // dynamic shared memory per CTA on sm_100
@@ -98,6 +96,7 @@ struct K1Params {
   int n_sub, N;   // MMAs per K step and their N (verify rows each; multiple of 16)
   int rot;        // 1: three MMAs of N <= 128 per K step whose accumulators rotate over the four 128-column units
   int pair256;    // rot with N = 128 exactly: two of the three units of a tile are adjacent and take ONE MMA of N = 256
+  int conv_group; // (on-chip expansion) converter warps that share one K block
   int tile_rows;  // vocabulary rows per CTA per tile (<= 128, multiple of 4): balances the tiles over the pairs
   int ldl;        // row pitch of the logits buffer, in floats
   const float* w_scale;   // 8-bit W_lm: fp32 scale per vocabulary row, applied to the accumulators
@@ -516,36 +515,35 @@ __device__ __forceinline__ uint32_t bf16x2_fma(uint32_t a, uint32_t b, uint32_t 
   return d;
 }
 
-// Sixteen int8 values (one 16-byte piece c of row `row` of the raw block) -> sixteen bf16 values at their place in
-// the 128-byte-swizzled K-major tile that starts at `tile`: chunk 2c and 2c+1 of the row, each XOR-ed with row % 8.
-__device__ __forceinline__ void expand_int8x16(const uint4 x, uint8_t* tile, int row, int c) {
+// Sixteen int8 values (one 16-byte piece of a row of the raw block) -> sixteen bf16 values, written as the two 16-byte
+// chunks d0, d1 of the 128-byte-swizzled K-major tile that the caller has located.
+__device__ __forceinline__ void expand_int8x16(const uint4 x, uint8_t* d0, uint8_t* d1) {
   const uint32_t w[4] = {x.x, x.y, x.z, x.w};
   uint32_t o[8];
-  // byte b as n = b + 128 in 0..255 = 128 hi + lo:  b = (128 + lo) - (hi ? 128 : 256); the subtrahend's bits are
-  // 0x4380 (256) with bit 7 cleared when hi is set (0x4300 = 128)
+  // byte b = (128 + its low seven bits) - (256 if its sign bit is set, else 128); as bf16 bit patterns the minuend is
+  // 0x4300 | low bits and the subtrahend 0x4300 | sign bit (0x4380 = 256), so one byte permutation each puts two of
+  // them in a register next to the constant high byte 0x43
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
-    const uint32_t u = w[j] ^ 0x80808080u;
-    const uint32_t t0 = __byte_perm(u, 0u, 0x4140), t1 = __byte_perm(u, 0u, 0x4342);   // bytes 0,1 and 2,3 in 16-bit lanes
-    o[2 * j] = bf16x2_sub((t0 & 0x007F007Fu) | 0x43004300u, (t0 & 0x00800080u) ^ 0x43804380u);
-    o[2 * j + 1] = bf16x2_sub((t1 & 0x007F007Fu) | 0x43004300u, (t1 & 0x00800080u) ^ 0x43804380u);
+    const uint32_t lo = w[j] & 0x7F7F7F7Fu, sg = w[j] & 0x80808080u;
+    o[2 * j] = bf16x2_sub(__byte_perm(lo, 0x43434343u, 0x4140), __byte_perm(sg, 0x43434343u, 0x4140));       // bytes 0, 1
+    o[2 * j + 1] = bf16x2_sub(__byte_perm(lo, 0x43434343u, 0x4342), __byte_perm(sg, 0x43434343u, 0x4342));   // bytes 2, 3
   }
-  uint8_t* drow = tile + (row >> 3) * 1024 + (row & 7) * 128;
-  *reinterpret_cast<uint4*>(drow + (((2 * c) ^ (row & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
-  *reinterpret_cast<uint4*>(drow + (((2 * c + 1) ^ (row & 7)) << 4)) = make_uint4(o[4], o[5], o[6], o[7]);
+  *reinterpret_cast<uint4*>(d0) = make_uint4(o[0], o[1], o[2], o[3]);
+  *reinterpret_cast<uint4*>(d1) = make_uint4(o[4], o[5], o[6], o[7]);
 }
 
-// Thirty-two 4-bit codes (one 16-byte piece c, 0 or 1, of row `row` of the raw block; two's complement nibbles, even
-// entry in the low nibble) -> thirty-two bf16 values  code << shift  at their place in the 128-byte-swizzled K-major
-// tile: chunks 4c .. 4c+3 of the row, each XOR-ed with row % 8.  Every value (magnitude <= 7 * 2^4) is exact in bf16.
-__device__ __forceinline__ void expand_int4x32(const uint4 x, uint8_t* tile, int row, int c, int shift) {
+// Thirty-two 4-bit codes (one 16-byte piece of a row of the raw block; two's complement nibbles, even entry in the low
+// nibble) -> thirty-two bf16 values  code << shift, written as four 16-byte chunks of the 128-byte-swizzled K-major
+// tile: chunk j goes to d + ((16 j) ^ x3), d and x3 = 16 (row % 4) located by the caller.  Every value (magnitude
+// <= 7 * 2^4) is exact in bf16.
+__device__ __forceinline__ void expand_int4x32(const uint4 x, uint8_t* d, uint32_t x3, int shift) {
   const uint32_t w[4] = {x.x, x.y, x.z, x.w};
   // nibble n with its sign bit flipped is code + 8; (128 + code + 8) * 2^shift - 136 * 2^shift = code * 2^shift
   const uint32_t mul1 = static_cast<uint32_t>(127 + shift) << 7;           // bf16 bits of 2^shift
   const uint32_t mul = mul1 | (mul1 << 16);
   const uint32_t sub1 = 0xC308u + (static_cast<uint32_t>(shift) << 7);     // bf16 bits of -136 * 2^shift
   const uint32_t sub = sub1 | (sub1 << 16);
-  uint8_t* drow = tile + (row >> 3) * 1024 + (row & 7) * 128;
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
     const uint32_t u = w[j] ^ 0x88888888u;
@@ -555,7 +553,7 @@ __device__ __forceinline__ void expand_int4x32(const uint4 x, uint8_t* tile, int
     const uint32_t r2 = bf16x2_fma(((u >> 8) & 0x000F000Fu) | 0x43004300u, mul, sub);
     const uint32_t r3 = bf16x2_fma(((u >> 12) & 0x000F000Fu) | 0x43004300u, mul, sub);
     // back into channel order: (0,1) (2,3) (4,5) (6,7)
-    *reinterpret_cast<uint4*>(drow + (((4 * c + j) ^ (row & 7)) << 4)) =
+    *reinterpret_cast<uint4*>(d + ((16u * j) ^ x3)) =
         make_uint4(__byte_perm(r0, r1, 0x5410), __byte_perm(r2, r3, 0x5410), __byte_perm(r0, r1, 0x7632),
                    __byte_perm(r2, r3, 0x7632));
   }
@@ -637,11 +635,11 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < p.stages; ++i) {
-      mbar_init(full_bar + 8 * i, kW8 ? 2 + 2 * kConvWarps : 2);   // + every converter warp of the pair with 8-bit W_lm
+      mbar_init(full_bar + 8 * i, kW8 ? 2 + 2 * p.conv_group : 2);   // + the converter warps of a K block, both CTAs
       mbar_init(empty_bar + 8 * i, 1);
       if (kW8) {
         mbar_init(rawfull_bar + 8 * i, 1);
-        mbar_init(rawempty_bar + 8 * i, kConvWarps);
+        mbar_init(rawempty_bar + 8 * i, p.conv_group);
       }
     }
     for (int i = 0; i < 2; ++i) mbar_init(tfull_bar + 8 * i, 1);
@@ -678,20 +676,23 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
       uint32_t phase = 0;
       bool ok = true;
       grid_dependency_wait();                            // W_lm and the hidden rows may come from the kernel before
-      for (int t = 0; t < my_tiles && ok; ++t) {
-        const int v0 = (pair + t * npairs) * pair_rows + static_cast<int>(rank) * p.tile_rows;
-        int tile_width = 8, w_row = v0;                  // (mode 1) width of this tile's rows and where they are stored
-        if (kW8 && p.group_width) {
-          const int g = pair + t * npairs;
-          tile_width = p.group_width[g];
-          w_row = p.group_row[g] + static_cast<int>(rank) * p.tile_rows;
-        }
-        int kx = 0;                                      // K coordinate of the block, in elements
-        for (int kb = 0; kb < p.n_kblocks; ++kb, kx += kKStep) {
-          const uint32_t sa = base + stage * stage_bytes;
-          if (kW8) {
-            // only the raw tile: its slot is free again as soon as the converters have read it
+      if (kW8) {
+        // On-chip expansion: only the raw W_lm blocks.  The raw block of a slot may be refilled as soon as the
+        // converters have read it (16-bit rows, which go straight into the tile the MMA reads: once the MMAs of the
+        // slot's previous use are done as well).  The hidden blocks of a slot are fetched by the converter group that
+        // owns the K block, which waits for those MMAs anyway.
+        for (int t = 0; t < my_tiles && ok; ++t) {
+          int tile_width = 8;                              // width of this tile's rows and where they are stored
+          int w_row = (pair + t * npairs) * pair_rows + static_cast<int>(rank) * p.tile_rows;
+          if (p.group_width) {
+            const int g = pair + t * npairs;
+            tile_width = p.group_width[g];
+            w_row = p.group_row[g] + static_cast<int>(rank) * p.tile_rows;
+          }
+          int kx = 0;
+          for (int kb = 0; kb < p.n_kblocks; ++kb, kx += kKStep) {
             if (!mbar_wait(rawempty_bar + 8 * stage, phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
+            const uint32_t sa = base + stage * stage_bytes;
             const uint32_t rb = own_rawfull + 8 * stage;
             if (tile_width == 8) {
               mbar_expect_tx_cluster(rb, raw_tx_bytes);
@@ -699,31 +700,38 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
             } else if (tile_width == 4) {                  // two codes per byte: 32 bytes per row and K block
               mbar_expect_tx_cluster(rb, raw_tx_bytes >> 1);
               tma_load_2d(sa + raw_off, &tmap_w4, rb, kx >> 1, w_row, pol_w);
-            } else {                                       // bf16 rows go straight into the tile the MMA reads,
+            } else {
               if (!mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
-              mbar_expect_tx_cluster(rb, raw_tx_bytes << 1);   // once the MMAs of its previous use are done
+              mbar_expect_tx_cluster(rb, raw_tx_bytes << 1);
               tma_load_2d(sa, &tmap_w16, rb, kx, w_row, pol_w);
             }
+            if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+          }
+        }
+      } else
+      for (int t = 0; t < my_tiles && ok; ++t) {
+        const int v0 = (pair + t * npairs) * pair_rows + static_cast<int>(rank) * p.tile_rows;
+        int kx = 0;                                      // K coordinate of the block, in elements
+        for (int kb = 0; kb < p.n_kblocks; ++kb, kx += kKStep) {
+          const uint32_t sa = base + stage * stage_bytes;
+          if (!mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
+          const uint32_t fb = leader_full + 8 * stage;
+          mbar_expect_tx_cluster(fb, tx_bytes);
+          tma_load_2d(sa, &tmap_w, fb, kx, v0, pol_w);
+          if (kRot && p.pair256) {
+            // Row blocks 0, 1, 2 (128 rows each) sit on units (3t, 3t+1, 3t+2) mod 4.  Two of them that are adjacent
+            // without wrapping (blocks 0, 1, or blocks 1, 2 when the tile starts on unit 3) share one MMA of N = 256:
+            // this CTA then supplies ONE of the two blocks whole, and its half of the third block as before.
+            const bool late_pair = ((3 * t) & 3) == 3;
+            const int pair_row = (late_pair ? 128 : 0) + static_cast<int>(rank) * 128;
+            const int single_row = (late_pair ? 0 : 256) + static_cast<int>(rank) * 64;
+            tma_load_2d(sa + kWBlockBytes, &tmap_hidden, fb, kx, p.row0 + pair_row, pol_h);
+            tma_load_2d(sa + kWBlockBytes + hid_block_bytes, &tmap_hidden, fb, kx, p.row0 + pair_row + 64, pol_h);
+            tma_load_2d(sa + kWBlockBytes + 2 * hid_block_bytes, &tmap_hidden, fb, kx, p.row0 + single_row, pol_h);
           } else {
-            if (!mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
-            const uint32_t fb = leader_full + 8 * stage;
-            mbar_expect_tx_cluster(fb, tx_bytes);
-            tma_load_2d(sa, &tmap_w, fb, kx, v0, pol_w);
-            if (kRot && p.pair256) {
-              // Row blocks 0, 1, 2 (128 rows each) sit on units (3t, 3t+1, 3t+2) mod 4.  Two of them that are adjacent
-              // without wrapping (blocks 0, 1, or blocks 1, 2 when the tile starts on unit 3) share one MMA of N = 256:
-              // this CTA then supplies ONE of the two blocks whole, and its half of the third block as before.
-              const bool late_pair = ((3 * t) & 3) == 3;
-              const int pair_row = (late_pair ? 128 : 0) + static_cast<int>(rank) * 128;
-              const int single_row = (late_pair ? 0 : 256) + static_cast<int>(rank) * 64;
-              tma_load_2d(sa + kWBlockBytes, &tmap_hidden, fb, kx, p.row0 + pair_row, pol_h);
-              tma_load_2d(sa + kWBlockBytes + hid_block_bytes, &tmap_hidden, fb, kx, p.row0 + pair_row + 64, pol_h);
-              tma_load_2d(sa + kWBlockBytes + 2 * hid_block_bytes, &tmap_hidden, fb, kx, p.row0 + single_row, pol_h);
-            } else {
-              for (int s = 0; s < p.n_sub; ++s)
-                tma_load_2d(sa + kWBlockBytes + s * hid_block_bytes, &tmap_hidden, fb, kx,
-                            (kTwoPlane ? 2 : 1) * p.row0 + s * p.N + static_cast<int>(rank) * half_n, pol_h);
-            }
+            for (int s = 0; s < p.n_sub; ++s)
+              tma_load_2d(sa + kWBlockBytes + s * hid_block_bytes, &tmap_hidden, fb, kx,
+                          (kTwoPlane ? 2 : 1) * p.row0 + s * p.N + static_cast<int>(rank) * half_n, pol_h);
           }
           if (++stage == p.stages) { stage = 0; phase ^= 1u; }
         }
@@ -1112,84 +1120,125 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
         }
       }
     }
-  } else if (warp == kW8HiddenWarp) {
-    // ------------------------------------------------------------------ 8-bit W_lm: TMA producer of the hidden blocks
-    if (elect_one()) {
-      const uint64_t pol_h = l2_policy_evict_last();
-      const uint32_t leader_full = map_to_cta(full_bar, 0);
-      int stage = 0;
-      uint32_t phase = 0;
-      bool ok = true;
-      grid_dependency_wait();
-      for (int t = 0; t < my_tiles && ok; ++t) {
-        int kx = 0;
-        for (int kb = 0; kb < p.n_kblocks; ++kb, kx += kKStep) {
-          if (!mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
-          const uint32_t sa = base + stage * stage_bytes;
-          const uint32_t fb = leader_full + 8 * stage;
-          mbar_expect_tx_cluster(fb, hid_tx_bytes);
-          for (int s = 0; s < p.n_sub; ++s)
-            tma_load_2d(sa + kWBlockBytes + s * hid_block_bytes, &tmap_hidden, fb, kx,
-                        (kTwoPlane ? 2 : 1) * p.row0 + s * p.N + static_cast<int>(rank) * half_n, pol_h);
-          if (++stage == p.stages) { stage = 0; phase ^= 1u; }
-        }
-      }
-    }
-  } else {
+  } else if (kW8) {
     // ------------------------------------------------------------------ 8-bit W_lm: converter warps
     // int8 [tile_rows][64] (row pitch 64 bytes) -> bf16 [tile_rows][64] in the 128-byte-swizzled K-major layout the
     // MMA reads: 16-byte chunk c of row r sits at chunk position c ^ (r % 8) of its 128-byte row.  Every int8 value is
     // exact in bf16; the row's scale is applied to the accumulators by the epilogue warps.
-    // All converter warps share every K block (two independent 16-byte pieces per thread), in ring order.
-    const int cw = warp < kW8HiddenWarp ? warp - (2 + kW8EpiWarps) : warp - (kW8HiddenWarp + 1) + (kW8HiddenWarp - 2 - kW8EpiWarps);
-    const int ct = cw * 32 + lane;
+    // The converter warps form groups of conv_group warps; each group owns whole K blocks, every ngroups-th one of the
+    // CTA's sequence of blocks.  The waits, the expansion and the fence of one block are a chain of dependent steps:
+    // several groups run such chains side by side (ring slots permitting), several warps in a group shorten the chain.
+    const int cw = warp - (2 + kW8EpiWarps);
     const uint32_t leader_full = map_to_cta(full_bar, 0);
     const int units = p.tile_rows * 4;                   // 16-byte pieces of the int8 tile
-    int stage = 0;
-    uint32_t phase = 0;
-    bool ok = true;
+    const uint64_t pol_h = l2_policy_evict_last();       // hidden is re-read for every tile
+    const int total_blocks = my_tiles * p.n_kblocks;
     grid_dependency_wait();                              // the width table and the exponents may come from the kernel before
-    for (int t = 0; t < my_tiles && ok; ++t) {
-      int tile_width = 8, w_row = 0;                     // width of this tile's rows; first row in the 4-bit buffer
+    // No more groups than ring slots take part: a group that starts block i has finished block i - ngroups, whose slot
+    // had been freed by the MMAs of block i - ngroups - stages, so with ngroups <= stages every barrier it waits on is at
+    // most one phase behind and the parity waits below cannot mistake "two trips round the ring ago" for "done".
+    const int G = p.conv_group;
+    const int ngroups = min(kConvWarps / G, p.stages);
+    const int grp = cw / G, mem = cw - grp * G;          // warps beyond ngroups * G groups stay idle
+    const int step = 32 * G;                             // pieces the group expands per trip of its loops
+    const int first = mem * 32 + lane;                   // this lane's first piece
+    int t = 0, kb = grp;                                 // block i = t * n_kblocks + kb of the sequence, i % ngroups == grp
+    while (kb >= p.n_kblocks && t < my_tiles) { kb -= p.n_kblocks; ++t; }
+    // Where this lane's pieces go does not change from block to block.  8-bit: piece u is the 16 bytes c = u % 4 of row
+    // u / 4 and becomes chunks 2c, 2c+1 of the row's 128 bytes in the tile, each XOR-ed with row % 8 (128-byte swizzle;
+    // the row itself starts at row * 128); a step of the loop moves on by a multiple of 8 rows.  4-bit: piece u is half
+    // c = u % 2 of row u / 2 and becomes chunks 4c .. 4c+3.
+    const uint32_t off8 = static_cast<uint32_t>(first >> 2) * 128u + (((2u * (first & 3)) ^ ((first >> 2) & 7u)) << 4);
+    const uint32_t off4 = static_cast<uint32_t>(first >> 1) * 128u + (((4u * (first & 1)) ^ ((first >> 1) & 4u)) << 4);
+    const uint32_t x3 = ((first >> 1) & 3u) << 4;
+    const uint32_t raw_step = static_cast<uint32_t>(step) * 16u;          // bytes of the raw block per step
+    const uint32_t tile_step8 = static_cast<uint32_t>(step) * 32u;        // 8 G rows of the tile
+    const uint32_t tile_step4 = static_cast<uint32_t>(step) * 64u;        // 16 G rows of the tile
+    // Width of a tile's rows and where they start in the buffer of that width (4-bit: for the exponents).
+    auto tile_info = [&](int tt, int& width, int& wrow) {
+      width = 8; wrow = 0;
       if (p.group_width) {
-        const int g = pair + t * npairs;
-        tile_width = p.group_width[g];
-        w_row = p.group_row[g] + static_cast<int>(rank) * p.tile_rows;
+        const int g = pair + tt * npairs;
+        width = p.group_width[g];
+        wrow = p.group_row[g] + static_cast<int>(rank) * p.tile_rows;
       }
-      for (int kb = 0; kb < p.n_kblocks; ++kb) {
-        if (!mbar_wait_warp(rawfull_bar + 8 * stage, phase, abort_flag, p.status) ||
-            !mbar_wait_warp(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
-        uint8_t* slot = smem + stage * stage_bytes;
-        if (tile_width == 8) {
-          for (int u0 = ct; u0 < units; u0 += 2 * kConvThreads) {
-            const int u1 = u0 + kConvThreads;
-            const bool has1 = u1 < units;
-            const uint4 x0 = *reinterpret_cast<const uint4*>(slot + raw_off + (u0 >> 2) * 64 + (u0 & 3) * 16);
-            uint4 x1 = make_uint4(0u, 0u, 0u, 0u);
-            if (has1) x1 = *reinterpret_cast<const uint4*>(slot + raw_off + (u1 >> 2) * 64 + (u1 & 3) * 16);
-            expand_int8x16(x0, slot, u0 >> 2, u0 & 3);
-            if (has1) expand_int8x16(x1, slot, u1 >> 2, u1 & 3);
-          }
-        } else if (tile_width == 4) {
-          // 32-byte rows: two 16-byte pieces per row; a sub-block of 128 hidden channels spans two K blocks
-          const uint8_t* sh = p.shift4 + static_cast<size_t>(kb >> 1) * p.rows4;
-          for (int u0 = ct; u0 < (units >> 1); u0 += kConvThreads) {
-            const int row = u0 >> 1, c = u0 & 1;
-            const uint4 x0 = *reinterpret_cast<const uint4*>(slot + raw_off + row * 32 + c * 16);
-            const int r4 = w_row + row;
-            const int shift = (r4 >= 0 && r4 < p.rows4) ? min(static_cast<int>(sh[r4]), 4) : 0;
-            expand_int4x32(x0, slot, row, c, shift);
-          }
-        }
-        // (16-bit rows were loaded into the tile as they are)
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // generic-proxy writes, read by the MMA
-        __syncwarp();
-        if (lane == 0) {
-          mbar_arrive_cluster(leader_full + 8 * stage);  // this warp's share of the bf16 tile is in place
-          mbar_arrive(rawempty_bar + 8 * stage);         // and the raw block may be refilled
-        }
-        if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+    };
+    // (4-bit) the exponents of this lane's rows in K block kkb: a sub-block of 128 hidden channels spans two K blocks
+    auto fetch_shifts = [&](int kkb, int width, int wrow, uint32_t (&e)[8]) {
+      const uint8_t* sh = p.shift4 + static_cast<size_t>(kkb >> 1) * p.rows4;
+#pragma unroll
+      for (int n = 0; n < 8; ++n) {
+        const int row = (first + step * n) >> 1;
+        const int r4 = wrow + row;
+        e[n] = (width == 4 && row < p.tile_rows && r4 >= 0 && r4 < p.rows4) ? sh[r4] : 0u;
       }
+    };
+    int tile_width, w_row;
+    uint32_t e[8];
+    if (grp < ngroups && grp < total_blocks) {
+      tile_info(t, tile_width, w_row);
+      fetch_shifts(kb, tile_width, w_row, e);
+    }
+    for (int i = grp; i < total_blocks && grp < ngroups; i += ngroups) {
+      const int stage = i % p.stages;
+      const uint32_t phase = static_cast<uint32_t>(i / p.stages) & 1u;
+      uint8_t* slot = smem + stage * stage_bytes;
+      uint32_t shifts = 0;                               // one nibble per step
+#pragma unroll
+      for (int n = 0; n < 8; ++n) shifts |= min(e[n], 4u) << (4 * n);
+      // the group's next block: its exponents are fetched while this block is waited for and expanded
+      int t2 = t, kb2 = kb + ngroups, width2 = tile_width, w_row2 = w_row;
+      while (kb2 >= p.n_kblocks) { kb2 -= p.n_kblocks; ++t2; }
+      if (i + ngroups < total_blocks) {
+        if (t2 != t) tile_info(t2, width2, w_row2);
+        fetch_shifts(kb2, width2, w_row2, e);
+      }
+      // first the slot's previous use (which implies that its raw block's previous phase is over), then this block's bytes
+      if (!mbar_wait_warp(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.status)) break;
+      if (mem == 0 && lane == 0) {                       // the slot is free: its hidden blocks arrive while the W_lm block is expanded
+        const uint32_t sa = base + stage * stage_bytes;
+        const uint32_t fb = leader_full + 8 * stage;
+        mbar_expect_tx_cluster(fb, hid_tx_bytes);
+        for (int sb = 0; sb < p.n_sub; ++sb)
+          tma_load_2d(sa + kWBlockBytes + sb * hid_block_bytes, &tmap_hidden, fb, kb * kKStep,
+                      p.row0 + sb * p.N + static_cast<int>(rank) * half_n, pol_h);
+      }
+      if (!mbar_wait_warp(rawfull_bar + 8 * stage, phase, abort_flag, p.status)) break;
+      // Two pieces per trip of a loop that is kept rolled: the expansion of a whole block written out is some ten
+      // thousand bytes of straight-line code per width, which a warp would fetch anew for every block (measured: rolled
+      // is faster, and four pieces per trip are no faster than two).
+      const uint8_t* src = slot + raw_off + first * 16;
+      if (tile_width == 8) {
+        uint32_t o = off8;
+#pragma unroll 1
+        for (int u0 = first; u0 < units; u0 += 2 * step, src += 2 * raw_step, o += 2 * tile_step8) {
+          const bool two = u0 + step < units;
+          const uint4 x0 = *reinterpret_cast<const uint4*>(src);
+          const uint4 x1 = two ? *reinterpret_cast<const uint4*>(src + raw_step) : make_uint4(0u, 0u, 0u, 0u);
+          expand_int8x16(x0, slot + o, slot + (o ^ 16u));
+          if (two) expand_int8x16(x1, slot + o + tile_step8, slot + ((o + tile_step8) ^ 16u));
+        }
+      } else if (tile_width == 4) {
+        uint32_t o = off4;
+#pragma unroll 1
+        for (int n = 0; n < 8; n += 2, src += 2 * raw_step, o += 2 * tile_step4) {   // 32-byte rows: two pieces per row
+          const int u0 = first + step * n;
+          if (u0 >= (units >> 1)) break;
+          const bool two = u0 + step < (units >> 1);
+          const uint4 x0 = *reinterpret_cast<const uint4*>(src);
+          const uint4 x1 = two ? *reinterpret_cast<const uint4*>(src + raw_step) : make_uint4(0u, 0u, 0u, 0u);
+          expand_int4x32(x0, slot + o, x3, static_cast<int>((shifts >> (4 * n)) & 15u));
+          if (two) expand_int4x32(x1, slot + o + tile_step4, x3, static_cast<int>((shifts >> (4 * n + 4)) & 15u));
+        }
+      }
+      // (16-bit rows were loaded into the tile as they are)
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // generic-proxy writes, read by the MMA
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive_cluster(leader_full + 8 * stage);    // this warp's share of the bf16 tile is in place
+        mbar_arrive(rawempty_bar + 8 * stage);           // and the raw block may be refilled
+      }
+      t = t2; kb = kb2; tile_width = width2; w_row = w_row2;
     }
   }
 
@@ -1963,6 +2012,7 @@ struct hola_ctx {
   int no_rot;                 // tuning override: never use the rotating accumulator units
   int force_passes;           // tuning override: passes over W_lm (0: chosen by cost)
   int no_pair256;             // tuning override: rotating units always as three MMAs of N = 128
+  int conv_group;             // tuning override (0 = by plan): converter warps per K block in the on-chip expansion
   int host_in_place;          // hola_verify_host: read draft rows not sent ahead in place from pinned host memory
   cudaStream_t copy_stream;   // hola_verify_host: the draft tensor travels here while the GEMM runs
   cudaEvent_t copy_done;
@@ -2242,6 +2292,7 @@ hola_status run_lm_head(hola_ctx* ctx, const hola_verify_args* a, float* logits,
   K1Params kp;
   kp.M = M; kp.V = a->V; kp.n_ptiles = pl.n_ptiles; kp.n_kblocks = pl.n_kblocks;
   kp.pair256 = (pl.rot && pl.N == 128 && !ctx->no_pair256) ? 1 : 0;
+  kp.conv_group = ctx->conv_group > 0 ? ctx->conv_group : 2;
   kp.stages = pl.stages; kp.nbuf = pl.nbuf; kp.rot = pl.rot; kp.n_sub = pl.n_sub; kp.N = pl.N; kp.tile_rows = pl.tile_rows; kp.ldl = ldl;
   kp.logits = logits; kp.partials = ctx->partials; kp.part_stride = ctx->max_rows;
   kp.status = a->status_word ? a->status_word : ctx->status;
@@ -2548,6 +2599,10 @@ hola_status hola_set_option(hola_ctx* ctx, int option, int value) {
     case HOLA_OPT_ROTATING_UNITS: ctx->no_rot = value == 0; break;
     case HOLA_OPT_PAIR_MMA: ctx->no_pair256 = value == 0; break;
     case HOLA_OPT_HOST_IN_PLACE: ctx->host_in_place = value != 0; break;
+    case HOLA_OPT_CONVERTER_GROUP:
+      if (value < 0 || value > kConvWarps) return HOLA_ERR_INVALID_ARG;
+      ctx->conv_group = value;
+      break;
     case HOLA_OPT_PASSES:
       if (value < 0 || value > 64) return HOLA_ERR_INVALID_ARG;
       ctx->force_passes = value;

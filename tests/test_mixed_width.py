@@ -149,3 +149,29 @@ def test_mixed_width_on_the_bandwidth_bound_shapes(binding, name):
                           _np(out.entropy[pick]), _np(out.logZ[pick]), _np(out.logits[pick]))
     print(name, rep.summary())
     assert rep.ok, rep.summary()
+
+
+def test_converter_group_size_changes_speed_not_results(binding):
+    """The number of converter warps that share a K block is a speed knob: the expansion is exact whoever does it, so
+    every setting gives the same logits bit for bit (few K blocks, many K blocks, more groups than ring slots in use)."""
+    for B, k, H, V in ((3, 2, 128, 1300), (40, 4, 1024, 2600)):
+        w = workloads.gaussian_head("conv-group", B, k, H, V, seed=V, device=DEV, w_std=0.3, sigma=1.0, tau=1.7)
+        head = binding.hola_quantize_mixed(w.W_lm, _widths(V, [4, 8, 16, 8, 4]))
+        with binding.HolaVerify(B, k, H, V) as ctx:
+            base = ctx.hola_verify(w.hidden, head, w.draft_tok, w.draft_q, w.uniforms, w.tau, want_logits=True)
+            torch.cuda.synchronize()
+            assert int(base.status.item()) == 0
+            for G in (1, 2, 3, 4, 8, 0):
+                ctx.hola_set_option(binding.HOLA_OPT_CONVERTER_GROUP, G)
+                out = ctx.hola_verify(w.hidden, head, w.draft_tok, w.draft_q, w.uniforms, w.tau, want_logits=True)
+                torch.cuda.synchronize()
+                assert int(out.status.item()) == 0, G
+                assert torch.equal(out.logits, base.logits), G
+                assert torch.equal(out.accept_len, base.accept_len) and torch.equal(out.next_tok, base.next_tok)
+            for bad in (-1, 9):
+                with pytest.raises(binding.HolaError):
+                    ctx.hola_set_option(binding.HOLA_OPT_CONVERTER_GROUP, bad)
+    orc = _mixed_oracle(w, _widths(V, [4, 8, 16, 8, 4]))
+    rep = compare.compare(orc, _np(w.draft_q), _np(w.uniforms), _np(base.accept_len), _np(base.next_tok),
+                          _np(base.entropy), _np(base.logZ), _np(base.logits))
+    assert rep.ok, rep.summary()
