@@ -576,7 +576,7 @@ def run_vocab_parallel(args, rank: int, world: int, local: int, dev):
                 "clocks": clocks,
                 "e2e": {"value": w.M * args.e2e_steps / (e2e_total * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                         "d2h_bytes_per_step": d2h, "ms_per_step": e2e_total / args.e2e_steps},
-                "gpu_launches": (sh.ctx.hola_plan(w.B, w.k)["passes"] + 3) * args.steps,
+                "gpu_launches": (sh.ctx.hola_plan(w.B, w.k)["kernels_per_call"] + 2) * args.steps,
                 "accepted_tokens_per_s": accepted * args.steps / (ms_total * 1e-3),
                 "roofline": roof}
         print(json.dumps(line), flush=True)

@@ -20,7 +20,7 @@ HOLA_FALLBACK_SAMPLE, HOLA_FALLBACK_GREEDY = 0, 1
 HOLA_W_BF16, HOLA_W_INT8, HOLA_W8A8, HOLA_W8A16, HOLA_W_MIXED = 0, 1, 2, 3, 4
 GROUP_ROWS, SUB_BLOCK = 256, 128
 FLAG_BAD_TOKEN, FLAG_BAD_UNIFORM, FLAG_TIMEOUT, FLAG_R_ZERO = 1, 2, 4, 8
-HOLA_OPT_RING_SLOTS, HOLA_OPT_ROTATING_UNITS, HOLA_OPT_HOST_OVERLAP, HOLA_OPT_HOST_ROWS_ON_DEMAND, HOLA_OPT_PASSES, HOLA_OPT_PAIR_MMA, HOLA_OPT_HOST_IN_PLACE, HOLA_OPT_CONVERTER_GROUP = 1, 2, 3, 4, 5, 6, 7, 8
+HOLA_OPT_RING_SLOTS, HOLA_OPT_ROTATING_UNITS, HOLA_OPT_HOST_OVERLAP, HOLA_OPT_HOST_ROWS_ON_DEMAND, HOLA_OPT_PASSES, HOLA_OPT_PAIR_MMA, HOLA_OPT_HOST_IN_PLACE, HOLA_OPT_CONVERTER_GROUP, HOLA_OPT_FUSED_PASSES = 1, 2, 3, 4, 5, 6, 7, 8, 9
 
 EXPORTS = ["hola_create", "hola_destroy", "hola_workspace_bytes", "hola_verify", "hola_verify_host",
            "hola_lm_head_entropy", "hola_accept_sample", "hola_host_traffic", "hola_shard_record_bytes", "hola_shard_lm_head",

@@ -92,6 +92,8 @@ struct K1Params {
   int M;          // total verify rows B(k+1)
   int row0;       // first row of this pass
   int rows;       // rows of this pass (<= n_sub * N)
+  int n_pass;     // > 1: all passes in this launch; CTA pair i works on pass i % n_pass (rows from row0 + that many
+  int rows_per_pass;   // times rows_per_pass on) and shares the vocabulary tiles with the pairs i / n_pass, see the kernel
   int V, n_ptiles, n_kblocks, stages, nbuf;
   int n_sub, N;   // MMAs per K step and their N (verify rows each; multiple of 16)
   int rot;        // 1: three MMAs of N <= 128 per K step whose accumulators rotate over the four 128-column units
@@ -247,6 +249,11 @@ __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, vo
 __device__ __forceinline__ uint64_t l2_policy_evict_first() {
   uint64_t pol;
   asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_normal() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(pol));
   return pol;
 }
 __device__ __forceinline__ uint64_t l2_policy_evict_last() {
@@ -613,8 +620,14 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
   const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0);   // same value in all lanes, and the compiler knows it
   const int lane = threadIdx.x & 31;
   const uint32_t rank = cluster_cta_rank();              // 0 = leader of the pair
-  const int pair = blockIdx.x >> 1;
-  const int npairs = gridDim.x >> 1;
+  // One pass per launch: pair i of npairs takes the vocabulary tiles i, i + npairs, ...  All passes in one launch
+  // (n_pass > 1): n_pass neighbouring pairs form a group that walks the same tiles at the same time, one pass of the
+  // verify rows each, so that a tile of W_lm comes from HBM once and reaches the other pairs of the group out of the L2.
+  const int pair_of_grid = blockIdx.x >> 1;
+  const int pair = p.n_pass > 1 ? pair_of_grid / p.n_pass : pair_of_grid;          // which tiles
+  const int npairs = p.n_pass > 1 ? (gridDim.x >> 1) / p.n_pass : gridDim.x >> 1;
+  const int row0 = p.n_pass > 1 ? (pair_of_grid - pair * p.n_pass) * p.rows_per_pass : p.row0;
+  const int rows = p.n_pass > 1 ? min(p.rows_per_pass, p.M - row0) : p.rows;
   const int half_n = p.N >> 1;                           // hidden rows this CTA supplies per MMA
   const uint32_t hid_block_bytes = static_cast<uint32_t>(half_n) * 128u;
   const uint32_t raw_off = kWBlockBytes + p.n_sub * hid_block_bytes;     // int8 block of the slot (8-bit W_lm only)
@@ -668,7 +681,8 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (one per CTA)
     if (elect_one()) {
-      const uint64_t pol_w = l2_policy_evict_first();    // W_lm is streamed once
+      // W_lm is streamed once; with all passes in one launch the other pairs of the group read the tile out of the L2
+      const uint64_t pol_w = p.n_pass > 1 ? l2_policy_evict_normal() : l2_policy_evict_first();
       const uint64_t pol_h = l2_policy_evict_last();     // hidden is re-read for every tile
       const uint32_t leader_full = map_to_cta(full_bar, 0);
       const uint32_t own_rawfull = map_to_cta(rawfull_bar, rank);
@@ -725,13 +739,13 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
             const bool late_pair = ((3 * t) & 3) == 3;
             const int pair_row = (late_pair ? 128 : 0) + static_cast<int>(rank) * 128;
             const int single_row = (late_pair ? 0 : 256) + static_cast<int>(rank) * 64;
-            tma_load_2d(sa + kWBlockBytes, &tmap_hidden, fb, kx, p.row0 + pair_row, pol_h);
-            tma_load_2d(sa + kWBlockBytes + hid_block_bytes, &tmap_hidden, fb, kx, p.row0 + pair_row + 64, pol_h);
-            tma_load_2d(sa + kWBlockBytes + 2 * hid_block_bytes, &tmap_hidden, fb, kx, p.row0 + single_row, pol_h);
+            tma_load_2d(sa + kWBlockBytes, &tmap_hidden, fb, kx, row0 + pair_row, pol_h);
+            tma_load_2d(sa + kWBlockBytes + hid_block_bytes, &tmap_hidden, fb, kx, row0 + pair_row + 64, pol_h);
+            tma_load_2d(sa + kWBlockBytes + 2 * hid_block_bytes, &tmap_hidden, fb, kx, row0 + single_row, pol_h);
           } else {
             for (int s = 0; s < p.n_sub; ++s)
               tma_load_2d(sa + kWBlockBytes + s * hid_block_bytes, &tmap_hidden, fb, kx,
-                          (kTwoPlane ? 2 : 1) * p.row0 + s * p.N + static_cast<int>(rank) * half_n, pol_h);
+                          (kTwoPlane ? 2 : 1) * row0 + s * p.N + static_cast<int>(rank) * half_n, pol_h);
           }
           if (++stage == p.stages) { stage = 0; phase ^= 1u; }
         }
@@ -892,7 +906,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
             const int pr = group + slot * kGroups;
             const int sub = (64 * pr) / p.N, col = 64 * pr - sub * p.N;
             const uint32_t taddr = lane_addr + buf * 256 + sub * 256 + col;
-            const int vr0 = p.row0 + 32 * pr;            // verify row of the pair's first column
+            const int vr0 = row0 + 32 * pr;            // verify row of the pair's first column
             const int n_ok = min(32, p.M - vr0);
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
@@ -972,7 +986,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
 #pragma unroll
           for (int slot = 0; slot < 3; ++slot) {
             const int c0 = group * 32;                   // first column of the chunk inside its MMA
-            const int r0 = p.row0 + slot * p.N + c0;     // verify row of column c0
+            const int r0 = row0 + slot * p.N + c0;     // verify row of column c0
             const int n_ok = min(32, min(p.N - c0, p.M - r0));   // columns that are real rows
             if (n_ok > 0) {
 #pragma unroll
@@ -1045,7 +1059,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
             if (lane == 0) mbar_arrive_cluster(leader_tempty + 8 * (rot ? unit : buf));
           }
           const int c0 = j * 32;                         // first column of the chunk inside its MMA
-          const int r0 = p.row0 + sub * p.N + c0;        // verify row of column c0
+          const int r0 = row0 + sub * p.N + c0;        // verify row of column c0
           const int n_ok = min(32, min(p.N - c0, p.M - r0));   // columns that are real rows
           if (n_ok > 0) {
 #pragma unroll
@@ -1109,14 +1123,14 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
         a = stats_merge(a, o);
         if (kTwoPlane) {
           const int r = 32 * (group + slot * kGroups) + half * kTransRows + trow;   // row inside the pass
-          if (slot < 2 && thalf == 0 && r < p.rows)
-            merge[quarter * p.rows + r] = make_float4(a.m, a.s, a.t, __int_as_float(a.arg));
+          if (slot < 2 && thalf == 0 && r < rows)
+            merge[quarter * rows + r] = make_float4(a.m, a.s, a.t, __int_as_float(a.arg));
         } else if (slot < my_chunks && thalf == 0) {
           const int ch = rot ? slot * sub_chunks + group : group + slot * kGroups;
           const int sub = ch / sub_chunks, j = ch - sub * sub_chunks;
           const int c = j * 32 + half * kTransRows + trow;           // column inside its MMA
           const int r = sub * p.N + c;                               // row inside the pass
-          if (c < p.N && r < p.rows) merge[quarter * p.rows + r] = make_float4(a.m, a.s, a.t, __int_as_float(a.arg));
+          if (c < p.N && r < rows) merge[quarter * rows + r] = make_float4(a.m, a.s, a.t, __int_as_float(a.arg));
         }
       }
     }
@@ -1201,7 +1215,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
         mbar_expect_tx_cluster(fb, hid_tx_bytes);
         for (int sb = 0; sb < p.n_sub; ++sb)
           tma_load_2d(sa + kWBlockBytes + sb * hid_block_bytes, &tmap_hidden, fb, kb * kKStep,
-                      p.row0 + sb * p.N + static_cast<int>(rank) * half_n, pol_h);
+                      row0 + sb * p.N + static_cast<int>(rank) * half_n, pol_h);
       }
       if (!mbar_wait_warp(rawfull_bar + 8 * stage, phase, abort_flag, p.status)) break;
       // Two pieces per trip of a loop that is kept rolled: the expansion of a whole block written out is some ten
@@ -1250,15 +1264,22 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
   if (!*abort_flag) {
     // one partial per CTA and row: the four quarters merged
     const float4* merge = reinterpret_cast<const float4*>(trans_base);
-    for (int r = threadIdx.x; r < p.rows; r += kK1Threads) {
+    for (int r = threadIdx.x; r < rows; r += kK1Threads) {
       Stats a = stats_empty();
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
-        const float4 x = merge[q * p.rows + r];
+        const float4 x = merge[q * rows + r];
         a = stats_merge(a, Stats{x.x, x.y, x.z, __float_as_int(x.w)});
       }
-      p.partials[static_cast<size_t>(blockIdx.x) * p.part_stride + p.row0 + r] =
+      p.partials[static_cast<size_t>(blockIdx.x) * p.part_stride + row0 + r] =
           make_float4(a.m, a.s, a.t, __int_as_float(a.arg));
+    }
+    if (p.n_pass > 1) {
+      // the accept/sample kernel merges the partials of every CTA for every row: this CTA has seen only its pass
+      const Stats none = stats_empty();
+      const float4 blank = make_float4(none.m, none.s, none.t, __int_as_float(none.arg));
+      for (int r = threadIdx.x; r < p.M; r += kK1Threads)
+        if (r < row0 || r >= row0 + rows) p.partials[static_cast<size_t>(blockIdx.x) * p.part_stride + r] = blank;
     }
   }
   cluster_sync_execution_only();                         // the peer no longer signals this CTA's barriers or tensor memory
@@ -1978,6 +1999,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 struct Plan {
   int n_sub, N, rows_per_pass, passes, grid, stages, nbuf, rot, n_ptiles, n_kblocks, smem_bytes, tile_rows;
+  int fused;            // all passes in one launch, groups of `passes` CTA pairs sharing the vocabulary tiles
   double est_seconds;   // rough duration of all passes (the cost the split was chosen by)
 };
 
@@ -2012,6 +2034,7 @@ struct hola_ctx {
   int no_rot;                 // tuning override: never use the rotating accumulator units
   int force_passes;           // tuning override: passes over W_lm (0: chosen by cost)
   int no_pair256;             // tuning override: rotating units always as three MMAs of N = 128
+  int no_fuse;                // tuning override: several passes always as one launch each
   int conv_group;             // tuning override (0 = by plan): converter warps per K block in the on-chip expansion
   int host_in_place;          // hola_verify_host: read draft rows not sent ahead in place from pinned host memory
   cudaStream_t copy_stream;   // hola_verify_host: the draft tensor travels here while the GEMM runs
@@ -2106,7 +2129,8 @@ Plan make_plan(const hola_ctx* ctx, int M, int w_dtype = HOLA_W_BF16) {
   const int max_rows_per_pass = (w8 || two) ? kMaxN : kMaxRowsPerPass;
   const int p_min = (rows + max_rows_per_pass - 1) / max_rows_per_pass;
   const double t_hbm = (w8 || i8 ? 1.0 : 2.0) * ctx->V * static_cast<double>(ctx->H) / 6.4e12;
-  for (int passes = p_min; passes <= p_min + 3; ++passes) {
+  const int p_max = ctx->force_passes > p_min + 3 ? ctx->force_passes : p_min + 3;
+  for (int passes = p_min; passes <= p_max; ++passes) {
     if (ctx->force_passes && passes != ctx->force_passes && ctx->force_passes >= p_min) continue;
     const int r = (rows + passes - 1) / passes;
     // up to 256 rows: one MMA, two accumulator buffers; up to 384: three MMAs of N <= 128 on rotating 128-column
@@ -2140,7 +2164,11 @@ Plan make_plan(const hola_ctx* ctx, int M, int w_dtype = HOLA_W_BF16) {
   // Vocabulary rows per CTA per tile: the smallest multiple of 4 that covers V in the fewest whole rounds over
   // all pairs, so that every pair streams the same number of bytes (V = 32000 on 74 pairs: 2 rounds of 112 + 112
   // rows instead of 1.69 rounds of 128 + 128).
-  const int pairs = ctx->num_sms / 2 > 0 ? ctx->num_sms / 2 : 1;
+  const int all_pairs = ctx->num_sms / 2 > 0 ? ctx->num_sms / 2 : 1;
+  // Several passes: one launch in which `passes` neighbouring pairs walk the same tiles together, one pass each (W_lm
+  // then leaves HBM once, not once per pass), as long as every pass gets a pair.
+  best.fused = (best.passes > 1 && !ctx->no_fuse && all_pairs / best.passes >= 1) ? 1 : 0;
+  const int pairs = best.fused ? all_pairs / best.passes : all_pairs;     // pairs that divide the tiles among them
   const int rounds = (ctx->V + pairs * kPairTile - 1) / (pairs * kPairTile);
   int tile_rows = round_up((ctx->V + 2 * pairs * rounds - 1) / (2 * pairs * rounds), 4);
   if (tile_rows < 8) tile_rows = 8;
@@ -2148,7 +2176,7 @@ Plan make_plan(const hola_ctx* ctx, int M, int w_dtype = HOLA_W_BF16) {
   if (mixed) tile_rows = kLanes;                 // a pair's tile is one group of 256 rows of one width
   best.tile_rows = tile_rows;
   best.n_ptiles = (ctx->V + 2 * tile_rows - 1) / (2 * tile_rows);
-  best.grid = 2 * (best.n_ptiles < pairs ? best.n_ptiles : pairs);
+  best.grid = 2 * (best.n_ptiles < pairs ? best.n_ptiles : pairs) * (best.fused ? best.passes : 1);
   best.n_kblocks = i8 ? (ctx->H + 2 * kBlockK - 1) / (2 * kBlockK) : (ctx->H + kBlockK - 1) / kBlockK;
   best.smem_bytes = stages * stage_bytes + kBarrierBytes + trans_bytes + 1024;
   return best;
@@ -2321,7 +2349,9 @@ hola_status run_lm_head(hola_ctx* ctx, const hola_verify_args* a, float* logits,
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  for (int pass = 0; pass < pl.passes; ++pass) {
+  kp.n_pass = pl.fused ? pl.passes : 1;
+  kp.rows_per_pass = pl.rows_per_pass;
+  for (int pass = 0; pass < (pl.fused ? 1 : pl.passes); ++pass) {
     kp.row0 = pass * pl.rows_per_pass;
     kp.rows = M - kp.row0 < pl.rows_per_pass ? M - kp.row0 : pl.rows_per_pass;
     if (kp.rows <= 0) break;
@@ -2581,7 +2611,7 @@ hola_status hola_plan_ex(const hola_ctx* ctx, int B, int k, int w_dtype, hola_pl
   if (B > ctx->maxB || k > ctx->maxK) return HOLA_ERR_UNSUPPORTED_SHAPE;
   const Plan pl = make_plan(ctx, B * (k + 1), w_dtype);
   out->tile_v = 2 * pl.tile_rows; out->grid = pl.grid; out->stages = pl.stages; out->rows_per_pass = pl.rows_per_pass;
-  out->passes = pl.passes; out->kernels_per_call = pl.passes + 1;
+  out->passes = pl.passes; out->kernels_per_call = (pl.fused ? 1 : pl.passes) + 1;
   return HOLA_OK;
 }
 
@@ -2599,6 +2629,7 @@ hola_status hola_set_option(hola_ctx* ctx, int option, int value) {
     case HOLA_OPT_ROTATING_UNITS: ctx->no_rot = value == 0; break;
     case HOLA_OPT_PAIR_MMA: ctx->no_pair256 = value == 0; break;
     case HOLA_OPT_HOST_IN_PLACE: ctx->host_in_place = value != 0; break;
+    case HOLA_OPT_FUSED_PASSES: ctx->no_fuse = value == 0; break;
     case HOLA_OPT_CONVERTER_GROUP:
       if (value < 0 || value > kConvWarps) return HOLA_ERR_INVALID_ARG;
       ctx->conv_group = value;

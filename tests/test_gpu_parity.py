@@ -898,3 +898,47 @@ def test_wide_head_config(binding):
     check_ranges(w, out)
     H = _np(out.entropy).reshape(-1)
     assert (H[0::2] < 1.5).mean() > 0.9 and (H[1::2] > 10).mean() > 0.9     # peaked and flat rows
+
+
+@pytest.mark.parametrize("B,k,H,V,weights", [
+    (150, 5, 256, 9000, "bf16"),       # 900 rows: several passes, the last one ragged; more tiles than groups of pairs
+    (150, 5, 256, 700, "bf16"),        # three tiles only: fewer tiles than groups of pairs
+    (100, 7, 128, 5000, "w8a8"),       # 800 rows on the 8-bit kind
+    (130, 3, 256, 4000, "mixed"),      # 520 rows, at most 256 per pass in the on-chip expansion
+])
+def test_all_passes_in_one_launch_match_the_oracle_and_the_launch_per_pass(binding, B, k, H, V, weights):
+    """More verify rows than one pass over W_lm holds: by default every pass runs in the same launch (groups of CTA
+    pairs share the vocabulary tiles, one pass each); the option brings back one launch per pass.  Same results, and
+    both agree with the oracle."""
+    w = workloads.gaussian_head("fused-passes", B, k, H, V, seed=B + V, device=DEV, w_std=0.3, sigma=1.0, sigma_far=0.2,
+                                tau=1.6)
+    kw, head, orc = {}, w.W_lm, None
+    if weights == "w8a8":
+        head, sc = binding.hola_quantize_w8(w.W_lm)
+        kw = dict(w_scale=sc, a8=True)
+    elif weights == "mixed":
+        widths = [[4, 8, 16][g % 3] for g in range(-(-V // 256))]
+        head = binding.hola_quantize_mixed(w.W_lm, widths)
+    with binding.HolaVerify(B, k, H, V) as ctx:
+        wd = {"bf16": binding.HOLA_W_BF16, "w8a8": binding.HOLA_W8A8, "mixed": binding.HOLA_W_MIXED}[weights]
+        plan = ctx.hola_plan(B, k, wd)
+        assert plan["passes"] >= 2 and plan["kernels_per_call"] == 2
+        one = ctx.hola_verify(w.hidden, head, w.draft_tok, w.draft_q, w.uniforms, w.tau, want_logits=True, **kw)
+        torch.cuda.synchronize()
+        ctx.hola_set_option(binding.HOLA_OPT_FUSED_PASSES, 0)
+        assert ctx.hola_plan(B, k, wd)["kernels_per_call"] == plan["passes"] + 1
+        per = ctx.hola_verify(w.hidden, head, w.draft_tok, w.draft_q, w.uniforms, w.tau, want_logits=True, **kw)
+        torch.cuda.synchronize()
+    assert int(one.status.item()) == 0 and int(per.status.item()) == 0
+    assert torch.equal(one.logits, per.logits)
+    assert torch.equal(one.accept_len, per.accept_len) and torch.equal(one.next_tok, per.next_tok)
+    assert torch.allclose(one.entropy, per.entropy, atol=2e-5) and torch.allclose(one.logZ, per.logZ, atol=2e-5)
+    if weights == "bf16":
+        check_against_oracle(binding, w, out=one, seqs=range(0, B, 7))
+    elif weights == "w8a8":
+        orc = _w8_oracle(w.slice(range(0, B, 9)), head, sc, a8=True)
+        pick = torch.arange(0, B, 9, device=DEV)
+        sub = w.slice(range(0, B, 9))
+        rep = compare.compare(orc, _np(sub.draft_q), _np(sub.uniforms), _np(one.accept_len[pick]), _np(one.next_tok[pick]),
+                              _np(one.entropy[pick]), _np(one.logZ[pick]), _np(one.logits[pick]))
+        assert rep.ok, rep.summary()
