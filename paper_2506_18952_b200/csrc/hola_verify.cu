@@ -72,6 +72,7 @@ constexpr int kW8EpiWarps = 8;
 constexpr int kConvWarps = kK1Warps - 2 - kW8EpiWarps;   // 8
 constexpr int kTmemCols = 512;
 constexpr int kMaxStages = 12;
+constexpr int kMaxPaceGroups = 128;              // groups of CTA pairs of a launch that holds all passes
 constexpr int kSmemBudget = 227 * 1024;          // dynamic shared memory per CTA on sm_100
 constexpr int kBarrierBytes = 512;
 constexpr long long kWaitLimitCycles = 4000000000ll;   // about 2 s of SM clock per wait, far above any legitimate wait
@@ -116,6 +117,7 @@ struct K1Params {
   float4* partials;   // [grid][part_stride] (m, s, t, arg-max index)
   int part_stride;
   unsigned* status;
+  unsigned* pace;     // n_pass > 1: one counter per group of pairs (zero at launch), by which the group keeps in step
 };
 
 struct K3Params {
@@ -251,11 +253,6 @@ __device__ __forceinline__ uint64_t l2_policy_evict_first() {
   asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
   return pol;
 }
-__device__ __forceinline__ uint64_t l2_policy_evict_normal() {
-  uint64_t pol;
-  asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(pol));
-  return pol;
-}
 __device__ __forceinline__ uint64_t l2_policy_evict_last() {
   uint64_t pol;
   asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
@@ -271,6 +268,21 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       " [%0], [%1, {%3, %4}], [%2], %5;"
       ::"r"(dst), "l"(map), "r"(cluster_bar), "r"(x), "r"(y), "l"(policy)
       : "memory");
+}
+
+// All passes in one launch: the pairs of a group read the same tile of W_lm, and only those that read it within the
+// few tens of microseconds a line stays in the L2 are spared the trip to HBM.  So before a new tile every producer
+// thread of the group counts itself in and waits, for a bounded time, until the others have done so too.  A pace
+// maker, not a barrier: when the time is up the thread goes on, and nothing depends on the others having arrived.
+constexpr long long kPaceLimitCycles = 60000;
+__device__ __forceinline__ void keep_pace(unsigned* counter, unsigned target) {
+  atomicAdd(counter, 1u);
+  const long long t0 = clock64();
+  while (true) {
+    unsigned seen;
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
+    if (seen >= target || clock64() - t0 > kPaceLimitCycles) break;
+  }
 }
 
 // Programmatic dependent launch: the grid may have been started while the kernel before it in the stream was still
@@ -681,8 +693,10 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (one per CTA)
     if (elect_one()) {
-      // W_lm is streamed once; with all passes in one launch the other pairs of the group read the tile out of the L2
-      const uint64_t pol_w = p.n_pass > 1 ? l2_policy_evict_normal() : l2_policy_evict_first();
+      // W_lm is streamed once.  (With all passes in one launch the other pairs of the group read the tile out of the L2
+      // within microseconds, the group keeping in step; measured, the lines still do best as the first to be evicted:
+      // they then never displace the hidden rows, which every pair re-reads for every tile.)
+      const uint64_t pol_w = l2_policy_evict_first();
       const uint64_t pol_h = l2_policy_evict_last();     // hidden is re-read for every tile
       const uint32_t leader_full = map_to_cta(full_bar, 0);
       const uint32_t own_rawfull = map_to_cta(rawfull_bar, rank);
@@ -696,6 +710,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
         // slot's previous use are done as well).  The hidden blocks of a slot are fetched by the converter group that
         // owns the K block, which waits for those MMAs anyway.
         for (int t = 0; t < my_tiles && ok; ++t) {
+          if (p.n_pass > 1 && p.pace && t > 0) keep_pace(p.pace + pair, static_cast<unsigned>(2 * p.n_pass * t));
           int tile_width = 8;                              // width of this tile's rows and where they are stored
           int w_row = (pair + t * npairs) * pair_rows + static_cast<int>(rank) * p.tile_rows;
           if (p.group_width) {
@@ -725,6 +740,7 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
       } else
       for (int t = 0; t < my_tiles && ok; ++t) {
         const int v0 = (pair + t * npairs) * pair_rows + static_cast<int>(rank) * p.tile_rows;
+        if (p.n_pass > 1 && p.pace && t > 0) keep_pace(p.pace + pair, static_cast<unsigned>(2 * p.n_pass * t));
         int kx = 0;                                      // K coordinate of the block, in elements
         for (int kb = 0; kb < p.n_kblocks; ++kb, kx += kKStep) {
           const uint32_t sa = base + stage * stage_bytes;
@@ -2023,6 +2039,7 @@ struct hola_ctx {
   float* logits;            // [max_rows][ldl]
   float4* partials;         // [num_sms][max_rows]
   unsigned* status;         // [1]
+  unsigned* pace;           // [kMaxPaceGroups] counters of the groups of pairs when all passes share a launch
   double* hq;               // [max_rows][kHqSlices] slice sums of q ln q over the draft rows
   signed char* hid8;        // [max_rows][H] int8 hidden rows (8-bit activation mode)
   float* hid_scale;         // [max_rows]
@@ -2035,6 +2052,7 @@ struct hola_ctx {
   int force_passes;           // tuning override: passes over W_lm (0: chosen by cost)
   int no_pair256;             // tuning override: rotating units always as three MMAs of N = 128
   int no_fuse;                // tuning override: several passes always as one launch each
+  int no_pace;                // tuning override: the groups of pairs of a fused launch do not keep in step
   int conv_group;             // tuning override (0 = by plan): converter warps per K block in the on-chip expansion
   int host_in_place;          // hola_verify_host: read draft rows not sent ahead in place from pinned host memory
   cudaStream_t copy_stream;   // hola_verify_host: the draft tensor travels here while the GEMM runs
@@ -2079,7 +2097,7 @@ OutBlock out_block(int B, int k) {
 }
 
 struct WsLayout {
-  size_t logits, partials, status, hq, hid8, hid_scale, st_hidden, st_tok, st_q, st_u, st_out, st_qtok, st_small_end, total;
+  size_t logits, partials, status, pace, hq, hid8, hid_scale, st_hidden, st_tok, st_q, st_u, st_out, st_qtok, st_small_end, total;
 };
 
 WsLayout ws_layout(int maxB, int maxK, int H, int V, int num_sms) {
@@ -2091,6 +2109,7 @@ WsLayout ws_layout(int maxB, int maxK, int H, int V, int num_sms) {
   w.logits = take(rows * ldl * 4);
   w.partials = take(static_cast<size_t>(num_sms) * rows * 16);
   w.status = take(4);
+  w.pace = take(4 * kMaxPaceGroups);
   w.hq = take(rows * kHqSlices * 8);
   w.hid8 = take(2 * align_up(rows, 32) * static_cast<size_t>(H));     // one or two 8-bit planes of the hidden rows
   w.hid_scale = take(2 * rows * 4);                                   // their scales (second plane after the first)
@@ -2351,6 +2370,12 @@ hola_status run_lm_head(hola_ctx* ctx, const hola_verify_args* a, float* logits,
   cfg.numAttrs = 2;
   kp.n_pass = pl.fused ? pl.passes : 1;
   kp.rows_per_pass = pl.rows_per_pass;
+  kp.pace = nullptr;
+  if (pl.fused && ctx->pace && !ctx->no_pace && pl.grid / (2 * pl.passes) <= kMaxPaceGroups) {
+    kp.pace = ctx->pace;
+    e = cudaMemsetAsync(ctx->pace, 0, sizeof(unsigned) * static_cast<size_t>(pl.grid / (2 * pl.passes)), stream);
+    if (e != cudaSuccess) { set_error(ctx, "reset of the pace counters", e); return HOLA_ERR_CUDA; }
+  }
   for (int pass = 0; pass < (pl.fused ? 1 : pl.passes); ++pass) {
     kp.row0 = pass * pl.rows_per_pass;
     kp.rows = M - kp.row0 < pl.rows_per_pass ? M - kp.row0 : pl.rows_per_pass;
@@ -2557,6 +2582,7 @@ hola_status hola_create(hola_ctx** out, int device, int maxB, int maxK, int H, i
   ctx->logits = reinterpret_cast<float*>(ctx->ws + w.logits);
   ctx->partials = reinterpret_cast<float4*>(ctx->ws + w.partials);
   ctx->status = reinterpret_cast<unsigned*>(ctx->ws + w.status);
+  ctx->pace = reinterpret_cast<unsigned*>(ctx->ws + w.pace);
   ctx->hq = reinterpret_cast<double*>(ctx->ws + w.hq);
   ctx->hid8 = reinterpret_cast<signed char*>(ctx->ws + w.hid8);
   ctx->hid_scale = reinterpret_cast<float*>(ctx->ws + w.hid_scale);
