@@ -423,7 +423,8 @@ def main():
         step()
     prof = ctx.hola_profile_end()
     clocks = sampler.summary(t_wall0, t_wall1)
-    k1_ms = prof["lm_head_ms"] / max(1, prof["calls"]) / plan["passes"]
+    k1_launches = plan["kernels_per_call"] - 1            # one per pass, or one in all when the passes share a launch
+    k1_ms = prof["lm_head_ms"] / max(1, prof["calls"]) / k1_launches
     k3_ms = prof["accept_sample_ms"] / max(1, prof["calls"])
 
     # end to end through hola_verify_host: pinned host inputs, copies and read-back inside the timed region
@@ -457,13 +458,13 @@ def main():
             work["step_bytes"] += delta
         # the 8-bit tensor-core kinds have twice the nominal rate of bf16: measured bf16 peak x 2 for --weights w8a8
         # (w8a16 runs two 8-bit rows per verify row: per algorithmic flop its peak is the bf16 one again)
-        roof = fractions(work, peaks, k1_ms * 1e-3 * plan["passes"], ms_max / args.steps * 1e-3,
+        roof = fractions(work, peaks, k1_ms * 1e-3 * k1_launches, ms_max / args.steps * 1e-3,
                          2.0 if a8 is True else 1.0)
         traffic = ncu_traffic_bytes(w) if args.weights == "bf16" else None
         roof["traffic"] = traffic
         roof["traffic_source"] = ("ncu capture summarised under profiles/ (a constant of this file, not measured by this "
                                   "run)") if traffic is not None else None
-        roof.update({"kernel": "lm_head_entropy_kernel", "kernel_ms": k1_ms, "launches_per_step": plan["passes"],
+        roof.update({"kernel": "lm_head_entropy_kernel", "kernel_ms": k1_ms, "launches_per_step": k1_launches,
                      "peak_source": f"of {peak_kind}", "accept_sample_ms": k3_ms,
                      "kernel_ms_note": "events between the launches of a separate loop: they keep the accept/sample "
                                        "kernel from starting under the GEMM kernel's tail as it does in the timed steps"})
