@@ -165,7 +165,8 @@ typedef enum {
                                      * in turn.  0 = the default (2)                                                  */
   HOLA_OPT_FUSED_PASSES = 9,        /* more verify rows than one pass over W_lm holds: 1 = all passes in one launch, in
                                      * which as many neighbouring CTA pairs as there are passes walk the same vocabulary
-                                     * tiles together (default), 0 = one launch per pass                             */
+                                     * tiles together and keep in step (default), 2 = the same without keeping in
+                                     * step, 0 = one launch per pass                                                 */
   HOLA_OPT_PASSES = 5               /* passes over W_lm the verify rows are split into: 0 = chosen by estimated cost
                                      * (default), else that many when the rows fit (at most 512 per pass)             */
 } hola_option;

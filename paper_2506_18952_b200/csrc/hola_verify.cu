@@ -2655,7 +2655,11 @@ hola_status hola_set_option(hola_ctx* ctx, int option, int value) {
     case HOLA_OPT_ROTATING_UNITS: ctx->no_rot = value == 0; break;
     case HOLA_OPT_PAIR_MMA: ctx->no_pair256 = value == 0; break;
     case HOLA_OPT_HOST_IN_PLACE: ctx->host_in_place = value != 0; break;
-    case HOLA_OPT_FUSED_PASSES: ctx->no_fuse = value == 0; break;
+    case HOLA_OPT_FUSED_PASSES:
+      if (value < 0 || value > 2) return HOLA_ERR_INVALID_ARG;
+      ctx->no_fuse = value == 0;
+      ctx->no_pace = value == 2;
+      break;
     case HOLA_OPT_CONVERTER_GROUP:
       if (value < 0 || value > kConvWarps) return HOLA_ERR_INVALID_ARG;
       ctx->conv_group = value;

@@ -930,6 +930,14 @@ def test_all_passes_in_one_launch_match_the_oracle_and_the_launch_per_pass(bindi
         per = ctx.hola_verify(w.hidden, head, w.draft_tok, w.draft_q, w.uniforms, w.tau, want_logits=True, **kw)
         torch.cuda.synchronize()
     assert int(one.status.item()) == 0 and int(per.status.item()) == 0
+    with binding.HolaVerify(B, k, H, V) as ctx:            # all passes in one launch, the groups of pairs free-running
+        ctx.hola_set_option(binding.HOLA_OPT_FUSED_PASSES, 2)
+        free = ctx.hola_verify(w.hidden, head, w.draft_tok, w.draft_q, w.uniforms, w.tau, want_logits=True, **kw)
+        torch.cuda.synchronize()
+        with pytest.raises(binding.HolaError):
+            ctx.hola_set_option(binding.HOLA_OPT_FUSED_PASSES, 3)
+    assert int(free.status.item()) == 0 and torch.equal(free.logits, one.logits)
+    assert torch.equal(free.accept_len, one.accept_len) and torch.equal(free.next_tok, one.next_tok)
     assert torch.equal(one.logits, per.logits)
     assert torch.equal(one.accept_len, per.accept_len) and torch.equal(one.next_tok, per.next_tok)
     assert torch.allclose(one.entropy, per.entropy, atol=2e-5) and torch.allclose(one.logZ, per.logZ, atol=2e-5)
