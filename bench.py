@@ -44,10 +44,12 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 NOMINAL_PEAKS = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of lm_head_entropy_kernel<0>, from the ncu captures
-# summarised under profiles/: "batched" (--set full capture) and "large_vocab" (a capture of the three DRAM / time
-# counters on the full-size launch; its logits are stored with the streaming hint, so most of the 197 MB reach DRAM
-# inside the kernel).  Other workloads, and the other weight modes, report null.
-NCU_TRAFFIC = {"batched": 265922304 + 8190720, "large_vocab": 1055559936 + 172039680}
+# summarised under profiles/: "batched" (--set full capture), "large_vocab" and "wide" (captures of the three DRAM /
+# time counters on the full-size launch; their logits are stored with the streaming hint, so most of them reach DRAM
+# inside the kernel; "wide" is the one launch that holds all six passes).  Other workloads, and the other weight modes,
+# report null.
+NCU_TRAFFIC = {"batched": 265923328 + 8595200, "large_vocab": 1055559936 + 172039680,
+               "wide": 2809281024 + 1177498112}
 
 
 def ncu_traffic_bytes(w):
