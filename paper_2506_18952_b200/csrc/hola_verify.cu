@@ -565,12 +565,13 @@ __device__ __forceinline__ void expand_int4x32(const uint4 x, uint8_t* d, uint32
   const uint32_t sub = sub1 | (sub1 << 16);
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
-    const uint32_t u = w[j] ^ 0x88888888u;
-    // entries (0,4), (1,5), (2,6), (3,7) of this word side by side in 16-bit lanes
-    const uint32_t r0 = bf16x2_fma((u & 0x000F000Fu) | 0x43004300u, mul, sub);
-    const uint32_t r1 = bf16x2_fma(((u >> 4) & 0x000F000Fu) | 0x43004300u, mul, sub);
-    const uint32_t r2 = bf16x2_fma(((u >> 8) & 0x000F000Fu) | 0x43004300u, mul, sub);
-    const uint32_t r3 = bf16x2_fma(((u >> 12) & 0x000F000Fu) | 0x43004300u, mul, sub);
+    // entries (0,4), (1,5), (2,6), (3,7) of this word side by side in 16-bit lanes; flipping the sign bit of the nibble
+    // and setting the bits of 128 are one exclusive-or with 0x4308 (the masked nibble has no bits there)
+    const uint32_t u = w[j];
+    const uint32_t r0 = bf16x2_fma((u & 0x000F000Fu) ^ 0x43084308u, mul, sub);
+    const uint32_t r1 = bf16x2_fma(((u >> 4) & 0x000F000Fu) ^ 0x43084308u, mul, sub);
+    const uint32_t r2 = bf16x2_fma(((u >> 8) & 0x000F000Fu) ^ 0x43084308u, mul, sub);
+    const uint32_t r3 = bf16x2_fma(((u >> 12) & 0x000F000Fu) ^ 0x43084308u, mul, sub);
     // back into channel order: (0,1) (2,3) (4,5) (6,7)
     *reinterpret_cast<uint4*>(d + ((16u * j) ^ x3)) =
         make_uint4(__byte_perm(r0, r1, 0x5410), __byte_perm(r2, r3, 0x5410), __byte_perm(r0, r1, 0x7632),
@@ -1006,8 +1007,12 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
             const int n_ok = min(32, min(p.N - c0, p.M - r0));   // columns that are real rows
             if (n_ok > 0) {
 #pragma unroll
-              for (int i = 0; i < 32; ++i)
-                if (i < n_ok) v[i] = scaled<kMode>(v[i], w_scale, p.h_scale, r0 + i);
+              for (int i0 = 0; i0 < 32; i0 += 8) {
+#pragma unroll
+                for (int i = i0; i < i0 + 8; ++i)
+                  if (i < n_ok) v[i] = scaled<kMode>(v[i], w_scale, p.h_scale, r0 + i);
+                if (kMode >= 2) asm volatile("" ::: "memory");   // the row scales eight at a time, not all 32 ahead
+              }
               if (vocab_ok) {
                 float* dst = p.logits + static_cast<size_t>(r0) * p.ldl + vocab;
                 if (n_ok == 32 && p.stream_logits) {
@@ -1079,8 +1084,12 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
           const int n_ok = min(32, min(p.N - c0, p.M - r0));   // columns that are real rows
           if (n_ok > 0) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i)
-              if (i < n_ok) v[i] = scaled<kMode>(v[i], w_scale, p.h_scale, r0 + i);
+            for (int i0 = 0; i0 < 32; i0 += 8) {
+#pragma unroll
+              for (int i = i0; i < i0 + 8; ++i)
+                if (i < n_ok) v[i] = scaled<kMode>(v[i], w_scale, p.h_scale, r0 + i);
+              if (kMode >= 2) asm volatile("" ::: "memory");     // the row scales eight at a time, not all 32 ahead
+            }
             if (vocab_ok) {
               float* dst = p.logits + static_cast<size_t>(r0) * p.ldl + vocab;
               if (n_ok == 32 && p.stream_logits) {       // (the common cases without a test per store)
