@@ -297,6 +297,9 @@ typedef struct {
 } hola_plan_info;
 hola_status hola_plan(const hola_ctx* ctx, int B, int k, hola_plan_info* out);            /* bf16 W_lm */
 hola_status hola_plan_ex(const hola_ctx* ctx, int B, int k, int w_dtype, hola_plan_info* out);
+/* The same for a shape alone: no context and no device (host arithmetic only), default tuning options.  num_sms is
+ * the SM count the grid is cut for (148 on a B200), rows = B (k + 1) verify rows. */
+hola_status hola_plan_for_shape(int num_sms, int H, int V, int rows, int w_dtype, hola_plan_info* out);
 
 /* Per-kernel timing for reports.  Between hola_profile_begin and hola_profile_end every hola_verify call (at
  * most max_calls of them, max_calls <= 4096) records CUDA events on its stream around the LM-head GEMM launches

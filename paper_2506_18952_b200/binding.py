@@ -24,7 +24,7 @@ HOLA_OPT_RING_SLOTS, HOLA_OPT_ROTATING_UNITS, HOLA_OPT_HOST_OVERLAP, HOLA_OPT_HO
 
 EXPORTS = ["hola_create", "hola_destroy", "hola_workspace_bytes", "hola_verify", "hola_verify_host",
            "hola_lm_head_entropy", "hola_accept_sample", "hola_host_traffic", "hola_shard_record_bytes", "hola_shard_lm_head",
-           "hola_shard_accept", "hola_shard_sample", "hola_lm_head_entropy_static", "hola_quantize_w8", "hola_quantize_w4", "hola_plan", "hola_plan_ex", "hola_set_option", "hola_selftest_bounded_wait", "hola_profile_begin", "hola_profile_end", "hola_strerror", "hola_last_cuda_error",
+           "hola_shard_accept", "hola_shard_sample", "hola_lm_head_entropy_static", "hola_quantize_w8", "hola_quantize_w4", "hola_plan", "hola_plan_ex", "hola_plan_for_shape", "hola_set_option", "hola_selftest_bounded_wait", "hola_profile_begin", "hola_profile_end", "hola_strerror", "hola_last_cuda_error",
            "hola_version"]
 
 
@@ -90,6 +90,8 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
                                      ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p]
     lib.hola_plan.restype = ctypes.c_int
     lib.hola_plan.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.POINTER(hola_plan_info)]
+    lib.hola_plan_for_shape.restype = ctypes.c_int
+    lib.hola_plan_for_shape.argtypes = [ctypes.c_int] * 5 + [ctypes.POINTER(hola_plan_info)]
     lib.hola_plan_ex.restype = ctypes.c_int
     lib.hola_plan_ex.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.POINTER(hola_plan_info)]
     lib.hola_profile_begin.restype = ctypes.c_int
@@ -449,3 +451,13 @@ class HolaVerify:
         _check(self.lib, self._ctx, self.lib.hola_verify_host(self._ctx, ctypes.byref(a), _stream_ptr(stream)),
                "hola_verify_host")
         return out
+
+
+def hola_plan_for_shape(num_sms: int, H: int, V: int, rows: int, w_dtype: int = 0) -> dict:
+    """Launch geometry for a shape alone (host arithmetic; needs the library, not a device)."""
+    lib = load_library()
+    info = hola_plan_info()
+    st = lib.hola_plan_for_shape(int(num_sms), int(H), int(V), int(rows), int(w_dtype), ctypes.byref(info))
+    if st != 0:
+        raise HolaError(f"hola_plan_for_shape: status {st}")
+    return {n: getattr(info, n) for n, _ in hola_plan_info._fields_}

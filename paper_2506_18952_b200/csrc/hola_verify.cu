@@ -2640,6 +2640,20 @@ hola_status hola_destroy(hola_ctx* ctx) {
   return HOLA_OK;
 }
 
+hola_status hola_plan_for_shape(int num_sms, int H, int V, int rows, int w_dtype, hola_plan_info* out) {
+  if (!out || num_sms < 2 || H <= 0 || V <= 0 || rows <= 0) return HOLA_ERR_INVALID_ARG;
+  if (w_dtype < HOLA_W_BF16 || w_dtype > HOLA_W_MIXED) return HOLA_ERR_INVALID_ARG;
+  if (H % 8 != 0 || V > kMaxChunks * kChunk) return HOLA_ERR_UNSUPPORTED_SHAPE;
+  hola_ctx* c = static_cast<hola_ctx*>(calloc(1, sizeof(hola_ctx)));     // only the fields make_plan reads
+  if (!c) return HOLA_ERR_WORKSPACE;
+  c->num_sms = num_sms; c->H = H; c->V = V;
+  const Plan pl = make_plan(c, rows, w_dtype);
+  free(c);
+  out->tile_v = 2 * pl.tile_rows; out->grid = pl.grid; out->stages = pl.stages; out->rows_per_pass = pl.rows_per_pass;
+  out->passes = pl.passes; out->kernels_per_call = (pl.fused ? 1 : pl.passes) + 1;
+  return HOLA_OK;
+}
+
 hola_status hola_plan_ex(const hola_ctx* ctx, int B, int k, int w_dtype, hola_plan_info* out) {
   if (!ctx || !out || B < 0 || k < 0) return HOLA_ERR_INVALID_ARG;
   if (w_dtype < HOLA_W_BF16 || w_dtype > HOLA_W_MIXED) return HOLA_ERR_INVALID_ARG;

@@ -75,3 +75,43 @@ def test_product_package_does_not_touch_the_oracle():
                 src = open(os.path.join(dirpath, f)).read()
                 assert not re.search(r"^\s*(from|import)\s+oracle\b", src, flags=re.M), f"{f} imports the oracle"
                 assert "oracle/" not in src and "hola_verify_ref" not in src, f"{f} reaches into the oracle"
+
+
+def test_launch_geometry_for_shapes_without_a_device():
+    """hola_plan_for_shape is host arithmetic: the split of the verify rows into passes and of the grid into pairs (and,
+    when the passes share a launch, into groups of pairs that walk the same vocabulary tiles) must hold for any shape."""
+    from paper_2506_18952_b200 import binding as b
+    sms = 148
+    expansion = (b.HOLA_W_INT8, b.HOLA_W_MIXED)
+    for H, V in ((64, 8), (128, 700), (256, 4000), (4096, 32000), (4096, 128256), (8192, 128256), (1024, 524288)):
+        for rows in (1, 5, 16, 192, 256, 257, 384, 385, 512, 513, 900, 2304, 5000, 40000):
+            for wd in (b.HOLA_W_BF16, b.HOLA_W_INT8, b.HOLA_W8A8, b.HOLA_W8A16, b.HOLA_W_MIXED):
+                if wd == b.HOLA_W_MIXED and H % 128:
+                    continue
+                p = b.hola_plan_for_shape(sms, H, V, rows, wd)
+                what = (H, V, rows, wd, p)
+                cap = 256 if wd in expansion or wd == b.HOLA_W8A16 else 512
+                assert 1 <= p["rows_per_pass"] <= cap, what
+                assert p["passes"] == -(-rows // p["rows_per_pass"]), what            # no empty pass, every row covered
+                assert p["grid"] % 2 == 0 and 2 <= p["grid"] <= sms, what
+                assert 2 <= p["stages"] <= 12, what
+                assert 16 <= p["tile_v"] <= 256 and p["tile_v"] % 8 == 0, what
+                tiles = -(-V // p["tile_v"])
+                if p["passes"] > 1 and p["kernels_per_call"] == 2:                      # all passes in one launch
+                    assert p["passes"] <= sms // 2, what
+                    assert p["grid"] % (2 * p["passes"]) == 0, what
+                    groups = p["grid"] // (2 * p["passes"])
+                    assert 1 <= groups <= tiles, what                                   # every group has a tile
+                else:
+                    assert p["kernels_per_call"] == p["passes"] + 1, what
+                    assert p["grid"] // 2 <= tiles, what
+                if p["passes"] > sms // 2:
+                    assert p["kernels_per_call"] == p["passes"] + 1, what               # more passes than pairs: a launch each
+    # the shapes the bench runs
+    assert b.hola_plan_for_shape(sms, 4096, 128256, 384)["passes"] == 1
+    wide = b.hola_plan_for_shape(sms, 8192, 128256, 2304)
+    assert wide["passes"] == 6 and wide["rows_per_pass"] == 384 and wide["kernels_per_call"] == 2 and wide["grid"] == 144
+    for bad in ((1, 4096, 32000, 5, 0), (sms, 4097, 32000, 5, 0), (sms, 4096, 0, 5, 0), (sms, 4096, 32000, 0, 0),
+                (sms, 4096, 32000, 5, 9)):
+        with pytest.raises(b.HolaError):
+            b.hola_plan_for_shape(*bad)
