@@ -1216,21 +1216,23 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
     uint32_t e[8];
     if (grp < ngroups && grp < total_blocks) {
       tile_info(t, tile_width, w_row);
-      fetch_shifts(kb, tile_width, w_row, e);
+      if (tile_width == 4) fetch_shifts(kb, tile_width, w_row, e);
     }
+    int stage = grp;                                     // ring slot and phase of block i (grp < ngroups <= stages)
+    uint32_t phase = 0;
     for (int i = grp; i < total_blocks && grp < ngroups; i += ngroups) {
-      const int stage = i % p.stages;
-      const uint32_t phase = static_cast<uint32_t>(i / p.stages) & 1u;
       uint8_t* slot = smem + stage * stage_bytes;
       uint32_t shifts = 0;                               // one nibble per step
+      if (tile_width == 4) {
 #pragma unroll
-      for (int n = 0; n < 8; ++n) shifts |= min(e[n], 4u) << (4 * n);
+        for (int n = 0; n < 8; ++n) shifts |= min(e[n], 4u) << (4 * n);
+      }
       // the group's next block: its exponents are fetched while this block is waited for and expanded
       int t2 = t, kb2 = kb + ngroups, width2 = tile_width, w_row2 = w_row;
       while (kb2 >= p.n_kblocks) { kb2 -= p.n_kblocks; ++t2; }
       if (i + ngroups < total_blocks) {
         if (t2 != t) tile_info(t2, width2, w_row2);
-        fetch_shifts(kb2, width2, w_row2, e);
+        if (width2 == 4) fetch_shifts(kb2, width2, w_row2, e);
       }
       // first the slot's previous use (which implies that its raw block's previous phase is over), then this block's bytes
       if (!mbar_wait_warp(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.status)) break;
@@ -1278,6 +1280,8 @@ lm_head_entropy_kernel(const __grid_constant__ CUtensorMap tmap_hidden, const __
         mbar_arrive(rawempty_bar + 8 * stage);           // and the raw block may be refilled
       }
       t = t2; kb = kb2; tile_width = width2; w_row = w_row2;
+      stage += ngroups;
+      if (stage >= p.stages) { stage -= p.stages; phase ^= 1u; }
     }
   }
 
