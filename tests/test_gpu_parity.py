@@ -950,3 +950,26 @@ def test_all_passes_in_one_launch_match_the_oracle_and_the_launch_per_pass(bindi
         rep = compare.compare(orc, _np(sub.draft_q), _np(sub.uniforms), _np(one.accept_len[pick]), _np(one.next_tok[pick]),
                               _np(one.entropy[pick]), _np(one.logZ[pick]), _np(one.logits[pick]))
         assert rep.ok, rep.summary()
+
+
+def test_split_entry_points_on_a_shape_with_several_passes(binding):
+    """hola_lm_head_entropy (steps 1-2, statistics finished by the small finalising kernel) and hola_accept_sample
+    (steps 3-5 from given logits) on 600 verify rows, which take several passes in one launch: the same logits, entropy,
+    logZ and decisions as hola_verify, whose results the oracle checks."""
+    w = workloads.gaussian_head("split-passes", 100, 5, 256, 6000, seed=41, device=DEV, w_std=0.3, sigma=1.0, sigma_far=0.2,
+                                tau=1.6)
+    with binding.HolaVerify(w.B, w.k, w.H, w.V) as ctx:
+        assert ctx.hola_plan(w.B, w.k)["passes"] >= 2 and ctx.hola_plan(w.B, w.k)["kernels_per_call"] == 2
+        whole = ctx.hola_verify(w.hidden, w.W_lm, w.draft_tok, w.draft_q, w.uniforms, w.tau, want_logits=True)
+        torch.cuda.synchronize()
+        first = ctx.hola_lm_head_entropy(w.hidden, w.W_lm, want_logits=True)
+        torch.cuda.synchronize()
+        assert torch.equal(first.logits, whole.logits)
+        assert torch.allclose(first.entropy, whole.entropy, atol=2e-5) and torch.allclose(first.logZ, whole.logZ, atol=2e-5)
+        second = ctx.hola_accept_sample(first.logits, first.entropy, first.logZ, w.draft_tok, w.draft_q, w.uniforms, w.tau)
+        torch.cuda.synchronize()
+    # (the statistics went through fp32 outputs on the way: a decision within 2e-5 of a tie may differ)
+    same = (second.accept_len == whole.accept_len)
+    assert int((~same).sum().item()) <= 1
+    assert torch.equal(second.next_tok[same], whole.next_tok[same])
+    check_against_oracle(binding, w, out=whole, seqs=range(0, w.B, 9))
