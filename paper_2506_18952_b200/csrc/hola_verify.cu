@@ -10,11 +10,15 @@
 //       both halves.  Sixteen epilogue warps copy finished accumulators to the fp32 logits buffer and, from the
 //       same registers transposed through a small shared-memory buffer, keep per verify position the running
 //       softmax statistics (m, s, t) = (max, sum e^(l-m), sum e^(l-m)(l-m)) and the arg-max in registers, in the
-//       shadow of the next tile's MMAs.  W_lm is read from HBM once per pass; the logits are never read back.
+//       shadow of the next tile's MMAs.  W_lm is read from HBM once; the logits are never read back.  More verify
+//       rows than one pass holds (at most 512): all passes run in the same launch, on groups of neighbouring pairs
+//       that walk the same vocabulary tiles in step, one pass each, so that a tile still leaves HBM once and reaches
+//       the other pairs of its group out of the L2.
 //       With 257..384 verify rows the accumulators rotate over the four 128-column units of the tensor memory and a
 //       unit is handed back as soon as its chunk has gone to the logits buffer and a staging buffer.  In its
 //       on-chip-expansion mode the kernel streams groups of 256 vocabulary rows stored at 4, 8 or 16 bits and
-//       converter warps expand the codes exactly to bf16 (mixed-precision quantiser of the Lo-Bi Optimization section).
+//       converter warps (groups of two, each owning whole K blocks) expand the codes exactly to bf16 (mixed-precision
+//       quantiser of the Lo-Bi Optimization section).
 //   quantize_rows_int8_kernel   8-bit case of the Lo-Bi quantiser, per row (W_lm ahead of time, hidden rows per call).
 //   quantize_rows_w4_kernel     4-bit case: codes in [-7, 7] with one shared exponent per sub-block of 128 channels.
 //   bounded_wait_selftest_kernel  a wait that is made to run out, to exercise the give-up path without breaking anything.
