@@ -171,6 +171,15 @@ def test_converter_group_size_changes_speed_not_results(binding):
             for bad in (-1, 9):
                 with pytest.raises(binding.HolaError):
                     ctx.hola_set_option(binding.HOLA_OPT_CONVERTER_GROUP, bad)
+            # fewer ring slots than groups of converter warps: only as many groups as slots take part
+            for slots, G in ((2, 1), (3, 2), (2, 4)):
+                ctx.hola_set_option(binding.HOLA_OPT_RING_SLOTS, slots)
+                ctx.hola_set_option(binding.HOLA_OPT_CONVERTER_GROUP, G)
+                assert ctx.hola_plan(B, k, binding.HOLA_W_MIXED)["stages"] == slots
+                out = ctx.hola_verify(w.hidden, head, w.draft_tok, w.draft_q, w.uniforms, w.tau, want_logits=True)
+                torch.cuda.synchronize()
+                assert int(out.status.item()) == 0, (slots, G)
+                assert torch.equal(out.logits, base.logits), (slots, G)
     orc = _mixed_oracle(w, _widths(V, [4, 8, 16, 8, 4]))
     rep = compare.compare(orc, _np(w.draft_q), _np(w.uniforms), _np(base.accept_len), _np(base.next_tok),
                           _np(base.entropy), _np(base.logZ), _np(base.logits))
